@@ -1,0 +1,181 @@
+/*
+ * cafeq.h - C ABI of the CafeQ per-matrix optimisation path on one NVIDIA B200 (sm_100a).
+ *
+ * CafeQ (arXiv 2511.19705) quantises a weight matrix W after applying a learned invertible
+ * transform M, chosen without calibration data by minimising a proxy of the quantisation error:
+ *   single matrix  (Section 4, Eq. 3):   || M^-1 Q(M W) - W ||_F ,  M block-diagonal (Section 4.1)
+ *   coupled pair   (Section 4.2, Eq. 5): || Q(W1 M) Q(M^-1 W2) - W1 W2 ||_F  (PQE)
+ * trained through differentiable surrogates (Eq. 4; the LogSumExp of channel maxima, Section 4.2)
+ * and, for pairs, followed by the alternating adaptive rounding of Algorithm 1 (Section 5).
+ *
+ * Conventions of this library
+ *   - A weight is row-major [d_out, d_in] bf16 with `ld` elements between rows.  Quantisation
+ *     groups are `group` consecutive entries along d_in (0 = one group per row); one fp32 scale
+ *     per (row, group): s = absmax / qmax, qmax = 2^(bits-1) - 1, code = clamp(rne(u / s)).
+ *   - A block-diagonal operator is fp32 T[nbT][k][k] (row-major blocks).  On CAFEQ_AXIS_IN it acts
+ *     on the d_in index:  U[o, B*k+i] = sum_j T[B/replicas][i][j] W[o, B*k+j];  on CAFEQ_AXIS_OUT
+ *     on the d_out index: U[B*k+i, c] = sum_j T[B/replicas][i][j] W[B*k+j, c].  `replicas`
+ *     consecutive blocks of the matrix share one operator block (grouped-query heads).
+ *     CAFEQ_APPLY_TT applies the transpose of every block instead.
+ *   - Every operand of a transform product is rounded to bf16 first (the tensor-core operand
+ *     type); products accumulate in fp32.  The transform that is deployed is therefore bf16(M).
+ *   - All pointers are DEVICE pointers unless the comment says "host".  Every call only enqueues
+ *     work on `stream` (a cudaStream_t passed as void*; NULL = default stream) and returns; results
+ *     are valid after the caller synchronises that stream.  No call allocates or frees device
+ *     memory: scratch comes from the caller's workspace `ws` (size from cafeq_workspace_size,
+ *     256-byte aligned).  Calls that share a workspace must be ordered on one stream.
+ *   - Return value: a cafeq_status.  Argument errors are found on the host before anything is
+ *     launched and leave all outputs untouched.  Conditions found on the device (a singular block,
+ *     a non-finite value) are written to the int32 `status` word (first error wins; the caller
+ *     zeroes it) and later kernels of the same call skip their work.
+ */
+#ifndef CAFEQ_H_
+#define CAFEQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CAFEQ_OK = 0,
+  CAFEQ_ERR_INVALID_ARG = 1,
+  CAFEQ_ERR_UNSUPPORTED = 2, /* shape / bits / group combination not covered */
+  CAFEQ_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  CAFEQ_ERR_CUDA = 4,        /* a launch failed; cudaGetLastError has the detail */
+  CAFEQ_ERR_SINGULAR = 5,    /* device: a transform block has no usable pivot */
+  CAFEQ_ERR_NONFINITE = 6,   /* device: NaN or Inf met in a transformed weight */
+  CAFEQ_ERR_TIMEOUT = 7      /* device: a bounded wait inside a kernel ran out */
+} cafeq_status;
+
+enum { CAFEQ_AXIS_IN = 0, CAFEQ_AXIS_OUT = 1 };
+enum { CAFEQ_APPLY_T = 0, CAFEQ_APPLY_TT = 1 };
+enum { CAFEQ_PREC_BF16 = 0 };
+/* loss kinds: what the backward pass differentiates */
+enum {
+  CAFEQ_LOSS_SURROGATE = 0, /* single: Eq. 4 */
+  CAFEQ_LOSS_L2_STE = 1,    /* single: Eq. 3 with a straight-through rounding derivative */
+  CAFEQ_LOSS_LSE = 2,       /* pair: LogSumExp of group maxima (+ orthonormality penalty) */
+  CAFEQ_LOSS_PQE_STE = 3    /* pair: Eq. 5 squared, straight-through */
+};
+enum { CAFEQ_OPT_GD = 0, CAFEQ_OPT_ADAM = 1 };
+/* flags for the forward/backward calls */
+enum {
+  CAFEQ_FLAG_EXACT_LOSS = 1, /* also evaluate the quantised loss (l2 proxy / PQE) */
+  CAFEQ_FLAG_NO_GRAD = 2,    /* forward only */
+  CAFEQ_FLAG_GENERIC = 4     /* force the shape-agnostic kernels (debugging aid) */
+};
+enum { CAFEQ_ROUND_ALG1 = 0 };
+enum { CAFEQ_OFFSETS_NONE = 0, CAFEQ_OFFSETS_HARD_U8 = 1, CAFEQ_OFFSETS_SOFT_F32 = 2 };
+
+/* One weight matrix and how it is transformed and quantised. */
+typedef struct {
+  uint32_t struct_size; /* sizeof(cafeq_matrix_desc), for versioning */
+  int32_t d_out, d_in;  /* W is [d_out, d_in] row-major bf16 */
+  int64_t ld;           /* elements between rows, >= d_in */
+  int32_t bits;         /* 2..8 */
+  int32_t group;        /* along d_in; 0 => per-channel */
+  int32_t tblock;       /* transform block size k; 0 => no transform */
+  int32_t taxis;        /* CAFEQ_AXIS_IN | CAFEQ_AXIS_OUT */
+  int32_t trole;        /* CAFEQ_APPLY_T | CAFEQ_APPLY_TT (how cafeq_rtn uses the operator it is given) */
+  int32_t replicas;     /* consecutive matrix blocks sharing one operator block, >= 1 */
+  int32_t compute_prec; /* CAFEQ_PREC_BF16 */
+} cafeq_matrix_desc;
+
+/* Optimiser and loss settings (Section 4.1: gradient descent; Appendix D: Adam, t, lambda_orth). */
+typedef struct {
+  uint32_t struct_size;
+  int32_t loss_kind;  /* CAFEQ_LOSS_* */
+  int32_t optimizer;  /* CAFEQ_OPT_* */
+  float lr, beta1, beta2, eps;
+  float lambda_orth;  /* weight of ||M M^T - I||_F / sqrt(h) (pairs) */
+  float lse_t;        /* LogSumExp temperature t (pairs) */
+  float kappa;        /* constant of Eq. 4; <= 0 selects 1/(2^bits - 1)^2 */
+  int32_t steps;
+  int32_t eval_every; /* evaluate the quantised loss every n steps (0 = never) */
+} cafeq_opt_cfg;
+
+/* Scratch bytes needed by any call on d1 (and d2 for pair calls; NULL otherwise).  cfg may be NULL.
+ * `bytes` is a host pointer.  The same size serves every entry point below for these descriptors. */
+int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
+                         size_t* bytes);
+
+/* Round-to-nearest quantisation of T o W (Eq. 1 in its symmetric absmax form, after the transform of
+ * Section 4): codes int8 [d_out, d_in] (row stride d_in), scales fp32 [d_out, d_in/group].
+ * T = NULL or tblock = 0 quantises W itself.  T is used as given (CAFEQ_APPLY_T) or transposed; no
+ * inverse is taken here. */
+int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
+              void* ws, size_t ws_bytes, void* stream);
+
+/* One forward+backward evaluation for a single matrix (Section 4.1).
+ *   M       [nb,k,k] fp32 transform parameters; the transform applied is bf16(M).
+ *   Minv    optional out [nb,k,k]: inverse of bf16(M) as computed on the device.
+ *   offsets optional rounding offsets [d_out,d_in] (row stride d_in): uint8 {0,1} or fp32 in [0,1]
+ *           (offsets_kind); code = clamp(floor(u/s) + offset) instead of round-to-nearest.
+ *   losses  out fp32[4]: {surrogate (Eq. 4), ||M^-1 Q(MW) - W||_F^2 (Eq. 3), ||W||_F^2, 0};
+ *           entries 1,2 only with CAFEQ_FLAG_EXACT_LOSS or loss_kind = CAFEQ_LOSS_L2_STE.
+ *   gradM   out [nb,k,k] fp32 gradient of the chosen loss (ignored with CAFEQ_FLAG_NO_GRAD).
+ * The operator is M on d->taxis (trole is ignored: the parameter itself is applied). */
+int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* W, const float* M, float* Minv,
+                             const void* offsets, int offsets_kind, int loss_kind, float kappa, int flags,
+                             float* losses, float* gradM, int32_t* status, void* ws, size_t ws_bytes,
+                             void* stream);
+
+/* `cfg->steps` optimisation steps on a single matrix (Section 4.1: gradient descent on Eq. 4 from the
+ * caller's initial M; Adam selectable).  M is updated in place (fp32 master parameters).
+ * opt_state: fp32 [1 + 2*nb*k*k] = {step count, first moments, second moments} (Adam; may be NULL for GD);
+ * carrying it over between calls resumes a run exactly.  loss_history: out fp32 [steps, 2] =
+ * {surrogate, quantised loss or NaN when not evaluated at that step}. */
+int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, float* M, float* opt_state,
+                          const cafeq_opt_cfg* cfg, float* loss_history, int32_t* status, void* ws,
+                          size_t ws_bytes, void* stream);
+
+/* P = W1 W2 of Section 4.2 in stored layout: W1 is stored [h, d1] (= W1^T), W2 is stored [d3, r*h]
+ * (= W2^T), r = d2->replicas; P[x, y] = sum_j W1[(B/r)*k + j', x] W2[y, B*k + j'] over all blocks B of W2.
+ * P is fp32 [d1, d3] row-major. */
+int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                       const void* W2, float* P, void* ws, size_t ws_bytes, void* stream);
+
+/* One forward+backward evaluation for a coupled pair (Section 4.2).  d1 describes W1 (stored [h, d1],
+ * transformed on CAFEQ_AXIS_OUT by M^T, i.e. U = W1 M), d2 describes W2 (stored [d3, r*h], transformed
+ * on CAFEQ_AXIS_IN by bf16(inv(bf16(M))), i.e. V = M^-1 W2).  d1->tblock == d2->tblock == k,
+ * M is [h/k, k, k].
+ *   P       optional fp32 [d1, d3] from cafeq_pair_product; needed for PQE.
+ *   losses  out fp32[4]: {LSE + lambda*orth, LSE, orth penalty, PQE^2 (Eq. 5 squared) or 0}.
+ *   gradM   out [h/k, k, k]. */
+int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                            const void* W2, const float* M, const float* P, int loss_kind, float lse_t,
+                            float lambda_orth, int flags, float* losses, float* gradM, int32_t* status,
+                            void* ws, size_t ws_bytes, void* stream);
+
+/* `cfg->steps` optimisation steps on a pair (Appendix D: Adam on the LogSumExp surrogate with the
+ * orthonormality penalty).  loss_history: out fp32 [steps, 2] = {loss, PQE^2 or NaN}.  P as above
+ * (NULL => PQE never evaluated). */
+int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                        const void* W2, float* M, float* opt_state, const float* P, const cafeq_opt_cfg* cfg,
+                        float* loss_history, int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1 (Section 5) on the transformed pair U = W1 M, V = M^-1 W2 with Q = the group quantiser of
+ * each descriptor: codes1/scales1 for U (stored [h, d1]), codes2/scales2 for V (stored [d3, r*h]);
+ * pqe_history: out fp32 [2*iters + 1], the product error after independent rounding and after every
+ * half-iteration.  M = NULL rounds the untransformed pair. */
+int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                         const void* W2, const float* M, int iters, int mode, int8_t* codes1, float* scales1,
+                         int8_t* codes2, float* scales2, float* pqe_history, int32_t* status, void* ws,
+                         size_t ws_bytes, void* stream);
+
+/* Pack int8 codes [d_out, d_in] (row stride d_in) into `bits`-bit fields: u = q + qmax, little-endian bit
+ * stream along d_in per row, row stride d_in*bits/8 bytes (4-bit: low nibble first; 3-bit: code i at
+ * bits 3i..3i+2).  The paper fixes no layout (Section 5 only asks for fast dequantisation); this is the
+ * library's.  d_in*bits must be a multiple of 8. */
+int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed, void* stream);
+
+const char* cafeq_status_string(int status);
+int cafeq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAFEQ_H_ */

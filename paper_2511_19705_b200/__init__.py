@@ -1,0 +1,275 @@
+"""Thin Python binding of the CafeQ C-ABI library (include/cafeq.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of
+``libcafeq.so``.  PyTorch supplies device memory and the current stream.  There is
+no CPU fallback: if the library has not been built, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcafeq.so")
+
+AXIS_IN, AXIS_OUT = 0, 1
+APPLY_T, APPLY_TT = 0, 1
+LOSS_SURROGATE, LOSS_L2_STE, LOSS_LSE, LOSS_PQE_STE = 0, 1, 2, 3
+OPT_GD, OPT_ADAM = 0, 1
+FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC = 1, 2, 4
+OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
+
+EXPORTS = [
+    "cafeq_workspace_size", "cafeq_rtn", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
+    "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
+    "cafeq_pack", "cafeq_status_string", "cafeq_version",
+]
+
+
+class MatrixDesc(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("d_out", ctypes.c_int32), ("d_in", ctypes.c_int32),
+                ("ld", ctypes.c_int64), ("bits", ctypes.c_int32), ("group", ctypes.c_int32),
+                ("tblock", ctypes.c_int32), ("taxis", ctypes.c_int32), ("trole", ctypes.c_int32),
+                ("replicas", ctypes.c_int32), ("compute_prec", ctypes.c_int32)]
+
+
+class OptCfg(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("loss_kind", ctypes.c_int32), ("optimizer", ctypes.c_int32),
+                ("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+                ("eps", ctypes.c_float), ("lambda_orth", ctypes.c_float), ("lse_t", ctypes.c_float),
+                ("kappa", ctypes.c_float), ("steps", ctypes.c_int32), ("eval_every", ctypes.c_int32)]
+
+
+class CafeqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2511_19705_b200.build` (nvcc, sm_100a)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.cafeq_status_string.restype = ctypes.c_char_p
+        L.cafeq_status_string.argtypes = [ctypes.c_int]
+        L.cafeq_version.restype = ctypes.c_int
+        for name in EXPORTS[:-2]:
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().cafeq_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return lib().cafeq_version()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != 0:
+        raise CafeqError(rc, where)
+
+
+def _p(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    if isinstance(t, torch.Tensor):
+        return ctypes.c_void_p(t.data_ptr())
+    return ctypes.c_void_p(int(t))
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_desc(d_out, d_in, bits, group, tblock=0, taxis=AXIS_IN, trole=APPLY_T, replicas=1, ld=None) -> MatrixDesc:
+    return MatrixDesc(ctypes.sizeof(MatrixDesc), d_out, d_in, d_in if ld is None else ld, bits, group, tblock,
+                      taxis, trole, replicas, 0)
+
+
+def make_cfg(loss_kind=LOSS_SURROGATE, optimizer=OPT_GD, lr=0.5, beta1=0.1, beta2=0.999, eps=1e-8,
+             lambda_orth=0.1, lse_t=5.0, kappa=0.0, steps=1, eval_every=0) -> OptCfg:
+    return OptCfg(ctypes.sizeof(OptCfg), loss_kind, optimizer, lr, beta1, beta2, eps, lambda_orth, lse_t, kappa,
+                  steps, eval_every)
+
+
+def workspace_size(d1: MatrixDesc, d2: MatrixDesc | None = None, cfg: OptCfg | None = None) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().cafeq_workspace_size(ctypes.byref(d1), ctypes.byref(d2) if d2 is not None else None,
+                                    ctypes.byref(cfg) if cfg is not None else None, ctypes.byref(n))
+    _check(rc, "cafeq_workspace_size")
+    return int(n.value)
+
+
+_ws_cache: dict = {}
+
+
+def workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A cached uint8 scratch tensor of at least nbytes (torch allocations are 512-byte aligned)."""
+    key = str(device)
+    t = _ws_cache.get(key)
+    if t is None or t.numel() < nbytes:
+        _ws_cache[key] = t = torch.empty(int(nbytes), dtype=torch.uint8, device=device)
+    return t
+
+
+def _bits_tensor(W: torch.Tensor) -> torch.Tensor:
+    if W.dtype != torch.bfloat16 or not W.is_cuda or W.dim() != 2 or W.stride(1) != 1:
+        raise ValueError("W must be a 2-D CUDA bf16 tensor with unit inner stride")
+    return W
+
+
+def _f32(t, name):
+    if t is None:
+        return None
+    if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA float32 tensor")
+    return t
+
+
+# ----------------------------------------------------------------------------- entry points
+def cafeq_rtn(W, T=None, *, bits, group, tblock=0, taxis=AXIS_IN, trole=APPLY_T, replicas=1):
+    """Round-to-nearest codes (int8 [d_out,d_in]) and scales (fp32 [d_out, d_in/group]) of T o W."""
+    W = _bits_tensor(W)
+    d_out, d_in = W.shape
+    d = make_desc(d_out, d_in, bits, group, tblock if T is not None else 0, taxis, trole, replicas, W.stride(0))
+    g = group or d_in
+    codes = torch.empty((d_out, d_in), dtype=torch.int8, device=W.device)
+    scales = torch.empty((d_out, d_in // g), dtype=torch.float32, device=W.device)
+    ws = workspace(workspace_size(d), W.device)
+    rc = lib().cafeq_rtn(ctypes.byref(d), _p(W), _p(_f32(T, "T")), _p(codes), _p(scales), _p(ws),
+                         ctypes.c_size_t(ws.numel()), _stream())
+    _check(rc, "cafeq_rtn")
+    return codes, scales
+
+
+def cafeq_proxy_loss_fwd_bwd(W, M, *, bits, group, taxis=AXIS_IN, loss_kind=LOSS_SURROGATE, kappa=0.0, flags=0,
+                             offsets=None, want_minv=False):
+    """Returns dict(losses[4], gradM or None, Minv or None, status int tensor)."""
+    W = _bits_tensor(W)
+    M = _f32(M, "M")
+    d_out, d_in = W.shape
+    k = M.shape[-1]
+    d = make_desc(d_out, d_in, bits, group, k, taxis, APPLY_T, 1, W.stride(0))
+    losses = torch.zeros(4, dtype=torch.float32, device=W.device)
+    gradM = None if (flags & FLAG_NO_GRAD) else torch.empty_like(M)
+    Minv = torch.empty_like(M) if want_minv else None
+    status = torch.zeros(1, dtype=torch.int32, device=W.device)
+    okind = OFFSETS_NONE
+    if offsets is not None:
+        okind = OFFSETS_HARD_U8 if offsets.dtype == torch.uint8 else OFFSETS_SOFT_F32
+        if not offsets.is_contiguous() or tuple(offsets.shape) != (d_out, d_in):
+            raise ValueError("offsets must be contiguous [d_out, d_in]")
+    ws = workspace(workspace_size(d), W.device)
+    rc = lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(d), _p(W), _p(M), _p(Minv), _p(offsets), ctypes.c_int(okind),
+                                        ctypes.c_int(loss_kind), ctypes.c_float(kappa), ctypes.c_int(flags),
+                                        _p(losses), _p(gradM), _p(status), _p(ws), ctypes.c_size_t(ws.numel()),
+                                        _stream())
+    _check(rc, "cafeq_proxy_loss_fwd_bwd")
+    return dict(losses=losses, gradM=gradM, Minv=Minv, status=status)
+
+
+def cafeq_optimize_single(W, M, cfg: OptCfg, *, bits, group, taxis=AXIS_IN, opt_state=None):
+    """Updates M in place; returns (loss_history [steps,2], status, opt_state)."""
+    W = _bits_tensor(W)
+    M = _f32(M, "M")
+    d_out, d_in = W.shape
+    d = make_desc(d_out, d_in, bits, group, M.shape[-1], taxis, APPLY_T, 1, W.stride(0))
+    hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W.device)
+    status = torch.zeros(1, dtype=torch.int32, device=W.device)
+    if cfg.optimizer == OPT_ADAM and opt_state is None:
+        opt_state = torch.zeros(1 + 2 * M.numel(), dtype=torch.float32, device=W.device)
+    ws = workspace(workspace_size(d, None, cfg), W.device)
+    rc = lib().cafeq_optimize_single(ctypes.byref(d), _p(W), _p(M), _p(opt_state), ctypes.byref(cfg), _p(hist),
+                                     _p(status), _p(ws), ctypes.c_size_t(ws.numel()), _stream())
+    _check(rc, "cafeq_optimize_single")
+    return hist, status, opt_state
+
+
+def _pair_descs(W1, W2, k, bits, group1, group2, replicas):
+    W1 = _bits_tensor(W1)
+    W2 = _bits_tensor(W2)
+    d1 = make_desc(W1.shape[0], W1.shape[1], bits, group1, k, AXIS_OUT, APPLY_TT, 1, W1.stride(0))
+    d2 = make_desc(W2.shape[0], W2.shape[1], bits, group2, k, AXIS_IN, APPLY_T, replicas, W2.stride(0))
+    return d1, d2
+
+
+def cafeq_pair_product(W1, W2, *, k, bits=4, group1=0, group2=0, replicas=1):
+    d1, d2 = _pair_descs(W1, W2, k, bits, group1, group2, replicas)
+    P = torch.empty((W1.shape[1], W2.shape[0]), dtype=torch.float32, device=W1.device)
+    rc = lib().cafeq_pair_product(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(P), _p(None),
+                                  ctypes.c_size_t(0), _stream())
+    _check(rc, "cafeq_pair_product")
+    return P
+
+
+def cafeq_pair_loss_fwd_bwd(W1, W2, M, *, bits, group1, group2, replicas=1, P=None, loss_kind=LOSS_LSE, lse_t=5.0,
+                            lambda_orth=0.0, flags=0):
+    M = _f32(M, "M")
+    d1, d2 = _pair_descs(W1, W2, M.shape[-1], bits, group1, group2, replicas)
+    losses = torch.zeros(4, dtype=torch.float32, device=W1.device)
+    gradM = None if (flags & FLAG_NO_GRAD) else torch.empty_like(M)
+    status = torch.zeros(1, dtype=torch.int32, device=W1.device)
+    ws = workspace(workspace_size(d1, d2), W1.device)
+    rc = lib().cafeq_pair_loss_fwd_bwd(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(M), _p(_f32(P, "P")),
+                                       ctypes.c_int(loss_kind), ctypes.c_float(lse_t), ctypes.c_float(lambda_orth),
+                                       ctypes.c_int(flags), _p(losses), _p(gradM), _p(status), _p(ws),
+                                       ctypes.c_size_t(ws.numel()), _stream())
+    _check(rc, "cafeq_pair_loss_fwd_bwd")
+    return dict(losses=losses, gradM=gradM, status=status)
+
+
+def cafeq_optimize_pair(W1, W2, M, cfg: OptCfg, *, bits, group1, group2, replicas=1, P=None, opt_state=None):
+    M = _f32(M, "M")
+    d1, d2 = _pair_descs(W1, W2, M.shape[-1], bits, group1, group2, replicas)
+    hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W1.device)
+    status = torch.zeros(1, dtype=torch.int32, device=W1.device)
+    if cfg.optimizer == OPT_ADAM and opt_state is None:
+        opt_state = torch.zeros(1 + 2 * M.numel(), dtype=torch.float32, device=W1.device)
+    ws = workspace(workspace_size(d1, d2, cfg), W1.device)
+    rc = lib().cafeq_optimize_pair(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(M), _p(opt_state),
+                                   _p(_f32(P, "P")), ctypes.byref(cfg), _p(hist), _p(status), _p(ws),
+                                   ctypes.c_size_t(ws.numel()), _stream())
+    _check(rc, "cafeq_optimize_pair")
+    return hist, status, opt_state
+
+
+def cafeq_adaptive_round(W1, W2, M, *, iters, bits, group1, group2, replicas=1, k=None, mode=0):
+    k = M.shape[-1] if M is not None else k
+    d1, d2 = _pair_descs(W1, W2, k, bits, group1, group2, replicas)
+    dev = W1.device
+    g1 = group1 or W1.shape[1]
+    g2 = group2 or W2.shape[1]
+    codes1 = torch.empty(tuple(W1.shape), dtype=torch.int8, device=dev)
+    codes2 = torch.empty(tuple(W2.shape), dtype=torch.int8, device=dev)
+    scales1 = torch.empty((W1.shape[0], W1.shape[1] // g1), dtype=torch.float32, device=dev)
+    scales2 = torch.empty((W2.shape[0], W2.shape[1] // g2), dtype=torch.float32, device=dev)
+    hist = torch.zeros(2 * iters + 1, dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = workspace(workspace_size(d1, d2), dev)
+    rc = lib().cafeq_adaptive_round(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(_f32(M, "M")),
+                                    ctypes.c_int(iters), ctypes.c_int(mode), _p(codes1), _p(scales1), _p(codes2),
+                                    _p(scales2), _p(hist), _p(status), _p(ws), ctypes.c_size_t(ws.numel()), _stream())
+    _check(rc, "cafeq_adaptive_round")
+    return dict(codes1=codes1, scales1=scales1, codes2=codes2, scales2=scales2, pqe=hist, status=status)
+
+
+def cafeq_pack(codes, *, bits):
+    if codes.dtype != torch.int8 or not codes.is_cuda or not codes.is_contiguous():
+        raise ValueError("codes must be a contiguous CUDA int8 tensor")
+    d_out, d_in = codes.shape
+    d = make_desc(d_out, d_in, bits, 0)
+    packed = torch.empty((d_out, d_in * bits // 8), dtype=torch.uint8, device=codes.device)
+    rc = lib().cafeq_pack(ctypes.byref(d), _p(codes), _p(packed), _stream())
+    _check(rc, "cafeq_pack")
+    return packed

@@ -1,0 +1,689 @@
+// C-ABI entry points of the CafeQ optimisation path (declared in include/cafeq.h).
+// Host side only validates arguments, carves the caller's workspace and enqueues kernels.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "cafeq.h"
+#include "kernels_generic.cuh"
+
+namespace cafeq {
+
+// ------------------------------------------------------------------------------------------------
+// workspace carving
+// ------------------------------------------------------------------------------------------------
+struct Bump {
+  char* base;
+  size_t cap, used;
+  bool overflow;
+  Bump(void* b, size_t c) : base((char*)b), cap(c), used(0), overflow(false) {}
+  template <typename T>
+  T* take(size_t count) {
+    size_t bytes = (count * sizeof(T) + 255) & ~(size_t)255;
+    if (used + bytes > cap) { overflow = true; used += bytes; return nullptr; }
+    T* p = (T*)(base + used);
+    used += bytes;
+    return p;
+  }
+};
+
+static inline int grid_for(long long n, int threads = 256, int cap = 148 * 16) {
+  long long b = (n + threads - 1) / threads;
+  if (b < 1) b = 1;
+  if (b > cap) b = cap;
+  return (int)b;
+}
+
+static inline float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
+
+struct Geo {  // derived geometry of one descriptor
+  int d_out, d_in, g, ng, k, r, axis, nbq, nbT;
+  long long ld, n;
+};
+
+static int make_geo(const cafeq_matrix_desc* d, Geo* o, bool need_transform) {
+  if (!d || d->struct_size != sizeof(cafeq_matrix_desc)) return CAFEQ_ERR_INVALID_ARG;
+  if (d->d_out <= 0 || d->d_in <= 0 || d->ld < d->d_in) return CAFEQ_ERR_INVALID_ARG;
+  if (d->bits < 2 || d->bits > 8) return CAFEQ_ERR_INVALID_ARG;
+  if (d->group < 0 || d->tblock < 0 || d->replicas < 1) return CAFEQ_ERR_INVALID_ARG;
+  if (d->taxis != CAFEQ_AXIS_IN && d->taxis != CAFEQ_AXIS_OUT) return CAFEQ_ERR_INVALID_ARG;
+  if (d->compute_prec != CAFEQ_PREC_BF16) return CAFEQ_ERR_UNSUPPORTED;
+  o->d_out = d->d_out;
+  o->d_in = d->d_in;
+  o->ld = d->ld;
+  o->n = (long long)d->d_out * d->d_in;
+  o->g = d->group ? d->group : d->d_in;
+  if (d->d_in % o->g) return CAFEQ_ERR_INVALID_ARG;
+  o->ng = d->d_in / o->g;
+  o->k = d->tblock;
+  o->r = d->replicas;
+  o->axis = d->taxis;
+  o->nbq = 0;
+  o->nbT = 0;
+  if (o->k > 0) {
+    int dim = (o->axis == CAFEQ_AXIS_IN) ? d->d_in : d->d_out;
+    if (dim % o->k) return CAFEQ_ERR_INVALID_ARG;
+    o->nbq = dim / o->k;
+    if (o->nbq % o->r) return CAFEQ_ERR_INVALID_ARG;
+    o->nbT = o->nbq / o->r;
+    if (o->k > 1024) return CAFEQ_ERR_UNSUPPORTED;
+  } else if (need_transform) {
+    return CAFEQ_ERR_INVALID_ARG;
+  }
+  return CAFEQ_OK;
+}
+
+// scratch that one matrix needs in any call
+static size_t matrix_scratch_bytes(const Geo& G) {
+  size_t kk = (size_t)(G.nbT > 0 ? G.nbT : 1) * (size_t)(G.k > 0 ? G.k : 1) * (size_t)(G.k > 0 ? G.k : 1);
+  size_t rows_ng = (size_t)G.d_out * G.ng;
+  size_t b = 0;
+  b += 3 * ((size_t)G.n * 4 + 256);                   // U, Delta / gDelta, E / Uhat
+  b += 3 * (rows_ng * 4 + 256);                       // a, idx, coef
+  b += ((size_t)G.ng + G.d_out + G.d_in) * 4 + 1024;  // cw, Agrp
+  b += 8 * (kk * 4 + 256);                            // Mc, Minv, Minv_c, gMinv, tmp, RM, ...
+  b += 4 * ((size_t)(G.nbT + 1) * (G.k + 1) * 4 + 256);  // c, A
+  b += 4096;                                          // accumulators
+  return b;
+}
+
+// ------------------------------------------------------------------------------------------------
+// launch helpers
+// ------------------------------------------------------------------------------------------------
+static void launch_gemm(cudaStream_t st, const GemmArgs& g) {
+  dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, g.batch);
+  if (g.a_bf16 && g.b_bf16) gemm_kernel<true, true><<<grid, 256, 0, st>>>(g);
+  else if (g.a_bf16) gemm_kernel<true, false><<<grid, 256, 0, st>>>(g);
+  else if (g.b_bf16) gemm_kernel<false, true><<<grid, 256, 0, st>>>(g);
+  else gemm_kernel<false, false><<<grid, 256, 0, st>>>(g);
+}
+
+static GemmArgs gemm_defaults(const int32_t* status) {
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.divA = g.divB = g.divC = 1;
+  g.alpha = 1.f;
+  g.mode = GEMM_STORE;
+  g.batch = 1;
+  g.status = status;
+  return g;
+}
+
+// Out = T o X along `axis`; X is bf16 (x_bf16) or fp32; T fp32 blocks [nbT,k,k]; transposed uses T^T.
+static void launch_apply(cudaStream_t st, const void* X, int x_bf16, long long ldx, const Geo& G, const float* T,
+                         int transposed, float* Out, long long ldo, int mode, double* sq, const int32_t* status,
+                         float alpha = 1.f) {
+  GemmArgs g = gemm_defaults(status);
+  const int k = G.k;
+  g.alpha = alpha;
+  g.C = Out;
+  g.mode = mode;
+  g.sq = sq;
+  g.batch = G.nbq;
+  if (G.axis == CAFEQ_AXIS_IN) {
+    g.M = G.d_out; g.N = k; g.K = k;
+    g.A = X; g.a_bf16 = x_bf16; g.sAm = ldx; g.sAk = 1; g.sAb = k;
+    g.B = T; g.b_bf16 = 0; g.sBb = (long long)k * k; g.divB = G.r;
+    if (!transposed) { g.sBk = 1; g.sBn = k; } else { g.sBk = k; g.sBn = 1; }
+    g.sCm = ldo; g.sCn = 1; g.sCb = k;
+  } else {
+    g.M = k; g.N = G.d_in; g.K = k;
+    g.A = T; g.a_bf16 = 0; g.sAb = (long long)k * k; g.divA = G.r;
+    if (!transposed) { g.sAm = k; g.sAk = 1; } else { g.sAm = 1; g.sAk = k; }
+    g.B = X; g.b_bf16 = x_bf16; g.sBk = ldx; g.sBn = 1; g.sBb = (long long)k * ldx;
+    g.sCm = ldo; g.sCn = 1; g.sCb = (long long)k * ldo;
+  }
+  launch_gemm(st, g);
+}
+
+// gT[b / r][i][j] += alpha * sum_free Gm[.., i] X[.., j]  (atomic accumulation; caller zeroes gT)
+static void launch_opgrad(cudaStream_t st, const float* Gm, long long ldg, const void* X, int x_bf16, long long ldx,
+                          const Geo& G, float* gT, int transpose_out, float alpha, const int32_t* status) {
+  GemmArgs g = gemm_defaults(status);
+  const int k = G.k;
+  g.M = k; g.N = k; g.batch = G.nbq;
+  g.A = Gm; g.a_bf16 = 0;
+  g.B = X; g.b_bf16 = x_bf16;
+  g.C = gT; g.sCb = (long long)k * k; g.divC = G.r;
+  if (!transpose_out) { g.sCm = k; g.sCn = 1; } else { g.sCm = 1; g.sCn = k; }
+  g.alpha = alpha;
+  g.mode = GEMM_STORE | GEMM_ATOMIC;
+  if (G.axis == CAFEQ_AXIS_IN) {
+    g.K = G.d_out;
+    g.sAm = 1; g.sAk = ldg; g.sAb = k;
+    g.sBk = ldx; g.sBn = 1; g.sBb = k;
+  } else {
+    g.K = G.d_in;
+    g.sAm = ldg; g.sAk = 1; g.sAb = (long long)k * ldg;
+    g.sBk = 1; g.sBn = ldx; g.sBb = (long long)k * ldx;
+  }
+  launch_gemm(st, g);
+}
+
+// C[b] (op)= alpha * opA(A[b]) * opB(B[b]) for k x k blocks
+static void launch_kk(cudaStream_t st, const float* A, int tA, const float* B, int tB, float* C, int nb, int k, float alpha,
+                      int mode, const int32_t* status) {
+  GemmArgs g = gemm_defaults(status);
+  g.M = g.N = g.K = k;
+  g.batch = nb;
+  g.A = A; g.B = B; g.C = C;
+  g.sAb = g.sBb = g.sCb = (long long)k * k;
+  if (!tA) { g.sAm = k; g.sAk = 1; } else { g.sAm = 1; g.sAk = k; }
+  if (!tB) { g.sBk = k; g.sBn = 1; } else { g.sBk = 1; g.sBn = k; }
+  g.sCm = k; g.sCn = 1;
+  g.alpha = alpha;
+  g.mode = mode;
+  launch_gemm(st, g);
+}
+
+static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float* cnorm, int nb, int k, int32_t* status) {
+  int threads = k * k >= 1024 ? 1024 : ((k * k + 31) / 32) * 32;
+  size_t sh = (size_t)3 * k * sizeof(float);
+  block_inverse_kernel<<<nb, threads, sh, st>>>(Mc, Minv, cnorm, k, status);
+}
+
+static void launch_absmax(cudaStream_t st, const float* U, long long ld, const Geo& G, float* a, int* idx, int32_t* status) {
+  long long warps = (long long)G.d_out * G.ng;
+  long long blocks = (warps * 32 + 255) / 256;
+  absmax_kernel<<<(unsigned)blocks, 256, 0, st>>>(U, ld, G.d_out, G.ng, G.g, a, idx, status);
+}
+
+static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const float* coef, const int* idx, float* gT,
+                           int transpose_out, const int32_t* status) {
+  const int k = G.k;
+  size_t sh = (size_t)k * SCATTER_JS * sizeof(float);
+  if (sh > 48 * 1024) {
+    cudaFuncSetAttribute(scatter_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
+    cudaFuncSetAttribute(scatter_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
+  }
+  int strips = (k + SCATTER_JS - 1) / SCATTER_JS;
+  if (G.axis == CAFEQ_AXIS_IN) {
+    int want = (148 * 4) / (G.nbq * strips) + 1;
+    int splits = want < 1 ? 1 : want;
+    int rows_per = (G.d_out + splits - 1) / splits;
+    if (rows_per < 8) rows_per = 8;
+    splits = (G.d_out + rows_per - 1) / rows_per;
+    dim3 grid(G.nbq, strips, splits);
+    scatter_in_kernel<<<grid, 256, sh, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
+                                             transpose_out, rows_per, status);
+  } else {
+    int want = (148 * 4) / (G.nbq * strips) + 1;
+    int splits = want < 1 ? 1 : want;
+    int per = (G.ng + splits - 1) / splits;
+    if (per < 1) per = 1;
+    splits = (G.ng + per - 1) / per;
+    dim3 grid(G.nbq, strips, splits);
+    scatter_out_kernel<<<grid, 256, sh, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
+                                              transpose_out, per, status);
+  }
+}
+
+__global__ void bf16_to_f32_kernel(const uint16_t* __restrict__ W, long long ld, int rows, int cols, float* __restrict__ U) {
+  const long long n = (long long)rows * cols;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
+    U[e] = bf16_bits_to_float(W[row * ld + col]);
+  }
+}
+
+__global__ void resid_sq_kernel(float* __restrict__ R, const float* __restrict__ P, long long n, double* acc,
+                                const int32_t* status) {
+  if (status && *status) return;
+  __shared__ double red[32];
+  double local = 0.0;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    float v = R[i] - P[i];
+    R[i] = v;
+    local += (double)v * v;
+  }
+  double s = block_sum_double(local, red);
+  if (threadIdx.x == 0) atomicAdd(acc, s);
+}
+
+__global__ void store_sqrt_kernel(const double* acc, float* out) { *out = (float)sqrt(*acc); }
+
+// ------------------------------------------------------------------------------------------------
+// per-matrix scratch
+// ------------------------------------------------------------------------------------------------
+struct MatWS {
+  float *U, *D, *E;
+  float *a, *coef, *cw, *agrp;
+  int* idx;
+};
+
+static void carve_matrix(Bump& b, const Geo& G, MatWS* w, bool need_E) {
+  w->U = b.take<float>(G.n);
+  w->D = b.take<float>(G.n);
+  w->E = need_E ? b.take<float>(G.n) : nullptr;
+  size_t rows_ng = (size_t)G.d_out * G.ng;
+  w->a = b.take<float>(rows_ng);
+  w->idx = b.take<int>(rows_ng);
+  w->coef = b.take<float>(rows_ng);
+  w->cw = b.take<float>((size_t)(G.ng > G.d_out ? G.ng : G.d_out));
+  w->agrp = b.take<float>((size_t)G.ng);
+}
+
+// U = T o W, group absmax / arg-max, and (optionally) the quantiser outputs.
+static void forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits, const float* Tc, int transposed,
+                          const MatWS& w, const void* offsets, int off_kind, bool want_delta, float* Uhat, int8_t* codes,
+                          int32_t* status) {
+  if (Tc) launch_apply(st, W, 1, G.ld, G, Tc, transposed, w.U, G.d_in, GEMM_STORE, nullptr, status);
+  else bf16_to_f32_kernel<<<grid_for(G.n), 256, 0, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, w.U);
+  launch_absmax(st, w.U, G.d_in, G, w.a, w.idx, status);
+  if (want_delta || Uhat || codes)
+    quant_kernel<<<grid_for(G.n), 256, 0, st>>>(w.U, G.d_in, G.d_out, G.d_in, G.g, w.a, qmax_of(bits), offsets, off_kind,
+                                                want_delta ? w.D : nullptr, Uhat, codes, status);
+}
+
+}  // namespace cafeq
+
+using namespace cafeq;
+
+// ------------------------------------------------------------------------------------------------
+extern "C" const char* cafeq_status_string(int s) {
+  switch (s) {
+    case CAFEQ_OK: return "ok";
+    case CAFEQ_ERR_INVALID_ARG: return "invalid argument";
+    case CAFEQ_ERR_UNSUPPORTED: return "unsupported shape or mode";
+    case CAFEQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case CAFEQ_ERR_CUDA: return "CUDA launch failed";
+    case CAFEQ_ERR_SINGULAR: return "singular transform block";
+    case CAFEQ_ERR_NONFINITE: return "non-finite value";
+    case CAFEQ_ERR_TIMEOUT: return "bounded device wait expired";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int cafeq_version(void) { return 100; }
+
+extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
+                                    size_t* bytes) {
+  (void)cfg;
+  if (!bytes) return CAFEQ_ERR_INVALID_ARG;
+  Geo G1, G2;
+  int rc = make_geo(d1, &G1, false);
+  if (rc) return rc;
+  size_t b = matrix_scratch_bytes(G1);
+  if (d2) {
+    rc = make_geo(d2, &G2, false);
+    if (rc) return rc;
+    b += matrix_scratch_bytes(G2);
+    // product-sized buffers: residual R and two pseudo-inverse work matrices of adaptive rounding
+    size_t d1n = (size_t)d1->d_in, d3n = (size_t)d2->d_out, H = (size_t)d2->d_in;
+    b += (d1n * d3n * 4 + 256);
+    b += 6 * ((d1n > d3n ? d1n : d3n) * H * 4 + 256);
+    b += 4 * (H * H * 4 + 256);
+  }
+  *bytes = b;
+  return CAFEQ_OK;
+}
+
+static int check_ws(void* ws, size_t ws_bytes) {
+  if (!ws || ((uintptr_t)ws & 255)) return CAFEQ_ERR_WORKSPACE;
+  (void)ws_bytes;
+  return CAFEQ_OK;
+}
+
+static int last_launch() { return cudaGetLastError() == cudaSuccess ? CAFEQ_OK : CAFEQ_ERR_CUDA; }
+
+// ------------------------------------------------------------------------------------------------
+extern "C" int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
+                         void* ws, size_t ws_bytes, void* stream) {
+  Geo G;
+  int rc = make_geo(d, &G, false);
+  if (rc) return rc;
+  if (!W || !codes || !scales) return CAFEQ_ERR_INVALID_ARG;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool has_T = (T != nullptr && G.k > 0);
+  Bump b(ws, ws_bytes);
+  MatWS w;
+  carve_matrix(b, G, &w, false);
+  float* Tc = has_T ? b.take<float>((size_t)G.nbT * G.k * G.k) : nullptr;
+  if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  if (has_T) round_bf16_kernel<<<grid_for((long long)G.nbT * G.k * G.k), 256, 0, st>>>(T, Tc, (long long)G.nbT * G.k * G.k, nullptr);
+  forward_quant(st, W, G, d->bits, Tc, d->trole == CAFEQ_APPLY_TT, w, nullptr, CAFEQ_OFFSETS_NONE, false, nullptr, codes,
+                nullptr);
+  scales_kernel<<<grid_for((long long)G.d_out * G.ng), 256, 0, st>>>(w.a, scales, (long long)G.d_out * G.ng,
+                                                                     qmax_of(d->bits), nullptr);
+  return last_launch();
+}
+
+// ------------------------------------------------------------------------------------------------
+// single matrix forward + backward
+// ------------------------------------------------------------------------------------------------
+namespace cafeq {
+
+struct SingleWS {
+  MatWS m;
+  float *Mc, *Minv, *gMinv, *tmp, *c, *A;
+  double* acc;
+};
+
+static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
+  carve_matrix(b, G, &s->m, need_E);
+  size_t kk = (size_t)G.nbT * G.k * G.k;
+  s->Mc = b.take<float>(kk);
+  s->Minv = b.take<float>(kk);
+  s->gMinv = b.take<float>(kk);
+  s->tmp = b.take<float>(kk);
+  s->c = b.take<float>((size_t)G.nbT * G.k);
+  s->A = b.take<float>((size_t)G.nbT * G.k);
+  s->acc = b.take<double>(8);
+  return !b.overflow;
+}
+
+// Enqueue one forward(+backward) for a single matrix; gradM may be null.  hist is an optional [2] slot.
+static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& G, const void* W, const float* M,
+                        float* Minv_out, const void* offsets, int off_kind, int loss_kind, float kappa, bool want_exact,
+                        float* losses, float* hist, float* gradM, int32_t* status, const SingleWS& s) {
+  const int k = G.k;
+  const long long kk = (long long)G.nbT * k * k;
+  const float qm = qmax_of(d->bits);
+  const bool ste = (loss_kind == CAFEQ_LOSS_L2_STE);
+  const bool need_l2 = want_exact || ste;
+  zero_f64_kernel<<<1, 32, 0, st>>>(s.acc, 8);
+  round_bf16_kernel<<<grid_for(kk), 256, 0, st>>>(M, s.Mc, kk, status);
+  launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
+  if (Minv_out) copy_f32_kernel<<<grid_for(kk), 256, 0, st>>>(s.Minv, Minv_out, kk);
+  forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, status);
+  if (need_l2) {
+    // E = Minv o Delta, L2 = sum E^2
+    launch_apply(st, s.m.D, 0, G.d_in, G, s.Minv, 0, s.m.E, G.d_in, (ste ? GEMM_STORE : 0) | GEMM_SQSUM, s.acc + 1, status);
+    sqsum_bf16_kernel<<<grid_for(G.n), 256, 0, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);
+  }
+  // surrogate value, arg-max coefficients and A_t
+  const bool want_grad = (gradM != nullptr);
+  if (G.axis == CAFEQ_AXIS_IN) cw_in_kernel<<<(G.ng + 127) / 128, 128, 0, st>>>(s.c, G.d_in, G.g, k, G.r, s.m.cw);
+  else cw_out_kernel<<<(G.d_out + 127) / 128, 128, 0, st>>>(s.c, G.d_out, G.g, k, G.r, s.m.cw);
+  fill_f32_kernel<<<grid_for(G.nbT * k), 256, 0, st>>>(s.A, 0.f, (long long)G.nbT * k);
+  fill_f32_kernel<<<grid_for(G.ng), 256, 0, st>>>(s.m.agrp, 0.f, G.ng);
+  surrogate_rows_kernel<<<(G.d_out + 127) / 128, 128, 0, st>>>(s.m.a, s.m.idx, s.m.U, G.d_in, G.d_out, G.ng, G.g, G.axis,
+                                                               s.m.cw, kappa, k, G.r, (want_grad && !ste) ? s.m.coef : nullptr,
+                                                               s.m.agrp, s.A, s.acc + 0, status);
+  if (G.axis == CAFEQ_AXIS_IN) expand_agrp_kernel<<<(G.d_in + 127) / 128, 128, 0, st>>>(s.m.agrp, G.d_in, G.g, k, G.r, s.A);
+  finalize_single_kernel<<<1, 1, 0, st>>>(s.acc, losses, hist, need_l2 ? 1 : 0);
+  if (!want_grad) return;
+  fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(gradM, 0.f, kk);
+  if (!ste) {
+    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
+    scale_cols_kernel<<<grid_for(kk), 256, 0, st>>>(s.Minv, s.A, 2.f * kappa, k, kk, s.gMinv);
+  } else {
+    // gMinv = 2 * sum_free E Delta^T ; gDelta = 2 Minv^T o E (overwrites Delta) ; scale path through arg-max
+    fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(s.gMinv, 0.f, kk);
+    launch_opgrad(st, s.m.E, G.d_in, s.m.D, 0, G.d_in, G, s.gMinv, 0, 2.f, status);
+    launch_apply(st, s.m.E, 0, G.d_in, G, s.Minv, 1, s.m.D, G.d_in, GEMM_STORE, nullptr, status, 2.f);
+    ste_scale_path_kernel<<<(unsigned)(((long long)G.d_out * G.ng * 32 + 255) / 256), 256, 0, st>>>(
+        s.m.U, s.m.D, G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.idx, qm, offsets, off_kind, G.d_in, s.m.coef, status);
+    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
+  }
+  // gradM -= Minv^T gMinv Minv^T
+  launch_kk(st, s.Minv, 1, s.gMinv, 0, s.tmp, G.nbT, k, 1.f, GEMM_STORE, status);
+  launch_kk(st, s.tmp, 0, s.Minv, 1, gradM, G.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+}
+
+}  // namespace cafeq
+
+extern "C" int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* W, const float* M, float* Minv,
+                                        const void* offsets, int offsets_kind, int loss_kind, float kappa, int flags,
+                                        float* losses, float* gradM, int32_t* status, void* ws, size_t ws_bytes,
+                                        void* stream) {
+  Geo G;
+  int rc = make_geo(d, &G, true);
+  if (rc) return rc;
+  if (!W || !M || !losses) return CAFEQ_ERR_INVALID_ARG;
+  if (loss_kind != CAFEQ_LOSS_SURROGATE && loss_kind != CAFEQ_LOSS_L2_STE) return CAFEQ_ERR_INVALID_ARG;
+  if (offsets_kind < CAFEQ_OFFSETS_NONE || offsets_kind > CAFEQ_OFFSETS_SOFT_F32) return CAFEQ_ERR_INVALID_ARG;
+  if (offsets_kind != CAFEQ_OFFSETS_NONE && !offsets) return CAFEQ_ERR_INVALID_ARG;
+  const bool want_grad = !(flags & CAFEQ_FLAG_NO_GRAD);
+  if (want_grad && !gradM) return CAFEQ_ERR_INVALID_ARG;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  if (kappa <= 0.f) kappa = 1.f / (float)(((1 << d->bits) - 1) * ((1 << d->bits) - 1));
+  cudaStream_t st = (cudaStream_t)stream;
+  Bump b(ws, ws_bytes);
+  SingleWS s;
+  if (!carve_single(b, G, &s, true)) return CAFEQ_ERR_WORKSPACE;
+  single_step(st, d, G, W, M, Minv, offsets, offsets_kind, loss_kind, kappa, (flags & CAFEQ_FLAG_EXACT_LOSS) != 0, losses,
+              nullptr, want_grad ? gradM : nullptr, status, s);
+  return last_launch();
+}
+
+extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, float* M, float* opt_state,
+                                     const cafeq_opt_cfg* cfg, float* loss_history, int32_t* status, void* ws,
+                                     size_t ws_bytes, void* stream) {
+  Geo G;
+  int rc = make_geo(d, &G, true);
+  if (rc) return rc;
+  if (!W || !M || !cfg || cfg->struct_size != sizeof(cafeq_opt_cfg) || !loss_history) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->steps < 0) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->loss_kind != CAFEQ_LOSS_SURROGATE && cfg->loss_kind != CAFEQ_LOSS_L2_STE) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->optimizer == CAFEQ_OPT_ADAM && !opt_state) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->optimizer != CAFEQ_OPT_ADAM && cfg->optimizer != CAFEQ_OPT_GD) return CAFEQ_ERR_INVALID_ARG;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  float kappa = cfg->kappa;
+  if (kappa <= 0.f) kappa = 1.f / (float)(((1 << d->bits) - 1) * ((1 << d->bits) - 1));
+  cudaStream_t st = (cudaStream_t)stream;
+  Bump b(ws, ws_bytes);
+  SingleWS s;
+  if (!carve_single(b, G, &s, true)) return CAFEQ_ERR_WORKSPACE;
+  const long long kk = (long long)G.nbT * G.k * G.k;
+  float* grad = b.take<float>(kk);
+  if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  for (int it = 0; it < cfg->steps; ++it) {
+    bool eval = cfg->eval_every > 0 && (it % cfg->eval_every == 0);
+    single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
+                loss_history + 2 * (size_t)it, grad, status, s);
+    if (cfg->optimizer == CAFEQ_OPT_GD) {
+      gd_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, cfg->lr, kk, status);
+    } else {
+      adam_tick_kernel<<<1, 1, 0, st>>>(opt_state, status);
+      adam_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
+                                                       status);
+    }
+  }
+  return last_launch();
+}
+
+// ------------------------------------------------------------------------------------------------
+// pair
+// ------------------------------------------------------------------------------------------------
+namespace cafeq {
+
+static int make_pair_geo(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, Geo* G1, Geo* G2) {
+  int rc = make_geo(d1, G1, true);
+  if (rc) return rc;
+  if ((rc = make_geo(d2, G2, true))) return rc;
+  if (G1->axis != CAFEQ_AXIS_OUT || G2->axis != CAFEQ_AXIS_IN) return CAFEQ_ERR_INVALID_ARG;
+  if (G1->k != G2->k || G1->r != 1) return CAFEQ_ERR_INVALID_ARG;
+  if (G1->nbT != G2->nbT) return CAFEQ_ERR_INVALID_ARG;  // h / k operator blocks on both sides
+  if (d1->bits != d2->bits) return CAFEQ_ERR_UNSUPPORTED;
+  return CAFEQ_OK;
+}
+
+// Cm[x][y] = sum over blocks B of W2:  A1[(B/r)k + j][x] * A2[y][B k + j]   (A1 stored [h, d1], A2 stored [d3, r h])
+static void launch_pair_product(cudaStream_t st, const void* A1, int a1_bf16, long long ld1, const void* A2, int a2_bf16,
+                                long long ld2, const Geo& G1, const Geo& G2, float* Cm, const int32_t* status) {
+  const int d1n = G1.d_in, d3n = G2.d_out, k = G1.k;
+  GemmArgs g = gemm_defaults(status);
+  g.M = d1n; g.N = d3n;
+  g.A = A1; g.a_bf16 = a1_bf16; g.sAm = 1; g.sAk = ld1;
+  g.B = A2; g.b_bf16 = a2_bf16; g.sBk = 1; g.sBn = ld2;
+  g.C = Cm; g.sCm = d3n; g.sCn = 1; g.sCb = 0;
+  if (G2.r == 1) {
+    g.K = G1.d_out; g.batch = 1;
+    g.mode = GEMM_STORE;
+  } else {
+    fill_f32_kernel<<<grid_for((long long)d1n * d3n), 256, 0, st>>>(Cm, 0.f, (long long)d1n * d3n);
+    g.K = k; g.batch = G2.nbq;
+    g.sAb = (long long)k * ld1; g.divA = G2.r;
+    g.sBb = k;
+    g.mode = GEMM_STORE | GEMM_ATOMIC;
+  }
+  launch_gemm(st, g);
+}
+
+struct PairWS {
+  MatWS m1, m2;
+  float *Mc, *Minv, *Minv_c, *gMinv, *tmp, *RM, *amax, *R;
+  double* acc;
+};
+
+static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool need_R) {
+  carve_matrix(b, G1, &p->m1, true);
+  carve_matrix(b, G2, &p->m2, true);
+  size_t kk = (size_t)G1.nbT * G1.k * G1.k;
+  p->Mc = b.take<float>(kk);
+  p->Minv = b.take<float>(kk);
+  p->Minv_c = b.take<float>(kk);
+  p->gMinv = b.take<float>(kk);
+  p->tmp = b.take<float>(kk);
+  p->RM = b.take<float>(kk);
+  p->amax = b.take<float>(64);
+  p->acc = b.take<double>(8);
+  p->R = need_R ? b.take<float>((size_t)G1.d_in * G2.d_out) : nullptr;
+  return !b.overflow;
+}
+
+static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
+                      const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
+                      float* losses, float* hist, float* gradM, int32_t* status, const PairWS& p) {
+  const int k = G1.k;
+  const long long kk = (long long)G1.nbT * k * k;
+  const float sqrt_h = sqrtf((float)G1.d_out);
+  zero_f64_kernel<<<1, 32, 0, st>>>(p.acc, 8);
+  fill_f32_kernel<<<1, 32, 0, st>>>(p.amax, 0.f, 1);
+  round_bf16_kernel<<<grid_for(kk), 256, 0, st>>>(M, p.Mc, kk, status);
+  launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
+  round_bf16_kernel<<<grid_for(kk), 256, 0, st>>>(p.Minv, p.Minv_c, kk, status);
+  // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
+  forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
+                status);
+  forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
+                nullptr, status);
+  const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
+  max_f32_kernel<<<grid_for(n1), 256, 0, st>>>(p.m1.a, n1, p.amax, status);
+  max_f32_kernel<<<grid_for(n2), 256, 0, st>>>(p.m2.a, n2, p.amax, status);
+  sumexp_kernel<<<grid_for(n1), 256, 0, st>>>(p.m1.a, n1, p.amax, t, p.acc + 0, status);
+  sumexp_kernel<<<grid_for(n2), 256, 0, st>>>(p.m2.a, n2, p.amax, t, p.acc + 0, status);
+  // orthonormality penalty on the fp32 parameters: R = M M^T - I
+  launch_kk(st, M, 0, M, 1, p.tmp, G1.nbT, k, 1.f, GEMM_STORE, status);
+  sub_identity_kernel<<<grid_for(kk), 256, 0, st>>>(p.tmp, k, kk);
+  sqsum_f32_kernel<<<grid_for(kk), 256, 0, st>>>(p.tmp, kk, p.acc + 1);
+  if (want_pqe) {
+    launch_pair_product(st, p.m1.E, 0, G1.d_in, p.m2.E, 0, G2.d_in, G1, G2, p.R, status);
+    resid_sq_kernel<<<grid_for((long long)G1.d_in * G2.d_out), 256, 0, st>>>(p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
+                                                                             status);
+  }
+  finalize_pair_kernel<<<1, 1, 0, st>>>(p.acc, p.amax, t, lambda, sqrt_h, losses, hist, want_pqe ? 1 : 0);
+  if (!gradM) return;
+  lse_coef_kernel<<<grid_for(n1), 256, 0, st>>>(p.m1.a, p.m1.idx, p.m1.U, G1.d_in, G1.d_out, G1.ng, G1.g, p.amax, t, p.acc + 0,
+                                                p.m1.coef, status);
+  lse_coef_kernel<<<grid_for(n2), 256, 0, st>>>(p.m2.a, p.m2.idx, p.m2.U, G2.d_in, G2.d_out, G2.ng, G2.g, p.amax, t, p.acc + 0,
+                                                p.m2.coef, status);
+  fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(gradM, 0.f, kk);
+  fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(p.gMinv, 0.f, kk);
+  // U side: operator is M^T, so the block gradient is stored transposed
+  launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status);
+  // V side: gradient with respect to Minv, then through the inverse
+  launch_scatter(st, W2, G2, p.m2.coef, p.m2.idx, p.gMinv, 0, status);
+  launch_kk(st, p.Minv, 1, p.gMinv, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
+  launch_kk(st, p.RM, 0, p.Minv, 1, gradM, G1.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+  if (lambda != 0.f) {
+    launch_kk(st, p.tmp, 0, M, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
+    orth_grad_kernel<<<grid_for(kk), 256, 0, st>>>(gradM, p.RM, p.acc + 1, lambda, sqrt_h, kk);
+  }
+}
+
+}  // namespace cafeq
+
+extern "C" int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                                  const void* W2, float* P, void* ws, size_t ws_bytes, void* stream) {
+  Geo G1, G2;
+  int rc = make_pair_geo(d1, d2, &G1, &G2);
+  if (rc) return rc;
+  if (!W1 || !W2 || !P) return CAFEQ_ERR_INVALID_ARG;
+  (void)ws;
+  (void)ws_bytes;
+  launch_pair_product((cudaStream_t)stream, W1, 1, G1.ld, W2, 1, G2.ld, G1, G2, P, nullptr);
+  return last_launch();
+}
+
+extern "C" int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                                       const void* W2, const float* M, const float* P, int loss_kind, float lse_t,
+                                       float lambda_orth, int flags, float* losses, float* gradM, int32_t* status,
+                                       void* ws, size_t ws_bytes, void* stream) {
+  Geo G1, G2;
+  int rc = make_pair_geo(d1, d2, &G1, &G2);
+  if (rc) return rc;
+  if (!W1 || !W2 || !M || !losses) return CAFEQ_ERR_INVALID_ARG;
+  if (loss_kind == CAFEQ_LOSS_PQE_STE) return CAFEQ_ERR_UNSUPPORTED;
+  if (loss_kind != CAFEQ_LOSS_LSE) return CAFEQ_ERR_INVALID_ARG;
+  if (!(lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
+  const bool want_grad = !(flags & CAFEQ_FLAG_NO_GRAD);
+  const bool want_pqe = (flags & CAFEQ_FLAG_EXACT_LOSS) != 0;
+  if (want_grad && !gradM) return CAFEQ_ERR_INVALID_ARG;
+  if (want_pqe && !P) return CAFEQ_ERR_INVALID_ARG;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  Bump b(ws, ws_bytes);
+  PairWS p;
+  if (!carve_pair(b, G1, G2, &p, want_pqe)) return CAFEQ_ERR_WORKSPACE;
+  pair_step((cudaStream_t)stream, d1, d2, G1, G2, W1, W2, M, P, lse_t, lambda_orth, want_pqe, losses, nullptr,
+            want_grad ? gradM : nullptr, status, p);
+  return last_launch();
+}
+
+extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                                   const void* W2, float* M, float* opt_state, const float* P, const cafeq_opt_cfg* cfg,
+                                   float* loss_history, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+  Geo G1, G2;
+  int rc = make_pair_geo(d1, d2, &G1, &G2);
+  if (rc) return rc;
+  if (!W1 || !W2 || !M || !cfg || cfg->struct_size != sizeof(cafeq_opt_cfg) || !loss_history) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->loss_kind == CAFEQ_LOSS_PQE_STE) return CAFEQ_ERR_UNSUPPORTED;
+  if (cfg->loss_kind != CAFEQ_LOSS_LSE || cfg->steps < 0 || !(cfg->lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->optimizer == CAFEQ_OPT_ADAM && !opt_state) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->optimizer != CAFEQ_OPT_ADAM && cfg->optimizer != CAFEQ_OPT_GD) return CAFEQ_ERR_INVALID_ARG;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool any_pqe = (P != nullptr) && cfg->eval_every > 0;
+  Bump b(ws, ws_bytes);
+  PairWS p;
+  if (!carve_pair(b, G1, G2, &p, any_pqe)) return CAFEQ_ERR_WORKSPACE;
+  const long long kk = (long long)G1.nbT * G1.k * G1.k;
+  float* grad = b.take<float>(kk);
+  if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  for (int it = 0; it < cfg->steps; ++it) {
+    bool eval = any_pqe && (it % cfg->eval_every == 0);
+    pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
+              grad, status, p);
+    if (cfg->optimizer == CAFEQ_OPT_GD) {
+      gd_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, cfg->lr, kk, status);
+    } else {
+      adam_tick_kernel<<<1, 1, 0, st>>>(opt_state, status);
+      adam_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
+                                                       status);
+    }
+  }
+  return last_launch();
+}
+
+extern "C" int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
+                                    const void* W2, const float* M, int iters, int mode, int8_t* codes1, float* scales1,
+                                    int8_t* codes2, float* scales2, float* pqe_history, int32_t* status, void* ws,
+                                    size_t ws_bytes, void* stream) {
+  (void)d1; (void)W1; (void)d2; (void)W2; (void)M; (void)iters; (void)mode; (void)codes1; (void)scales1;
+  (void)codes2; (void)scales2; (void)pqe_history; (void)status; (void)ws; (void)ws_bytes; (void)stream;
+  return CAFEQ_ERR_UNSUPPORTED;
+}
+
+extern "C" int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed, void* stream) {
+  Geo G;
+  int rc = make_geo(d, &G, false);
+  if (rc) return rc;
+  if (!codes || !packed) return CAFEQ_ERR_INVALID_ARG;
+  if (G.d_in % 8) return CAFEQ_ERR_UNSUPPORTED;
+  pack_kernel<<<grid_for(G.n / 8), 256, 0, (cudaStream_t)stream>>>(codes, packed, G.d_out, G.d_in, d->bits);
+  return last_launch();
+}

@@ -1,0 +1,715 @@
+// Shape-agnostic CUDA kernels of the CafeQ path: a strided batched GEMM with fp32 accumulation and the
+// element-wise / reduction steps around it.  They cover every shape (tiny test matrices, odd block
+// sizes) and serve as the on-device cross-check of the fused tensor-core kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "cafeq.h"
+
+namespace cafeq {
+
+// ------------------------------------------------------------------------------------------------
+// small helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
+
+__device__ __forceinline__ float round_to_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+__device__ __forceinline__ void raise_status(int32_t* status, int code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ double block_sum_double(double v, double* sh) {
+  // sh: at least 32 doubles of shared memory
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  int nw = (blockDim.x + 31) >> 5;
+  v = (threadIdx.x < nw) ? sh[threadIdx.x] : 0.0;
+  if (w == 0)
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;  // valid in thread 0
+}
+
+// ------------------------------------------------------------------------------------------------
+// fill / copy / round
+// ------------------------------------------------------------------------------------------------
+__global__ void fill_f32_kernel(float* p, float v, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    p[i] = v;
+}
+
+__global__ void zero_f64_kernel(double* p, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = 0.0;
+}
+
+// out = float(bf16(in)): the operand actually fed to the transform products.
+__global__ void round_bf16_kernel(const float* __restrict__ in, float* __restrict__ out, long long n,
+                                  const int32_t* status) {
+  if (status && *status) return;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    out[i] = round_to_bf16(in[i]);
+}
+
+__global__ void copy_f32_kernel(const float* __restrict__ in, float* __restrict__ out, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    out[i] = in[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// strided batched GEMM:  C[b][m][n] (op)= alpha * sum_k A[b/divA][m][k] * B[b/divB][k][n]
+// ------------------------------------------------------------------------------------------------
+enum { GEMM_STORE = 1, GEMM_ACCUM = 2, GEMM_ATOMIC = 4, GEMM_SUBP = 8, GEMM_SQSUM = 16 };
+
+struct GemmArgs {
+  const void* A;
+  const void* B;
+  float* C;
+  const float* P;  // optional matrix subtracted before the square sum / store
+  double* sq;      // optional accumulator of sum(v^2)
+  int M, N, K, batch;
+  long long sAm, sAk, sAb;
+  long long sBk, sBn, sBb;
+  long long sCm, sCn, sCb;
+  long long sPm, sPn, sPb;
+  int a_bf16, b_bf16;
+  int divA, divB, divC;
+  float alpha;
+  int mode;
+  const int32_t* status;
+};
+
+template <bool ABF, bool BBF>
+__global__ void __launch_bounds__(256) gemm_kernel(GemmArgs g) {
+  if (g.status && *g.status) return;
+  constexpr int BM = 64, BN = 64, BK = 16;
+  __shared__ float As[BK][BM + 4];
+  __shared__ float Bs[BK][BN + 4];
+  __shared__ double red[32];
+  const int tid = threadIdx.x;
+  const int b = blockIdx.z;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const long long ab = (long long)(b / g.divA) * g.sAb, bb = (long long)(b / g.divB) * g.sBb;
+  const bool a_kfast = (g.sAk == 1), b_nfast = (g.sBn == 1);
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < g.K; k0 += BK) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      int t = tid + q * 256;
+      int m, kk;
+      if (a_kfast) { kk = t & 15; m = t >> 4; } else { m = t & 63; kk = t >> 6; }
+      int gm = m0 + m, gk = k0 + kk;
+      float v = 0.f;
+      if (gm < g.M && gk < g.K) {
+        long long off = ab + gm * g.sAm + gk * g.sAk;
+        v = ABF ? bf16_bits_to_float(((const uint16_t*)g.A)[off]) : ((const float*)g.A)[off];
+      }
+      As[kk][m] = v;
+      int n;
+      if (b_nfast) { n = t & 63; kk = t >> 6; } else { kk = t & 15; n = t >> 4; }
+      int gn = n0 + n;
+      gk = k0 + kk;
+      v = 0.f;
+      if (gn < g.N && gk < g.K) {
+        long long off = bb + gk * g.sBk + gn * g.sBn;
+        v = BBF ? bf16_bits_to_float(((const uint16_t*)g.B)[off]) : ((const float*)g.B)[off];
+      }
+      Bs[kk][n] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+
+  double local = 0.0;
+  const long long cb = (long long)(b / g.divC) * g.sCb;
+  const long long pb = (long long)b * g.sPb;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int gm = m0 + ty * 4 + i;
+    if (gm >= g.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int gn = n0 + tx * 4 + j;
+      if (gn >= g.N) continue;
+      float v = g.alpha * acc[i][j];
+      if (g.mode & GEMM_SUBP) v -= g.P[pb + gm * g.sPm + gn * g.sPn];
+      if (g.mode & GEMM_SQSUM) local += (double)v * (double)v;
+      if (g.mode & GEMM_STORE) {
+        float* c = g.C + cb + gm * g.sCm + gn * g.sCn;
+        if (g.mode & GEMM_ATOMIC) atomicAdd(c, v);
+        else if (g.mode & GEMM_ACCUM) *c += v;
+        else *c = v;
+      }
+    }
+  }
+  if (g.mode & GEMM_SQSUM) {
+    double s = block_sum_double(local, red);
+    if (tid == 0) atomicAdd(g.sq, s);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// block inverse: Gauss-Jordan with partial pivoting, one CTA per k x k block, matrix kept in the output
+// buffer (global memory, L2 resident).  Also emits the column square norms c[t] = sum_i Minv[i][t]^2.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) block_inverse_kernel(const float* __restrict__ Min, float* __restrict__ Out,
+                                                             float* __restrict__ cnorm, int k, int32_t* status) {
+  if (status && *status) return;
+  extern __shared__ float sm[];  // prow[k], fcol[k], piv (int) [k], red
+  float* prow = sm;
+  float* fcol = sm + k;
+  int* piv = (int*)(sm + 2 * k);
+  __shared__ float rv[32];
+  __shared__ int ri[32];
+  __shared__ int s_r;
+  __shared__ int s_bad;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const float* A0 = Min + (size_t)blockIdx.x * k * k;
+  float* A = Out + (size_t)blockIdx.x * k * k;
+  for (int e = tid; e < k * k; e += nt) A[e] = A0[e];
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  for (int p = 0; p < k; ++p) {
+    // pivot search over rows >= p of column p
+    float best = -1.f;
+    int bi = p;
+    for (int i = p + tid; i < k; i += nt) {
+      float v = fabsf(A[(size_t)i * k + p]);
+      if (v > best) { best = v; bi = i; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if ((tid & 31) == 0) { rv[tid >> 5] = best; ri[tid >> 5] = bi; }
+    __syncthreads();
+    if (tid < 32) {
+      int nw = (nt + 31) >> 5;
+      best = (tid < nw) ? rv[tid] : -1.f;
+      bi = (tid < nw) ? ri[tid] : p;
+      for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+      }
+      if (tid == 0) {
+        s_r = bi;
+        piv[p] = bi;
+        if (!(best > 1e-30f) || !isfinite(best)) s_bad = 1;
+      }
+    }
+    __syncthreads();
+    if (s_bad) {
+      if (tid == 0) raise_status(status, CAFEQ_ERR_SINGULAR);
+      return;
+    }
+    const int r = s_r;
+    // exchange rows p and r; keep the (new) pivot row in shared memory
+    for (int j = tid; j < k; j += nt) {
+      float vr = A[(size_t)r * k + j], vp = A[(size_t)p * k + j];
+      A[(size_t)r * k + j] = vp;
+      prow[j] = vr;
+    }
+    __syncthreads();
+    const float d = 1.0f / prow[p];
+    // column p after the exchange (factors); row p itself handled separately
+    for (int i = tid; i < k; i += nt) fcol[i] = (i == p) ? 0.f : A[(size_t)i * k + p];
+    __syncthreads();
+    for (int e = tid; e < k * k; e += nt) {
+      int i = e / k, j = e - i * k;
+      float sp = (j == p) ? d : prow[j] * d;
+      if (i == p) {
+        A[e] = sp;
+      } else {
+        float cur = (j == p) ? 0.f : A[e];
+        A[e] = fmaf(-fcol[i], sp, cur);
+      }
+    }
+    __syncthreads();
+  }
+  // undo the row exchanges as column exchanges in reverse order
+  for (int p = k - 1; p >= 0; --p) {
+    int r = piv[p];
+    if (r != p) {
+      for (int i = tid; i < k; i += nt) {
+        float a = A[(size_t)i * k + p];
+        A[(size_t)i * k + p] = A[(size_t)i * k + r];
+        A[(size_t)i * k + r] = a;
+      }
+    }
+    __syncthreads();
+  }
+  if (cnorm) {
+    for (int t = tid; t < k; t += nt) {
+      float s = 0.f;
+      for (int i = 0; i < k; ++i) {
+        float v = A[(size_t)i * k + t];
+        s = fmaf(v, v, s);
+      }
+      cnorm[(size_t)blockIdx.x * k + t] = s;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// group absmax with arg-max (lowest index on ties): one warp per (row, group)
+// ------------------------------------------------------------------------------------------------
+__global__ void absmax_kernel(const float* __restrict__ U, long long ld, int rows, int ng, int g,
+                              float* __restrict__ a, int* __restrict__ idx, int32_t* status) {
+  if (status && *status) return;
+  long long w = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const long long total = (long long)rows * ng;
+  if (w >= total) return;
+  const int row = (int)(w / ng), G = (int)(w - (long long)row * ng);
+  const float* p = U + row * ld + (long long)G * g;
+  float best = -1.f;
+  int bi = 0x7fffffff;
+  bool bad = false;
+  for (int e = lane; e < g; e += 32) {
+    float v = fabsf(p[e]);
+    if (!(v <= 3.0e38f)) bad = true;
+    if (v > best) { best = v; bi = e; }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+  }
+  if (__any_sync(0xffffffffu, bad)) {
+    if (lane == 0) raise_status(status, CAFEQ_ERR_NONFINITE);
+    return;
+  }
+  if (lane == 0) {
+    a[w] = best;
+    idx[w] = bi;
+  }
+}
+
+__global__ void scales_kernel(const float* __restrict__ a, float* __restrict__ s, long long n, float qmax,
+                              const int32_t* status) {
+  if (status && *status) return;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    s[i] = __fdiv_rn(a[i], qmax);
+}
+
+// ------------------------------------------------------------------------------------------------
+// quantise: code, dequantised value, residual Delta = Uhat - U
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float quantise_one(float u, float s, float qmax, float off, int off_kind) {
+  float x = (s > 0.f) ? __fdiv_rn(u, s) : 0.f;
+  float q = (off_kind == CAFEQ_OFFSETS_NONE) ? rintf(x) : floorf(x) + off;
+  return fminf(fmaxf(q, -qmax), qmax);
+}
+
+__global__ void quant_kernel(const float* __restrict__ U, long long ld, int rows, int cols, int g,
+                             const float* __restrict__ a, float qmax, const void* __restrict__ offsets, int off_kind,
+                             float* __restrict__ Delta, float* __restrict__ Uhat, int8_t* __restrict__ codes,
+                             const int32_t* status) {
+  if (status && *status) return;
+  const int ng = cols / g;
+  const long long n = (long long)rows * cols;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
+    float u = U[row * ld + col];
+    float s = __fdiv_rn(a[(long long)row * ng + col / g], qmax);
+    float off = 0.f;
+    if (off_kind == CAFEQ_OFFSETS_HARD_U8) off = (float)((const uint8_t*)offsets)[e];
+    else if (off_kind == CAFEQ_OFFSETS_SOFT_F32) off = ((const float*)offsets)[e];
+    float q = quantise_one(u, s, qmax, off, off_kind);
+    float uh = s * q;
+    if (Delta) Delta[row * ld + col] = uh - u;
+    if (Uhat) Uhat[row * ld + col] = uh;
+    if (codes) codes[e] = (int8_t)q;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// surrogate (Eq. 4 per entry): weights cw, loss, arg-max coefficients, A_t
+// ------------------------------------------------------------------------------------------------
+// axis IN:  cw[Gc] = sum_{t in group Gc} c[t'],  t' = (B / r) * k + (t mod k), B = t / k
+__global__ void cw_in_kernel(const float* __restrict__ c, int d_in, int g, int k, int r, float* __restrict__ cw) {
+  int Gc = blockIdx.x * blockDim.x + threadIdx.x;
+  if (Gc >= d_in / g) return;
+  float s = 0.f;
+  for (int e = 0; e < g; ++e) {
+    int t = Gc * g + e;
+    int B = t / k;
+    s += c[(B / r) * k + (t - B * k)];
+  }
+  cw[Gc] = s;
+}
+
+// axis OUT: cw[row] = g * c[t'(row)]
+__global__ void cw_out_kernel(const float* __restrict__ c, int d_out, int g, int k, int r, float* __restrict__ cw) {
+  int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= d_out) return;
+  int B = row / k;
+  cw[row] = (float)g * c[(B / r) * k + (row - B * k)];
+}
+
+// one thread per row: loss partial sum and arg-max coefficients  coef = scale * cw * a * sign(U[e*]).
+// A_t accumulation: axis IN  Agrp[Gc] += a^2 (per column group, expanded later);
+//                   axis OUT A[t'(row)] += g * sum_G a^2.
+__global__ void surrogate_rows_kernel(const float* __restrict__ a, const int* __restrict__ idx,
+                                      const float* __restrict__ U, long long ld, int rows, int ng, int g, int axis,
+                                      const float* __restrict__ cw, float kappa, int k, int r, float* __restrict__ coef,
+                                      float* __restrict__ Agrp, float* __restrict__ A, double* __restrict__ acc,
+                                      const int32_t* status) {
+  if (status && *status) return;
+  __shared__ double red[32];
+  int row = blockIdx.x * blockDim.x + threadIdx.x;
+  double local = 0.0;
+  if (row < rows) {
+    float srow = 0.f;
+    for (int G = 0; G < ng; ++G) {
+      long long w = (long long)row * ng + G;
+      float av = a[w];
+      float u = U[row * ld + (long long)G * g + idx[w]];
+      float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
+      float wgt = (axis == CAFEQ_AXIS_IN) ? cw[G] : cw[row];
+      local += (double)wgt * (double)av * (double)av;
+      if (coef) coef[w] = 2.f * kappa * wgt * av * sgn;
+      if (axis == CAFEQ_AXIS_IN) {
+        if (Agrp) atomicAdd(&Agrp[G], av * av);
+      } else {
+        srow += av * av;
+      }
+    }
+    if (axis == CAFEQ_AXIS_OUT && A) {
+      int B = row / k;
+      atomicAdd(&A[(B / r) * k + (row - B * k)], (float)g * srow);
+    }
+  }
+  double s = block_sum_double(local, red);
+  if (threadIdx.x == 0) atomicAdd(acc, (double)kappa * s);
+}
+
+// axis IN: A[t'] += Agrp[group of t]
+__global__ void expand_agrp_kernel(const float* __restrict__ Agrp, int d_in, int g, int k, int r, float* __restrict__ A) {
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= d_in) return;
+  int B = t / k;
+  atomicAdd(&A[(B / r) * k + (t - B * k)], Agrp[t / g]);
+}
+
+// gMinv[b][i][t] = scale * Minv[b][i][t] * A[b][t]
+__global__ void scale_cols_kernel(const float* __restrict__ Minv, const float* __restrict__ A, float scale, int k,
+                                  long long n, float* __restrict__ out) {
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    long long b = e / ((long long)k * k);
+    int t = (int)(e % k);
+    out[e] = scale * Minv[e] * A[b * k + t];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// straight-through scale path: coef[row, G] = sign(U[e*]) / qmax * sum_{e in G} gDelta_e (q_e - U_e / s_G)
+// (+ optionally, for the pair PQE loss, the direct term stays in gU and is handled by a dense product)
+// ------------------------------------------------------------------------------------------------
+__global__ void ste_scale_path_kernel(const float* __restrict__ U, const float* __restrict__ gD, long long ld, int rows,
+                                      int ng, int g, const float* __restrict__ a, const int* __restrict__ idx, float qmax,
+                                      const void* __restrict__ offsets, int off_kind, int cols, float* __restrict__ coef,
+                                      const int32_t* status) {
+  if (status && *status) return;
+  long long w = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= (long long)rows * ng) return;
+  const int row = (int)(w / ng), G = (int)(w - (long long)row * ng);
+  const float av = a[w];
+  const float s = __fdiv_rn(av, qmax);
+  float sum = 0.f;
+  for (int e = lane; e < g; e += 32) {
+    long long col = (long long)G * g + e;
+    float u = U[row * ld + col];
+    float off = 0.f;
+    if (off_kind == CAFEQ_OFFSETS_HARD_U8) off = (float)((const uint8_t*)offsets)[(long long)row * cols + col];
+    else if (off_kind == CAFEQ_OFFSETS_SOFT_F32) off = ((const float*)offsets)[(long long)row * cols + col];
+    float q = quantise_one(u, s, qmax, off, off_kind);
+    float x = (s > 0.f) ? __fdiv_rn(u, s) : 0.f;
+    sum = fmaf(gD[row * ld + col], q - x, sum);
+  }
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) {
+    float u = U[row * ld + (long long)G * g + idx[w]];
+    float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
+    coef[w] = sum * sgn / qmax;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// sparse backward: gradT[B/r][i][j] += sum over (row, group) pairs routed through their arg-max entry
+//   axis IN : pair (o, G) in block B adds coef * W[o, B*k + j] to row i* = (G*g + idx) mod k
+//   axis OUT: pair (B*k + i, G) adds coef * W[B*k + j, G*g + idx] to row i
+// transpose_out stores into gradT[..][j][i] instead (operator applied transposed).
+// One CTA owns a strip of JS columns j of one block and accumulates it in shared memory.
+// ------------------------------------------------------------------------------------------------
+constexpr int SCATTER_JS = 32;
+
+__global__ void __launch_bounds__(256) scatter_in_kernel(const uint16_t* __restrict__ W, long long ld, int d_out, int d_in,
+                                                         int g, int k, int r, const float* __restrict__ coef,
+                                                         const int* __restrict__ idx, float* __restrict__ gradT,
+                                                         int transpose_out, int rows_per_cta, const int32_t* status) {
+  if (status && *status) return;
+  extern __shared__ float acc[];  // [k][SCATTER_JS]
+  const int B = blockIdx.x, js = blockIdx.y * SCATTER_JS;
+  const int r0 = blockIdx.z * rows_per_cta, r1 = min(d_out, r0 + rows_per_cta);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+  for (int e = tid; e < k * SCATTER_JS; e += blockDim.x) acc[e] = 0.f;
+  __syncthreads();
+  const int ng = d_in / g;
+  const int j = js + lane;
+  // groups that intersect this block: columns [B*k, B*k + k)
+  const int G0 = (B * k) / g, G1 = (B * k + k - 1) / g;
+  for (int o = r0 + warp; o < r1; o += nw) {
+    float w = (j < k) ? bf16_bits_to_float(W[o * ld + (long long)B * k + j]) : 0.f;
+    for (int G = G0; G <= G1; ++G) {
+      long long p = (long long)o * ng + G;
+      int col = G * g + idx[p];          // arg-max column of the group
+      if (col < B * k || col >= B * k + k) continue;  // group larger than the block: arg-max in another block
+      float cf = coef[p];
+      if (j < k && cf != 0.f) atomicAdd(&acc[(col - B * k) * SCATTER_JS + lane], cf * w);
+    }
+  }
+  __syncthreads();
+  float* out = gradT + (size_t)(B / r) * k * k;
+  for (int e = tid; e < k * SCATTER_JS; e += blockDim.x) {
+    int i = e / SCATTER_JS, jj = js + (e - i * SCATTER_JS);
+    if (jj < k && acc[e] != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], acc[e]);
+  }
+}
+
+__global__ void __launch_bounds__(256) scatter_out_kernel(const uint16_t* __restrict__ W, long long ld, int d_out, int d_in,
+                                                          int g, int k, int r, const float* __restrict__ coef,
+                                                          const int* __restrict__ idx, float* __restrict__ gradT,
+                                                          int transpose_out, int groups_per_cta, const int32_t* status) {
+  if (status && *status) return;
+  extern __shared__ float acc[];  // [k][SCATTER_JS]
+  const int B = blockIdx.x, js = blockIdx.y * SCATTER_JS;
+  const int ng = d_in / g;
+  const int G0 = blockIdx.z * groups_per_cta, G1 = min(ng, G0 + groups_per_cta);
+  const int tid = threadIdx.x;
+  for (int e = tid; e < k * SCATTER_JS; e += blockDim.x) acc[e] = 0.f;
+  __syncthreads();
+  // thread handles (i, jj) pairs: i over rows of the block, jj over the strip
+  for (int e = tid; e < k * SCATTER_JS; e += blockDim.x) {
+    int i = e / SCATTER_JS, jj = e - i * SCATTER_JS;
+    int j = js + jj;
+    if (j >= k) continue;
+    float s = 0.f;
+    long long row = (long long)B * k + i;
+    for (int G = G0; G < G1; ++G) {
+      long long p = row * ng + G;
+      float cf = coef[p];
+      if (cf != 0.f) s = fmaf(cf, bf16_bits_to_float(W[((long long)B * k + j) * ld + (long long)G * g + idx[p]]), s);
+    }
+    acc[e] = s;
+  }
+  __syncthreads();
+  float* out = gradT + (size_t)(B / r) * k * k;
+  for (int e = tid; e < k * SCATTER_JS; e += blockDim.x) {
+    int i = e / SCATTER_JS, jj = js + (e - i * SCATTER_JS);
+    if (jj < k && acc[e] != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], acc[e]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// optimiser updates and bookkeeping
+// ------------------------------------------------------------------------------------------------
+__global__ void gd_update_kernel(float* __restrict__ M, const float* __restrict__ g, float lr, long long n,
+                                 const int32_t* status) {
+  if (status && *status) return;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    M[i] = M[i] - lr * g[i];
+}
+
+// state = {step, m[n], v[n]}; the step counter is advanced by adam_tick_kernel before the update.
+__global__ void adam_tick_kernel(float* state, const int32_t* status) {
+  if (status && *status) return;
+  state[0] += 1.f;
+}
+
+__global__ void adam_update_kernel(float* __restrict__ M, const float* __restrict__ g, float* __restrict__ state, float lr,
+                                   float b1, float b2, float eps, long long n, const int32_t* status) {
+  if (status && *status) return;
+  const float step = state[0];
+  const float c1 = 1.f - powf(b1, step), c2 = 1.f - powf(b2, step);
+  float* m = state + 1;
+  float* v = state + 1 + n;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    float gi = g[i];
+    float mi = b1 * m[i] + (1.f - b1) * gi;
+    float vi = b2 * v[i] + (1.f - b2) * gi * gi;
+    m[i] = mi;
+    v[i] = vi;
+    M[i] = M[i] - lr * (mi / c1) / (sqrtf(vi / c2) + eps);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// reductions: sum of squares of bf16 / fp32 arrays
+// ------------------------------------------------------------------------------------------------
+__global__ void sqsum_bf16_kernel(const uint16_t* __restrict__ W, long long ld, int rows, int cols, double* acc,
+                                  const int32_t* status) {
+  if (status && *status) return;
+  __shared__ double red[32];
+  double local = 0.0;
+  const long long n = (long long)rows * cols;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
+    float v = bf16_bits_to_float(W[row * ld + col]);
+    local += (double)v * v;
+  }
+  double s = block_sum_double(local, red);
+  if (threadIdx.x == 0) atomicAdd(acc, s);
+}
+
+// ------------------------------------------------------------------------------------------------
+// pair: LogSumExp over group maxima (two passes), orthonormality penalty
+// ------------------------------------------------------------------------------------------------
+__global__ void max_f32_kernel(const float* __restrict__ a, long long n, float* __restrict__ out_max,
+                               const int32_t* status) {
+  // a >= 0, so an integer atomicMax on the bit pattern orders correctly
+  if (status && *status) return;
+  float m = 0.f;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    m = fmaxf(m, a[i]);
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) atomicMax((int*)out_max, __float_as_int(m));
+}
+
+__global__ void sumexp_kernel(const float* __restrict__ a, long long n, const float* __restrict__ amax, float t,
+                              double* __restrict__ acc, const int32_t* status) {
+  if (status && *status) return;
+  __shared__ double red[32];
+  const float mx = *amax;
+  double local = 0.0;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    local += (double)expf(t * (a[i] - mx));
+  double s = block_sum_double(local, red);
+  if (threadIdx.x == 0) atomicAdd(acc, s);
+}
+
+// coef[w] = exp(t (a - max)) / Z * sign(U[arg-max])
+__global__ void lse_coef_kernel(const float* __restrict__ a, const int* __restrict__ idx, const float* __restrict__ U,
+                                long long ld, int rows, int ng, int g, const float* __restrict__ amax, float t,
+                                const double* __restrict__ Z, float* __restrict__ coef, const int32_t* status) {
+  if (status && *status) return;
+  const long long n = (long long)rows * ng;
+  const float mx = *amax;
+  const float zinv = (float)(1.0 / *Z);
+  for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < n; w += (long long)gridDim.x * blockDim.x) {
+    int row = (int)(w / ng), G = (int)(w - (long long)row * ng);
+    float u = U[row * ld + (long long)G * g + idx[w]];
+    float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
+    coef[w] = expf(t * (a[w] - mx)) * zinv * sgn;
+  }
+}
+
+// R = M M^T - I in place on a [nb,k,k] buffer that already holds M M^T
+__global__ void sub_identity_kernel(float* __restrict__ R, int k, long long n) {
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    long long q = e % ((long long)k * k);
+    if (q / k == q % k) R[e] -= 1.f;
+  }
+}
+
+__global__ void sqsum_f32_kernel(const float* __restrict__ x, long long n, double* acc) {
+  __shared__ double red[32];
+  double local = 0.0;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    local += (double)x[i] * x[i];
+  double s = block_sum_double(local, red);
+  if (threadIdx.x == 0) atomicAdd(acc, s);
+}
+
+// gradM += lambda * 2 (R M) / (||R||_F sqrt(h));  RM holds R M;  nothing when the norm is below 1e-12
+__global__ void orth_grad_kernel(float* __restrict__ gradM, const float* __restrict__ RM, const double* __restrict__ r2,
+                                 float lambda, float sqrt_h, long long n) {
+  const double nrm = sqrt(*r2);
+  if (nrm < 1e-12) return;
+  const float f = (float)(2.0 * lambda / (nrm * sqrt_h));
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    gradM[i] += f * RM[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// finalisers: double accumulators -> the fp32 outputs of the API
+// ------------------------------------------------------------------------------------------------
+// single: acc = {surrogate, L2, ||W||^2}
+__global__ void finalize_single_kernel(const double* acc, float* losses, float* hist /*[2] or NULL*/, int want_exact) {
+  if (losses) {
+    losses[0] = (float)acc[0];
+    losses[1] = want_exact ? (float)acc[1] : 0.f;
+    losses[2] = want_exact ? (float)acc[2] : 0.f;
+    losses[3] = 0.f;
+  }
+  if (hist) {
+    hist[0] = (float)acc[0];
+    hist[1] = want_exact ? (float)acc[1] : nanf("");
+  }
+}
+
+// pair: acc = {Z, ||R_orth||^2, PQE^2}; amax = running max
+__global__ void finalize_pair_kernel(const double* acc, const float* amax, float t, float lambda, float sqrt_h,
+                                     float* losses, float* hist, int want_pqe) {
+  float lse = *amax + (float)(log(acc[0]) / (double)t);
+  float orth = (float)(sqrt(acc[1]) / (double)sqrt_h);
+  if (losses) {
+    losses[0] = lse + lambda * orth;
+    losses[1] = lse;
+    losses[2] = orth;
+    losses[3] = want_pqe ? (float)acc[2] : 0.f;
+  }
+  if (hist) {
+    hist[0] = lse + lambda * orth;
+    hist[1] = want_pqe ? (float)acc[2] : nanf("");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// pack: u = q + qmax, little-endian bit stream per row; one thread per output 32-bit word group
+// ------------------------------------------------------------------------------------------------
+__global__ void pack_kernel(const int8_t* __restrict__ codes, uint8_t* __restrict__ packed, int rows, int cols, int bits) {
+  // one thread packs 8 consecutive codes into `bits` bytes
+  const long long chunks_per_row = cols / 8;
+  const long long n = (long long)rows * chunks_per_row;
+  const int qmax = (1 << (bits - 1)) - 1;
+  for (long long c = blockIdx.x * (long long)blockDim.x + threadIdx.x; c < n; c += (long long)gridDim.x * blockDim.x) {
+    long long row = c / chunks_per_row, ch = c - row * chunks_per_row;
+    const int8_t* src = codes + row * cols + ch * 8;
+    unsigned long long v = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v |= (unsigned long long)((unsigned)(src[i] + qmax) & ((1u << bits) - 1u)) << (bits * i);
+    uint8_t* dst = packed + row * ((long long)cols * bits / 8) + ch * bits;
+    for (int b = 0; b < bits; ++b) dst[b] = (uint8_t)(v >> (8 * b));
+  }
+}
+
+}  // namespace cafeq
