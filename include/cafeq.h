@@ -174,6 +174,16 @@ int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed,
 
 const char* cafeq_status_string(int status);
 int cafeq_version(void);
+/* Number of kernels this library has launched in the calling process so far (host counter, for
+ * benchmarks that must state how many of the library's kernels ran inside a timed region). */
+long long cafeq_debug_launch_count(void);
+/* Benchmark aid: time selected kernels of later calls with CUDA events recorded on the launching stream.
+ * begin() creates `capacity` event pairs (host objects, no device memory); read() waits for the recorded
+ * events, writes up to `capacity` durations in milliseconds and kernel kinds (1 transform pass, 2 sparse
+ * backward, 3 block inverse, 4 dense pair product) to HOST arrays, sets *count and releases the events.
+ * Not thread-safe; launches beyond the capacity are simply not timed. */
+int cafeq_debug_timer_begin(int capacity);
+int cafeq_debug_timer_read(float* ms, int* kinds, int* count);
 
 #ifdef __cplusplus
 }

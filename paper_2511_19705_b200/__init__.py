@@ -24,7 +24,8 @@ OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_status_string", "cafeq_version",
+    "cafeq_pack", "cafeq_debug_timer_begin", "cafeq_debug_timer_read", "cafeq_debug_launch_count",
+    "cafeq_status_string", "cafeq_version",
 ]
 
 
@@ -61,8 +62,9 @@ def lib() -> ctypes.CDLL:
         L.cafeq_status_string.restype = ctypes.c_char_p
         L.cafeq_status_string.argtypes = [ctypes.c_int]
         L.cafeq_version.restype = ctypes.c_int
-        for name in EXPORTS[:-2]:
+        for name in EXPORTS[:-3]:
             getattr(L, name).restype = ctypes.c_int
+        L.cafeq_debug_launch_count.restype = ctypes.c_longlong
         _lib = L
     return _lib
 
@@ -73,6 +75,24 @@ def status_string(code: int) -> str:
 
 def version() -> int:
     return lib().cafeq_version()
+
+
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(lib().cafeq_debug_launch_count())
+
+
+def timer_begin(capacity: int) -> None:
+    _check(lib().cafeq_debug_timer_begin(ctypes.c_int(capacity)), "cafeq_debug_timer_begin")
+
+
+def timer_read(capacity: int):
+    """Returns (durations_ms list, kinds list) of the kernels timed since timer_begin."""
+    ms = (ctypes.c_float * max(capacity, 1))()
+    kinds = (ctypes.c_int * max(capacity, 1))()
+    n = ctypes.c_int(0)
+    _check(lib().cafeq_debug_timer_read(ms, kinds, ctypes.byref(n)), "cafeq_debug_timer_read")
+    return [ms[i] for i in range(n.value)], [kinds[i] for i in range(n.value)]
 
 
 def _check(rc: int, where: str) -> None:

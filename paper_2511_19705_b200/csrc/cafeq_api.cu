@@ -6,10 +6,43 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <atomic>
+#include <vector>
+
 #include "cafeq.h"
 #include "kernels_generic.cuh"
 
 namespace cafeq {
+
+// Process-wide count of kernel launches made by this library (read by benchmarks through
+// cafeq_debug_launch_count; it has no effect on any result).
+static std::atomic<long long> g_launches{0};
+#define CQ_LAUNCH(kernel, grid, block, smem, st, ...)       \
+  do {                                                      \
+    g_launches.fetch_add(1, std::memory_order_relaxed);     \
+    kernel<<<grid, block, smem, st>>>(__VA_ARGS__);         \
+  } while (0)
+
+// Optional per-launch timing of selected kernels with CUDA events on the launching stream (benchmarks
+// only; off unless cafeq_debug_timer_begin was called).  Kinds: 1 transform pass, 2 sparse backward,
+// 3 block inverse, 4 dense pair product.
+struct KernelTimer {
+  std::vector<cudaEvent_t> a, b;
+  std::vector<int> kind;
+  int used = 0;
+  bool on = false;
+};
+static KernelTimer g_kt;
+static inline int kt_begin(int kind, cudaStream_t st) {
+  if (!g_kt.on || g_kt.used >= (int)g_kt.a.size()) return -1;
+  int i = g_kt.used++;
+  g_kt.kind[i] = kind;
+  cudaEventRecord(g_kt.a[i], st);
+  return i;
+}
+static inline void kt_end(int i, cudaStream_t st) {
+  if (i >= 0) cudaEventRecord(g_kt.b[i], st);
+}
 
 // ------------------------------------------------------------------------------------------------
 // workspace carving
@@ -94,10 +127,10 @@ static size_t matrix_scratch_bytes(const Geo& G) {
 // ------------------------------------------------------------------------------------------------
 static void launch_gemm(cudaStream_t st, const GemmArgs& g) {
   dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, g.batch);
-  if (g.a_bf16 && g.b_bf16) gemm_kernel<true, true><<<grid, 256, 0, st>>>(g);
-  else if (g.a_bf16) gemm_kernel<true, false><<<grid, 256, 0, st>>>(g);
-  else if (g.b_bf16) gemm_kernel<false, true><<<grid, 256, 0, st>>>(g);
-  else gemm_kernel<false, false><<<grid, 256, 0, st>>>(g);
+  if (g.a_bf16 && g.b_bf16) CQ_LAUNCH((gemm_kernel<true, true>), grid, 256, 0, st, g);
+  else if (g.a_bf16) CQ_LAUNCH((gemm_kernel<true, false>), grid, 256, 0, st, g);
+  else if (g.b_bf16) CQ_LAUNCH((gemm_kernel<false, true>), grid, 256, 0, st, g);
+  else CQ_LAUNCH((gemm_kernel<false, false>), grid, 256, 0, st, g);
 }
 
 static GemmArgs gemm_defaults(const int32_t* status) {
@@ -135,7 +168,9 @@ static void launch_apply(cudaStream_t st, const void* X, int x_bf16, long long l
     g.B = X; g.b_bf16 = x_bf16; g.sBk = ldx; g.sBn = 1; g.sBb = (long long)k * ldx;
     g.sCm = ldo; g.sCn = 1; g.sCb = (long long)k * ldo;
   }
+  int ti = kt_begin(1, st);
   launch_gemm(st, g);
+  kt_end(ti, st);
 }
 
 // gT[b / r][i][j] += alpha * sum_free Gm[.., i] X[.., j]  (atomic accumulation; caller zeroes gT)
@@ -181,13 +216,15 @@ static void launch_kk(cudaStream_t st, const float* A, int tA, const float* B, i
 static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float* cnorm, int nb, int k, int32_t* status) {
   int threads = k * k >= 1024 ? 1024 : ((k * k + 31) / 32) * 32;
   size_t sh = (size_t)3 * k * sizeof(float);
-  block_inverse_kernel<<<nb, threads, sh, st>>>(Mc, Minv, cnorm, k, status);
+  int ti = kt_begin(3, st);
+  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status);
+  kt_end(ti, st);
 }
 
 static void launch_absmax(cudaStream_t st, const float* U, long long ld, const Geo& G, float* a, int* idx, int32_t* status) {
   long long warps = (long long)G.d_out * G.ng;
   long long blocks = (warps * 32 + 255) / 256;
-  absmax_kernel<<<(unsigned)blocks, 256, 0, st>>>(U, ld, G.d_out, G.ng, G.g, a, idx, status);
+  CQ_LAUNCH(absmax_kernel, (unsigned)blocks, 256, 0, st, U, ld, G.d_out, G.ng, G.g, a, idx, status);
 }
 
 static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const float* coef, const int* idx, float* gT,
@@ -199,6 +236,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     cudaFuncSetAttribute(scatter_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
   }
   int strips = (k + SCATTER_JS - 1) / SCATTER_JS;
+  int ti = kt_begin(2, st);
   if (G.axis == CAFEQ_AXIS_IN) {
     int want = (148 * 4) / (G.nbq * strips) + 1;
     int splits = want < 1 ? 1 : want;
@@ -206,7 +244,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     if (rows_per < 8) rows_per = 8;
     splits = (G.d_out + rows_per - 1) / rows_per;
     dim3 grid(G.nbq, strips, splits);
-    scatter_in_kernel<<<grid, 256, sh, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
+    CQ_LAUNCH(scatter_in_kernel, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
                                              transpose_out, rows_per, status);
   } else {
     int want = (148 * 4) / (G.nbq * strips) + 1;
@@ -215,9 +253,10 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     if (per < 1) per = 1;
     splits = (G.ng + per - 1) / per;
     dim3 grid(G.nbq, strips, splits);
-    scatter_out_kernel<<<grid, 256, sh, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
+    CQ_LAUNCH(scatter_out_kernel, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
                                               transpose_out, per, status);
   }
+  kt_end(ti, st);
 }
 
 __global__ void bf16_to_f32_kernel(const uint16_t* __restrict__ W, long long ld, int rows, int cols, float* __restrict__ U) {
@@ -270,10 +309,10 @@ static void forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits
                           const MatWS& w, const void* offsets, int off_kind, bool want_delta, float* Uhat, int8_t* codes,
                           int32_t* status) {
   if (Tc) launch_apply(st, W, 1, G.ld, G, Tc, transposed, w.U, G.d_in, GEMM_STORE, nullptr, status);
-  else bf16_to_f32_kernel<<<grid_for(G.n), 256, 0, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, w.U);
+  else CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, w.U);
   launch_absmax(st, w.U, G.d_in, G, w.a, w.idx, status);
   if (want_delta || Uhat || codes)
-    quant_kernel<<<grid_for(G.n), 256, 0, st>>>(w.U, G.d_in, G.d_out, G.d_in, G.g, w.a, qmax_of(bits), offsets, off_kind,
+    CQ_LAUNCH(quant_kernel, grid_for(G.n), 256, 0, st, w.U, G.d_in, G.d_out, G.d_in, G.g, w.a, qmax_of(bits), offsets, off_kind,
                                                 want_delta ? w.D : nullptr, Uhat, codes, status);
 }
 
@@ -297,6 +336,42 @@ extern "C" const char* cafeq_status_string(int s) {
 }
 
 extern "C" int cafeq_version(void) { return 100; }
+
+extern "C" long long cafeq_debug_launch_count(void) { return g_launches.load(); }
+
+extern "C" int cafeq_debug_timer_begin(int capacity) {
+  if (capacity < 0 || g_kt.on) return CAFEQ_ERR_INVALID_ARG;
+  g_kt.a.resize(capacity);
+  g_kt.b.resize(capacity);
+  g_kt.kind.assign(capacity, 0);
+  for (int i = 0; i < capacity; ++i) {
+    if (cudaEventCreate(&g_kt.a[i]) != cudaSuccess || cudaEventCreate(&g_kt.b[i]) != cudaSuccess) return CAFEQ_ERR_CUDA;
+  }
+  g_kt.used = 0;
+  g_kt.on = true;
+  return CAFEQ_OK;
+}
+
+extern "C" int cafeq_debug_timer_read(float* ms, int* kinds, int* count) {
+  if (!g_kt.on || !ms || !kinds || !count) return CAFEQ_ERR_INVALID_ARG;
+  int rc = CAFEQ_OK;
+  for (int i = 0; i < g_kt.used; ++i) {
+    if (cudaEventSynchronize(g_kt.b[i]) != cudaSuccess || cudaEventElapsedTime(&ms[i], g_kt.a[i], g_kt.b[i]) != cudaSuccess)
+      rc = CAFEQ_ERR_CUDA;
+    kinds[i] = g_kt.kind[i];
+  }
+  *count = g_kt.used;
+  for (size_t i = 0; i < g_kt.a.size(); ++i) {
+    cudaEventDestroy(g_kt.a[i]);
+    cudaEventDestroy(g_kt.b[i]);
+  }
+  g_kt.a.clear();
+  g_kt.b.clear();
+  g_kt.kind.clear();
+  g_kt.used = 0;
+  g_kt.on = false;
+  return rc;
+}
 
 extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
                                     size_t* bytes) {
@@ -343,10 +418,10 @@ extern "C" int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float*
   carve_matrix(b, G, &w, false);
   float* Tc = has_T ? b.take<float>((size_t)G.nbT * G.k * G.k) : nullptr;
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
-  if (has_T) round_bf16_kernel<<<grid_for((long long)G.nbT * G.k * G.k), 256, 0, st>>>(T, Tc, (long long)G.nbT * G.k * G.k, nullptr);
+  if (has_T) CQ_LAUNCH(round_bf16_kernel, grid_for((long long)G.nbT * G.k * G.k), 256, 0, st, T, Tc, (long long)G.nbT * G.k * G.k, nullptr);
   forward_quant(st, W, G, d->bits, Tc, d->trole == CAFEQ_APPLY_TT, w, nullptr, CAFEQ_OFFSETS_NONE, false, nullptr, codes,
                 nullptr);
-  scales_kernel<<<grid_for((long long)G.d_out * G.ng), 256, 0, st>>>(w.a, scales, (long long)G.d_out * G.ng,
+  CQ_LAUNCH(scales_kernel, grid_for((long long)G.d_out * G.ng), 256, 0, st, w.a, scales, (long long)G.d_out * G.ng,
                                                                      qmax_of(d->bits), nullptr);
   return last_launch();
 }
@@ -384,38 +459,38 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   const float qm = qmax_of(d->bits);
   const bool ste = (loss_kind == CAFEQ_LOSS_L2_STE);
   const bool need_l2 = want_exact || ste;
-  zero_f64_kernel<<<1, 32, 0, st>>>(s.acc, 8);
-  round_bf16_kernel<<<grid_for(kk), 256, 0, st>>>(M, s.Mc, kk, status);
+  CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, s.acc, 8);
+  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, s.Mc, kk, status);
   launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
-  if (Minv_out) copy_f32_kernel<<<grid_for(kk), 256, 0, st>>>(s.Minv, Minv_out, kk);
+  if (Minv_out) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, Minv_out, kk);
   forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, status);
   if (need_l2) {
     // E = Minv o Delta, L2 = sum E^2
     launch_apply(st, s.m.D, 0, G.d_in, G, s.Minv, 0, s.m.E, G.d_in, (ste ? GEMM_STORE : 0) | GEMM_SQSUM, s.acc + 1, status);
-    sqsum_bf16_kernel<<<grid_for(G.n), 256, 0, st>>>((const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);
+    CQ_LAUNCH(sqsum_bf16_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);
   }
   // surrogate value, arg-max coefficients and A_t
   const bool want_grad = (gradM != nullptr);
-  if (G.axis == CAFEQ_AXIS_IN) cw_in_kernel<<<(G.ng + 127) / 128, 128, 0, st>>>(s.c, G.d_in, G.g, k, G.r, s.m.cw);
-  else cw_out_kernel<<<(G.d_out + 127) / 128, 128, 0, st>>>(s.c, G.d_out, G.g, k, G.r, s.m.cw);
-  fill_f32_kernel<<<grid_for(G.nbT * k), 256, 0, st>>>(s.A, 0.f, (long long)G.nbT * k);
-  fill_f32_kernel<<<grid_for(G.ng), 256, 0, st>>>(s.m.agrp, 0.f, G.ng);
-  surrogate_rows_kernel<<<(G.d_out + 127) / 128, 128, 0, st>>>(s.m.a, s.m.idx, s.m.U, G.d_in, G.d_out, G.ng, G.g, G.axis,
+  if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, s.c, G.d_in, G.g, k, G.r, s.m.cw);
+  else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(G.nbT * k), 256, 0, st, s.A, 0.f, (long long)G.nbT * k);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(G.ng), 256, 0, st, s.m.agrp, 0.f, G.ng);
+  CQ_LAUNCH(surrogate_rows_kernel, (G.d_out + 127) / 128, 128, 0, st, s.m.a, s.m.idx, s.m.U, G.d_in, G.d_out, G.ng, G.g, G.axis,
                                                                s.m.cw, kappa, k, G.r, (want_grad && !ste) ? s.m.coef : nullptr,
                                                                s.m.agrp, s.A, s.acc + 0, status);
-  if (G.axis == CAFEQ_AXIS_IN) expand_agrp_kernel<<<(G.d_in + 127) / 128, 128, 0, st>>>(s.m.agrp, G.d_in, G.g, k, G.r, s.A);
-  finalize_single_kernel<<<1, 1, 0, st>>>(s.acc, losses, hist, need_l2 ? 1 : 0);
+  if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, s.m.agrp, G.d_in, G.g, k, G.r, s.A);
+  CQ_LAUNCH(finalize_single_kernel, 1, 1, 0, st, s.acc, losses, hist, need_l2 ? 1 : 0);
   if (!want_grad) return;
-  fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(gradM, 0.f, kk);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
   if (!ste) {
     launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
-    scale_cols_kernel<<<grid_for(kk), 256, 0, st>>>(s.Minv, s.A, 2.f * kappa, k, kk, s.gMinv);
+    CQ_LAUNCH(scale_cols_kernel, grid_for(kk), 256, 0, st, s.Minv, s.A, 2.f * kappa, k, kk, s.gMinv);
   } else {
     // gMinv = 2 * sum_free E Delta^T ; gDelta = 2 Minv^T o E (overwrites Delta) ; scale path through arg-max
-    fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(s.gMinv, 0.f, kk);
+    CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, s.gMinv, 0.f, kk);
     launch_opgrad(st, s.m.E, G.d_in, s.m.D, 0, G.d_in, G, s.gMinv, 0, 2.f, status);
     launch_apply(st, s.m.E, 0, G.d_in, G, s.Minv, 1, s.m.D, G.d_in, GEMM_STORE, nullptr, status, 2.f);
-    ste_scale_path_kernel<<<(unsigned)(((long long)G.d_out * G.ng * 32 + 255) / 256), 256, 0, st>>>(
+    CQ_LAUNCH(ste_scale_path_kernel, (unsigned)(((long long)G.d_out * G.ng * 32 + 255) / 256), 256, 0, st, 
         s.m.U, s.m.D, G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.idx, qm, offsets, off_kind, G.d_in, s.m.coef, status);
     launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
   }
@@ -476,10 +551,10 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
     single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
                 loss_history + 2 * (size_t)it, grad, status, s);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
-      gd_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, cfg->lr, kk, status);
+      CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
-      adam_tick_kernel<<<1, 1, 0, st>>>(opt_state, status);
-      adam_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
+      CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
+      CQ_LAUNCH(adam_update_kernel, grid_for(kk), 256, 0, st, M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
                                                        status);
     }
   }
@@ -515,7 +590,7 @@ static void launch_pair_product(cudaStream_t st, const void* A1, int a1_bf16, lo
     g.K = G1.d_out; g.batch = 1;
     g.mode = GEMM_STORE;
   } else {
-    fill_f32_kernel<<<grid_for((long long)d1n * d3n), 256, 0, st>>>(Cm, 0.f, (long long)d1n * d3n);
+    CQ_LAUNCH(fill_f32_kernel, grid_for((long long)d1n * d3n), 256, 0, st, Cm, 0.f, (long long)d1n * d3n);
     g.K = k; g.batch = G2.nbq;
     g.sAb = (long long)k * ld1; g.divA = G2.r;
     g.sBb = k;
@@ -552,38 +627,38 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   const int k = G1.k;
   const long long kk = (long long)G1.nbT * k * k;
   const float sqrt_h = sqrtf((float)G1.d_out);
-  zero_f64_kernel<<<1, 32, 0, st>>>(p.acc, 8);
-  fill_f32_kernel<<<1, 32, 0, st>>>(p.amax, 0.f, 1);
-  round_bf16_kernel<<<grid_for(kk), 256, 0, st>>>(M, p.Mc, kk, status);
+  CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, p.acc, 8);
+  CQ_LAUNCH(fill_f32_kernel, 1, 32, 0, st, p.amax, 0.f, 1);
+  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, p.Mc, kk, status);
   launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
-  round_bf16_kernel<<<grid_for(kk), 256, 0, st>>>(p.Minv, p.Minv_c, kk, status);
+  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, p.Minv, p.Minv_c, kk, status);
   // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
   forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
                 status);
   forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
                 nullptr, status);
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
-  max_f32_kernel<<<grid_for(n1), 256, 0, st>>>(p.m1.a, n1, p.amax, status);
-  max_f32_kernel<<<grid_for(n2), 256, 0, st>>>(p.m2.a, n2, p.amax, status);
-  sumexp_kernel<<<grid_for(n1), 256, 0, st>>>(p.m1.a, n1, p.amax, t, p.acc + 0, status);
-  sumexp_kernel<<<grid_for(n2), 256, 0, st>>>(p.m2.a, n2, p.amax, t, p.acc + 0, status);
+  CQ_LAUNCH(max_f32_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, status);
+  CQ_LAUNCH(max_f32_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.amax, status);
+  CQ_LAUNCH(sumexp_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, t, p.acc + 0, status);
+  CQ_LAUNCH(sumexp_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.amax, t, p.acc + 0, status);
   // orthonormality penalty on the fp32 parameters: R = M M^T - I
   launch_kk(st, M, 0, M, 1, p.tmp, G1.nbT, k, 1.f, GEMM_STORE, status);
-  sub_identity_kernel<<<grid_for(kk), 256, 0, st>>>(p.tmp, k, kk);
-  sqsum_f32_kernel<<<grid_for(kk), 256, 0, st>>>(p.tmp, kk, p.acc + 1);
+  CQ_LAUNCH(sub_identity_kernel, grid_for(kk), 256, 0, st, p.tmp, k, kk);
+  CQ_LAUNCH(sqsum_f32_kernel, grid_for(kk), 256, 0, st, p.tmp, kk, p.acc + 1);
   if (want_pqe) {
     launch_pair_product(st, p.m1.E, 0, G1.d_in, p.m2.E, 0, G2.d_in, G1, G2, p.R, status);
-    resid_sq_kernel<<<grid_for((long long)G1.d_in * G2.d_out), 256, 0, st>>>(p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
+    CQ_LAUNCH(resid_sq_kernel, grid_for((long long)G1.d_in * G2.d_out), 256, 0, st, p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
                                                                              status);
   }
-  finalize_pair_kernel<<<1, 1, 0, st>>>(p.acc, p.amax, t, lambda, sqrt_h, losses, hist, want_pqe ? 1 : 0);
+  CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, want_pqe ? 1 : 0);
   if (!gradM) return;
-  lse_coef_kernel<<<grid_for(n1), 256, 0, st>>>(p.m1.a, p.m1.idx, p.m1.U, G1.d_in, G1.d_out, G1.ng, G1.g, p.amax, t, p.acc + 0,
+  CQ_LAUNCH(lse_coef_kernel, grid_for(n1), 256, 0, st, p.m1.a, p.m1.idx, p.m1.U, G1.d_in, G1.d_out, G1.ng, G1.g, p.amax, t, p.acc + 0,
                                                 p.m1.coef, status);
-  lse_coef_kernel<<<grid_for(n2), 256, 0, st>>>(p.m2.a, p.m2.idx, p.m2.U, G2.d_in, G2.d_out, G2.ng, G2.g, p.amax, t, p.acc + 0,
+  CQ_LAUNCH(lse_coef_kernel, grid_for(n2), 256, 0, st, p.m2.a, p.m2.idx, p.m2.U, G2.d_in, G2.d_out, G2.ng, G2.g, p.amax, t, p.acc + 0,
                                                 p.m2.coef, status);
-  fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(gradM, 0.f, kk);
-  fill_f32_kernel<<<grid_for(kk), 256, 0, st>>>(p.gMinv, 0.f, kk);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
   // U side: operator is M^T, so the block gradient is stored transposed
   launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status);
   // V side: gradient with respect to Minv, then through the inverse
@@ -592,7 +667,7 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   launch_kk(st, p.RM, 0, p.Minv, 1, gradM, G1.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
   if (lambda != 0.f) {
     launch_kk(st, p.tmp, 0, M, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
-    orth_grad_kernel<<<grid_for(kk), 256, 0, st>>>(gradM, p.RM, p.acc + 1, lambda, sqrt_h, kk);
+    CQ_LAUNCH(orth_grad_kernel, grid_for(kk), 256, 0, st, gradM, p.RM, p.acc + 1, lambda, sqrt_h, kk);
   }
 }
 
@@ -659,10 +734,10 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
               grad, status, p);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
-      gd_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, cfg->lr, kk, status);
+      CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
-      adam_tick_kernel<<<1, 1, 0, st>>>(opt_state, status);
-      adam_update_kernel<<<grid_for(kk), 256, 0, st>>>(M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
+      CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
+      CQ_LAUNCH(adam_update_kernel, grid_for(kk), 256, 0, st, M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
                                                        status);
     }
   }
@@ -684,6 +759,6 @@ extern "C" int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8
   if (rc) return rc;
   if (!codes || !packed) return CAFEQ_ERR_INVALID_ARG;
   if (G.d_in % 8) return CAFEQ_ERR_UNSUPPORTED;
-  pack_kernel<<<grid_for(G.n / 8), 256, 0, (cudaStream_t)stream>>>(codes, packed, G.d_out, G.d_in, d->bits);
+  CQ_LAUNCH(pack_kernel, grid_for(G.n / 8), 256, 0, (cudaStream_t)stream, codes, packed, G.d_out, G.d_in, d->bits);
   return last_launch();
 }
