@@ -320,14 +320,17 @@ def pair_product(A1s, A2s, k: int, r: int):
 
 
 def orth_penalty(M):
-    """||M M^T - I||_F / sqrt(d) on the whole block-diagonal M, and its gradient."""
+    """||M M^T - I||_F / sqrt(d) on the whole block-diagonal M, and its gradient.
+
+    The norm is not squared, so its gradient has no limit at M M^T = I; below 1e-5 (the noise floor
+    of an fp32 product of a rotation stored in fp32) the gradient is taken as zero."""
     M = np.asarray(M, dtype=np.float64)
     nb, k, _ = M.shape
     R = M @ np.transpose(M, (0, 2, 1)) - np.eye(k)
     nrm = np.sqrt(np.sum(R * R))
     d = nb * k
-    if nrm < 1e-12:
-        return 0.0, np.zeros_like(M)
+    if nrm / np.sqrt(d) < 1e-5:
+        return float(nrm / np.sqrt(d)), np.zeros_like(M)
     return float(nrm / np.sqrt(d)), (2.0 * R @ M) / (nrm * np.sqrt(d))
 
 

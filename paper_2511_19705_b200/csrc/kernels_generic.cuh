@@ -649,11 +649,12 @@ __global__ void sqsum_f32_kernel(const float* __restrict__ x, long long n, doubl
   if (threadIdx.x == 0) atomicAdd(acc, s);
 }
 
-// gradM += lambda * 2 (R M) / (||R||_F sqrt(h));  RM holds R M;  nothing when the norm is below 1e-12
+// gradM += lambda * 2 (R M) / (||R||_F sqrt(h));  RM holds R M;  nothing when ||R||_F / sqrt(h) < 1e-5
+// (the un-squared norm has no gradient at R = 0 and below the fp32 noise floor its direction is noise)
 __global__ void orth_grad_kernel(float* __restrict__ gradM, const float* __restrict__ RM, const double* __restrict__ r2,
                                  float lambda, float sqrt_h, long long n) {
   const double nrm = sqrt(*r2);
-  if (nrm < 1e-12) return;
+  if (nrm < 1e-5 * (double)sqrt_h) return;
   const float f = (float)(2.0 * lambda / (nrm * sqrt_h));
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
     gradM[i] += f * RM[i];

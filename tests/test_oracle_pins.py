@@ -392,6 +392,8 @@ def test_orth_penalty_value_and_gradient():
     assert val == pytest.approx(np.linalg.norm(D @ D.T - np.eye(8)) / np.sqrt(8), rel=1e-12)
     assert np.allclose(g, _fd(lambda X: orc.orth_penalty(X)[0], M), rtol=1e-5, atol=1e-9)
     assert orc.orth_penalty(syn.identity_blocks(2, 4))[0] == 0.0
+    v, g0 = orc.orth_penalty(syn.haar_blocks(2, 4, 1))          # a rotation stored in fp32: value ~1e-8, no gradient
+    assert v < 1e-6 and not g0.any()
 
 
 # ------------------------------------------------------------------ LogSumExp (P8)
