@@ -179,8 +179,9 @@ int cafeq_version(void);
 long long cafeq_debug_launch_count(void);
 /* Benchmark aid: time selected kernels of later calls with CUDA events recorded on the launching stream.
  * begin() creates `capacity` event pairs (host objects, no device memory); read() waits for the recorded
- * events, writes up to `capacity` durations in milliseconds and kernel kinds (1 transform pass, 2 sparse
- * backward, 3 block inverse, 4 dense pair product) to HOST arrays, sets *count and releases the events.
+ * events, writes up to `capacity` durations in milliseconds and kernel kinds (1 transform pass on the
+ * shape-agnostic kernels, 2 sparse backward, 3 block inverse, 4 dense pair product, 5 fused tensor-core
+ * transform pass) to HOST arrays, sets *count and releases the events.
  * Not thread-safe; launches beyond the capacity are simply not timed. */
 int cafeq_debug_timer_begin(int capacity);
 int cafeq_debug_timer_read(float* ms, int* kinds, int* count);

@@ -11,6 +11,7 @@
 
 #include "cafeq.h"
 #include "kernels_generic.cuh"
+#include "kernels_fused.cuh"
 
 namespace cafeq {
 
@@ -24,8 +25,8 @@ static std::atomic<long long> g_launches{0};
   } while (0)
 
 // Optional per-launch timing of selected kernels with CUDA events on the launching stream (benchmarks
-// only; off unless cafeq_debug_timer_begin was called).  Kinds: 1 transform pass, 2 sparse backward,
-// 3 block inverse, 4 dense pair product.
+// only; off unless cafeq_debug_timer_begin was called).  Kinds: 1 transform pass (shape-agnostic kernels),
+// 2 sparse backward, 3 block inverse, 4 dense pair product, 5 fused tensor-core transform pass.
 struct KernelTimer {
   std::vector<cudaEvent_t> a, b;
   std::vector<int> kind;
@@ -114,7 +115,8 @@ static size_t matrix_scratch_bytes(const Geo& G) {
   size_t rows_ng = (size_t)G.d_out * G.ng;
   size_t b = 0;
   b += 3 * ((size_t)G.n * 4 + 256);                   // U, Delta / gDelta, E / Uhat
-  b += 3 * (rows_ng * 4 + 256);                       // a, idx, coef
+  b += (size_t)G.n * 2 + 256;                         // bf16 residual of the fused pass
+  b += 4 * (rows_ng * 4 + 256);                       // a, usel, idx, coef
   b += ((size_t)G.ng + G.d_out + G.d_in) * 4 + 1024;  // cw, Agrp
   b += 8 * (kk * 4 + 256);                            // Mc, Minv, Minv_c, gMinv, tmp, RM, ...
   b += 4 * ((size_t)(G.nbT + 1) * (G.k + 1) * 4 + 256);  // c, A
@@ -221,10 +223,11 @@ static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float*
   kt_end(ti, st);
 }
 
-static void launch_absmax(cudaStream_t st, const float* U, long long ld, const Geo& G, float* a, int* idx, int32_t* status) {
+static void launch_absmax(cudaStream_t st, const float* U, long long ld, const Geo& G, float* a, float* usel, int* idx,
+                          int32_t* status) {
   long long warps = (long long)G.d_out * G.ng;
   long long blocks = (warps * 32 + 255) / 256;
-  CQ_LAUNCH(absmax_kernel, (unsigned)blocks, 256, 0, st, U, ld, G.d_out, G.ng, G.g, a, idx, status);
+  CQ_LAUNCH(absmax_kernel, (unsigned)blocks, 256, 0, st, U, ld, G.d_out, G.ng, G.g, a, usel, idx, status);
 }
 
 static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const float* coef, const int* idx, float* gT,
@@ -287,33 +290,69 @@ __global__ void store_sqrt_kernel(const double* acc, float* out) { *out = (float
 // per-matrix scratch
 // ------------------------------------------------------------------------------------------------
 struct MatWS {
+  uint16_t *Tb, *Dbf;  // fused pass: bf16 operator blocks (applied orientation) and bf16 residual
   float *U, *D, *E;
-  float *a, *coef, *cw, *agrp;
+  float *a, *usel, *coef, *cw, *agrp;
   int* idx;
 };
 
 static void carve_matrix(Bump& b, const Geo& G, MatWS* w, bool need_E) {
+  w->Tb = b.take<uint16_t>((size_t)(G.nbT > 0 ? G.nbT : 1) * (G.k > 0 ? G.k : 1) * (G.k > 0 ? G.k : 1));
+  w->Dbf = b.take<uint16_t>(G.n);
   w->U = b.take<float>(G.n);
   w->D = b.take<float>(G.n);
   w->E = need_E ? b.take<float>(G.n) : nullptr;
   size_t rows_ng = (size_t)G.d_out * G.ng;
   w->a = b.take<float>(rows_ng);
+  w->usel = b.take<float>(rows_ng);
   w->idx = b.take<int>(rows_ng);
   w->coef = b.take<float>(rows_ng);
   w->cw = b.take<float>((size_t)(G.ng > G.d_out ? G.ng : G.d_out));
   w->agrp = b.take<float>((size_t)G.ng);
 }
 
-// U = T o W, group absmax / arg-max, and (optionally) the quantiser outputs.
-static void forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits, const float* Tc, int transposed,
+// One fused tensor-core pass (see kernels_fused.cuh); returns false when the shape is not covered.
+static bool fused_pass(cudaStream_t st, const void* X, long long ldx, const Geo& G, const float* Top, int transposed,
+                       uint16_t* Tb, BdParams p, int32_t* status) {
+  const int form = (G.axis == CAFEQ_AXIS_IN) ? BD_IN : BD_OUT;
+  if (!bd_supported(form, G.d_out, G.d_in, ldx, G.k, G.g, X)) return false;
+  const long long kk = (long long)G.nbT * G.k * G.k;
+  CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Top, Tb, G.k, kk, transposed, status);
+  p.d_out = G.d_out;
+  p.d_in = G.d_in;
+  p.r = G.r;
+  p.status = status;
+  int ti = kt_begin(5, st);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  int rc = bd_launch(st, form, G.k, G.g, X, ldx, Tb, G.nbT, p);
+  kt_end(ti, st);
+  return rc == CAFEQ_OK;
+}
+
+// U = T o W, group absmax / arg-max, and (optionally) the quantiser outputs.  Returns true when the fused
+// tensor-core pass ran (then the residual is in w.Dbf as bf16 instead of w.D as fp32, and U is not stored).
+static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits, const float* Tc, int transposed,
                           const MatWS& w, const void* offsets, int off_kind, bool want_delta, float* Uhat, int8_t* codes,
-                          int32_t* status) {
+                          float* scales, int32_t* status, bool allow_fused) {
+  if (Tc && allow_fused && off_kind == CAFEQ_OFFSETS_NONE && !Uhat) {
+    BdParams p;
+    memset(&p, 0, sizeof(p));
+    p.epi = EPI_ABSMAX | (want_delta ? EPI_DELTA : 0) | (codes ? EPI_CODES : 0);
+    p.qmax = qmax_of(bits);
+    p.a = w.a; p.usel = w.usel; p.idx = w.idx;
+    p.delta = w.Dbf; p.codes = codes; p.scales = scales;
+    if (fused_pass(st, W, G.ld, G, Tc, transposed, w.Tb, p, status)) return true;
+  }
   if (Tc) launch_apply(st, W, 1, G.ld, G, Tc, transposed, w.U, G.d_in, GEMM_STORE, nullptr, status);
   else CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, w.U);
-  launch_absmax(st, w.U, G.d_in, G, w.a, w.idx, status);
+  launch_absmax(st, w.U, G.d_in, G, w.a, w.usel, w.idx, status);
   if (want_delta || Uhat || codes)
     CQ_LAUNCH(quant_kernel, grid_for(G.n), 256, 0, st, w.U, G.d_in, G.d_out, G.d_in, G.g, w.a, qmax_of(bits), offsets, off_kind,
-                                                want_delta ? w.D : nullptr, Uhat, codes, status);
+              want_delta ? w.D : nullptr, Uhat, codes, status);
+  if (scales)
+    CQ_LAUNCH(scales_kernel, grid_for((long long)G.d_out * G.ng), 256, 0, st, w.a, scales, (long long)G.d_out * G.ng,
+              qmax_of(bits), status);
+  return false;
 }
 
 }  // namespace cafeq
@@ -420,9 +459,7 @@ extern "C" int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float*
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
   if (has_T) CQ_LAUNCH(round_bf16_kernel, grid_for((long long)G.nbT * G.k * G.k), 256, 0, st, T, Tc, (long long)G.nbT * G.k * G.k, nullptr);
   forward_quant(st, W, G, d->bits, Tc, d->trole == CAFEQ_APPLY_TT, w, nullptr, CAFEQ_OFFSETS_NONE, false, nullptr, codes,
-                nullptr);
-  CQ_LAUNCH(scales_kernel, grid_for((long long)G.d_out * G.ng), 256, 0, st, w.a, scales, (long long)G.d_out * G.ng,
-                                                                     qmax_of(d->bits), nullptr);
+                scales, nullptr, true);
   return last_launch();
 }
 
@@ -453,7 +490,7 @@ static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
 // Enqueue one forward(+backward) for a single matrix; gradM may be null.  hist is an optional [2] slot.
 static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& G, const void* W, const float* M,
                         float* Minv_out, const void* offsets, int off_kind, int loss_kind, float kappa, bool want_exact,
-                        float* losses, float* hist, float* gradM, int32_t* status, const SingleWS& s) {
+                        float* losses, float* hist, float* gradM, int32_t* status, const SingleWS& s, bool force_generic) {
   const int k = G.k;
   const long long kk = (long long)G.nbT * k * k;
   const float qm = qmax_of(d->bits);
@@ -463,10 +500,20 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, s.Mc, kk, status);
   launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
   if (Minv_out) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, Minv_out, kk);
-  forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, status);
+  const bool fused = forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, nullptr,
+                                   status, !ste && !force_generic);
   if (need_l2) {
     // E = Minv o Delta, L2 = sum E^2
-    launch_apply(st, s.m.D, 0, G.d_in, G, s.Minv, 0, s.m.E, G.d_in, (ste ? GEMM_STORE : 0) | GEMM_SQSUM, s.acc + 1, status);
+    bool done = false;
+    if (fused) {
+      BdParams bp;
+      memset(&bp, 0, sizeof(bp));
+      bp.epi = EPI_SQSUM;
+      bp.sqacc = s.acc + 1;
+      done = fused_pass(st, s.m.Dbf, G.d_in, G, s.Minv, 0, s.m.Tb, bp, status);
+    }
+    if (!done)
+      launch_apply(st, s.m.D, 0, G.d_in, G, s.Minv, 0, s.m.E, G.d_in, (ste ? GEMM_STORE : 0) | GEMM_SQSUM, s.acc + 1, status);
     CQ_LAUNCH(sqsum_bf16_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);
   }
   // surrogate value, arg-max coefficients and A_t
@@ -475,7 +522,7 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
   CQ_LAUNCH(fill_f32_kernel, grid_for(G.nbT * k), 256, 0, st, s.A, 0.f, (long long)G.nbT * k);
   CQ_LAUNCH(fill_f32_kernel, grid_for(G.ng), 256, 0, st, s.m.agrp, 0.f, G.ng);
-  CQ_LAUNCH(surrogate_rows_kernel, (G.d_out + 127) / 128, 128, 0, st, s.m.a, s.m.idx, s.m.U, G.d_in, G.d_out, G.ng, G.g, G.axis,
+  CQ_LAUNCH(surrogate_rows_kernel, (G.d_out + 127) / 128, 128, 0, st, s.m.a, s.m.usel, G.d_out, G.ng, G.g, G.axis,
                                                                s.m.cw, kappa, k, G.r, (want_grad && !ste) ? s.m.coef : nullptr,
                                                                s.m.agrp, s.A, s.acc + 0, status);
   if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, s.m.agrp, G.d_in, G.g, k, G.r, s.A);
@@ -491,7 +538,7 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
     launch_opgrad(st, s.m.E, G.d_in, s.m.D, 0, G.d_in, G, s.gMinv, 0, 2.f, status);
     launch_apply(st, s.m.E, 0, G.d_in, G, s.Minv, 1, s.m.D, G.d_in, GEMM_STORE, nullptr, status, 2.f);
     CQ_LAUNCH(ste_scale_path_kernel, (unsigned)(((long long)G.d_out * G.ng * 32 + 255) / 256), 256, 0, st, 
-        s.m.U, s.m.D, G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.idx, qm, offsets, off_kind, G.d_in, s.m.coef, status);
+        s.m.U, s.m.D, G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.usel, qm, offsets, off_kind, G.d_in, s.m.coef, status);
     launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
   }
   // gradM -= Minv^T gMinv Minv^T
@@ -521,7 +568,7 @@ extern "C" int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* 
   SingleWS s;
   if (!carve_single(b, G, &s, true)) return CAFEQ_ERR_WORKSPACE;
   single_step(st, d, G, W, M, Minv, offsets, offsets_kind, loss_kind, kappa, (flags & CAFEQ_FLAG_EXACT_LOSS) != 0, losses,
-              nullptr, want_grad ? gradM : nullptr, status, s);
+              nullptr, want_grad ? gradM : nullptr, status, s, (flags & CAFEQ_FLAG_GENERIC) != 0);
   return last_launch();
 }
 
@@ -549,7 +596,7 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = cfg->eval_every > 0 && (it % cfg->eval_every == 0);
     single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
-                loss_history + 2 * (size_t)it, grad, status, s);
+                loss_history + 2 * (size_t)it, grad, status, s, false);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
@@ -623,7 +670,7 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
 
 static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
                       const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
-                      float* losses, float* hist, float* gradM, int32_t* status, const PairWS& p) {
+                      float* losses, float* hist, float* gradM, int32_t* status, const PairWS& p, bool force_generic) {
   const int k = G1.k;
   const long long kk = (long long)G1.nbT * k * k;
   const float sqrt_h = sqrtf((float)G1.d_out);
@@ -634,9 +681,9 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, p.Minv, p.Minv_c, kk, status);
   // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
   forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
-                status);
+                nullptr, status, !force_generic);
   forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
-                nullptr, status);
+                nullptr, nullptr, status, !force_generic);
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
   CQ_LAUNCH(max_f32_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, status);
   CQ_LAUNCH(max_f32_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.amax, status);
@@ -653,9 +700,9 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   }
   CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, want_pqe ? 1 : 0);
   if (!gradM) return;
-  CQ_LAUNCH(lse_coef_kernel, grid_for(n1), 256, 0, st, p.m1.a, p.m1.idx, p.m1.U, G1.d_in, G1.d_out, G1.ng, G1.g, p.amax, t, p.acc + 0,
+  CQ_LAUNCH(lse_coef_kernel, grid_for(n1), 256, 0, st, p.m1.a, p.m1.usel, n1, p.amax, t, p.acc + 0,
                                                 p.m1.coef, status);
-  CQ_LAUNCH(lse_coef_kernel, grid_for(n2), 256, 0, st, p.m2.a, p.m2.idx, p.m2.U, G2.d_in, G2.d_out, G2.ng, G2.g, p.amax, t, p.acc + 0,
+  CQ_LAUNCH(lse_coef_kernel, grid_for(n2), 256, 0, st, p.m2.a, p.m2.usel, n2, p.amax, t, p.acc + 0,
                                                 p.m2.coef, status);
   CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
   CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
@@ -705,7 +752,7 @@ extern "C" int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* 
   PairWS p;
   if (!carve_pair(b, G1, G2, &p, want_pqe)) return CAFEQ_ERR_WORKSPACE;
   pair_step((cudaStream_t)stream, d1, d2, G1, G2, W1, W2, M, P, lse_t, lambda_orth, want_pqe, losses, nullptr,
-            want_grad ? gradM : nullptr, status, p);
+            want_grad ? gradM : nullptr, status, p, (flags & CAFEQ_FLAG_GENERIC) != 0);
   return last_launch();
 }
 
@@ -732,7 +779,7 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = any_pqe && (it % cfg->eval_every == 0);
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
-              grad, status, p);
+              grad, status, p, false);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {

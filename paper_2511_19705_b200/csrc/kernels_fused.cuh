@@ -1,0 +1,522 @@
+// Fused block-diagonal transform pass on the 5th-generation tensor cores (sm_100a):
+//   U = T o X on one axis of a bf16 matrix X, accumulated in tensor memory, followed in the same kernel by
+//   the per-group work the method needs on U -- absmax / arg-max (Eq. 1's scale, Eq. 4's ||.||_inf, the
+//   LogSumExp maxima), round-to-nearest codes, the residual Delta = Q(U) - U, or a sum of squares.
+// U never goes to HBM.  One CTA keeps its operator block(s) resident in shared memory and streams tiles of
+// X through a TMA ring; accumulators are double-buffered in tensor memory so the epilogue of tile t overlaps
+// the products of tile t+1.
+//
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer (and tensor-memory owner),
+// warps 2..9 = epilogue (two warps per 32-lane quarter, each owning 128 accumulator columns).
+// Every wait on an mbarrier is bounded; when one runs out the kernel raises CAFEQ_ERR_TIMEOUT in the status
+// word, all roles leave their loops, tensor memory is released and the kernel returns.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cafeq.h"
+#include "kernels_generic.cuh"
+
+namespace cafeq {
+
+enum { BD_IN = 0, BD_OUT = 1 };
+enum { EPI_ABSMAX = 1, EPI_DELTA = 2, EPI_CODES = 4, EPI_SQSUM = 8 };
+
+struct BdParams {
+  int d_out, d_in;     // shape of X
+  int r;               // matrix blocks per operator block
+  int n_major;         // IN: tile columns (256 d_in columns each); OUT: row blocks (k rows each)
+  int n_minor;         // IN: row tiles of 128; OUT: column tiles of NC
+  int ctas_per_major;
+  int epi;
+  float qmax;
+  float* a;            // [d_out, d_in / G] group absmax
+  float* usel;         // signed value at the arg-max
+  int* idx;            // arg-max position inside the group
+  uint16_t* delta;     // bf16 [d_out, d_in], row stride d_in
+  int8_t* codes;       // [d_out, d_in]
+  float* scales;       // [d_out, d_in / G]
+  double* sqacc;
+  int32_t* status;
+};
+
+constexpr int BD_THREADS = 320;
+constexpr int BD_STAGE_BYTES = 16384;  // one TMA box: 64 columns x 128 rows of bf16
+constexpr int BD_STAGES_PER_TILE = 4;
+constexpr uint64_t BD_WAIT_NS = 2000000000ull;
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when the limit ran out here or in another role (abort flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > BD_WAIT_NS) {
+        *abort_flag = 1;
+        raise_status(status, CAFEQ_ERR_TIMEOUT);
+        return false;
+      }
+      __nanosleep(32);
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 bytes apart.
+// K-major operands step along K by moving the start address inside the swizzled row; MN-major operands
+// step along K by whole 8-row groups.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;              // leading byte offset (unused: one swizzle chunk along the leading dim)
+  d |= (uint64_t)(1024 >> 4) << 32;    // stride byte offset: next 8-row group
+  d |= (uint64_t)1 << 46;              // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;              // SWIZZLE_128B
+  return d;
+}
+
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
+         ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------------
+template <int FORM, int K, int G>
+struct BdCfg {
+  static constexpr int NBLK = (FORM == BD_IN) ? 256 / K : 1;          // operator blocks resident per CTA
+  static constexpr int T_BYTES = NBLK * K * K * 2;
+  static constexpr int KH = (K >= 128) ? K / 128 : 1;                 // OUT: 128-row halves of the block
+  static constexpr int NC = 256 / KH;                                 // OUT: d_in columns per tile
+  static constexpr int NSTAGE = (T_BYTES >= 131072) ? 5 : 6;
+  static constexpr int SMEM = 1024 + T_BYTES + NSTAGE * BD_STAGE_BYTES + 256;
+};
+
+template <int FORM, int K, int G>
+__global__ void __launch_bounds__(BD_THREADS, 1)
+bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmT, const BdParams p) {
+  using C = BdCfg<FORM, K, G>;
+  static_assert(K == 64 || K == 128 || K == 256, "block size");
+  static_assert(FORM == BD_IN || K >= 128, "output-axis form needs k >= 128");
+  static_assert(G == 64 || G == 128, "group size");
+  if (p.status && *p.status) return;
+
+  const int major = blockIdx.x / p.ctas_per_major;
+  const int sub = blockIdx.x - major * p.ctas_per_major;
+  const int m_begin = (int)(((long long)sub * p.n_minor) / p.ctas_per_major);
+  const int m_end = (int)(((long long)(sub + 1) * p.n_minor) / p.ctas_per_major);
+  if (m_begin >= m_end) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sT = smem;
+  uint8_t* sStage = smem + C::T_BYTES;
+  uint64_t* bars = (uint64_t*)(sStage + C::NSTAGE * BD_STAGE_BYTES);
+  // barrier slots: full[NSTAGE], empty[NSTAGE], tfull, accf[2], acce[2]
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8 * C::NSTAGE;
+  const uint32_t bar_tfull = bar_empty + 8 * C::NSTAGE;
+  const uint32_t bar_accf = bar_tfull + 8;
+  const uint32_t bar_acce = bar_accf + 16;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 5);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::NSTAGE; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    mbar_init(bar_tfull, 1);
+    mbar_init(bar_accf, 1);
+    mbar_init(bar_accf + 8, 1);
+    mbar_init(bar_acce, 8);
+    mbar_init(bar_acce + 8, 8);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(bar_tfull, C::T_BYTES);
+      for (int bi = 0; bi < C::NBLK; ++bi) {
+        const int tb = (FORM == BD_IN) ? (major * C::NBLK + bi) / p.r : major / p.r;
+        for (int ci = 0; ci < K / 64; ++ci)
+          tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), &tmT, ci * 64, tb * K, bar_tfull);
+      }
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = m_begin; t < m_end && ok; ++t) {
+        for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
+          const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          mbar_expect_tx(bar_full + 8 * s, BD_STAGE_BYTES);
+          int x, y;
+          if constexpr (FORM == BD_IN) {
+            x = major * 256 + sidx * 64;
+            y = t * 128;
+          } else {
+            const int nc = sidx / C::KH, kh = sidx % C::KH;
+            x = t * C::NC + nc * 64;
+            y = major * K + kh * 128;
+          }
+          tma_load_2d(smem_u32(sStage + s * BD_STAGE_BYTES), &tmX, x, y, bar_full + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      bool ok = mbar_wait(bar_tfull, 0, abort_flag, p.status);
+      tc_fence_after();
+      constexpr uint32_t idesc_in = umma_idesc_bf16(128, K, 0, 0);
+      constexpr uint32_t idesc_out = umma_idesc_bf16(128, 64, 0, 1);
+      const uint32_t sT_u = smem_u32(sT), sSt_u = smem_u32(sStage);
+      uint32_t it = 0, tl = 0;
+      for (int t = m_begin; t < m_end && ok; ++t, ++tl) {
+        const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
+        if (!mbar_wait(bar_acce + 8 * buf, aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t dbase = tmem_base + buf * 256u;
+        for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
+          const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+          if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
+          if constexpr (FORM == BD_IN) {
+            const int bi = (sidx * 64) / K, ci = ((sidx * 64) % K) / 64;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const uint64_t ad = umma_desc_sw128(stage + kk * 32);
+              const uint64_t bd = umma_desc_sw128(sT_u + bi * K * K * 2 + ci * K * 128 + kk * 32);
+              tc_mma_bf16(dbase + bi * K, ad, bd, idesc_in, (ci | kk) != 0 ? 1u : 0u);
+            }
+          } else {
+            const int nc = sidx / C::KH, kh = sidx % C::KH;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint64_t bd = umma_desc_sw128(stage + ks * 2048);
+#pragma unroll
+              for (int mh = 0; mh < C::KH; ++mh) {
+                const uint64_t ad = umma_desc_sw128(sT_u + (kh * 2 + ks / 4) * K * 128 + mh * 128 * 128 + (ks % 4) * 32);
+                tc_mma_bf16(dbase + mh * C::NC + nc * 64, ad, bd, idesc_out, (kh | ks) != 0 ? 1u : 0u);
+              }
+            }
+          }
+          tc_commit(bar_empty + 8 * s);
+        }
+        if (ok) tc_commit(bar_accf + 8 * buf);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3, hw = (warp - 2) >> 2;
+    const int L = q * 32 + lane;
+    uint32_t tl = 0;
+    bool ok = true;
+    double sq_local = 0.0;
+    bool bad = false;
+    constexpr int NG = 128 / G;
+    const int ng_row = p.d_in / G;
+    for (int t = m_begin; t < m_end && ok; ++t, ++tl) {
+      const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
+      ok = mbar_wait(bar_accf + 8 * buf, aph, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256u + hw * 128u;
+      int row, col0;
+      if constexpr (FORM == BD_IN) {
+        row = t * 128 + L;
+        col0 = major * 256 + hw * 128;
+      } else if constexpr (K == 256) {
+        row = major * 256 + hw * 128 + L;
+        col0 = t * 128;
+      } else {
+        row = major * 128 + L;
+        col0 = t * 256 + hw * 128;
+      }
+      const bool valid = (row < p.d_out) && (col0 < p.d_in);
+      float v[32];
+      float best[NG], bval[NG];
+      int bidx[NG];
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) { best[gi] = -1.f; bval[gi] = 0.f; bidx[gi] = 0; }
+      float sq = 0.f;
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        tc_ld32(taddr + ch * 32, v);
+        const int gi = (G == 128) ? 0 : (ch >> 1);
+        const int e0 = (G == 128) ? ch * 32 : (ch & 1) * 32;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float av = fabsf(v[e]);
+          if (av > best[gi]) { best[gi] = av; bval[gi] = v[e]; bidx[gi] = e0 + e; }
+          sq = fmaf(v[e], v[e], sq);
+        }
+      }
+      if (p.epi & EPI_SQSUM) sq_local += valid ? (double)sq : 0.0;
+      if (p.epi & (EPI_ABSMAX | EPI_DELTA | EPI_CODES)) {
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi)
+          if (valid && !(best[gi] <= 3.0e38f)) bad = true;
+        if (valid && (p.epi & EPI_ABSMAX)) {
+#pragma unroll
+          for (int gi = 0; gi < NG; ++gi) {
+            const long long w = (long long)row * ng_row + (col0 / G + gi);
+            p.a[w] = best[gi];
+            p.usel[w] = bval[gi];
+            p.idx[w] = bidx[gi];
+          }
+        }
+        if (p.epi & (EPI_DELTA | EPI_CODES)) {
+          float sc[NG];
+#pragma unroll
+          for (int gi = 0; gi < NG; ++gi) {
+            sc[gi] = __fdiv_rn(best[gi], p.qmax);
+            if (valid && (p.epi & EPI_CODES)) p.scales[(long long)row * ng_row + (col0 / G + gi)] = sc[gi];
+          }
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            tc_ld32(taddr + ch * 32, v);
+            const float s = sc[(G == 128) ? 0 : (ch >> 1)];
+            uint32_t dpk[16];
+            uint32_t cpk[8];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float q0 = (s > 0.f) ? rintf(__fdiv_rn(v[e], s)) : 0.f;
+              float q1 = (s > 0.f) ? rintf(__fdiv_rn(v[e + 1], s)) : 0.f;
+              q0 = fminf(fmaxf(q0, -p.qmax), p.qmax);
+              q1 = fminf(fmaxf(q1, -p.qmax), p.qmax);
+              const float d0 = s * q0 - v[e], d1 = s * q1 - v[e + 1];
+              const uint32_t lo = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d0));
+              const uint32_t hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d1));
+              dpk[e >> 1] = lo | (hi << 16);
+              const uint32_t c0 = (uint32_t)((int)q0) & 0xFFu, c1 = (uint32_t)((int)q1) & 0xFFu;
+              if ((e & 2) == 0) cpk[e >> 2] = c0 | (c1 << 8);
+              else cpk[e >> 2] |= (c0 << 16) | (c1 << 24);
+            }
+            if (valid && (p.epi & EPI_DELTA)) {
+              uint4* dst = reinterpret_cast<uint4*>(p.delta + (long long)row * p.d_in + col0 + ch * 32);
+#pragma unroll
+              for (int w4 = 0; w4 < 4; ++w4) dst[w4] = make_uint4(dpk[4 * w4], dpk[4 * w4 + 1], dpk[4 * w4 + 2], dpk[4 * w4 + 3]);
+            }
+            if (valid && (p.epi & EPI_CODES)) {
+              uint4* dst = reinterpret_cast<uint4*>(p.codes + (long long)row * p.d_in + col0 + ch * 32);
+              dst[0] = make_uint4(cpk[0], cpk[1], cpk[2], cpk[3]);
+              dst[1] = make_uint4(cpk[4], cpk[5], cpk[6], cpk[7]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+    }
+    if (p.epi & EPI_SQSUM) {
+      for (int o = 16; o > 0; o >>= 1) sq_local += __shfl_xor_sync(0xffffffffu, sq_local, o);
+      if (lane == 0 && sq_local != 0.0) atomicAdd(p.sqacc, sq_local);
+    }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) raise_status(p.status, CAFEQ_ERR_NONFINITE);
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side: tensor maps and launch
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor map: `cols` contiguous elements per row, `rows` rows, row pitch in elements, box 64 x box_rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+static bool make_map_bf16(CUtensorMap* m, const void* base, long long cols, long long rows, long long pitch, int box_rows) {
+  EncodeTiledFn enc = get_encode_tiled();
+  if (!enc) return false;
+  if (((uintptr_t)base & 15) || ((pitch * 2) & 15)) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Shapes the fused pass covers; everything else runs on the shape-agnostic kernels.
+static bool bd_supported(int form, int d_out, int d_in, long long ld, int k, int g, const void* X) {
+  if (!(g == 64 || g == 128)) return false;
+  if (form == BD_IN) {
+    if (!(k == 64 || k == 128 || k == 256)) return false;
+    if (d_in % 256) return false;
+  } else {
+    if (!(k == 128 || k == 256)) return false;
+    if (d_out % k || d_in % 128) return false;
+  }
+  if ((ld % 8) || ((uintptr_t)X & 15)) return false;
+  return true;
+}
+
+template <int FORM, int K, int G>
+static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmT, BdParams p) {
+  using C = BdCfg<FORM, K, G>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(bd_pass_kernel<FORM, K, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+      return CAFEQ_ERR_CUDA;
+    attr_done = true;
+  }
+  if (FORM == BD_IN) {
+    p.n_major = p.d_in / 256;
+    p.n_minor = (p.d_out + 127) / 128;
+  } else {
+    p.n_major = p.d_out / K;
+    p.n_minor = (p.d_in + C::NC - 1) / C::NC;
+  }
+  int cpm = 148 / p.n_major;
+  if (cpm < 1) cpm = 1;
+  if (cpm > p.n_minor) cpm = p.n_minor;
+  p.ctas_per_major = cpm;
+  bd_pass_kernel<FORM, K, G><<<p.n_major * cpm, BD_THREADS, C::SMEM, st>>>(tmX, tmT, p);
+  return CAFEQ_OK;
+}
+
+// X: bf16 [d_out, d_in] with pitch ld; Tb: bf16 operator blocks [nbT * k, k] in applied orientation.
+static int bd_launch(cudaStream_t st, int form, int k, int g, const void* X, long long ld, const void* Tb, int nbT, BdParams p) {
+  CUtensorMap tmX, tmT;
+  if (!make_map_bf16(&tmX, X, p.d_in, p.d_out, ld, 128)) return CAFEQ_ERR_UNSUPPORTED;
+  if (!make_map_bf16(&tmT, Tb, k, (long long)nbT * k, k, k)) return CAFEQ_ERR_UNSUPPORTED;
+#define BD_CASE(F, KK, GG) \
+  if (form == F && k == KK && g == GG) return bd_launch_t<F, KK, GG>(st, tmX, tmT, p);
+  BD_CASE(BD_IN, 64, 64)
+  BD_CASE(BD_IN, 64, 128)
+  BD_CASE(BD_IN, 128, 64)
+  BD_CASE(BD_IN, 128, 128)
+  BD_CASE(BD_IN, 256, 64)
+  BD_CASE(BD_IN, 256, 128)
+  BD_CASE(BD_OUT, 128, 64)
+  BD_CASE(BD_OUT, 128, 128)
+  BD_CASE(BD_OUT, 256, 64)
+  BD_CASE(BD_OUT, 256, 128)
+#undef BD_CASE
+  return CAFEQ_ERR_UNSUPPORTED;
+}
+
+// fp32 operator blocks -> bf16 in applied orientation (transposed when the role asks for T^T)
+__global__ void operator_to_bf16_kernel(const float* __restrict__ T, uint16_t* __restrict__ out, int k, long long n, int transpose,
+                                        const int32_t* status) {
+  if (status && *status) return;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    long long b = e / ((long long)k * k);
+    int i = (int)((e / k) % k), j = (int)(e % k);
+    float v = transpose ? T[b * k * k + (long long)j * k + i] : T[e];
+    out[e] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+  }
+}
+
+}  // namespace cafeq

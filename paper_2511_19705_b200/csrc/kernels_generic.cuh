@@ -281,7 +281,7 @@ __global__ void __launch_bounds__(1024) block_inverse_kernel(const float* __rest
 // group absmax with arg-max (lowest index on ties): one warp per (row, group)
 // ------------------------------------------------------------------------------------------------
 __global__ void absmax_kernel(const float* __restrict__ U, long long ld, int rows, int ng, int g,
-                              float* __restrict__ a, int* __restrict__ idx, int32_t* status) {
+                              float* __restrict__ a, float* __restrict__ usel, int* __restrict__ idx, int32_t* status) {
   if (status && *status) return;
   long long w = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
@@ -309,6 +309,7 @@ __global__ void absmax_kernel(const float* __restrict__ U, long long ld, int row
   if (lane == 0) {
     a[w] = best;
     idx[w] = bi;
+    usel[w] = p[bi];  // signed value at the arg-max
   }
 }
 
@@ -377,8 +378,8 @@ __global__ void cw_out_kernel(const float* __restrict__ c, int d_out, int g, int
 // one thread per row: loss partial sum and arg-max coefficients  coef = scale * cw * a * sign(U[e*]).
 // A_t accumulation: axis IN  Agrp[Gc] += a^2 (per column group, expanded later);
 //                   axis OUT A[t'(row)] += g * sum_G a^2.
-__global__ void surrogate_rows_kernel(const float* __restrict__ a, const int* __restrict__ idx,
-                                      const float* __restrict__ U, long long ld, int rows, int ng, int g, int axis,
+__global__ void surrogate_rows_kernel(const float* __restrict__ a, const float* __restrict__ usel, int rows, int ng,
+                                      int g, int axis,
                                       const float* __restrict__ cw, float kappa, int k, int r, float* __restrict__ coef,
                                       float* __restrict__ Agrp, float* __restrict__ A, double* __restrict__ acc,
                                       const int32_t* status) {
@@ -391,7 +392,7 @@ __global__ void surrogate_rows_kernel(const float* __restrict__ a, const int* __
     for (int G = 0; G < ng; ++G) {
       long long w = (long long)row * ng + G;
       float av = a[w];
-      float u = U[row * ld + (long long)G * g + idx[w]];
+      float u = usel[w];
       float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
       float wgt = (axis == CAFEQ_AXIS_IN) ? cw[G] : cw[row];
       local += (double)wgt * (double)av * (double)av;
@@ -434,7 +435,7 @@ __global__ void scale_cols_kernel(const float* __restrict__ Minv, const float* _
 // (+ optionally, for the pair PQE loss, the direct term stays in gU and is handled by a dense product)
 // ------------------------------------------------------------------------------------------------
 __global__ void ste_scale_path_kernel(const float* __restrict__ U, const float* __restrict__ gD, long long ld, int rows,
-                                      int ng, int g, const float* __restrict__ a, const int* __restrict__ idx, float qmax,
+                                      int ng, int g, const float* __restrict__ a, const float* __restrict__ usel, float qmax,
                                       const void* __restrict__ offsets, int off_kind, int cols, float* __restrict__ coef,
                                       const int32_t* status) {
   if (status && *status) return;
@@ -457,7 +458,7 @@ __global__ void ste_scale_path_kernel(const float* __restrict__ U, const float* 
   }
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
   if (lane == 0) {
-    float u = U[row * ld + (long long)G * g + idx[w]];
+    float u = usel[w];
     float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
     coef[w] = sum * sgn / qmax;
   }
@@ -617,16 +618,14 @@ __global__ void sumexp_kernel(const float* __restrict__ a, long long n, const fl
 }
 
 // coef[w] = exp(t (a - max)) / Z * sign(U[arg-max])
-__global__ void lse_coef_kernel(const float* __restrict__ a, const int* __restrict__ idx, const float* __restrict__ U,
-                                long long ld, int rows, int ng, int g, const float* __restrict__ amax, float t,
-                                const double* __restrict__ Z, float* __restrict__ coef, const int32_t* status) {
+__global__ void lse_coef_kernel(const float* __restrict__ a, const float* __restrict__ usel, long long n,
+                                const float* __restrict__ amax, float t, const double* __restrict__ Z,
+                                float* __restrict__ coef, const int32_t* status) {
   if (status && *status) return;
-  const long long n = (long long)rows * ng;
   const float mx = *amax;
   const float zinv = (float)(1.0 / *Z);
   for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < n; w += (long long)gridDim.x * blockDim.x) {
-    int row = (int)(w / ng), G = (int)(w - (long long)row * ng);
-    float u = U[row * ld + (long long)G * g + idx[w]];
+    float u = usel[w];
     float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
     coef[w] = expf(t * (a[w] - mx)) * zinv * sgn;
   }

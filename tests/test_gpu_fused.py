@@ -1,0 +1,151 @@
+"""GPU parity of the fused tensor-core transform pass (both axes, every block/group variant, ragged and
+multi-tile shapes) against the CPU oracle, at shapes up to the Gemma-2-9B matrices the benchmark times."""
+import numpy as np
+import pytest
+
+import cafeq_synth as syn
+from oracle import cafeq_oracle as orc
+from parity_utils import assert_codes_tie_aware, f32_dev, rel_err, to_dev, w64
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def cq():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2511_19705_b200 as m
+    m.lib()
+    return m
+
+
+def _axis(name, cq):
+    return cq.AXIS_IN if name == "in" else cq.AXIS_OUT
+
+
+# shapes chosen so that the fused pass is selected: d_in % 256 == 0 (input axis) or d_out % k == 0 and
+# d_in % 128 == 0 (output axis); several have a ragged last row tile or more tiles than CTAs
+FUSED_SHAPES = [("in", 64, 64, (128, 256)), ("in", 64, 128, (300, 512)), ("in", 128, 64, (130, 256)),
+                ("in", 128, 128, (256, 512)), ("in", 256, 64, (520, 512)), ("in", 256, 128, (200, 768)),
+                ("out", 128, 64, (256, 384)), ("out", 128, 128, (384, 640)), ("out", 256, 64, (512, 128)),
+                ("out", 256, 128, (768, 384))]
+
+
+@pytest.mark.parametrize("axis,k,group,shape", FUSED_SHAPES)
+@pytest.mark.parametrize("kind", ["identity", "perm", "pow2"])
+def test_fused_rtn_exact_transforms_bit_exact(cq, axis, k, group, shape, kind):
+    d_out, d_in = shape
+    Wb = syn.weight_student_t(d_out, d_in, 21, 2, 10.0)
+    Wb[0, :group] = 0
+    nb = (d_in if axis == "in" else d_out) // k
+    T = {"identity": syn.identity_blocks(nb, k), "perm": syn.signed_perm_blocks(nb, k, 3),
+         "pow2": syn.pow2_diag_blocks(nb, k, 4)}[kind]
+    codes, scales = cq.cafeq_rtn(to_dev(Wb), f32_dev(T), bits=4, group=group, tblock=k, taxis=_axis(axis, cq))
+    U = orc.apply_blocks(w64(Wb), T.astype(np.float64), axis)
+    Q = orc.quant_sym(U, 4, group)
+    assert np.array_equal(codes.cpu().numpy().astype(np.int32), Q["q"])
+    assert np.array_equal(scales.cpu().numpy(), Q["s"])
+
+
+@pytest.mark.parametrize("axis,k,group,shape", FUSED_SHAPES)
+@pytest.mark.parametrize("transposed", [False, True])
+def test_fused_rtn_general_transform_tie_aware(cq, axis, k, group, shape, transposed):
+    d_out, d_in = shape
+    Wb = syn.weight_student_t(d_out, d_in, 31, 2, 10.0)
+    nb = (d_in if axis == "in" else d_out) // k
+    T = syn.perturbed_blocks(nb, k, 9, 0.2)
+    codes, scales = cq.cafeq_rtn(to_dev(Wb), f32_dev(T), bits=3, group=group, tblock=k, taxis=_axis(axis, cq),
+                                 trole=cq.APPLY_TT if transposed else cq.APPLY_T)
+    Tc = orc.round_bf16(T)
+    if transposed:
+        Tc = np.transpose(Tc, (0, 2, 1))
+    U = orc.apply_blocks(w64(Wb), Tc, axis)
+    Q = orc.quant_sym(U, 3, group)
+    assert_codes_tie_aware(codes.cpu().numpy(), scales.cpu().numpy(), Q, U, group)
+
+
+def test_fused_replicas(cq):
+    Wb = syn.weight_student_t(192, 1024, 33)
+    T = syn.perturbed_blocks(2, 256, 5, 0.2)                     # 4 matrix blocks share 2 operator blocks
+    codes, scales = cq.cafeq_rtn(to_dev(Wb), f32_dev(T), bits=4, group=128, tblock=256, replicas=2)
+    U = orc.apply_blocks(w64(Wb), orc.round_bf16(T), "in", 2)
+    assert_codes_tie_aware(codes.cpu().numpy(), scales.cpu().numpy(), orc.quant_sym(U, 4, 128), U, 128)
+
+
+@pytest.mark.parametrize("axis,k,group,shape", FUSED_SHAPES)
+def test_fused_single_matches_oracle_and_generic(cq, axis, k, group, shape):
+    d_out, d_in = shape
+    Wb = syn.weight_student_t(d_out, d_in, 41, 2, 10.0)
+    nb = (d_in if axis == "in" else d_out) // k
+    M = syn.perturbed_blocks(nb, k, 13, 0.1)
+    kw = dict(bits=3, group=group, taxis=_axis(axis, cq))
+    out = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), flags=cq.FLAG_EXACT_LOSS, **kw)
+    gen = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), flags=cq.FLAG_EXACT_LOSS | cq.FLAG_GENERIC, **kw)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0 and int(gen["status"].item()) == 0
+    W = w64(Wb)
+    f = orc.single_forward(W, M, 3, group, axis)
+    g = orc.single_grad_surrogate(W, f, group, axis)
+    for o in (out, gen):
+        L = o["losses"].cpu().numpy()
+        assert abs(L[0] - f["surrogate"]) <= TOL * f["surrogate"]
+        assert abs(L[1] - f["L2"]) <= TOL * f["L2"]
+        gg = o["gradM"].cpu().numpy()
+        for b in range(nb):
+            assert rel_err(gg[b], g[b]) <= TOL, f"block {b}"
+
+
+def test_fused_pair_matches_oracle(cq):
+    k, r, h, d1, d3 = 256, 2, 512, 384, 300
+    W1b, W2b = syn.weight_student_t(h, d1, 51, 2, 10.0), syn.weight_student_t(d3, r * h, 52, 2, 10.0)
+    M = syn.perturbed_blocks(h // k, k, 17, 0.1)
+    out = cq.cafeq_pair_loss_fwd_bwd(to_dev(W1b), to_dev(W2b), f32_dev(M), bits=3, group1=128, group2=128, replicas=r,
+                                     lse_t=5.0, lambda_orth=0.1)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    W1, W2 = w64(W1b), w64(W2b)
+    f = orc.pair_forward(W1, W2, M, 3, 128, 128, r, 5.0, 0.1, False)
+    L = out["losses"].cpu().numpy()
+    assert abs(L[0] - f["loss"]) <= TOL * abs(f["loss"]) and abs(L[1] - f["lse"]) <= TOL * abs(f["lse"])
+    assert rel_err(out["gradM"].cpu().numpy(), orc.pair_grad_lse(W1, W2, f, 128, 128)) <= TOL
+
+
+# ------------------------------------------------------------------ full-size matrices of the benchmark workload
+def test_fused_full_size_q_matrix_bit_exact_and_sampled(cq):
+    """q of the 9B-shaped layer (4096 x 3584, k = 256, 3-bit, g = 128) in the launch configuration the
+    benchmark uses: identity transform bit-exact on every entry; a rotation checked on sampled rows."""
+    name, d_out, d_in = "q", 4096, 3584
+    Wb = syn.make_weight(3, name, d_out, d_in)
+    Wd = to_dev(Wb)
+    codes, scales = cq.cafeq_rtn(Wd, f32_dev(syn.identity_blocks(d_in // 256, 256)), bits=3, group=128, tblock=256)
+    Q = orc.quant_sym(w64(Wb), 3, 128)
+    assert np.array_equal(codes.cpu().numpy().astype(np.int32), Q["q"])
+    assert np.array_equal(scales.cpu().numpy(), Q["s"])
+    M = syn.make_transform(name, d_in // 256, 256)
+    codes, scales = cq.cafeq_rtn(Wd, f32_dev(M), bits=3, group=128, tblock=256)
+    rows = np.random.default_rng(0).choice(d_out, size=96, replace=False)
+    rows = np.sort(np.concatenate([rows, [0, 127, 128, d_out - 1]]))
+    U = orc.apply_blocks(w64(Wb[rows]), orc.round_bf16(M), "in")
+    Qs = orc.quant_sym(U, 3, 128)
+    assert_codes_tie_aware(codes.cpu().numpy()[rows], scales.cpu().numpy()[rows], Qs, U, 128)
+    # losses and gradient of the full matrix
+    out = cq.cafeq_proxy_loss_fwd_bwd(Wd, f32_dev(M), bits=3, group=128, flags=cq.FLAG_EXACT_LOSS)
+    W = w64(Wb)
+    f = orc.single_forward(W, M, 3, 128, "in")
+    g = orc.single_grad_surrogate(W, f, 128, "in")
+    L = out["losses"].cpu().numpy()
+    assert abs(L[0] - f["surrogate"]) <= TOL * f["surrogate"] and abs(L[1] - f["L2"]) <= TOL * f["L2"]
+    assert rel_err(out["gradM"].cpu().numpy(), g) <= TOL
+
+
+def test_fused_full_size_v_matrix_output_axis(cq):
+    """v of the 9B-shaped layer (2048 x 3584) transformed on the output axis with k = 256."""
+    Wb = syn.make_weight(3, "v", 2048, 3584)
+    M = syn.make_transform("v", 8, 256)
+    codes, scales = cq.cafeq_rtn(to_dev(Wb), f32_dev(M), bits=3, group=128, tblock=256, taxis=cq.AXIS_OUT,
+                                 trole=cq.APPLY_TT)
+    U = orc.apply_blocks(w64(Wb), np.transpose(orc.round_bf16(M), (0, 2, 1)), "out")
+    assert_codes_tie_aware(codes.cpu().numpy(), scales.cpu().numpy(), orc.quant_sym(U, 3, 128), U, 128)
