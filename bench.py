@@ -240,11 +240,14 @@ def main():
     by_kind = {}
     for d, kd in zip(kms, kinds):
         by_kind.setdefault(kd, []).append(d)
-    names = {1: "transform_pass", 2: "sparse_backward", 3: "block_inverse", 4: "pair_product"}
+    names = {1: "transform_pass_generic", 2: "sparse_backward", 3: "block_inverse", 4: "pair_product",
+             5: "transform_pass_tcgen05"}
     kernel_ms = {names.get(kd, str(kd)): dict(launches_per_step=len(v) / args.steps, ms_per_step=sum(v) / args.steps)
                  for kd, v in by_kind.items()}
     roof = None
-    if 1 in by_kind:
+    tk = max((kd for kd in (1, 5) if kd in by_kind), key=lambda kd: sum(by_kind[kd]), default=None)
+    if tk is not None:
+        by_kind[1] = by_kind[tk]
         t_pass = sum(by_kind[1]) / args.steps * 1e-3            # seconds of transform passes per step
         passes = len(by_kind[1]) / args.steps / 7.0             # passes over the layer per step
         flops = 2.0 * k * layer.weights * passes                # 2k flop per weight per pass
@@ -258,7 +261,7 @@ def main():
             ach = byts / t_pass / 1e9
             roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
                         traffic=None)
-        roof.update(kernel="transform_pass", peak_source=peaks["source"] + (" sustained" if roof["bound"] == "tensor" else ""),
+        roof.update(kernel=names[tk], peak_source=peaks["source"] + (" sustained" if roof["bound"] == "tensor" else ""),
                     launches_per_step=len(by_kind[1]) / args.steps, avg_launch_ms=sum(by_kind[1]) / len(by_kind[1]),
                     algorithmic_gb_per_step=byts / 1e9, algorithmic_tflop_per_step=flops / 1e12)
 
