@@ -47,7 +47,8 @@ typedef enum {
   CAFEQ_ERR_CUDA = 4,        /* a launch failed; cudaGetLastError has the detail */
   CAFEQ_ERR_SINGULAR = 5,    /* device: a transform block has no usable pivot */
   CAFEQ_ERR_NONFINITE = 6,   /* device: NaN or Inf met in a transformed weight */
-  CAFEQ_ERR_TIMEOUT = 7      /* device: a bounded wait inside a kernel ran out */
+  CAFEQ_ERR_TIMEOUT = 7,     /* device: a bounded wait inside a kernel ran out */
+  CAFEQ_ERR_TOO_LARGE = 8    /* problem needs more scratch than the built-in buffer of cafeq_rtn_noalloc holds */
 } cafeq_status;
 
 enum { CAFEQ_AXIS_IN = 0, CAFEQ_AXIS_OUT = 1 };
@@ -108,6 +109,26 @@ int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d
  * inverse is taken here. */
 int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
               void* ws, size_t ws_bytes, void* stream);
+
+/* cafeq_rtn for callers that cannot allocate device memory and therefore have no workspace to hand
+ * over: code running inside a memory-pool or allocator callback, between the driver calls of another
+ * library that forbids allocation, in a process whose memory budget is already fixed, or anywhere a
+ * cudaMalloc (which synchronises the whole device) would stall other streams.  (The paper has no
+ * counterpart; the arithmetic and the outputs are exactly those of cafeq_rtn.)
+ *   - Scratch is a buffer of CAFEQ_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU
+ *     that loads the library holds it from then until the process exits.  Inputs and outputs are still
+ *     the caller's.  Neither this call nor anything under it calls cudaMalloc, cudaFree or an
+ *     allocating library routine.
+ *   - A descriptor whose cafeq_workspace_size exceeds CAFEQ_NOALLOC_SCRATCH_BYTES is refused with
+ *     CAFEQ_ERR_TOO_LARGE before anything is launched (use cafeq_rtn with your own workspace then).
+ *   - The first call on each device looks up the buffer's device address (with that device current);
+ *     make that first call outside any stream capture.  Later calls only enqueue kernels.
+ *   - All calls in the process share the one buffer per device, and it keeps whatever the last call
+ *     left there.  Nothing in this path reads scratch before writing it, so nothing needs clearing, but
+ *     two calls that can overlap on the GPU (different streams, no dependency) race on it: order them. */
+#define CAFEQ_NOALLOC_SCRATCH_BYTES (16u << 20)
+int cafeq_rtn_noalloc(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
+                      void* stream);
 
 /* One forward+backward evaluation for a single matrix (Section 4.1).
  *   M       [nb,k,k] fp32 transform parameters; the transform applied is bf16(M).

@@ -22,7 +22,7 @@ FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC = 1, 2, 4
 OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 
 EXPORTS = [
-    "cafeq_workspace_size", "cafeq_rtn", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
+    "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
     "cafeq_pack", "cafeq_debug_timer_begin", "cafeq_debug_timer_read", "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
@@ -170,6 +170,26 @@ def cafeq_rtn(W, T=None, *, bits, group, tblock=0, taxis=AXIS_IN, trole=APPLY_T,
     rc = lib().cafeq_rtn(ctypes.byref(d), _p(W), _p(_f32(T, "T")), _p(codes), _p(scales), _p(ws),
                          ctypes.c_size_t(ws.numel()), _stream())
     _check(rc, "cafeq_rtn")
+    return codes, scales
+
+
+NOALLOC_SCRATCH_BYTES = 16 << 20
+
+
+def cafeq_rtn_noalloc(W, T, codes, scales, *, bits, group, tblock=0, taxis=AXIS_IN, trole=APPLY_T, replicas=1):
+    """cafeq_rtn into caller-provided `codes` / `scales`, using the scratch buffer built into the library
+    (no workspace, no allocation anywhere on the way).  Raises CafeqError(8) when the matrix needs more than
+    NOALLOC_SCRATCH_BYTES of scratch."""
+    W = _bits_tensor(W)
+    d_out, d_in = W.shape
+    g = group or d_in
+    if codes.dtype != torch.int8 or tuple(codes.shape) != (d_out, d_in) or not codes.is_contiguous():
+        raise ValueError("codes must be a contiguous int8 [d_out, d_in] tensor")
+    if scales.dtype != torch.float32 or tuple(scales.shape) != (d_out, d_in // g) or not scales.is_contiguous():
+        raise ValueError("scales must be a contiguous float32 [d_out, d_in/group] tensor")
+    d = make_desc(d_out, d_in, bits, group, tblock if T is not None else 0, taxis, trole, replicas, W.stride(0))
+    rc = lib().cafeq_rtn_noalloc(ctypes.byref(d), _p(W), _p(_f32(T, "T")), _p(codes), _p(scales), _stream())
+    _check(rc, "cafeq_rtn_noalloc")
     return codes, scales
 
 

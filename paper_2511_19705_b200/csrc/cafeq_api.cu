@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "cafeq.h"
@@ -370,6 +371,7 @@ extern "C" const char* cafeq_status_string(int s) {
     case CAFEQ_ERR_SINGULAR: return "singular transform block";
     case CAFEQ_ERR_NONFINITE: return "non-finite value";
     case CAFEQ_ERR_TIMEOUT: return "bounded device wait expired";
+    case CAFEQ_ERR_TOO_LARGE: return "problem needs more scratch than the built-in buffer holds";
     default: return "unknown status";
   }
 }
@@ -808,4 +810,36 @@ extern "C" int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8
   if (G.d_in % 8) return CAFEQ_ERR_UNSUPPORTED;
   CQ_LAUNCH(pack_kernel, grid_for(G.n / 8), 256, 0, (cudaStream_t)stream, codes, packed, G.d_out, G.d_in, d->bits);
   return last_launch();
+}
+
+// ------------------------------------------------------------------------------------------------
+// cafeq_rtn without a caller workspace: scratch lives in the library image
+// ------------------------------------------------------------------------------------------------
+// In host code the name of a __device__ array is only a handle for the runtime, not an address a kernel can
+// use; the device address is looked up once per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CAFEQ_NOALLOC_SCRATCH_BYTES];
+static constexpr int kMaxDevices = 64;
+static void* g_noalloc_ptr[kMaxDevices] = {};
+static std::mutex g_noalloc_mu;
+
+extern "C" int cafeq_rtn_noalloc(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
+                                 void* stream) {
+  size_t need = 0;
+  int rc = cafeq_workspace_size(d, nullptr, nullptr, &need);
+  if (rc) return rc;
+  if (need > (size_t)CAFEQ_NOALLOC_SCRATCH_BYTES) return CAFEQ_ERR_TOO_LARGE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CAFEQ_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return CAFEQ_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return CAFEQ_ERR_CUDA;
+      g_noalloc_ptr[dev] = p;
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  return cafeq_rtn(d, W, T, codes, scales, scratch, (size_t)CAFEQ_NOALLOC_SCRATCH_BYTES, stream);
 }
