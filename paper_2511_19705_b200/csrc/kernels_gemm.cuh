@@ -1,0 +1,259 @@
+// Batched dense products on the 5th-generation tensor cores (sm_100a) for the k x k algebra around the
+// transform (Newton-Schulz refinement of M^-1, the M^-1 path of the gradient, M M^T of the orthonormality
+// penalty) and for the pairwise product term of Eq. 5 (PQE).
+//
+//   C[b][m][n] = alpha * sum_t sum_l A_t[b / divA][m][l] * B_t[b][n][l]  + beta * C0[b][m][n] + gamma * [m == n]
+//
+// Every operand is bf16, row-major with the contraction index l contiguous (both K-major), so one product is
+// the "A times B-transposed" form.  fp32 precision comes from summing up to three terms over bf16 splits
+// (x = hi + lo, hi = bf16(x), lo = bf16(x - hi)); the accumulator is fp32 in tensor memory.
+// The epilogue can write C as fp32, as bf16 hi / lo splits in row-major and / or transposed order (the
+// operand layouts the next product needs), and accumulate sum(C^2).
+//
+// One CTA computes one 128 x BN tile: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner,
+// warps 2..5 = epilogue (one accumulator row per thread).  Every mbarrier wait is bounded.
+#pragma once
+
+#include "kernels_fused.cuh"
+
+namespace cafeq {
+
+constexpr int TG_THREADS = 192;
+constexpr int TG_BK = 64;
+constexpr int TG_MAX_TERMS = 3;
+
+struct TgMaps {
+  CUtensorMap a[TG_MAX_TERMS];
+  CUtensorMap b[TG_MAX_TERMS];
+};
+
+struct TgParams {
+  int M, N, K, batch, nterms;
+  int rowsA_per_batch, rowsB_per_batch;  // row offset of batch b in the 2-D operand views (0 for a shared operand)
+  int divA;                              // batch b reads A rows of batch b / divA
+  int a_rep_k, a_rep_r;                  // replicated contraction blocks of A: chunk at l reads columns ((l / k) / r) * k + l % k
+  float alpha, beta, gamma;
+  const float* C0;
+  long long ldc0, sC0b;
+  float* C;
+  long long ldc, sCb;
+  uint16_t *Chi, *Clo;    // bf16 splits, row-major [batch][M][N] (ld = N)
+  uint16_t *Cthi, *Ctlo;  // bf16 splits, transposed [batch][N][M] (ld = M)
+  double* sq;             // sum of C^2: sq[b * sq_stride]
+  int sq_stride;
+  const int* run_flag;    // optional: skip the whole launch when *run_flag == 0
+  int32_t* status;
+};
+
+template <int BN>
+struct TgCfg {
+  static constexpr int A_BYTES = 128 * TG_BK * 2;
+  static constexpr int B_BYTES = BN * TG_BK * 2;
+  static constexpr int STAGE = A_BYTES + B_BYTES;
+  static constexpr int NSTAGE = 4;
+  static constexpr int SMEM = 1024 + NSTAGE * STAGE + 256;
+  static constexpr int TMEM_COLS = (BN < 32) ? 32 : BN;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(TG_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
+  using C = TgCfg<BN>;
+  if (p.status && *p.status) return;
+  if (p.run_flag && *p.run_flag == 0) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = (uint64_t*)(smem + C::NSTAGE * C::STAGE);
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8 * C::NSTAGE;
+  const uint32_t bar_acc = bar_empty + 8 * C::NSTAGE;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 1);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * 128, b = blockIdx.z;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::NSTAGE; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    mbar_init(bar_acc, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)C::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int kchunks = p.K / TG_BK;
+  const int total = kchunks * p.nterms;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int ya = (b / p.divA) * p.rowsA_per_batch + m0;
+      const int yb = b * p.rowsB_per_batch + n0;
+      for (int it = 0; it < total; ++it) {
+        const int t = it / kchunks, c = it - t * kchunks;
+        const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) break;
+        mbar_expect_tx(bar_full + 8 * s, C::STAGE);
+        const int l0 = c * TG_BK;
+        int xa = l0;
+        if (p.a_rep_r > 1) xa = ((l0 / p.a_rep_k) / p.a_rep_r) * p.a_rep_k + (l0 % p.a_rep_k);
+        uint8_t* st = smem + s * C::STAGE;
+        tma_load_2d(smem_u32(st), &maps.a[t], xa, ya, bar_full + 8 * s);
+        tma_load_2d(smem_u32(st + C::A_BYTES), &maps.b[t], l0, yb, bar_full + 8 * s);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(128, BN, 0, 0);
+      bool ok = true;
+      for (int it = 0; it < total && ok; ++it) {
+        const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + s * C::STAGE), sb = sa + C::A_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_bf16(tmem_base, umma_desc_sw128(sa + kk * 32), umma_desc_sw128(sb + kk * 32), idesc, (it | kk) != 0 ? 1u : 0u);
+        tc_commit(bar_empty + 8 * s);
+      }
+      if (ok) tc_commit(bar_acc);
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = m0 + q * 32 + lane;
+    bool ok = mbar_wait(bar_acc, 0, abort_flag, p.status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const bool rv = row < p.M;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      double sq = 0.0;
+      const long long cb = (long long)b * p.sCb, c0b = (long long)b * p.sC0b;
+      const long long sb_mn = (long long)b * p.M * p.N;
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        float v[32];
+        tc_ld32(taddr + ch * 32, v);
+        const int nb0 = n0 + ch * 32;
+        if (nb0 >= p.N) break;
+        const bool full = rv && (nb0 + 32 <= p.N);
+        float sqf = 0.f;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          float x = p.alpha * v[e];
+          const int n = nb0 + e;
+          if (p.C0 && rv && n < p.N) x = fmaf(p.beta, p.C0[c0b + (long long)row * p.ldc0 + n], x);
+          if (n == row) x += p.gamma;
+          v[e] = x;
+          if (rv && n < p.N) sqf = fmaf(x, x, sqf);
+        }
+        sq += (double)sqf;
+        if (p.C && rv) {
+          float* dst = p.C + cb + (long long)row * p.ldc + nb0;
+          if (full && ((p.ldc & 3) == 0) && (((uintptr_t)dst & 15) == 0)) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+          } else {
+            for (int e = 0; e < 32; ++e)
+              if (nb0 + e < p.N) dst[e] = v[e];
+          }
+        }
+        if (p.Chi || p.Cthi) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int n = nb0 + e;
+            const __nv_bfloat16 h = __float2bfloat16_rn(v[e]);
+            const __nv_bfloat16 l = __float2bfloat16_rn(v[e] - __bfloat162float(h));
+            if (rv && n < p.N) {
+              if (p.Chi) p.Chi[sb_mn + (long long)row * p.N + n] = __bfloat16_as_ushort(h);
+              if (p.Clo) p.Clo[sb_mn + (long long)row * p.N + n] = __bfloat16_as_ushort(l);
+              if (p.Cthi) p.Cthi[sb_mn + (long long)n * p.M + row] = __bfloat16_as_ushort(h);
+              if (p.Ctlo) p.Ctlo[sb_mn + (long long)n * p.M + row] = __bfloat16_as_ushort(l);
+            }
+          }
+        }
+      }
+      if (p.sq) {
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if (lane == 0 && sq != 0.0) atomicAdd(p.sq + (long long)b * p.sq_stride, sq);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+  }
+}
+
+// 2-D bf16 operand view for the product kernel: `rows` rows of `cols` contiguous elements.
+struct TgOperand {
+  const void* ptr;
+  long long rows, cols, pitch;
+};
+
+template <int BN>
+static int tg_launch_t(cudaStream_t st, const TgOperand* A, const TgOperand* B, TgParams p) {
+  using C = TgCfg<BN>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+      return CAFEQ_ERR_CUDA;
+    attr_done = true;
+  }
+  TgMaps maps;
+  memset(&maps, 0, sizeof(maps));
+  for (int t = 0; t < p.nterms; ++t) {
+    if (!make_map_bf16(&maps.a[t], A[t].ptr, A[t].cols, A[t].rows, A[t].pitch, 128)) return CAFEQ_ERR_UNSUPPORTED;
+    if (!make_map_bf16(&maps.b[t], B[t].ptr, B[t].cols, B[t].rows, B[t].pitch, BN)) return CAFEQ_ERR_UNSUPPORTED;
+  }
+  dim3 grid((p.N + BN - 1) / BN, (p.M + 127) / 128, p.batch);
+  tc_gemm_kernel<BN><<<grid, TG_THREADS, C::SMEM, st>>>(maps, p);
+  return CAFEQ_OK;
+}
+
+// K must be a multiple of 64; operands 16-byte aligned with pitches that are multiples of 8 elements.
+static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, const TgParams& p) {
+  if (p.K % TG_BK || p.nterms < 1 || p.nterms > TG_MAX_TERMS) return CAFEQ_ERR_UNSUPPORTED;
+  if (p.N <= 64) return tg_launch_t<64>(st, A, B, p);
+  if (p.N <= 128 || (p.batch > 1 && p.N <= 256 && p.batch * ((p.M + 127) / 128) < 74)) return tg_launch_t<128>(st, A, B, p);
+  return tg_launch_t<256>(st, A, B, p);
+}
+
+// fp32 [n] -> bf16 hi / lo splits in row-major and transposed block order (blocks of k x k)
+__global__ void split_bf16_kernel(const float* __restrict__ X, int k, long long n, uint16_t* __restrict__ hi,
+                                  uint16_t* __restrict__ lo, uint16_t* __restrict__ thi, uint16_t* __restrict__ tlo,
+                                  const int* run_flag, const int32_t* status) {
+  if (status && *status) return;
+  if (run_flag && *run_flag == 0) return;
+  const long long kk = (long long)k * k;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const float x = X[e];
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    const __nv_bfloat16 l = __float2bfloat16_rn(x - __bfloat162float(h));
+    if (hi) hi[e] = __bfloat16_as_ushort(h);
+    if (lo) lo[e] = __bfloat16_as_ushort(l);
+    if (thi || tlo) {
+      const long long b = e / kk, r = e - b * kk;
+      const int i = (int)(r / k), j = (int)(r - (long long)i * k);
+      const long long te = b * kk + (long long)j * k + i;
+      if (thi) thi[te] = __bfloat16_as_ushort(h);
+      if (tlo) tlo[te] = __bfloat16_as_ushort(l);
+    }
+  }
+}
+
+}  // namespace cafeq

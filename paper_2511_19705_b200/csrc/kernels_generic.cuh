@@ -178,8 +178,10 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs g) {
 // buffer (global memory, L2 resident).  Also emits the column square norms c[t] = sum_i Minv[i][t]^2.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) block_inverse_kernel(const float* __restrict__ Min, float* __restrict__ Out,
-                                                             float* __restrict__ cnorm, int k, int32_t* status) {
+                                                             float* __restrict__ cnorm, int k, int32_t* status,
+                                                             const int* run_flag) {
   if (status && *status) return;
+  if (run_flag && *run_flag == 0) return;
   extern __shared__ float sm[];  // prow[k], fcol[k], piv (int) [k], red
   float* prow = sm;
   float* fcol = sm + k;
