@@ -13,6 +13,7 @@
 #include "cafeq.h"
 #include "kernels_generic.cuh"
 #include "kernels_fused.cuh"
+#include "kernels_gemm.cuh"
 
 namespace cafeq {
 
@@ -216,12 +217,169 @@ static void launch_kk(cudaStream_t st, const float* A, int tA, const float* B, i
   launch_gemm(st, g);
 }
 
-static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float* cnorm, int nb, int k, int32_t* status) {
+static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float* cnorm, int nb, int k, int32_t* status,
+                           const int* run_flag = nullptr) {
   int threads = k * k >= 1024 ? 1024 : ((k * k + 31) / 32) * 32;
   size_t sh = (size_t)3 * k * sizeof(float);
-  int ti = kt_begin(3, st);
-  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status);
+  int ti = run_flag ? -1 : kt_begin(3, st);
+  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status, run_flag);
   kt_end(ti, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// k x k algebra on the tensor cores: split-precision products and the Newton-Schulz inverse
+// ------------------------------------------------------------------------------------------------
+struct KkWS {  // bf16 scratch, each [nbT * k * k]
+  uint16_t *Ab, *Xh[2], *Xl[2], *XTh[2], *XTl[2], *RTh, *RTl, *Ph, *Pl, *Qh, *Ql;
+  double* rn;  // [NS_MAX_ITERS][nbT] squared residual norms
+  int* flag;   // 1 => Newton-Schulz did not converge, the Gauss-Jordan kernel takes over
+  int cur;     // which of the ping-pong split sets holds the current inverse (host bookkeeping)
+};
+constexpr int NS_MAX_ITERS = 8;
+constexpr int NS_COLD_ITERS = 6;
+constexpr int NS_WARM_ITERS = 2;
+
+static bool kk_fast(int k) { return k == 64 || k == 128 || k == 256; }
+
+static void carve_kk(Bump& b, int nbT, int k, KkWS* w) {
+  const size_t kk = (size_t)nbT * k * k;
+  uint16_t** all[] = {&w->Ab, &w->Xh[0], &w->Xh[1], &w->Xl[0], &w->Xl[1], &w->XTh[0], &w->XTh[1], &w->XTl[0], &w->XTl[1],
+                      &w->RTh, &w->RTl, &w->Ph, &w->Pl, &w->Qh, &w->Ql};
+  for (auto pp : all) *pp = b.take<uint16_t>(kk);
+  w->rn = b.take<double>((size_t)NS_MAX_ITERS * nbT);
+  w->flag = b.take<int>(64);
+  w->cur = 0;
+}
+static size_t kk_scratch_bytes(int nbT, int k) {
+  const size_t kk = (size_t)(nbT > 0 ? nbT : 1) * (k > 0 ? k : 1) * (k > 0 ? k : 1);
+  return 15 * (kk * 2 + 256) + (size_t)NS_MAX_ITERS * (nbT + 1) * 8 + 1024;
+}
+
+// C[b] = alpha * sum_t A_t[b] B_t[b]^T + beta * C0[b] + gamma * I for nb blocks of k x k; operands bf16 [nb*k, k]
+static int launch_kk_tc(cudaStream_t st, int nterms, const uint16_t* const* A, const uint16_t* const* B, int nb, int k,
+                        float alpha, float beta, float gamma, const float* C0, float* C, uint16_t* Chi, uint16_t* Clo,
+                        uint16_t* Cthi, uint16_t* Ctlo, double* sq, const int* run_flag, int32_t* status, int sq_stride = 1) {
+  TgOperand oa[TG_MAX_TERMS], ob[TG_MAX_TERMS];
+  for (int t = 0; t < nterms; ++t) {
+    oa[t] = TgOperand{A[t], (long long)nb * k, k, k};
+    ob[t] = TgOperand{B[t], (long long)nb * k, k, k};
+  }
+  TgParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = p.N = p.K = k;
+  p.batch = nb;
+  p.nterms = nterms;
+  p.rowsA_per_batch = p.rowsB_per_batch = k;
+  p.divA = 1;
+  p.a_rep_k = k;
+  p.a_rep_r = 1;
+  p.alpha = alpha; p.beta = beta; p.gamma = gamma;
+  p.C0 = C0; p.ldc0 = k; p.sC0b = (long long)k * k;
+  p.C = C; p.ldc = k; p.sCb = (long long)k * k;
+  p.Chi = Chi; p.Clo = Clo; p.Cthi = Cthi; p.Ctlo = Ctlo;
+  p.sq = sq; p.sq_stride = sq_stride;
+  p.run_flag = run_flag;
+  p.status = status;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return tg_launch(st, oa, ob, p);
+}
+
+__global__ void transpose_blocks_kernel(const float* __restrict__ in, float* __restrict__ out, int k, long long n) {
+  const long long kk = (long long)k * k;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const long long b = e / kk, r = e - b * kk;
+    const int i = (int)(r / k), j = (int)(r - (long long)i * k);
+    out[e] = in[b * kk + (long long)j * k + i];
+  }
+}
+
+__global__ void zero_ns_kernel(double* rn, int n, int* flag) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) rn[i] = 0.0;
+  if (i == 0) *flag = 0;
+}
+
+// flag = 1 when any block's last squared residual is above tol2 or not finite
+__global__ void ns_check_kernel(const double* __restrict__ rn_last, int nb, double tol2, int* flag) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < nb) {
+    const double v = rn_last[i];
+    if (!(v <= tol2)) atomicExch(flag, 1);
+  }
+}
+
+// c[b][t] = sum_i X[b][i][t]^2
+__global__ void colnorm_kernel(const float* __restrict__ X, int k, int nb, float* __restrict__ c) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (t >= k || b >= nb) return;
+  const float* Xb = X + (size_t)b * k * k;
+  float s = 0.f;
+  for (int i = 0; i < k; ++i) {
+    const float v = Xb[(size_t)i * k + t];
+    s = fmaf(v, v, s);
+  }
+  c[(size_t)b * k + t] = s;
+}
+
+static void launch_split(cudaStream_t st, const float* X, int k, long long n, uint16_t* hi, uint16_t* lo, uint16_t* thi,
+                         uint16_t* tlo, const int* run_flag, const int32_t* status) {
+  CQ_LAUNCH(split_bf16_kernel, grid_for(n), 256, 0, st, X, k, n, hi, lo, thi, tlo, run_flag, status);
+}
+
+// Minv = inv(bf16(M)) by Newton-Schulz iteration X <- X + X (I - A X) on the tensor cores, from X0 = A^T
+// (cold: right for the near-orthogonal transforms the method starts from) or from the caller's previous
+// inverse (warm).  The last residual is checked on the device; if it is not small the Gauss-Jordan kernel
+// recomputes everything.  Leaves fp32 Minv in X, its bf16 splits in w.Xh/Xl/XTh/XTl[w.cur], and c = column
+// square norms of Minv (optional).
+static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm, int nb, int k, bool warm, KkWS& w,
+                       int32_t* status) {
+  const long long kk = (long long)nb * k * k;
+  const int iters = warm ? NS_WARM_ITERS : NS_COLD_ITERS;
+  int ti = kt_begin(3, st);
+  CQ_LAUNCH(zero_ns_kernel, (NS_MAX_ITERS * nb + 127) / 128, 128, 0, st, w.rn, NS_MAX_ITERS * nb, w.flag);
+  CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Mc, w.Ab, k, kk, 0, status);
+  if (!warm) CQ_LAUNCH(transpose_blocks_kernel, grid_for(kk), 256, 0, st, Mc, X, k, kk);
+  int cur = 0;
+  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
+  for (int it = 0; it < iters; ++it) {
+    const uint16_t* a1[2] = {w.Ab, w.Ab};
+    const uint16_t* b1[2] = {w.XTh[cur], w.XTl[cur]};
+    launch_kk_tc(st, 2, a1, b1, nb, k, -1.f, 0.f, 1.f, nullptr, nullptr, nullptr, nullptr, w.RTh, w.RTl, w.rn + (size_t)it * nb,
+                 nullptr, status);
+    const uint16_t* a2[3] = {w.Xh[cur], w.Xl[cur], w.Xh[cur]};
+    const uint16_t* b2[3] = {w.RTh, w.RTh, w.RTl};
+    launch_kk_tc(st, 3, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], w.Xl[cur ^ 1], w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr,
+                 nullptr, status);
+    cur ^= 1;
+  }
+  w.cur = cur;
+  // accept when ||I - A X||_F before the last update was below 3e-3 (the update squares it)
+  CQ_LAUNCH(ns_check_kernel, (nb + 127) / 128, 128, 0, st, w.rn + (size_t)(iters - 1) * nb, nb, 9e-6, w.flag);
+  launch_inverse(st, Mc, X, nullptr, nb, k, status, w.flag);
+  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], w.flag, status);
+  if (cnorm) {
+    dim3 grid((k + 127) / 128, nb);
+    CQ_LAUNCH(colnorm_kernel, grid, 128, 0, st, X, k, nb, cnorm);
+  }
+  kt_end(ti, st);
+}
+
+// G (op)= -X^T Gx X^T for every block, on the tensor cores with three-term bf16 splits; X = Minv with its
+// splits in w[w.cur]; Gx fp32 [nb,k,k] (dL/dMinv).  G += result when accumulate, else G = result.
+static void minv_path_tc(cudaStream_t st, const float* Gx, float* G, int nb, int k, bool accumulate, KkWS& w, int32_t* status) {
+  const long long kk = (long long)nb * k * k;
+  const int c = w.cur;
+  launch_split(st, Gx, k, kk, nullptr, nullptr, w.Ph, w.Pl, nullptr, status);  // Gx^T splits
+  // T1 = X^T Gx : T1[i][j] = sum_l XT[i][l] * GxT[j][l]
+  const uint16_t* a1[3] = {w.XTh[c], w.XTl[c], w.XTh[c]};
+  const uint16_t* b1[3] = {w.Ph, w.Ph, w.Pl};
+  launch_kk_tc(st, 3, a1, b1, nb, k, 1.f, 0.f, 0.f, nullptr, nullptr, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status);
+  // G -= T1 X^T : [i][j] = sum_l T1[i][l] * X[j][l]
+  const uint16_t* a2[3] = {w.Qh, w.Ql, w.Qh};
+  const uint16_t* b2[3] = {w.Xh[c], w.Xh[c], w.Xl[c]};
+  launch_kk_tc(st, 3, a2, b2, nb, k, -1.f, accumulate ? 1.f : 0.f, 0.f, accumulate ? G : nullptr, G, nullptr, nullptr, nullptr,
+               nullptr, nullptr, nullptr, status);
 }
 
 static void launch_absmax(cudaStream_t st, const float* U, long long ld, const Geo& G, float* a, float* usel, int* idx,
