@@ -66,7 +66,8 @@ enum { CAFEQ_OPT_GD = 0, CAFEQ_OPT_ADAM = 1 };
 enum {
   CAFEQ_FLAG_EXACT_LOSS = 1, /* also evaluate the quantised loss (l2 proxy / PQE) */
   CAFEQ_FLAG_NO_GRAD = 2,    /* forward only */
-  CAFEQ_FLAG_GENERIC = 4     /* force the shape-agnostic kernels (debugging aid) */
+  CAFEQ_FLAG_GENERIC = 4,    /* force the shape-agnostic kernels (debugging aid) */
+  CAFEQ_FLAG_WARM_MINV = 8   /* Minv holds an approximate inverse (e.g. the previous step's) to refine */
 };
 enum { CAFEQ_ROUND_ALG1 = 0 };
 enum { CAFEQ_OFFSETS_NONE = 0, CAFEQ_OFFSETS_HARD_U8 = 1, CAFEQ_OFFSETS_SOFT_F32 = 2 };
@@ -96,6 +97,8 @@ typedef struct {
   float kappa;        /* constant of Eq. 4; <= 0 selects 1/(2^bits - 1)^2 */
   int32_t steps;
   int32_t eval_every; /* evaluate the quantised loss every n steps (0 = never) */
+  int32_t resume;     /* non-zero: opt_state comes from an earlier call on the same problem (its stored
+                         inverse is refined instead of inverting from scratch) */
 } cafeq_opt_cfg;
 
 /* Scratch bytes needed by any call on d1 (and d2 for pair calls; NULL otherwise).  cfg may be NULL.
@@ -132,7 +135,9 @@ int cafeq_rtn_noalloc(const cafeq_matrix_desc* d, const void* W, const float* T,
 
 /* One forward+backward evaluation for a single matrix (Section 4.1).
  *   M       [nb,k,k] fp32 transform parameters; the transform applied is bf16(M).
- *   Minv    optional out [nb,k,k]: inverse of bf16(M) as computed on the device.
+ *   Minv    optional out [nb,k,k]: inverse of bf16(M) as computed on the device; with
+ *           CAFEQ_FLAG_WARM_MINV also an input, a nearby inverse that Newton-Schulz steps refine (block sizes
+ *           64/128/256; the result is checked on the device and recomputed by elimination if it did not converge).
  *   offsets optional rounding offsets [d_out,d_in] (row stride d_in): uint8 {0,1} or fp32 in [0,1]
  *           (offsets_kind); code = clamp(floor(u/s) + offset) instead of round-to-nearest.
  *   losses  out fp32[4]: {surrogate (Eq. 4), ||M^-1 Q(MW) - W||_F^2 (Eq. 3), ||W||_F^2, 0};
@@ -146,8 +151,9 @@ int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* W, const fl
 
 /* `cfg->steps` optimisation steps on a single matrix (Section 4.1: gradient descent on Eq. 4 from the
  * caller's initial M; Adam selectable).  M is updated in place (fp32 master parameters).
- * opt_state: fp32 [1 + 2*nb*k*k] = {step count, first moments, second moments} (Adam; may be NULL for GD);
- * carrying it over between calls resumes a run exactly.  loss_history: out fp32 [steps, 2] =
+ * opt_state: fp32 [1 + 3*nb*k*k] = {step count, Adam first moments, Adam second moments, inverse of the last
+ * step's transform}; required for Adam, optional for gradient descent.  Carrying it over between calls with
+ * cfg->resume = 1 resumes a run; the caller zeroes it before the first call.  loss_history: out fp32 [steps, 2] =
  * {surrogate, quantised loss or NaN when not evaluated at that step}. */
 int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, float* M, float* opt_state,
                           const cafeq_opt_cfg* cfg, float* loss_history, int32_t* status, void* ws,

@@ -18,7 +18,7 @@ AXIS_IN, AXIS_OUT = 0, 1
 APPLY_T, APPLY_TT = 0, 1
 LOSS_SURROGATE, LOSS_L2_STE, LOSS_LSE, LOSS_PQE_STE = 0, 1, 2, 3
 OPT_GD, OPT_ADAM = 0, 1
-FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC = 1, 2, 4
+FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC, FLAG_WARM_MINV = 1, 2, 4, 8
 OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 
 EXPORTS = [
@@ -40,7 +40,8 @@ class OptCfg(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("loss_kind", ctypes.c_int32), ("optimizer", ctypes.c_int32),
                 ("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
                 ("eps", ctypes.c_float), ("lambda_orth", ctypes.c_float), ("lse_t", ctypes.c_float),
-                ("kappa", ctypes.c_float), ("steps", ctypes.c_int32), ("eval_every", ctypes.c_int32)]
+                ("kappa", ctypes.c_float), ("steps", ctypes.c_int32), ("eval_every", ctypes.c_int32),
+                ("resume", ctypes.c_int32)]
 
 
 class CafeqError(RuntimeError):
@@ -118,9 +119,9 @@ def make_desc(d_out, d_in, bits, group, tblock=0, taxis=AXIS_IN, trole=APPLY_T, 
 
 
 def make_cfg(loss_kind=LOSS_SURROGATE, optimizer=OPT_GD, lr=0.5, beta1=0.1, beta2=0.999, eps=1e-8,
-             lambda_orth=0.1, lse_t=5.0, kappa=0.0, steps=1, eval_every=0) -> OptCfg:
+             lambda_orth=0.1, lse_t=5.0, kappa=0.0, steps=1, eval_every=0, resume=0) -> OptCfg:
     return OptCfg(ctypes.sizeof(OptCfg), loss_kind, optimizer, lr, beta1, beta2, eps, lambda_orth, lse_t, kappa,
-                  steps, eval_every)
+                  steps, eval_every, resume)
 
 
 def workspace_size(d1: MatrixDesc, d2: MatrixDesc | None = None, cfg: OptCfg | None = None) -> int:
@@ -194,7 +195,7 @@ def cafeq_rtn_noalloc(W, T, codes, scales, *, bits, group, tblock=0, taxis=AXIS_
 
 
 def cafeq_proxy_loss_fwd_bwd(W, M, *, bits, group, taxis=AXIS_IN, loss_kind=LOSS_SURROGATE, kappa=0.0, flags=0,
-                             offsets=None, want_minv=False):
+                             offsets=None, want_minv=False, Minv=None):
     """Returns dict(losses[4], gradM or None, Minv or None, status int tensor)."""
     W = _bits_tensor(W)
     M = _f32(M, "M")
@@ -203,7 +204,10 @@ def cafeq_proxy_loss_fwd_bwd(W, M, *, bits, group, taxis=AXIS_IN, loss_kind=LOSS
     d = make_desc(d_out, d_in, bits, group, k, taxis, APPLY_T, 1, W.stride(0))
     losses = torch.zeros(4, dtype=torch.float32, device=W.device)
     gradM = None if (flags & FLAG_NO_GRAD) else torch.empty_like(M)
-    Minv = torch.empty_like(M) if want_minv else None
+    if Minv is None:
+        Minv = torch.empty_like(M) if want_minv else None
+    else:
+        Minv = _f32(Minv, "Minv")
     status = torch.zeros(1, dtype=torch.int32, device=W.device)
     okind = OFFSETS_NONE
     if offsets is not None:
@@ -228,7 +232,7 @@ def cafeq_optimize_single(W, M, cfg: OptCfg, *, bits, group, taxis=AXIS_IN, opt_
     hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W.device)
     status = torch.zeros(1, dtype=torch.int32, device=W.device)
     if cfg.optimizer == OPT_ADAM and opt_state is None:
-        opt_state = torch.zeros(1 + 2 * M.numel(), dtype=torch.float32, device=W.device)
+        opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W.device)
     ws = workspace(workspace_size(d, None, cfg), W.device)
     rc = lib().cafeq_optimize_single(ctypes.byref(d), _p(W), _p(M), _p(opt_state), ctypes.byref(cfg), _p(hist),
                                      _p(status), _p(ws), ctypes.c_size_t(ws.numel()), _stream())
@@ -275,7 +279,7 @@ def cafeq_optimize_pair(W1, W2, M, cfg: OptCfg, *, bits, group1, group2, replica
     hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W1.device)
     status = torch.zeros(1, dtype=torch.int32, device=W1.device)
     if cfg.optimizer == OPT_ADAM and opt_state is None:
-        opt_state = torch.zeros(1 + 2 * M.numel(), dtype=torch.float32, device=W1.device)
+        opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W1.device)
     ws = workspace(workspace_size(d1, d2, cfg), W1.device)
     rc = lib().cafeq_optimize_pair(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(M), _p(opt_state),
                                    _p(_f32(P, "P")), ctypes.byref(cfg), _p(hist), _p(status), _p(ws),

@@ -111,6 +111,8 @@ static int make_geo(const cafeq_matrix_desc* d, Geo* o, bool need_transform) {
   return CAFEQ_OK;
 }
 
+static size_t kk_scratch_bytes(int nbT, int k);
+
 // scratch that one matrix needs in any call
 static size_t matrix_scratch_bytes(const Geo& G) {
   size_t kk = (size_t)(G.nbT > 0 ? G.nbT : 1) * (size_t)(G.k > 0 ? G.k : 1) * (size_t)(G.k > 0 ? G.k : 1);
@@ -123,6 +125,7 @@ static size_t matrix_scratch_bytes(const Geo& G) {
   b += 8 * (kk * 4 + 256);                            // Mc, Minv, Minv_c, gMinv, tmp, RM, ...
   b += 4 * ((size_t)(G.nbT + 1) * (G.k + 1) * 4 + 256);  // c, A
   b += 4096;                                          // accumulators
+  b += kk_scratch_bytes(G.nbT, G.k);                  // bf16 splits of the k x k algebra
   return b;
 }
 
@@ -632,6 +635,7 @@ struct SingleWS {
   MatWS m;
   float *Mc, *Minv, *gMinv, *tmp, *c, *A;
   double* acc;
+  KkWS kk;
 };
 
 static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
@@ -644,21 +648,25 @@ static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
   s->c = b.take<float>((size_t)G.nbT * G.k);
   s->A = b.take<float>((size_t)G.nbT * G.k);
   s->acc = b.take<double>(8);
+  carve_kk(b, G.nbT, G.k, &s->kk);
   return !b.overflow;
 }
 
 // Enqueue one forward(+backward) for a single matrix; gradM may be null.  hist is an optional [2] slot.
 static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& G, const void* W, const float* M,
                         float* Minv_out, const void* offsets, int off_kind, int loss_kind, float kappa, bool want_exact,
-                        float* losses, float* hist, float* gradM, int32_t* status, const SingleWS& s, bool force_generic) {
+                        float* losses, float* hist, float* gradM, int32_t* status, SingleWS& s, bool force_generic,
+                        bool warm = false) {
   const int k = G.k;
+  const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G.nbT * k * k;
   const float qm = qmax_of(d->bits);
   const bool ste = (loss_kind == CAFEQ_LOSS_L2_STE);
   const bool need_l2 = want_exact || ste;
   CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, s.acc, 8);
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, s.Mc, kk, status);
-  launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
+  if (tc) ns_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, warm, s.kk, status);
+  else launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
   if (Minv_out) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, Minv_out, kk);
   const bool fused = forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, nullptr,
                                    status, !ste && !force_generic);
@@ -702,8 +710,12 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
     launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
   }
   // gradM -= Minv^T gMinv Minv^T
-  launch_kk(st, s.Minv, 1, s.gMinv, 0, s.tmp, G.nbT, k, 1.f, GEMM_STORE, status);
-  launch_kk(st, s.tmp, 0, s.Minv, 1, gradM, G.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+  if (tc) {
+    minv_path_tc(st, s.gMinv, gradM, G.nbT, k, true, s.kk, status);
+  } else {
+    launch_kk(st, s.Minv, 1, s.gMinv, 0, s.tmp, G.nbT, k, 1.f, GEMM_STORE, status);
+    launch_kk(st, s.tmp, 0, s.Minv, 1, gradM, G.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+  }
 }
 
 }  // namespace cafeq
@@ -727,8 +739,10 @@ extern "C" int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* 
   Bump b(ws, ws_bytes);
   SingleWS s;
   if (!carve_single(b, G, &s, true)) return CAFEQ_ERR_WORKSPACE;
+  const bool warm = (flags & CAFEQ_FLAG_WARM_MINV) && Minv;
+  if (warm) CQ_LAUNCH(copy_f32_kernel, grid_for((long long)G.nbT * G.k * G.k), 256, 0, st, Minv, s.Minv, (long long)G.nbT * G.k * G.k);
   single_step(st, d, G, W, M, Minv, offsets, offsets_kind, loss_kind, kappa, (flags & CAFEQ_FLAG_EXACT_LOSS) != 0, losses,
-              nullptr, want_grad ? gradM : nullptr, status, s, (flags & CAFEQ_FLAG_GENERIC) != 0);
+              nullptr, want_grad ? gradM : nullptr, status, s, (flags & CAFEQ_FLAG_GENERIC) != 0, warm);
   return last_launch();
 }
 
@@ -753,11 +767,14 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
   const long long kk = (long long)G.nbT * G.k * G.k;
   float* grad = b.take<float>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  const bool resume = cfg->resume && opt_state;
+  if (resume) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, opt_state + 1 + 2 * kk, s.Minv, kk);
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = cfg->eval_every > 0 && (it % cfg->eval_every == 0);
     single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
-                loss_history + 2 * (size_t)it, grad, status, s, false);
+                loss_history + 2 * (size_t)it, grad, status, s, false, resume || it > 0);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
+      if (opt_state) CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
       CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
@@ -765,6 +782,7 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
                                                        status);
     }
   }
+  if (opt_state && cfg->steps > 0) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, opt_state + 1 + 2 * kk, kk);
   return last_launch();
 }
 
@@ -810,6 +828,7 @@ struct PairWS {
   MatWS m1, m2;
   float *Mc, *Minv, *Minv_c, *gMinv, *tmp, *RM, *amax, *R;
   double* acc;
+  KkWS kk;
 };
 
 static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool need_R) {
@@ -825,19 +844,23 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
   p->amax = b.take<float>(64);
   p->acc = b.take<double>(8);
   p->R = need_R ? b.take<float>((size_t)G1.d_in * G2.d_out) : nullptr;
+  carve_kk(b, G1.nbT, G1.k, &p->kk);
   return !b.overflow;
 }
 
 static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
                       const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
-                      float* losses, float* hist, float* gradM, int32_t* status, const PairWS& p, bool force_generic) {
+                      float* losses, float* hist, float* gradM, int32_t* status, PairWS& p, bool force_generic,
+                      bool warm = false) {
   const int k = G1.k;
+  const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G1.nbT * k * k;
   const float sqrt_h = sqrtf((float)G1.d_out);
   CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, p.acc, 8);
   CQ_LAUNCH(fill_f32_kernel, 1, 32, 0, st, p.amax, 0.f, 1);
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, p.Mc, kk, status);
-  launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
+  if (tc) ns_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, warm, p.kk, status);
+  else launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, p.Minv, p.Minv_c, kk, status);
   // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
   forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
@@ -850,9 +873,25 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   CQ_LAUNCH(sumexp_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, t, p.acc + 0, status);
   CQ_LAUNCH(sumexp_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.amax, t, p.acc + 0, status);
   // orthonormality penalty on the fp32 parameters: R = M M^T - I
-  launch_kk(st, M, 0, M, 1, p.tmp, G1.nbT, k, 1.f, GEMM_STORE, status);
-  CQ_LAUNCH(sub_identity_kernel, grid_for(kk), 256, 0, st, p.tmp, k, kk);
-  CQ_LAUNCH(sqsum_f32_kernel, grid_for(kk), 256, 0, st, p.tmp, kk, p.acc + 1);
+  if (tc) {
+    // R = M M^T - I (symmetric) with its bf16 splits, ||R||_F^2, and R M for the gradient
+    KkWS& w = p.kk;
+    launch_split(st, M, k, kk, w.Ph, w.Pl, w.Qh, w.Ql, nullptr, status);
+    const uint16_t* a1[3] = {w.Ph, w.Pl, w.Ph};
+    const uint16_t* b1[3] = {w.Ph, w.Ph, w.Pl};
+    launch_kk_tc(st, 3, a1, b1, G1.nbT, k, 1.f, 0.f, -1.f, nullptr, nullptr, w.RTh, w.RTl, nullptr, nullptr, p.acc + 1, nullptr,
+                 status, 0);
+    if (gradM && lambda != 0.f) {
+      const uint16_t* a2[3] = {w.RTh, w.RTl, w.RTh};
+      const uint16_t* b2[3] = {w.Qh, w.Qh, w.Ql};
+      launch_kk_tc(st, 3, a2, b2, G1.nbT, k, 1.f, 0.f, 0.f, nullptr, p.RM, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                   status);
+    }
+  } else {
+    launch_kk(st, M, 0, M, 1, p.tmp, G1.nbT, k, 1.f, GEMM_STORE, status);
+    CQ_LAUNCH(sub_identity_kernel, grid_for(kk), 256, 0, st, p.tmp, k, kk);
+    CQ_LAUNCH(sqsum_f32_kernel, grid_for(kk), 256, 0, st, p.tmp, kk, p.acc + 1);
+  }
   if (want_pqe) {
     launch_pair_product(st, p.m1.E, 0, G1.d_in, p.m2.E, 0, G2.d_in, G1, G2, p.R, status);
     CQ_LAUNCH(resid_sq_kernel, grid_for((long long)G1.d_in * G2.d_out), 256, 0, st, p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
@@ -870,10 +909,14 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status);
   // V side: gradient with respect to Minv, then through the inverse
   launch_scatter(st, W2, G2, p.m2.coef, p.m2.idx, p.gMinv, 0, status);
-  launch_kk(st, p.Minv, 1, p.gMinv, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
-  launch_kk(st, p.RM, 0, p.Minv, 1, gradM, G1.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+  if (tc) {
+    minv_path_tc(st, p.gMinv, gradM, G1.nbT, k, true, p.kk, status);
+  } else {
+    launch_kk(st, p.Minv, 1, p.gMinv, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
+    launch_kk(st, p.RM, 0, p.Minv, 1, gradM, G1.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+  }
   if (lambda != 0.f) {
-    launch_kk(st, p.tmp, 0, M, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
+    if (!tc) launch_kk(st, p.tmp, 0, M, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
     CQ_LAUNCH(orth_grad_kernel, grid_for(kk), 256, 0, st, gradM, p.RM, p.acc + 1, lambda, sqrt_h, kk);
   }
 }
@@ -936,11 +979,14 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   const long long kk = (long long)G1.nbT * G1.k * G1.k;
   float* grad = b.take<float>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  const bool resume = cfg->resume && opt_state;
+  if (resume) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, opt_state + 1 + 2 * kk, p.Minv, kk);
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = any_pqe && (it % cfg->eval_every == 0);
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
-              grad, status, p, false);
+              grad, status, p, false, resume || it > 0);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
+      if (opt_state) CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
       CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
@@ -948,6 +994,7 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
                                                        status);
     }
   }
+  if (opt_state && cfg->steps > 0) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, p.Minv, opt_state + 1 + 2 * kk, kk);
   return last_launch();
 }
 

@@ -37,7 +37,7 @@ def test_every_declared_symbol_is_exported(cq):
 def test_struct_sizes_match_header_layout(cq):
     # uint32 + 2*int32 + (pad) int64 + 7*int32 -> 56 bytes with natural alignment
     assert ctypes.sizeof(cq.MatrixDesc) == 56
-    assert ctypes.sizeof(cq.OptCfg) == 48
+    assert ctypes.sizeof(cq.OptCfg) == 52
 
 
 def test_workspace_size_and_argument_errors(cq):
