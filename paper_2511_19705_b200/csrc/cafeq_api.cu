@@ -327,7 +327,8 @@ __global__ void colnorm_kernel(const float* __restrict__ X, int k, int nb, float
 
 static void launch_split(cudaStream_t st, const float* X, int k, long long n, uint16_t* hi, uint16_t* lo, uint16_t* thi,
                          uint16_t* tlo, const int* run_flag, const int32_t* status) {
-  CQ_LAUNCH(split_bf16_kernel, grid_for(n), 256, 0, st, X, k, n, hi, lo, thi, tlo, run_flag, status);
+  dim3 grid(k / 32, k / 32, (unsigned)(n / ((long long)k * k)));
+  CQ_LAUNCH(split_bf16_kernel, grid, dim3(32, 8), 0, st, X, k, hi, lo, thi, tlo, run_flag, status);
 }
 
 // Minv = inv(bf16(M)) by Newton-Schulz iteration X <- X + X (I - A X) on the tensor cores, from X0 = A^T
@@ -395,13 +396,46 @@ static void launch_absmax(cudaStream_t st, const float* U, long long ld, const G
 static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const float* coef, const int* idx, float* gT,
                            int transpose_out, const int32_t* status) {
   const int k = G.k;
+  int ti = kt_begin(2, st);
+  const bool aligned = ((uintptr_t)W % 4 == 0) && (G.ld % 2 == 0);
+  if (k % SC2_JS == 0 && G.g % 2 == 0 && aligned && G.axis == CAFEQ_AXIS_IN && (k + G.g - 1) / G.g + 1 <= SC2_MAXG + 1 &&
+      ((k >= G.g) ? k / G.g : 1) <= SC2_MAXG && (k % G.g == 0 || G.g % k == 0)) {
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(scatter_in_strip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4); attr = true; }
+    const int strips = k / SC2_JS;
+    int splits = (148 * 3) / (G.nbq * strips);
+    if (splits < 1) splits = 1;
+    int rows_per = (G.d_out + splits - 1) / splits;
+    rows_per = ((rows_per + 31) / 32) * 32;
+    splits = (G.d_out + rows_per - 1) / rows_per;
+    dim3 grid(G.nbq, strips, splits);
+    CQ_LAUNCH(scatter_in_strip_kernel, grid, 256, (size_t)k * SC2_JS * 4, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r,
+              coef, idx, gT, transpose_out, rows_per, status);
+    kt_end(ti, st);
+    return;
+  }
+  if (k % SC2_JS == 0 && k <= 256 && G.g % 2 == 0 && G.g <= 128 && aligned && G.axis == CAFEQ_AXIS_OUT) {
+    static bool attr = false;
+    const size_t shmax = (size_t)256 * SC2_JS * 4 + (size_t)SC2_JS * (128 + 2) * 2;
+    if (!attr) { cudaFuncSetAttribute(scatter_out_strip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shmax); attr = true; }
+    const int strips = k / SC2_JS;
+    int splits = (148 * 2) / (G.nbq * strips);
+    if (splits < 1) splits = 1;
+    int per = (G.ng + splits - 1) / splits;
+    splits = (G.ng + per - 1) / per;
+    dim3 grid(G.nbq, strips, splits);
+    const size_t sh = (size_t)k * SC2_JS * 4 + (size_t)SC2_JS * (G.g + 2) * 2;
+    CQ_LAUNCH(scatter_out_strip_kernel, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
+              transpose_out, per, status);
+    kt_end(ti, st);
+    return;
+  }
   size_t sh = (size_t)k * SCATTER_JS * sizeof(float);
   if (sh > 48 * 1024) {
     cudaFuncSetAttribute(scatter_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
     cudaFuncSetAttribute(scatter_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
   }
   int strips = (k + SCATTER_JS - 1) / SCATTER_JS;
-  int ti = kt_begin(2, st);
   if (G.axis == CAFEQ_AXIS_IN) {
     int want = (148 * 4) / (G.nbq * strips) + 1;
     int splits = want < 1 ? 1 : want;

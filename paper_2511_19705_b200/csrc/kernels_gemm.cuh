@@ -148,11 +148,26 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
         if (nb0 >= p.N) break;
         const bool full = rv && (nb0 + 32 <= p.N);
         float sqf = 0.f;
+        const float* c0p = p.C0 ? p.C0 + c0b + (long long)row * p.ldc0 + nb0 : nullptr;
+        const bool c0vec = full && c0p && ((p.ldc0 & 3) == 0) && (((uintptr_t)c0p & 15) == 0);
+        if (c0vec) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            const float4 c4 = *reinterpret_cast<const float4*>(c0p + e);
+            v[e] = fmaf(p.beta, c4.x, p.alpha * v[e]);
+            v[e + 1] = fmaf(p.beta, c4.y, p.alpha * v[e + 1]);
+            v[e + 2] = fmaf(p.beta, c4.z, p.alpha * v[e + 2]);
+            v[e + 3] = fmaf(p.beta, c4.w, p.alpha * v[e + 3]);
+          }
+        }
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-          float x = p.alpha * v[e];
+          float x = v[e];
           const int n = nb0 + e;
-          if (p.C0 && rv && n < p.N) x = fmaf(p.beta, p.C0[c0b + (long long)row * p.ldc0 + n], x);
+          if (!c0vec) {
+            x = p.alpha * x;
+            if (c0p && rv && n < p.N) x = fmaf(p.beta, c0p[e], x);
+          }
           if (n == row) x += p.gamma;
           v[e] = x;
           if (rv && n < p.N) sqf = fmaf(x, x, sqf);
@@ -169,17 +184,46 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
           }
         }
         if (p.Chi || p.Cthi) {
+          uint32_t hp[16], lp[16];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int n = nb0 + e;
-            const __nv_bfloat16 h = __float2bfloat16_rn(v[e]);
-            const __nv_bfloat16 l = __float2bfloat16_rn(v[e] - __bfloat162float(h));
-            if (rv && n < p.N) {
-              if (p.Chi) p.Chi[sb_mn + (long long)row * p.N + n] = __bfloat16_as_ushort(h);
-              if (p.Clo) p.Clo[sb_mn + (long long)row * p.N + n] = __bfloat16_as_ushort(l);
-              if (p.Cthi) p.Cthi[sb_mn + (long long)n * p.M + row] = __bfloat16_as_ushort(h);
-              if (p.Ctlo) p.Ctlo[sb_mn + (long long)n * p.M + row] = __bfloat16_as_ushort(l);
+          for (int e = 0; e < 32; e += 2) {
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(v[e]), h1 = __float2bfloat16_rn(v[e + 1]);
+            const __nv_bfloat16 l0 = __float2bfloat16_rn(v[e] - __bfloat162float(h0));
+            const __nv_bfloat16 l1 = __float2bfloat16_rn(v[e + 1] - __bfloat162float(h1));
+            hp[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            lp[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+          }
+          const long long ro = sb_mn + (long long)row * p.N + nb0;
+          const bool rvec = full && ((p.N & 7) == 0);
+          if (p.Chi && rv) {
+            if (rvec) {
+#pragma unroll
+              for (int w4 = 0; w4 < 4; ++w4)
+                *reinterpret_cast<uint4*>(p.Chi + ro + 8 * w4) = make_uint4(hp[4 * w4], hp[4 * w4 + 1], hp[4 * w4 + 2], hp[4 * w4 + 3]);
+            } else {
+              for (int e = 0; e < 32; ++e)
+                if (nb0 + e < p.N) p.Chi[ro + e] = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
             }
+          }
+          if (p.Clo && rv) {
+            if (rvec) {
+#pragma unroll
+              for (int w4 = 0; w4 < 4; ++w4)
+                *reinterpret_cast<uint4*>(p.Clo + ro + 8 * w4) = make_uint4(lp[4 * w4], lp[4 * w4 + 1], lp[4 * w4 + 2], lp[4 * w4 + 3]);
+            } else {
+              for (int e = 0; e < 32; ++e)
+                if (nb0 + e < p.N) p.Clo[ro + e] = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
+            }
+          }
+          if (p.Cthi && rv) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (nb0 + e < p.N) p.Cthi[sb_mn + (long long)(nb0 + e) * p.M + row] = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
+          }
+          if (p.Ctlo && rv) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (nb0 + e < p.N) p.Ctlo[sb_mn + (long long)(nb0 + e) * p.M + row] = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
           }
         }
       }
@@ -233,25 +277,36 @@ static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, co
   return tg_launch_t<256>(st, A, B, p);
 }
 
-// fp32 [n] -> bf16 hi / lo splits in row-major and transposed block order (blocks of k x k)
-__global__ void split_bf16_kernel(const float* __restrict__ X, int k, long long n, uint16_t* __restrict__ hi,
-                                  uint16_t* __restrict__ lo, uint16_t* __restrict__ thi, uint16_t* __restrict__ tlo,
-                                  const int* run_flag, const int32_t* status) {
+// fp32 blocks [nb][k][k] -> bf16 hi / lo splits in row-major and transposed order; one 32 x 32 tile per CTA
+// (grid: k/32, k/32, nb; block 32 x 8), transposed outputs staged through shared memory.  k % 32 == 0.
+__global__ void __launch_bounds__(256) split_bf16_kernel(const float* __restrict__ X, int k, uint16_t* __restrict__ hi,
+                                                         uint16_t* __restrict__ lo, uint16_t* __restrict__ thi,
+                                                         uint16_t* __restrict__ tlo, const int* run_flag, const int32_t* status) {
   if (status && *status) return;
   if (run_flag && *run_flag == 0) return;
-  const long long kk = (long long)k * k;
-  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
-    const float x = X[e];
+  __shared__ uint32_t tile[32][33];
+  const size_t base = (size_t)blockIdx.z * k * k;
+  const int j0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = i0 + ty + 8 * r, j = j0 + tx;
+    const float x = X[base + (size_t)i * k + j];
     const __nv_bfloat16 h = __float2bfloat16_rn(x);
     const __nv_bfloat16 l = __float2bfloat16_rn(x - __bfloat162float(h));
-    if (hi) hi[e] = __bfloat16_as_ushort(h);
-    if (lo) lo[e] = __bfloat16_as_ushort(l);
-    if (thi || tlo) {
-      const long long b = e / kk, r = e - b * kk;
-      const int i = (int)(r / k), j = (int)(r - (long long)i * k);
-      const long long te = b * kk + (long long)j * k + i;
-      if (thi) thi[te] = __bfloat16_as_ushort(h);
-      if (tlo) tlo[te] = __bfloat16_as_ushort(l);
+    const uint16_t hb = __bfloat16_as_ushort(h), lb = __bfloat16_as_ushort(l);
+    if (hi) hi[base + (size_t)i * k + j] = hb;
+    if (lo) lo[base + (size_t)i * k + j] = lb;
+    tile[ty + 8 * r][tx] = (uint32_t)hb | ((uint32_t)lb << 16);
+  }
+  __syncthreads();
+  if (thi || tlo) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int j = j0 + ty + 8 * r, i = i0 + tx;
+      const uint32_t v = tile[tx][ty + 8 * r];
+      if (thi) thi[base + (size_t)j * k + i] = (uint16_t)(v & 0xFFFFu);
+      if (tlo) tlo[base + (size_t)j * k + i] = (uint16_t)(v >> 16);
     }
   }
 }

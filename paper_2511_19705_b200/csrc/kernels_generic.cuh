@@ -543,6 +543,116 @@ __global__ void __launch_bounds__(256) scatter_out_kernel(const uint16_t* __rest
 }
 
 // ------------------------------------------------------------------------------------------------
+// sparse backward, strip form (k a multiple of 64).  One CTA owns 64 columns j of one block and a share of
+// the free axis, accumulates gradT[.][i][js..js+64) in shared memory and adds it to global memory once.
+// ------------------------------------------------------------------------------------------------
+constexpr int SC2_JS = 64;
+constexpr int SC2_MAXG = 4;  // groups of one row that can fall into one block (k / g)
+
+// axis IN: every (row o, group G) adds coef * W[o, B*k + j] to row i* = arg-max column - B*k (shared atomics:
+// the target row depends on the data)
+__global__ void __launch_bounds__(256) scatter_in_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out, int d_in,
+                                                               int g, int k, int r, const float* __restrict__ coef,
+                                                               const int* __restrict__ idx, float* __restrict__ gradT,
+                                                               int transpose_out, int rows_per_cta, const int32_t* status) {
+  if (status && *status) return;
+  extern __shared__ float acc[];  // [k][64]
+  const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
+  const int r0 = blockIdx.z * rows_per_cta, r1 = min(d_out, r0 + rows_per_cta);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < k * SC2_JS; e += 256) acc[e] = 0.f;
+  __syncthreads();
+  const int ng = d_in / g;
+  const int G0 = (B * k) / g, nG = (B * k + k - 1) / g - G0 + 1;  // nG <= SC2_MAXG (host checks)
+  const uint16_t* Wc = W + (long long)B * k + js + lane;
+  for (int ob = r0 + warp * 4; ob < r1; ob += 32) {
+    float w0[4], w1[4], cf[4][SC2_MAXG];
+    int ii[4][SC2_MAXG];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int o = ob + u;
+      const bool ok = o < r1;
+      w0[u] = ok ? bf16_bits_to_float(Wc[o * ld]) : 0.f;
+      w1[u] = ok ? bf16_bits_to_float(Wc[o * ld + 32]) : 0.f;
+#pragma unroll
+      for (int q = 0; q < SC2_MAXG; ++q) {
+        cf[u][q] = 0.f;
+        ii[u][q] = 0;
+        if (ok && q < nG) {
+          const long long p = (long long)o * ng + G0 + q;
+          const int col = (G0 + q) * g + idx[p] - B * k;
+          if (col >= 0 && col < k) { cf[u][q] = coef[p]; ii[u][q] = col; }
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int q = 0; q < SC2_MAXG; ++q)
+        if (cf[u][q] != 0.f) {
+          atomicAdd(&acc[ii[u][q] * SC2_JS + lane], cf[u][q] * w0[u]);
+          atomicAdd(&acc[ii[u][q] * SC2_JS + lane + 32], cf[u][q] * w1[u]);
+        }
+  }
+  __syncthreads();
+  float* out = gradT + (size_t)(B / r) * k * k;
+  for (int e = tid; e < k * SC2_JS; e += 256) {
+    const int i = e / SC2_JS, jj = js + (e - i * SC2_JS);
+    const float v = acc[e];
+    if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], v);
+  }
+}
+
+// axis OUT: pair (row B*k + i, group G) adds coef * W[B*k + j, G*g + idx] to gradT[i][j].  The CTA stages the
+// tile W[B*k + js .. +64, G*g .. +g] in shared memory (padded rows, so a column read is conflict-free) and every
+// (i, j) of the strip has exactly one owner thread: no atomics until the final add.  g <= 128.
+__global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
+                                                                int d_in, int g, int k, int r, const float* __restrict__ coef,
+                                                                const int* __restrict__ idx, float* __restrict__ gradT,
+                                                                int transpose_out, int groups_per_cta, const int32_t* status) {
+  if (status && *status) return;
+  extern __shared__ float acc[];                         // [k][64] then the tile
+  uint16_t* tile = (uint16_t*)(acc + (size_t)k * SC2_JS);  // [64][g + 2]
+  __shared__ float s_cf[256];
+  __shared__ int s_ix[256];
+  const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
+  const int ng = d_in / g;
+  const int Ga = blockIdx.z * groups_per_cta, Gb = min(ng, Ga + groups_per_cta);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tp = g + 2;
+  for (int e = tid; e < k * SC2_JS; e += 256) acc[e] = 0.f;
+  for (int G = Ga; G < Gb; ++G) {
+    __syncthreads();
+    // stage the tile: 64 rows x g columns, two columns per thread access
+    for (int e = tid; e < SC2_JS * (g / 2); e += 256) {
+      const int jr = e / (g / 2), c2 = e - jr * (g / 2);
+      const uint32_t v = *reinterpret_cast<const uint32_t*>(W + ((long long)B * k + js + jr) * ld + (long long)G * g + 2 * c2);
+      *reinterpret_cast<uint32_t*>(tile + jr * tp + 2 * c2) = v;
+    }
+    for (int i = tid; i < k; i += 256) {
+      const long long p = ((long long)B * k + i) * ng + G;
+      s_cf[i] = coef[p];
+      s_ix[i] = idx[p];
+    }
+    __syncthreads();
+    for (int i = warp; i < k; i += 8) {
+      const float cf = s_cf[i];
+      if (cf == 0.f) continue;
+      const int c = s_ix[i];
+      acc[i * SC2_JS + lane] = fmaf(cf, bf16_bits_to_float(tile[lane * tp + c]), acc[i * SC2_JS + lane]);
+      acc[i * SC2_JS + lane + 32] = fmaf(cf, bf16_bits_to_float(tile[(lane + 32) * tp + c]), acc[i * SC2_JS + lane + 32]);
+    }
+  }
+  __syncthreads();
+  float* out = gradT + (size_t)(B / r) * k * k;
+  for (int e = tid; e < k * SC2_JS; e += 256) {
+    const int i = e / SC2_JS, jj = js + (e - i * SC2_JS);
+    const float v = acc[e];
+    if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], v);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // optimiser updates and bookkeeping
 // ------------------------------------------------------------------------------------------------
 __global__ void gd_update_kernel(float* __restrict__ M, const float* __restrict__ g, float lr, long long n,
