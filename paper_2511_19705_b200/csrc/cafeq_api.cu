@@ -529,11 +529,12 @@ static bool fused_pass(cudaStream_t st, const void* X, long long ldx, const Geo&
 // tensor-core pass ran (then the residual is in w.Dbf as bf16 instead of w.D as fp32, and U is not stored).
 static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits, const float* Tc, int transposed,
                           const MatWS& w, const void* offsets, int off_kind, bool want_delta, float* Uhat, int8_t* codes,
-                          float* scales, int32_t* status, bool allow_fused) {
+                          float* scales, int32_t* status, bool allow_fused, const BdParams* surr = nullptr) {
   if (Tc && allow_fused && off_kind == CAFEQ_OFFSETS_NONE && !Uhat) {
     BdParams p;
     memset(&p, 0, sizeof(p));
-    p.epi = EPI_ABSMAX | (want_delta ? EPI_DELTA : 0) | (codes ? EPI_CODES : 0);
+    if (surr) p = *surr;
+    p.epi = EPI_ABSMAX | (want_delta ? EPI_DELTA : 0) | (codes ? EPI_CODES : 0) | (surr ? EPI_SURR : 0);
     p.qmax = qmax_of(bits);
     p.a = w.a; p.usel = w.usel; p.idx = w.idx;
     p.delta = w.Dbf; p.codes = codes; p.scales = scales;
@@ -702,8 +703,21 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   if (tc) ns_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, warm, s.kk, status);
   else launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
   if (Minv_out) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, Minv_out, kk);
+  // Eq. 4 weights per group, accumulators, then the pass (which evaluates Eq. 4 in its epilogue when it can)
+  const bool want_grad = (gradM != nullptr);
+  if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, s.c, G.d_in, G.g, k, G.r, s.m.cw);
+  else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(G.nbT * k), 256, 0, st, s.A, 0.f, (long long)G.nbT * k);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(G.ng), 256, 0, st, s.m.agrp, 0.f, G.ng);
+  BdParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.cw = s.m.cw;
+  sp.kappa = kappa;
+  sp.coef = (want_grad && !ste) ? s.m.coef : nullptr;
+  sp.lossacc = s.acc + 0;
+  sp.Aacc = (G.axis == CAFEQ_AXIS_IN) ? s.m.agrp : s.A;
   const bool fused = forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, nullptr,
-                                   status, !ste && !force_generic);
+                                   status, !ste && !force_generic, &sp);
   if (need_l2) {
     // E = Minv o Delta, L2 = sum E^2
     bool done = false;
@@ -718,15 +732,10 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
       launch_apply(st, s.m.D, 0, G.d_in, G, s.Minv, 0, s.m.E, G.d_in, (ste ? GEMM_STORE : 0) | GEMM_SQSUM, s.acc + 1, status);
     CQ_LAUNCH(sqsum_bf16_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);
   }
-  // surrogate value, arg-max coefficients and A_t
-  const bool want_grad = (gradM != nullptr);
-  if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, s.c, G.d_in, G.g, k, G.r, s.m.cw);
-  else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
-  CQ_LAUNCH(fill_f32_kernel, grid_for(G.nbT * k), 256, 0, st, s.A, 0.f, (long long)G.nbT * k);
-  CQ_LAUNCH(fill_f32_kernel, grid_for(G.ng), 256, 0, st, s.m.agrp, 0.f, G.ng);
-  CQ_LAUNCH(surrogate_rows_kernel, (G.d_out + 127) / 128, 128, 0, st, s.m.a, s.m.usel, G.d_out, G.ng, G.g, G.axis,
-                                                               s.m.cw, kappa, k, G.r, (want_grad && !ste) ? s.m.coef : nullptr,
-                                                               s.m.agrp, s.A, s.acc + 0, status);
+  if (!fused)
+    CQ_LAUNCH(surrogate_rows_kernel, (G.d_out + 127) / 128, 128, 0, st, s.m.a, s.m.usel, G.d_out, G.ng, G.g, G.axis,
+                                                                 s.m.cw, kappa, k, G.r, (want_grad && !ste) ? s.m.coef : nullptr,
+                                                                 s.m.agrp, s.A, s.acc + 0, status);
   if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, s.m.agrp, G.d_in, G.g, k, G.r, s.A);
   CQ_LAUNCH(finalize_single_kernel, 1, 1, 0, st, s.acc, losses, hist, need_l2 ? 1 : 0);
   if (!want_grad) return;

@@ -22,7 +22,7 @@
 namespace cafeq {
 
 enum { BD_IN = 0, BD_OUT = 1 };
-enum { EPI_ABSMAX = 1, EPI_DELTA = 2, EPI_CODES = 4, EPI_SQSUM = 8 };
+enum { EPI_ABSMAX = 1, EPI_DELTA = 2, EPI_CODES = 4, EPI_SQSUM = 8, EPI_SURR = 16 };
 
 struct BdParams {
   int d_out, d_in;     // shape of X
@@ -39,6 +39,12 @@ struct BdParams {
   int8_t* codes;       // [d_out, d_in]
   float* scales;       // [d_out, d_in / G]
   double* sqacc;
+  // EPI_SURR: Eq. 4 evaluated per entry inside the pass
+  const float* cw;     // input axis: sum of c_t over each column group [d_in / G]; output axis: G * c_t per row [d_out]
+  float kappa;
+  float* coef;         // [d_out, d_in / G] backward coefficient 2 kappa cw a sign(U at arg-max); may be null
+  double* lossacc;     // += kappa * sum cw a^2
+  float* Aacc;         // input axis: [d_in / G] += a^2 per column group; output axis: [nbT * k] += G * sum_G a^2 per operator row
   int32_t* status;
 };
 
@@ -296,7 +302,9 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int L = q * 32 + lane;
     uint32_t tl = 0;
     bool ok = true;
-    double sq_local = 0.0;
+    double sq_local = 0.0, sur_local = 0.0;
+    float srow = 0.f;
+    int srow_row = -1;
     bool bad = false;
     constexpr int NG = 128 / G;
     const int ng_row = p.d_in / G;
@@ -351,6 +359,29 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             p.idx[w] = bidx[gi];
           }
         }
+        if (p.epi & EPI_SURR) {
+          float surf = 0.f;
+#pragma unroll
+          for (int gi = 0; gi < NG; ++gi) {
+            const int Gc = col0 / G + gi;
+            const float av = valid ? best[gi] : 0.f;
+            const float wgt = valid ? ((FORM == BD_IN) ? p.cw[Gc] : p.cw[row]) : 0.f;
+            surf = fmaf(wgt * av, av, surf);
+            if (valid && p.coef) {
+              const float sg = (bval[gi] > 0.f) ? 1.f : ((bval[gi] < 0.f) ? -1.f : 0.f);
+              p.coef[(long long)row * ng_row + Gc] = 2.f * p.kappa * wgt * av * sg;
+            }
+            if constexpr (FORM == BD_IN) {
+              float a2 = av * av;
+              for (int o = 16; o > 0; o >>= 1) a2 += __shfl_xor_sync(0xffffffffu, a2, o);
+              if (lane == 0 && a2 != 0.f && col0 < p.d_in) atomicAdd(&p.Aacc[Gc], a2);
+            } else {
+              srow = fmaf(av, av, srow);
+            }
+          }
+          sur_local += (double)surf;
+          if (valid) srow_row = row;
+        }
         if (p.epi & (EPI_DELTA | EPI_CODES)) {
           float sc[NG];
 #pragma unroll
@@ -398,6 +429,16 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     if (p.epi & EPI_SQSUM) {
       for (int o = 16; o > 0; o >>= 1) sq_local += __shfl_xor_sync(0xffffffffu, sq_local, o);
       if (lane == 0 && sq_local != 0.0) atomicAdd(p.sqacc, sq_local);
+    }
+    if (p.epi & EPI_SURR) {
+      for (int o = 16; o > 0; o >>= 1) sur_local += __shfl_xor_sync(0xffffffffu, sur_local, o);
+      if (lane == 0 && sur_local != 0.0) atomicAdd(p.lossacc, (double)p.kappa * sur_local);
+      if constexpr (FORM == BD_OUT) {
+        if (srow_row >= 0 && srow != 0.f) {
+          const int Bq = srow_row / K;
+          atomicAdd(&p.Aacc[(Bq / p.r) * K + (srow_row - Bq * K)], (float)G * srow);
+        }
+      }
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) raise_status(p.status, CAFEQ_ERR_NONFINITE);
   }
