@@ -145,6 +145,7 @@ def main():
     ap.add_argument("--exact", action="store_true", help="also evaluate the quantised losses (Eq. 3 / Eq. 5) every step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--sample-frac", type=int, default=32)
     args = ap.parse_args()
 
@@ -190,9 +191,8 @@ def main():
         return torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
 
     sp = [SingleProblem(n, up_bf16(W), torch.from_numpy(M).to(dev), bits, group) for n, W, M in singles]
-    pp = [PairProblem(n, up_bf16(W1), up_bf16(W2), torch.from_numpy(M).to(dev), bits, group, group, r)
+    pp = [PairProblem(n, up_bf16(W1), up_bf16(W2), torch.from_numpy(M).to(dev), bits, group, group, r, lr=1e-4)
           for n, W1, W2, M, r in pairs]
-    flags = cq.FLAG_EXACT_LOSS if args.exact else 0
     if args.exact:
         for p in pp:
             p.P = cq.cafeq_pair_product(p.W1, p.W2, k=p.M.shape[-1], replicas=p.d2.replicas)
@@ -205,14 +205,23 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    # gradient-descent step size of the single matrices: a small fixed fraction of the first gradient's largest
+    # entry, so that the transforms move every step (the block inverse has real work) without leaving the
+    # neighbourhood of the initial rotations during the run
+    layer.step(0)
+    torch.cuda.synchronize()
+    for p in sp:
+        p.cfg.lr = float(1e-3 / max(float(p.grad.abs().max().item()), 1e-30))
+
+    def one_step():
+        layer.opt_step(eval_exact=args.exact)
+
     for _ in range(max(args.warmup, 3)):
-        layer.step(flags)
+        one_step()
     sync_all()
     assert all(s == 0 for s in layer.statuses()), layer.statuses()
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    time.sleep(0.3)
+    # ---- pass 1: eager launches with the library's in-stream event pairs around its main kernels
     n_timed = 64 * args.steps
     cq.timer_begin(n_timed)
     l0 = cq.launch_count()
@@ -220,19 +229,55 @@ def main():
     sync_all()
     e0.record()
     for _ in range(args.steps):
-        layer.step(flags)
+        one_step()
     e1.record()
     sync_all()
     launches = cq.launch_count() - l0
-    ms = e0.elapsed_time(e1)
+    ms_eager = e0.elapsed_time(e1)
     kms, kinds = cq.timer_read(n_timed)
+
+    # ---- pass 2 (the reported value): the same step captured once into a CUDA graph and replayed
+    graph = None
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                one_step()
+        except Exception as exc:  # capture refused: report the eager number
+            print(f"graph capture failed: {exc}", file=sys.stderr)
+            graph = None
+            torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    if graph is not None:
+        for _ in range(3):
+            graph.replay()
+        sync_all()
+        e0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record()
+        sync_all()
+        ms = e0.elapsed_time(e1)
+    else:
+        sync_all()
+        e0.record()
+        for _ in range(args.steps):
+            one_step()
+        e1.record()
+        sync_all()
+        ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
+    assert all(s == 0 for s in layer.statuses()), layer.statuses()
     if dist is not None:
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     ms_per_step = ms / args.steps
     value = world * args.steps / (ms * 1e-3)
+    cfg_json.update(launch="cuda_graph_replay" if graph is not None else "eager", eager_ms_per_step=ms_eager / args.steps,
+                    step="fwd+bwd+update (GD singles, Adam pairs), warm-started block inverse")
 
     # ---- roofline of the dominant kernel (the block-diagonal transform pass), from the in-stream event pairs
     peaks = load_peaks()
@@ -247,32 +292,33 @@ def main():
     roof = None
     tk = max((kd for kd in (1, 5) if kd in by_kind), key=lambda kd: sum(by_kind[kd]), default=None)
     if tk is not None:
-        by_kind[1] = by_kind[tk]
-        t_pass = sum(by_kind[1]) / args.steps * 1e-3            # seconds of transform passes per step
-        passes = len(by_kind[1]) / args.steps / 7.0             # passes over the layer per step
+        tp = by_kind[tk]
+        t_pass = sum(tp) / args.steps * 1e-3                    # seconds of transform passes per step
+        passes = len(tp) / args.steps / 7.0                     # passes over the layer per step
         flops = 2.0 * k * layer.weights * passes                # 2k flop per weight per pass
         byts = 2.0 * layer.weights * passes                     # bf16 weights read once per pass
-        t_hbm, t_tc = byts / (peaks["hbm_gbs"] * 1e9), flops / ((peaks["bf16_sus"] or peaks["bf16_tflops"]) * 1e12)
+        tc_peak = peaks["bf16_sus"] or peaks["bf16_tflops"]
+        t_hbm, t_tc = byts / (peaks["hbm_gbs"] * 1e9), flops / (tc_peak * 1e12)
         if t_tc >= t_hbm:
             ach = flops / t_pass / 1e12
-            roof = dict(bound="tensor", achieved=ach, peak=peaks["bf16_sus"] or peaks["bf16_tflops"], unit="TFLOP/s",
-                        frac=ach / (peaks["bf16_sus"] or peaks["bf16_tflops"]), traffic=None)
+            roof = dict(bound="tensor", achieved=ach, peak=tc_peak, unit="TFLOP/s", frac=ach / tc_peak, traffic=None)
         else:
             ach = byts / t_pass / 1e9
             roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
                         traffic=None)
         roof.update(kernel=names[tk], peak_source=peaks["source"] + (" sustained" if roof["bound"] == "tensor" else ""),
-                    launches_per_step=len(by_kind[1]) / args.steps, avg_launch_ms=sum(by_kind[1]) / len(by_kind[1]),
-                    algorithmic_gb_per_step=byts / 1e9, algorithmic_tflop_per_step=flops / 1e12)
+                    launches_per_step=len(tp) / args.steps, avg_launch_ms=sum(tp) / len(tp),
+                    algorithmic_gb_per_step=byts / 1e9, algorithmic_tflop_per_step=flops / 1e12,
+                    hbm_gbs_achieved=byts / t_pass / 1e9)
 
     # ---- end to end through the C ABI with host buffers (pinned): H2D of every weight and transform, the step,
-    #      D2H of losses and gradients, every step
+    #      D2H of the loss histories and the updated transforms, every step
     e2e = None
     if not args.no_e2e and rank == 0:
         hostW = [t.cpu().pin_memory() for p in sp for t in (p.W, p.M)] + \
                 [t.cpu().pin_memory() for p in pp for t in (p.W1, p.W2, p.M)]
         devW = [t for p in sp for t in (p.W, p.M)] + [t for p in pp for t in (p.W1, p.W2, p.M)]
-        outs = [t for p in sp + pp for t in (p.losses, p.grad)]
+        outs = [t for p in sp + pp for t in (p.hist, p.M)]
         hostO = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
         h2d = sum(t.numel() * t.element_size() for t in hostW)
         d2h = sum(t.numel() * t.element_size() for t in outs)
@@ -281,7 +327,7 @@ def main():
         def e2e_step():
             for h, d in zip(hostW, devW):
                 d.copy_(h, non_blocking=True)
-            layer.step(flags)
+            one_step()
             for h, d in zip(hostO, outs):
                 h.copy_(d, non_blocking=True)
 

@@ -2,6 +2,13 @@
 
 Holds descriptors, device buffers and workspaces for every matrix / pair of a layer so that a step is
 nothing but C-ABI calls on resident memory (no allocation inside the step).  Marshalling only.
+
+Two kinds of step:
+  * ``step(flags)``      forward + backward of the training objective at the current transform
+                         (cafeq_proxy_loss_fwd_bwd / cafeq_pair_loss_fwd_bwd);
+  * ``opt_step()``       forward + backward + parameter update (cafeq_optimize_single / _pair with
+                         steps = 1), resuming from the optimiser state of the previous call, which also
+                         carries the previous inverse so the block inverse is refined, not recomputed.
 """
 from __future__ import annotations
 
@@ -9,12 +16,12 @@ import ctypes
 
 import torch
 
-from . import (AXIS_IN, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, _check, _p, _pair_descs, _stream,
-               lib, make_desc, workspace_size)
+from . import (AXIS_IN, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, OPT_ADAM, OPT_GD, _check, _p,
+               _pair_descs, _stream, lib, make_cfg, make_desc, workspace_size)
 
 
 class SingleProblem:
-    def __init__(self, name, W, M, bits, group, taxis=AXIS_IN):
+    def __init__(self, name, W, M, bits, group, taxis=AXIS_IN, lr=1e-3):
         self.name, self.W, self.M = name, W, M
         d_out, d_in = W.shape
         self.desc = make_desc(d_out, d_in, bits, group, M.shape[-1], taxis, 0, 1, W.stride(0))
@@ -23,6 +30,9 @@ class SingleProblem:
         self.status = torch.zeros(1, dtype=torch.int32, device=W.device)
         self.ws_bytes = workspace_size(self.desc)
         self.weights = W.numel()
+        self.opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W.device)
+        self.hist = torch.zeros((1, 2), dtype=torch.float32, device=W.device)
+        self.cfg = make_cfg(loss_kind=LOSS_SURROGATE, optimizer=OPT_GD, lr=lr, steps=1, eval_every=0, resume=0)
 
     def step(self, ws, flags=0, loss_kind=LOSS_SURROGATE):
         rc = lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(self.desc), _p(self.W), _p(self.M), _p(None), _p(None),
@@ -31,9 +41,17 @@ class SingleProblem:
                                             _p(ws), ctypes.c_size_t(ws.numel()), _stream())
         _check(rc, "cafeq_proxy_loss_fwd_bwd")
 
+    def opt_step(self, ws, eval_exact=False):
+        self.cfg.eval_every = 1 if eval_exact else 0
+        rc = lib().cafeq_optimize_single(ctypes.byref(self.desc), _p(self.W), _p(self.M), _p(self.opt_state),
+                                         ctypes.byref(self.cfg), _p(self.hist), _p(self.status), _p(ws),
+                                         ctypes.c_size_t(ws.numel()), _stream())
+        _check(rc, "cafeq_optimize_single")
+        self.cfg.resume = 1
+
 
 class PairProblem:
-    def __init__(self, name, W1, W2, M, bits, group1, group2, replicas, lse_t=5.0, lambda_orth=0.1):
+    def __init__(self, name, W1, W2, M, bits, group1, group2, replicas, lse_t=5.0, lambda_orth=0.1, lr=1e-4):
         self.name, self.W1, self.W2, self.M = name, W1, W2, M
         self.d1, self.d2 = _pair_descs(W1, W2, M.shape[-1], bits, group1, group2, replicas)
         self.losses = torch.zeros(4, dtype=torch.float32, device=W1.device)
@@ -43,6 +61,10 @@ class PairProblem:
         self.lse_t, self.lambda_orth = lse_t, lambda_orth
         self.weights = W1.numel() + W2.numel()
         self.P = None
+        self.opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W1.device)
+        self.hist = torch.zeros((1, 2), dtype=torch.float32, device=W1.device)
+        self.cfg = make_cfg(loss_kind=LOSS_LSE, optimizer=OPT_ADAM, lr=lr, beta1=0.1, beta2=0.999, eps=1e-8,
+                            lambda_orth=lambda_orth, lse_t=lse_t, steps=1, eval_every=0, resume=0)
 
     def step(self, ws, flags=0):
         rc = lib().cafeq_pair_loss_fwd_bwd(ctypes.byref(self.d1), _p(self.W1), ctypes.byref(self.d2), _p(self.W2),
@@ -53,9 +75,18 @@ class PairProblem:
                                            _stream())
         _check(rc, "cafeq_pair_loss_fwd_bwd")
 
+    def opt_step(self, ws, eval_exact=False):
+        self.cfg.eval_every = 1 if (eval_exact and self.P is not None) else 0
+        rc = lib().cafeq_optimize_pair(ctypes.byref(self.d1), _p(self.W1), ctypes.byref(self.d2), _p(self.W2),
+                                       _p(self.M), _p(self.opt_state), _p(self.P if self.cfg.eval_every else None),
+                                       ctypes.byref(self.cfg), _p(self.hist), _p(self.status), _p(ws),
+                                       ctypes.c_size_t(ws.numel()), _stream())
+        _check(rc, "cafeq_optimize_pair")
+        self.cfg.resume = 1
+
 
 class LayerStep:
-    """All single matrices and pairs of one layer; step() = one forward+backward over every one of them."""
+    """All single matrices and pairs of one layer; step() / opt_step() run over every one of them."""
 
     def __init__(self, singles, pairs):
         self.singles, self.pairs = list(singles), list(pairs)
@@ -69,6 +100,10 @@ class LayerStep:
             p.step(self.ws, flags)
         for p in self.pairs:
             p.step(self.ws, flags)
+
+    def opt_step(self, eval_exact=False):
+        for p in self.singles + self.pairs:
+            p.opt_step(self.ws, eval_exact)
 
     def statuses(self):
         return [int(p.status.item()) for p in self.singles + self.pairs]
