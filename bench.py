@@ -145,6 +145,7 @@ def main():
     ap.add_argument("--exact", action="store_true", help="also evaluate the quantised losses (Eq. 3 / Eq. 5) every step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--serial", action="store_true", help="one stream and one shared workspace for the whole layer")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--sample-frac", type=int, default=32)
     args = ap.parse_args()
@@ -196,7 +197,7 @@ def main():
     if args.exact:
         for p in pp:
             p.P = cq.cafeq_pair_product(p.W1, p.W2, k=p.M.shape[-1], replicas=p.d2.replicas)
-    layer = LayerStep(sp, pp)
+    layer = LayerStep(sp, pp, parallel=not args.serial)
     cfg_json.update(weights_per_step=int(layer.weights), bits=bits, group=group, block=spec["k"])
 
     def sync_all():
@@ -221,7 +222,9 @@ def main():
     sync_all()
     assert all(s == 0 for s in layer.statuses()), layer.statuses()
 
-    # ---- pass 1: eager launches with the library's in-stream event pairs around its main kernels
+    # ---- pass 1: eager launches on one stream with the library's in-stream event pairs around its main kernels
+    par = layer.parallel
+    layer.parallel = False
     n_timed = 64 * args.steps
     cq.timer_begin(n_timed)
     l0 = cq.launch_count()
@@ -235,6 +238,7 @@ def main():
     launches = cq.launch_count() - l0
     ms_eager = e0.elapsed_time(e1)
     kms, kinds = cq.timer_read(n_timed)
+    layer.parallel = par
 
     # ---- pass 2 (the reported value): the same step captured once into a CUDA graph and replayed
     graph = None
@@ -276,7 +280,8 @@ def main():
         ms = float(t.item())
     ms_per_step = ms / args.steps
     value = world * args.steps / (ms * 1e-3)
-    cfg_json.update(launch="cuda_graph_replay" if graph is not None else "eager", eager_ms_per_step=ms_eager / args.steps,
+    cfg_json.update(launch="cuda_graph_replay" if graph is not None else "eager",
+                    streams=len(layer.streams) if layer.parallel else 1, eager_ms_per_step=ms_eager / args.steps,
                     step="fwd+bwd+update (GD singles, Adam pairs), warm-started block inverse")
 
     # ---- roofline of the dominant kernel (the block-diagonal transform pass), from the in-stream event pairs

@@ -221,11 +221,11 @@ static void launch_kk(cudaStream_t st, const float* A, int tA, const float* B, i
 }
 
 static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float* cnorm, int nb, int k, int32_t* status,
-                           const int* run_flag = nullptr) {
+                           const double* rn_check = nullptr, double tol2 = 0.0, int* redo_flag = nullptr) {
   int threads = k * k >= 1024 ? 1024 : ((k * k + 31) / 32) * 32;
   size_t sh = (size_t)3 * k * sizeof(float);
-  int ti = run_flag ? -1 : kt_begin(3, st);
-  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status, run_flag);
+  int ti = rn_check ? -1 : kt_begin(3, st);
+  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status, rn_check, tol2, redo_flag);
   kt_end(ti, st);
 }
 
@@ -302,15 +302,6 @@ __global__ void zero_ns_kernel(double* rn, int n, int* flag) {
   if (i == 0) *flag = 0;
 }
 
-// flag = 1 when any block's last squared residual is above tol2 or not finite
-__global__ void ns_check_kernel(const double* __restrict__ rn_last, int nb, double tol2, int* flag) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < nb) {
-    const double v = rn_last[i];
-    if (!(v <= tol2)) atomicExch(flag, 1);
-  }
-}
-
 // c[b][t] = sum_i X[b][i][t]^2
 __global__ void colnorm_kernel(const float* __restrict__ X, int k, int nb, float* __restrict__ c) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -359,8 +350,7 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   }
   w.cur = cur;
   // accept when ||I - A X||_F before the last update was below 1e-2 (the update squares it: <= 1e-4 after)
-  CQ_LAUNCH(ns_check_kernel, (nb + 127) / 128, 128, 0, st, w.rn + (size_t)(iters - 1) * nb, nb, 1e-4, w.flag);
-  launch_inverse(st, Mc, X, nullptr, nb, k, status, w.flag);
+  launch_inverse(st, Mc, X, nullptr, nb, k, status, w.rn + (size_t)(iters - 1) * nb, 1e-4, w.flag);
   launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], w.flag, status);
   if (cnorm) {
     dim3 grid((k + 127) / 128, nb);
@@ -398,19 +388,31 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
   const int k = G.k;
   int ti = kt_begin(2, st);
   const bool aligned = ((uintptr_t)W % 4 == 0) && (G.ld % 2 == 0);
-  if (k % SC2_JS == 0 && G.g % 2 == 0 && aligned && G.axis == CAFEQ_AXIS_IN && (k + G.g - 1) / G.g + 1 <= SC2_MAXG + 1 &&
-      ((k >= G.g) ? k / G.g : 1) <= SC2_MAXG && (k % G.g == 0 || G.g % k == 0)) {
+  const int nG = (k >= G.g) ? k / G.g : 1;  // groups of one row inside one block (g | k or k | g on this path)
+  if (k % SC2_JS == 0 && k <= 256 && aligned && G.axis == CAFEQ_AXIS_IN && (k % G.g == 0 || G.g % k == 0) &&
+      (nG == 1 || nG == 2 || nG == 4)) {
     static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(scatter_in_strip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4); attr = true; }
+    if (!attr) {
+      cudaFuncSetAttribute(scatter_in_strip_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4);
+      cudaFuncSetAttribute(scatter_in_strip_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4);
+      cudaFuncSetAttribute(scatter_in_strip_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4);
+      attr = true;
+    }
     const int strips = k / SC2_JS;
-    int splits = (148 * 3) / (G.nbq * strips);
+    int splits = (148 * 3 + G.nbq * strips - 1) / (G.nbq * strips);
     if (splits < 1) splits = 1;
     int rows_per = (G.d_out + splits - 1) / splits;
     rows_per = ((rows_per + 31) / 32) * 32;
     splits = (G.d_out + rows_per - 1) / rows_per;
     dim3 grid(G.nbq, strips, splits);
-    CQ_LAUNCH(scatter_in_strip_kernel, grid, 256, (size_t)k * SC2_JS * 4, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r,
-              coef, idx, gT, transpose_out, rows_per, status);
+    const size_t sh = (size_t)k * SC2_JS * 4;
+#define SC_IN(NGV)                                                                                                       \
+  CQ_LAUNCH(scatter_in_strip_kernel<NGV>, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, \
+            gT, transpose_out, rows_per, status)
+    if (nG == 1) SC_IN(1);
+    else if (nG == 2) SC_IN(2);
+    else SC_IN(4);
+#undef SC_IN
     kt_end(ti, st);
     return;
   }
@@ -419,7 +421,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     const size_t shmax = (size_t)256 * SC2_JS * 4 + (size_t)SC2_JS * (128 + 2) * 2;
     if (!attr) { cudaFuncSetAttribute(scatter_out_strip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shmax); attr = true; }
     const int strips = k / SC2_JS;
-    int splits = (148 * 2) / (G.nbq * strips);
+    int splits = (148 * 4 + G.nbq * strips - 1) / (G.nbq * strips);
     if (splits < 1) splits = 1;
     int per = (G.ng + splits - 1) / splits;
     splits = (G.ng + per - 1) / per;

@@ -50,7 +50,7 @@ struct TgCfg {
   static constexpr int A_BYTES = 128 * TG_BK * 2;
   static constexpr int B_BYTES = BN * TG_BK * 2;
   static constexpr int STAGE = A_BYTES + B_BYTES;
-  static constexpr int NSTAGE = 4;
+  static constexpr int NSTAGE = (BN <= 128) ? 6 : 4;
   static constexpr int SMEM = 1024 + NSTAGE * STAGE + 256;
   static constexpr int TMEM_COLS = (BN < 32) ? 32 : BN;
 };
@@ -74,6 +74,10 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * BN, m0 = blockIdx.y * 128, b = blockIdx.z;
 
+  if (threadIdx.x < 2 * TG_MAX_TERMS) {
+    const int t = threadIdx.x >> 1;
+    if (t < p.nterms) tma_prefetch_desc((threadIdx.x & 1) ? &maps.b[t] : &maps.a[t]);
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::NSTAGE; ++s) {
       mbar_init(bar_full + 8 * s, 1);

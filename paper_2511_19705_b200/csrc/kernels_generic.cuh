@@ -179,9 +179,14 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs g) {
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) block_inverse_kernel(const float* __restrict__ Min, float* __restrict__ Out,
                                                              float* __restrict__ cnorm, int k, int32_t* status,
-                                                             const int* run_flag) {
+                                                             const double* __restrict__ rn_check, double tol2, int* redo_flag) {
+  // rn_check: squared residual of an iterative inverse per block; the elimination only runs for blocks whose
+  // residual is above tol2 (or not finite) and then raises redo_flag for whoever depends on the result
   if (status && *status) return;
-  if (run_flag && *run_flag == 0) return;
+  if (rn_check) {
+    if (rn_check[blockIdx.x] <= tol2) return;
+    if (threadIdx.x == 0 && redo_flag) *redo_flag = 1;
+  }
   extern __shared__ float sm[];  // prow[k], fcol[k], piv (int) [k], red
   float* prow = sm;
   float* fcol = sm + k;
@@ -550,11 +555,14 @@ constexpr int SC2_JS = 64;
 constexpr int SC2_MAXG = 4;  // groups of one row that can fall into one block (k / g)
 
 // axis IN: every (row o, group G) adds coef * W[o, B*k + j] to row i* = arg-max column - B*k (shared atomics:
-// the target row depends on the data)
-__global__ void __launch_bounds__(256) scatter_in_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out, int d_in,
-                                                               int g, int k, int r, const float* __restrict__ coef,
-                                                               const int* __restrict__ idx, float* __restrict__ gradT,
-                                                               int transpose_out, int rows_per_cta, const int32_t* status) {
+// the target row depends on the data).  A lane owns the adjacent columns 2*lane and 2*lane+1 (one 32-bit load);
+// inside the accumulator the even columns sit in the first half of a row and the odd ones in the second, so
+// both atomics of a warp are bank-conflict free.  NG = groups of one row that fall into one block.
+template <int NG>
+__global__ void __launch_bounds__(256, 2) scatter_in_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
+                                                                  int d_in, int g, int k, int r, const float* __restrict__ coef,
+                                                                  const int* __restrict__ idx, float* __restrict__ gradT,
+                                                                  int transpose_out, int rows_per_cta, const int32_t* status) {
   if (status && *status) return;
   extern __shared__ float acc[];  // [k][64]
   const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
@@ -563,41 +571,55 @@ __global__ void __launch_bounds__(256) scatter_in_strip_kernel(const uint16_t* _
   for (int e = tid; e < k * SC2_JS; e += 256) acc[e] = 0.f;
   __syncthreads();
   const int ng = d_in / g;
-  const int G0 = (B * k) / g, nG = (B * k + k - 1) / g - G0 + 1;  // nG <= SC2_MAXG (host checks)
-  const uint16_t* Wc = W + (long long)B * k + js + lane;
-  for (int ob = r0 + warp * 4; ob < r1; ob += 32) {
-    float w0[4], w1[4], cf[4][SC2_MAXG];
-    int ii[4][SC2_MAXG];
+  const int G0 = (B * k) / g;
+  const int off = G0 * g - B * k;  // column of the first group's start relative to the block
+  const uint32_t* Wp = reinterpret_cast<const uint32_t*>(W + (long long)B * k + js) + lane;
+  const long long ldw = ld / 2;
+  struct Rec {
+    uint32_t w[4];
+    float cf[4][NG];
+    int ii[4][NG];
+  };
+  auto load = [&](int ob, Rec& R) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int o = ob + u;
-      const bool ok = o < r1;
-      w0[u] = ok ? bf16_bits_to_float(Wc[o * ld]) : 0.f;
-      w1[u] = ok ? bf16_bits_to_float(Wc[o * ld + 32]) : 0.f;
+      const int o = min(ob + u, r1 - 1);
+      const bool ok = ob + u < r1;
+      R.w[u] = Wp[o * ldw];
+      const float* cp = coef + (long long)o * ng + G0;
+      const int* ip = idx + (long long)o * ng + G0;
 #pragma unroll
-      for (int q = 0; q < SC2_MAXG; ++q) {
-        cf[u][q] = 0.f;
-        ii[u][q] = 0;
-        if (ok && q < nG) {
-          const long long p = (long long)o * ng + G0 + q;
-          const int col = (G0 + q) * g + idx[p] - B * k;
-          if (col >= 0 && col < k) { cf[u][q] = coef[p]; ii[u][q] = col; }
-        }
+      for (int q = 0; q < NG; ++q) {
+        const int col = q * g + ip[q] + off;
+        const bool in = ok && (unsigned)col < (unsigned)k;
+        R.cf[u][q] = in ? cp[q] : 0.f;
+        R.ii[u][q] = in ? col * SC2_JS + lane : lane;
       }
     }
+  };
+  Rec cur, nxt;
+  const int ob0 = r0 + warp * 4;
+  if (ob0 < r1) load(ob0, cur);
+  for (int ob = ob0; ob < r1; ob += 32) {
+    const bool more = ob + 32 < r1;
+    if (more) load(ob + 32, nxt);
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < 4; ++u) {
+      const float w0 = __uint_as_float(cur.w[u] << 16), w1 = __uint_as_float(cur.w[u] & 0xFFFF0000u);
 #pragma unroll
-      for (int q = 0; q < SC2_MAXG; ++q)
-        if (cf[u][q] != 0.f) {
-          atomicAdd(&acc[ii[u][q] * SC2_JS + lane], cf[u][q] * w0[u]);
-          atomicAdd(&acc[ii[u][q] * SC2_JS + lane + 32], cf[u][q] * w1[u]);
+      for (int q = 0; q < NG; ++q)
+        if (cur.cf[u][q] != 0.f) {
+          atomicAdd(&acc[cur.ii[u][q]], cur.cf[u][q] * w0);
+          atomicAdd(&acc[cur.ii[u][q] + 32], cur.cf[u][q] * w1);
         }
+    }
+    if (more) cur = nxt;
   }
   __syncthreads();
   float* out = gradT + (size_t)(B / r) * k * k;
   for (int e = tid; e < k * SC2_JS; e += 256) {
-    const int i = e / SC2_JS, jj = js + (e - i * SC2_JS);
+    const int i = e / SC2_JS, pos = e - i * SC2_JS;
+    const int jj = js + ((pos < 32) ? 2 * pos : 2 * (pos - 32) + 1);
     const float v = acc[e];
     if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], v);
   }
@@ -649,6 +671,89 @@ __global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* 
     const int i = e / SC2_JS, jj = js + (e - i * SC2_JS);
     const float v = acc[e];
     if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], v);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// step set-up in one launch: Mc = float(bf16(M)), Ab = bf16(M), every accumulator of the step cleared, the
+// optimiser's step counter advanced
+// ------------------------------------------------------------------------------------------------
+struct PrepArgs {
+  const float* M;
+  float* Mc;
+  uint16_t* Ab;
+  long long kk;
+  float* zero_f[4];      // fp32 arrays to clear
+  long long zero_fn[4];
+  double* zero_d[2];     // double arrays to clear
+  int zero_dn[2];
+  int* flag;             // cleared
+  float* step_counter;   // += 1 (optimiser state), may be null
+  const int32_t* status;
+};
+
+__global__ void step_prep_kernel(PrepArgs a) {
+  if (a.status && *a.status) return;
+  const long long stride = (long long)gridDim.x * blockDim.x, t0 = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  for (long long e = t0; e < a.kk; e += stride) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(a.M[e]);
+    if (a.Mc) a.Mc[e] = __bfloat162float(h);
+    if (a.Ab) a.Ab[e] = __bfloat16_as_ushort(h);
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    if (a.zero_f[q])
+      for (long long e = t0; e < a.zero_fn[q]; e += stride) a.zero_f[q][e] = 0.f;
+#pragma unroll
+  for (int q = 0; q < 2; ++q)
+    if (a.zero_d[q])
+      for (long long e = t0; e < a.zero_dn[q]; e += stride) a.zero_d[q][e] = 0.0;
+  if (t0 == 0) {
+    if (a.flag) *a.flag = 0;
+    if (a.step_counter) *a.step_counter += 1.f;
+  }
+}
+
+// c[b][t] = sum_i X[b][i][t]^2 for 32 columns t per CTA (grid: k/32, nb; block 32 x 8), and optionally the
+// input-axis group weights cw[Gc] += sum_{t in Gc} c[t] (cw cleared by the caller; groups are runs of g columns
+// of the concatenated blocks, r = 1)
+__global__ void __launch_bounds__(256) colnorm_cw_kernel(const float* __restrict__ X, int k, float* __restrict__ c,
+                                                         float* __restrict__ cw, int g) {
+  __shared__ float part[8][33];
+  const int b = blockIdx.y, t = blockIdx.x * 32 + threadIdx.x;
+  const float* Xb = X + (size_t)b * k * k;
+  float s = 0.f;
+  for (int i = threadIdx.y; i < k; i += 8) {
+    const float v = Xb[(size_t)i * k + t];
+    s = fmaf(v, v, s);
+  }
+  part[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) tot += part[q][threadIdx.x];
+    if (c) c[(size_t)b * k + t] = tot;
+    if (cw) {
+      const int col = b * k + t;  // position along the transformed axis
+      if (g >= 32) {
+        for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+        if (threadIdx.x == 0) atomicAdd(&cw[col / g], tot);
+      } else {
+        atomicAdd(&cw[col / g], tot);
+      }
+    }
+  }
+}
+
+// dL/dMinv of Eq. 4: out[b][i][t] = scale * Minv[b][i][t] * A_t; input axis with r = 1 reads A_t = Agrp[(b k + t) / g]
+__global__ void gminv_kernel(const float* __restrict__ Minv, const float* __restrict__ A, const float* __restrict__ Agrp,
+                             int g, float scale, int k, long long n, float* __restrict__ out) {
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const long long b = e / ((long long)k * k);
+    const int t = (int)(e % k);
+    const float At = Agrp ? Agrp[(b * k + t) / g] : A[b * k + t];
+    out[e] = scale * Minv[e] * At;
   }
 }
 

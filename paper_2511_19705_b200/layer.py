@@ -86,24 +86,54 @@ class PairProblem:
 
 
 class LayerStep:
-    """All single matrices and pairs of one layer; step() / opt_step() run over every one of them."""
+    """All single matrices and pairs of one layer; step() / opt_step() run over every one of them.
 
-    def __init__(self, singles, pairs):
+    The problems of a layer are independent, so with ``parallel=True`` every problem gets its own workspace
+    and its own stream: opt_step() forks from the current stream, enqueues each problem's calls on that
+    problem's stream and joins back, which lets the short, latency-bound kernels of one problem (block
+    inverse, k x k products) run beside the bandwidth-bound passes of another.  The fork/join uses events
+    only, so it can be captured into a CUDA graph."""
+
+    def __init__(self, singles, pairs, parallel=False):
         self.singles, self.pairs = list(singles), list(pairs)
-        need = max([p.ws_bytes for p in self.singles + self.pairs] + [256])
-        dev = (self.singles + self.pairs)[0].status.device
-        self.ws = torch.empty(need, dtype=torch.uint8, device=dev)
-        self.weights = sum(p.weights for p in self.singles + self.pairs)
+        probs = self.singles + self.pairs
+        dev = probs[0].status.device
+        self.parallel = parallel
+        if parallel:
+            for p in probs:
+                p.ws = torch.empty(max(p.ws_bytes, 256), dtype=torch.uint8, device=dev)
+            self.streams = [torch.cuda.Stream(device=dev) for _ in probs]
+            self.ws = None
+        else:
+            need = max([p.ws_bytes for p in probs] + [256])
+            self.ws = torch.empty(need, dtype=torch.uint8, device=dev)
+            for p in probs:
+                p.ws = self.ws
+        self.weights = sum(p.weights for p in probs)
 
     def step(self, flags=0):
-        for p in self.singles:
-            p.step(self.ws, flags)
-        for p in self.pairs:
-            p.step(self.ws, flags)
+        for p in self.singles + self.pairs:
+            p.step(p.ws, flags)
 
     def opt_step(self, eval_exact=False):
-        for p in self.singles + self.pairs:
-            p.opt_step(self.ws, eval_exact)
+        probs = self.singles + self.pairs
+        if not self.parallel:
+            for p in probs:
+                p.opt_step(p.ws, eval_exact)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        # largest problems first, so the long chains start early
+        order = sorted(range(len(probs)), key=lambda i: -probs[i].weights)
+        for i in order:
+            st = self.streams[i]
+            st.wait_event(fork)
+            with torch.cuda.stream(st):
+                probs[i].opt_step(probs[i].ws, eval_exact)
+                done = torch.cuda.Event()
+                done.record(st)
+            main.wait_event(done)
 
     def statuses(self):
         return [int(p.status.item()) for p in self.singles + self.pairs]
