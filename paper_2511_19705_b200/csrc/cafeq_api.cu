@@ -328,12 +328,14 @@ static void launch_split(cudaStream_t st, const float* X, int k, long long n, ui
 // recomputes everything.  Leaves fp32 Minv in X, its bf16 splits in w.Xh/Xl/XTh/XTl[w.cur], and c = column
 // square norms of Minv (optional).
 static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm, int nb, int k, bool warm, KkWS& w,
-                       int32_t* status) {
+                       int32_t* status, bool prepped = false) {
   const long long kk = (long long)nb * k * k;
   const int iters = warm ? NS_WARM_ITERS : NS_COLD_ITERS;
   int ti = kt_begin(3, st);
-  CQ_LAUNCH(zero_ns_kernel, (NS_MAX_ITERS * nb + 127) / 128, 128, 0, st, w.rn, NS_MAX_ITERS * nb, w.flag);
-  CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Mc, w.Ab, k, kk, 0, status);
+  if (!prepped) {  // otherwise step_prep_kernel has cleared rn / flag and written Ab
+    CQ_LAUNCH(zero_ns_kernel, (NS_MAX_ITERS * nb + 127) / 128, 128, 0, st, w.rn, NS_MAX_ITERS * nb, w.flag);
+    CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Mc, w.Ab, k, kk, 0, status);
+  }
   if (!warm) CQ_LAUNCH(transpose_blocks_kernel, grid_for(kk), 256, 0, st, Mc, X, k, kk);
   int cur = 0;
   launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
@@ -418,7 +420,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
   }
   if (k % SC2_JS == 0 && k <= 256 && G.g % 2 == 0 && G.g <= 128 && aligned && G.axis == CAFEQ_AXIS_OUT) {
     static bool attr = false;
-    const size_t shmax = (size_t)256 * SC2_JS * 4 + (size_t)SC2_JS * (128 + 2) * 2;
+    const size_t shmax = (size_t)256 * SC2_JS * 4 + (size_t)2 * SC2_JS * (128 + 2) * 2;
     if (!attr) { cudaFuncSetAttribute(scatter_out_strip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)shmax); attr = true; }
     const int strips = k / SC2_JS;
     int splits = (148 * 4 + G.nbq * strips - 1) / (G.nbq * strips);
@@ -426,7 +428,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     int per = (G.ng + splits - 1) / splits;
     splits = (G.ng + per - 1) / per;
     dim3 grid(G.nbq, strips, splits);
-    const size_t sh = (size_t)k * SC2_JS * 4 + (size_t)SC2_JS * (G.g + 2) * 2;
+    const size_t sh = (size_t)k * SC2_JS * 4 + (size_t)2 * SC2_JS * (G.g + 2) * 2;
     CQ_LAUNCH(scatter_out_strip_kernel, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
               transpose_out, per, status);
     kt_end(ti, st);
@@ -511,11 +513,12 @@ static void carve_matrix(Bump& b, const Geo& G, MatWS* w, bool need_E) {
 
 // One fused tensor-core pass (see kernels_fused.cuh); returns false when the shape is not covered.
 static bool fused_pass(cudaStream_t st, const void* X, long long ldx, const Geo& G, const float* Top, int transposed,
-                       uint16_t* Tb, BdParams p, int32_t* status) {
+                       uint16_t* Tb, BdParams p, int32_t* status, const uint16_t* Tb_ready = nullptr) {
   const int form = (G.axis == CAFEQ_AXIS_IN) ? BD_IN : BD_OUT;
   if (!bd_supported(form, G.d_out, G.d_in, ldx, G.k, G.g, X)) return false;
   const long long kk = (long long)G.nbT * G.k * G.k;
-  CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Top, Tb, G.k, kk, transposed, status);
+  if (Tb_ready && !transposed) Tb = const_cast<uint16_t*>(Tb_ready);  // bf16 operator already in applied orientation
+  else CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Top, Tb, G.k, kk, transposed, status);
   p.d_out = G.d_out;
   p.d_in = G.d_in;
   p.r = G.r;
@@ -531,7 +534,8 @@ static bool fused_pass(cudaStream_t st, const void* X, long long ldx, const Geo&
 // tensor-core pass ran (then the residual is in w.Dbf as bf16 instead of w.D as fp32, and U is not stored).
 static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits, const float* Tc, int transposed,
                           const MatWS& w, const void* offsets, int off_kind, bool want_delta, float* Uhat, int8_t* codes,
-                          float* scales, int32_t* status, bool allow_fused, const BdParams* surr = nullptr) {
+                          float* scales, int32_t* status, bool allow_fused, const BdParams* surr = nullptr,
+                          const uint16_t* Tb_ready = nullptr) {
   if (Tc && allow_fused && off_kind == CAFEQ_OFFSETS_NONE && !Uhat) {
     BdParams p;
     memset(&p, 0, sizeof(p));
@@ -540,7 +544,7 @@ static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits
     p.qmax = qmax_of(bits);
     p.a = w.a; p.usel = w.usel; p.idx = w.idx;
     p.delta = w.Dbf; p.codes = codes; p.scales = scales;
-    if (fused_pass(st, W, G.ld, G, Tc, transposed, w.Tb, p, status)) return true;
+    if (fused_pass(st, W, G.ld, G, Tc, transposed, w.Tb, p, status, Tb_ready)) return true;
   }
   if (Tc) launch_apply(st, W, 1, G.ld, G, Tc, transposed, w.U, G.d_in, GEMM_STORE, nullptr, status);
   else CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, w.U);
@@ -693,24 +697,48 @@ static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
 static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& G, const void* W, const float* M,
                         float* Minv_out, const void* offsets, int off_kind, int loss_kind, float kappa, bool want_exact,
                         float* losses, float* hist, float* gradM, int32_t* status, SingleWS& s, bool force_generic,
-                        bool warm = false) {
+                        bool warm = false, float* step_counter = nullptr) {
   const int k = G.k;
   const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G.nbT * k * k;
   const float qm = qmax_of(d->bits);
   const bool ste = (loss_kind == CAFEQ_LOSS_L2_STE);
   const bool need_l2 = want_exact || ste;
-  CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, s.acc, 8);
-  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, s.Mc, kk, status);
-  if (tc) ns_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, warm, s.kk, status);
-  else launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
-  if (Minv_out) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, Minv_out, kk);
-  // Eq. 4 weights per group, accumulators, then the pass (which evaluates Eq. 4 in its epilogue when it can)
   const bool want_grad = (gradM != nullptr);
-  if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, s.c, G.d_in, G.g, k, G.r, s.m.cw);
-  else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
-  CQ_LAUNCH(fill_f32_kernel, grid_for(G.nbT * k), 256, 0, st, s.A, 0.f, (long long)G.nbT * k);
-  CQ_LAUNCH(fill_f32_kernel, grid_for(G.ng), 256, 0, st, s.m.agrp, 0.f, G.ng);
+  const bool in_r1 = (G.axis == CAFEQ_AXIS_IN && G.r == 1);
+  if (tc) {
+    PrepArgs pa;
+    memset(&pa, 0, sizeof(pa));
+    pa.M = M; pa.Mc = s.Mc; pa.Ab = s.kk.Ab; pa.kk = kk;
+    pa.zero_f[0] = s.A; pa.zero_fn[0] = (long long)G.nbT * k;
+    pa.zero_f[1] = s.m.agrp; pa.zero_fn[1] = G.ng;
+    if (in_r1) { pa.zero_f[2] = s.m.cw; pa.zero_fn[2] = G.ng; }
+    if (want_grad) { pa.zero_f[3] = gradM; pa.zero_fn[3] = kk; }
+    pa.zero_d[0] = s.acc; pa.zero_dn[0] = 8;
+    pa.zero_d[1] = s.kk.rn; pa.zero_dn[1] = NS_MAX_ITERS * G.nbT;
+    pa.flag = s.kk.flag;
+    pa.step_counter = step_counter;
+    pa.status = status;
+    CQ_LAUNCH(step_prep_kernel, grid_for(kk), 256, 0, st, pa);
+    ns_inverse(st, s.Mc, s.Minv, nullptr, G.nbT, k, warm, s.kk, status, true);
+    dim3 cg(k / 32, G.nbT);
+    CQ_LAUNCH(colnorm_cw_kernel, cg, dim3(32, 8), 0, st, s.Minv, k, s.c, in_r1 ? s.m.cw : nullptr, G.g);
+    if (!in_r1) {
+      if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, s.c, G.d_in, G.g, k, G.r, s.m.cw);
+      else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
+    }
+  } else {
+    CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, s.acc, 8);
+    CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, s.Mc, kk, status);
+    if (step_counter) CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, step_counter, status);
+    launch_inverse(st, s.Mc, s.Minv, s.c, G.nbT, k, status);
+    if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, s.c, G.d_in, G.g, k, G.r, s.m.cw);
+    else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, s.c, G.d_out, G.g, k, G.r, s.m.cw);
+    CQ_LAUNCH(fill_f32_kernel, grid_for(G.nbT * k), 256, 0, st, s.A, 0.f, (long long)G.nbT * k);
+    CQ_LAUNCH(fill_f32_kernel, grid_for(G.ng), 256, 0, st, s.m.agrp, 0.f, G.ng);
+    if (want_grad) CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
+  }
+  if (Minv_out && Minv_out != s.Minv) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, Minv_out, kk);
   BdParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.cw = s.m.cw;
@@ -719,7 +747,7 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   sp.lossacc = s.acc + 0;
   sp.Aacc = (G.axis == CAFEQ_AXIS_IN) ? s.m.agrp : s.A;
   const bool fused = forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, nullptr,
-                                   status, !ste && !force_generic, &sp);
+                                   status, !ste && !force_generic, &sp, tc ? s.kk.Ab : nullptr);
   if (need_l2) {
     // E = Minv o Delta, L2 = sum E^2
     bool done = false;
@@ -738,13 +766,13 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
     CQ_LAUNCH(surrogate_rows_kernel, (G.d_out + 127) / 128, 128, 0, st, s.m.a, s.m.usel, G.d_out, G.ng, G.g, G.axis,
                                                                  s.m.cw, kappa, k, G.r, (want_grad && !ste) ? s.m.coef : nullptr,
                                                                  s.m.agrp, s.A, s.acc + 0, status);
-  if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, s.m.agrp, G.d_in, G.g, k, G.r, s.A);
+  if (G.axis == CAFEQ_AXIS_IN && !in_r1)
+    CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, s.m.agrp, G.d_in, G.g, k, G.r, s.A);
   CQ_LAUNCH(finalize_single_kernel, 1, 1, 0, st, s.acc, losses, hist, need_l2 ? 1 : 0);
   if (!want_grad) return;
-  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
   if (!ste) {
     launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
-    CQ_LAUNCH(scale_cols_kernel, grid_for(kk), 256, 0, st, s.Minv, s.A, 2.f * kappa, k, kk, s.gMinv);
+    CQ_LAUNCH(gminv_kernel, grid_for(kk), 256, 0, st, s.Minv, s.A, in_r1 ? s.m.agrp : nullptr, G.g, 2.f * kappa, k, kk, s.gMinv);
   } else {
     // gMinv = 2 * sum_free E Delta^T ; gDelta = 2 Minv^T o E (overwrites Delta) ; scale path through arg-max
     CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, s.gMinv, 0.f, kk);
@@ -812,22 +840,20 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
   const long long kk = (long long)G.nbT * G.k * G.k;
   float* grad = b.take<float>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  // the inverse of the last step's transform lives in the optimiser state, so a resumed run refines it
   const bool resume = cfg->resume && opt_state;
-  if (resume) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, opt_state + 1 + 2 * kk, s.Minv, kk);
+  if (opt_state) s.Minv = opt_state + 1 + 2 * kk;
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = cfg->eval_every > 0 && (it % cfg->eval_every == 0);
     single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
-                loss_history + 2 * (size_t)it, grad, status, s, false, resume || it > 0);
+                loss_history + 2 * (size_t)it, grad, status, s, false, resume || it > 0, opt_state);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
-      if (opt_state) CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
-      CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
       CQ_LAUNCH(adam_update_kernel, grid_for(kk), 256, 0, st, M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
                                                        status);
     }
   }
-  if (opt_state && cfg->steps > 0) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, s.Minv, opt_state + 1 + 2 * kk, kk);
   return last_launch();
 }
 

@@ -11,14 +11,14 @@
 // operand layouts the next product needs), and accumulate sum(C^2).
 //
 // One CTA computes one 128 x BN tile: warp 0 = TMA producer, warp 1 = MMA issuer and tensor-memory owner,
-// warps 2..5 = epilogue (one accumulator row per thread).  Every mbarrier wait is bounded.
+// warps 2..9 = epilogue (one accumulator row and half of the tile's columns per thread).  Every mbarrier wait is bounded.
 #pragma once
 
 #include "kernels_fused.cuh"
 
 namespace cafeq {
 
-constexpr int TG_THREADS = 192;
+constexpr int TG_THREADS = 320;
 constexpr int TG_BK = 64;
 constexpr int TG_MAX_TERMS = 3;
 
@@ -134,7 +134,8 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
       if (ok) tc_commit(bar_acc);
     }
   } else {
-    const int q = warp & 3;
+    // eight epilogue warps: two per 32-lane quarter of the accumulator, each taking half of the columns
+    const int q = warp & 3, half = (warp - 2) >> 2;
     const int row = m0 + q * 32 + lane;
     bool ok = mbar_wait(bar_acc, 0, abort_flag, p.status);
     ok = __all_sync(0xffffffffu, ok);
@@ -145,13 +146,15 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
       double sq = 0.0;
       const long long cb = (long long)b * p.sCb, c0b = (long long)b * p.sC0b;
       const long long sb_mn = (long long)b * p.M * p.N;
-      for (int ch = 0; ch < BN / 32; ++ch) {
+      constexpr int CH = BN / 64;  // 32-column chunks per warp
+      for (int ci = 0; ci < CH; ++ci) {
+        const int ch = half * CH + ci;
         float v[32];
         tc_ld32(taddr + ch * 32, v);
         const int nb0 = n0 + ch * 32;
         if (nb0 >= p.N) break;
+        const bool inner = (nb0 + 32 <= p.N) && (m0 + 128 <= p.M);  // no edge in this chunk: no per-element checks
         const bool full = rv && (nb0 + 32 <= p.N);
-        float sqf = 0.f;
         const float* c0p = p.C0 ? p.C0 + c0b + (long long)row * p.ldc0 + nb0 : nullptr;
         const bool c0vec = full && c0p && ((p.ldc0 & 3) == 0) && (((uintptr_t)c0p & 15) == 0);
         if (c0vec) {
@@ -163,20 +166,31 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
             v[e + 2] = fmaf(p.beta, c4.z, p.alpha * v[e + 2]);
             v[e + 3] = fmaf(p.beta, c4.w, p.alpha * v[e + 3]);
           }
-        }
+        } else {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float x = v[e];
-          const int n = nb0 + e;
-          if (!c0vec) {
-            x = p.alpha * x;
-            if (c0p && rv && n < p.N) x = fmaf(p.beta, c0p[e], x);
+          for (int e = 0; e < 32; ++e) {
+            float x = p.alpha * v[e];
+            if (c0p && rv && nb0 + e < p.N) x = fmaf(p.beta, c0p[e], x);
+            v[e] = x;
           }
-          if (n == row) x += p.gamma;
-          v[e] = x;
-          if (rv && n < p.N) sqf = fmaf(x, x, sqf);
         }
-        sq += (double)sqf;
+        if (p.gamma != 0.f && row >= nb0 && row < nb0 + 32) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (nb0 + e == row) v[e] += p.gamma;
+        }
+        if (p.sq) {
+          float sqf = 0.f;
+          if (inner) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) sqf = fmaf(v[e], v[e], sqf);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (rv && nb0 + e < p.N) sqf = fmaf(v[e], v[e], sqf);
+          }
+          sq += (double)sqf;
+        }
         if (p.C && rv) {
           float* dst = p.C + cb + (long long)row * p.ldc + nb0;
           if (full && ((p.ldc & 3) == 0) && (((uintptr_t)dst & 15) == 0)) {
@@ -220,14 +234,26 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
             }
           }
           if (p.Cthi && rv) {
+            uint16_t* ct = p.Cthi + sb_mn + (long long)nb0 * p.M + row;
+            if (inner) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (nb0 + e < p.N) p.Cthi[sb_mn + (long long)(nb0 + e) * p.M + row] = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
+              for (int e = 0; e < 32; ++e, ct += p.M) *ct = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e, ct += p.M)
+                if (nb0 + e < p.N) *ct = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
+            }
           }
           if (p.Ctlo && rv) {
+            uint16_t* ct = p.Ctlo + sb_mn + (long long)nb0 * p.M + row;
+            if (inner) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (nb0 + e < p.N) p.Ctlo[sb_mn + (long long)(nb0 + e) * p.M + row] = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
+              for (int e = 0; e < 32; ++e, ct += p.M) *ct = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e, ct += p.M)
+                if (nb0 + e < p.N) *ct = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
+            }
           }
         }
       }

@@ -625,45 +625,70 @@ __global__ void __launch_bounds__(256, 2) scatter_in_strip_kernel(const uint16_t
   }
 }
 
-// axis OUT: pair (row B*k + i, group G) adds coef * W[B*k + j, G*g + idx] to gradT[i][j].  The CTA stages the
-// tile W[B*k + js .. +64, G*g .. +g] in shared memory (padded rows, so a column read is conflict-free) and every
-// (i, j) of the strip has exactly one owner thread: no atomics until the final add.  g <= 128.
+// axis OUT: pair (row B*k + i, group G) adds coef * W[B*k + j, G*g + idx] to gradT[i][j].  The CTA stages
+// the tile W[B*k + js .. +64, G*g .. +g] in shared memory (padded rows, so a column read is conflict-free) and every
+// (i, j) of the strip has exactly one owner thread: no atomics until the final add.  Tiles and the (coef, idx)
+// records of the next group are fetched with asynchronous copies while the current group is accumulated.
+// g <= 128, g even, k <= 256.
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 __global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
                                                                 int d_in, int g, int k, int r, const float* __restrict__ coef,
                                                                 const int* __restrict__ idx, float* __restrict__ gradT,
                                                                 int transpose_out, int groups_per_cta, const int32_t* status) {
   if (status && *status) return;
-  extern __shared__ float acc[];                         // [k][64] then the tile
-  uint16_t* tile = (uint16_t*)(acc + (size_t)k * SC2_JS);  // [64][g + 2]
-  __shared__ float s_cf[256];
-  __shared__ int s_ix[256];
+  extern __shared__ float acc[];  // [k][64], then two tiles [64][g + 2]
+  const int tp = g + 2;
+  uint16_t* tile0 = (uint16_t*)(acc + (size_t)k * SC2_JS);
+  __shared__ float s_cf[2][256];
+  __shared__ int s_ix[2][256];
   const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
   const int ng = d_in / g;
   const int Ga = blockIdx.z * groups_per_cta, Gb = min(ng, Ga + groups_per_cta);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tp = g + 2;
   for (int e = tid; e < k * SC2_JS; e += 256) acc[e] = 0.f;
-  for (int G = Ga; G < Gb; ++G) {
-    __syncthreads();
-    // stage the tile: 64 rows x g columns, two columns per thread access
-    for (int e = tid; e < SC2_JS * (g / 2); e += 256) {
-      const int jr = e / (g / 2), c2 = e - jr * (g / 2);
-      const uint32_t v = *reinterpret_cast<const uint32_t*>(W + ((long long)B * k + js + jr) * ld + (long long)G * g + 2 * c2);
-      *reinterpret_cast<uint32_t*>(tile + jr * tp + 2 * c2) = v;
+  const int half_g = g / 2;
+  auto stage = [&](int G, int buf) {
+    uint16_t* tile = tile0 + (size_t)buf * SC2_JS * tp;
+    const uint16_t* src = W + ((long long)B * k + js) * ld + (long long)G * g;
+    for (int e = tid; e < SC2_JS * half_g; e += 256) {
+      const int jr = e / half_g, c2 = e - jr * half_g;
+      cp_async4(tile + jr * tp + 2 * c2, src + jr * ld + 2 * c2);
     }
     for (int i = tid; i < k; i += 256) {
       const long long p = ((long long)B * k + i) * ng + G;
-      s_cf[i] = coef[p];
-      s_ix[i] = idx[p];
+      cp_async4(&s_cf[buf][i], coef + p);
+      cp_async4(&s_ix[buf][i], idx + p);
+    }
+    cp_async_commit();
+  };
+  int buf = 0;
+  if (Ga < Gb) stage(Ga, 0);
+  for (int G = Ga; G < Gb; ++G) {
+    if (G + 1 < Gb) {
+      stage(G + 1, buf ^ 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
     __syncthreads();
+    const uint16_t* tile = tile0 + (size_t)buf * SC2_JS * tp;
     for (int i = warp; i < k; i += 8) {
-      const float cf = s_cf[i];
+      const float cf = s_cf[buf][i];
       if (cf == 0.f) continue;
-      const int c = s_ix[i];
+      const int c = s_ix[buf][i];
       acc[i * SC2_JS + lane] = fmaf(cf, bf16_bits_to_float(tile[lane * tp + c]), acc[i * SC2_JS + lane]);
       acc[i * SC2_JS + lane + 32] = fmaf(cf, bf16_bits_to_float(tile[(lane + 32) * tp + c]), acc[i * SC2_JS + lane + 32]);
     }
+    __syncthreads();
+    buf ^= 1;
   }
   __syncthreads();
   float* out = gradT + (size_t)(B / r) * k * k;
