@@ -555,11 +555,13 @@ constexpr int SC2_JS = 64;
 constexpr int SC2_MAXG = 4;  // groups of one row that can fall into one block (k / g)
 
 // axis IN: every (row o, group G) adds coef * W[o, B*k + j] to row i* = arg-max column - B*k (shared atomics:
-// the target row depends on the data).  A lane owns the adjacent columns 2*lane and 2*lane+1 (one 32-bit load);
-// inside the accumulator the even columns sit in the first half of a row and the odd ones in the second, so
-// both atomics of a warp are bank-conflict free.  NG = groups of one row that fall into one block.
+// the target row depends on the data).  A warp takes 32 consecutive rows: each lane fetches the records
+// (target row, coefficient) of one row, then the warp walks the 32 rows, broadcasting a record by shuffle and
+// adding the row's 64 strip columns.  A lane owns the adjacent columns 2*lane and 2*lane+1 (one 32-bit load);
+// inside the accumulator the even columns sit in the first half of a row and the odd ones in the second, so both
+// atomics of a warp are bank-conflict free.  NG = groups of one row that fall into one block.
 template <int NG>
-__global__ void __launch_bounds__(256, 2) scatter_in_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
+__global__ void __launch_bounds__(256, 3) scatter_in_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
                                                                   int d_in, int g, int k, int r, const float* __restrict__ coef,
                                                                   const int* __restrict__ idx, float* __restrict__ gradT,
                                                                   int transpose_out, int rows_per_cta, const int32_t* status) {
@@ -575,45 +577,44 @@ __global__ void __launch_bounds__(256, 2) scatter_in_strip_kernel(const uint16_t
   const int off = G0 * g - B * k;  // column of the first group's start relative to the block
   const uint32_t* Wp = reinterpret_cast<const uint32_t*>(W + (long long)B * k + js) + lane;
   const long long ldw = ld / 2;
-  struct Rec {
-    uint32_t w[4];
-    float cf[4][NG];
-    int ii[4][NG];
-  };
-  auto load = [&](int ob, Rec& R) {
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int o = min(ob + u, r1 - 1);
-      const bool ok = ob + u < r1;
-      R.w[u] = Wp[o * ldw];
-      const float* cp = coef + (long long)o * ng + G0;
-      const int* ip = idx + (long long)o * ng + G0;
+  float* accl = acc + lane;
+  for (int base = r0 + warp * 32; base < r1; base += 256) {
+    int ii[NG];
+    float cf[NG];
+    {
+      const int o = base + lane;
+      const bool ok = o < r1;
+      const long long p = (long long)(ok ? o : r0) * ng + G0;
 #pragma unroll
       for (int q = 0; q < NG; ++q) {
-        const int col = q * g + ip[q] + off;
+        const int ix = __ldg(idx + p + q);
+        const float c = __ldg(coef + p + q);
+        const int col = q * g + ix + off;
         const bool in = ok && (unsigned)col < (unsigned)k;
-        R.cf[u][q] = in ? cp[q] : 0.f;
-        R.ii[u][q] = in ? col * SC2_JS + lane : lane;
+        cf[q] = in ? c : 0.f;
+        ii[q] = in ? col * SC2_JS : 0;
       }
     }
-  };
-  Rec cur, nxt;
-  const int ob0 = r0 + warp * 4;
-  if (ob0 < r1) load(ob0, cur);
-  for (int ob = ob0; ob < r1; ob += 32) {
-    const bool more = ob + 32 < r1;
-    if (more) load(ob + 32, nxt);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float w0 = __uint_as_float(cur.w[u] << 16), w1 = __uint_as_float(cur.w[u] & 0xFFFF0000u);
+    for (int c8 = 0; c8 < 32; c8 += 8) {
+      uint32_t w[8];
 #pragma unroll
-      for (int q = 0; q < NG; ++q)
-        if (cur.cf[u][q] != 0.f) {
-          atomicAdd(&acc[cur.ii[u][q]], cur.cf[u][q] * w0);
-          atomicAdd(&acc[cur.ii[u][q] + 32], cur.cf[u][q] * w1);
+      for (int u = 0; u < 8; ++u) {
+        const int row = base + c8 + u;
+        w[u] = (row < r1) ? __ldg(Wp + row * ldw) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float w0 = __uint_as_float(w[u] << 16), w1 = __uint_as_float(w[u] & 0xFFFF0000u);
+#pragma unroll
+        for (int q = 0; q < NG; ++q) {
+          const int io = __shfl_sync(0xffffffffu, ii[q], c8 + u);
+          const float c = __shfl_sync(0xffffffffu, cf[q], c8 + u);
+          atomicAdd(accl + io, c * w0);
+          atomicAdd(accl + io + 32, c * w1);
         }
+      }
     }
-    if (more) cur = nxt;
   }
   __syncthreads();
   float* out = gradT + (size_t)(B / r) * k * k;
@@ -625,11 +626,14 @@ __global__ void __launch_bounds__(256, 2) scatter_in_strip_kernel(const uint16_t
   }
 }
 
-// axis OUT: pair (row B*k + i, group G) adds coef * W[B*k + j, G*g + idx] to gradT[i][j].  The CTA stages
-// the tile W[B*k + js .. +64, G*g .. +g] in shared memory (padded rows, so a column read is conflict-free) and every
-// (i, j) of the strip has exactly one owner thread: no atomics until the final add.  Tiles and the (coef, idx)
-// records of the next group are fetched with asynchronous copies while the current group is accumulated.
-// g <= 128, g even, k <= 256.
+// axis OUT: pair (row B*k + i, group G) adds coef * W[B*k + j, G*g + idx] to gradT[i][j].  The CTA stages the
+// tile W[B*k + js .. +64, G*g .. +g] in shared memory; warp w owns the rows i = w, w+8, ... of the block and a
+// lane the strip columns lane and lane+32, with the K/8 x 2 accumulators in registers: every (i, j) has exactly
+// one owner, so nothing is atomic until the final add to global memory.  Tiles and the (coef, idx) records of
+// the next group arrive by asynchronous copies while the current group is accumulated.  g <= 128, g % 4 == 0.
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
 __device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
 }
@@ -639,31 +643,34 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+template <int K>
 __global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
-                                                                int d_in, int g, int k, int r, const float* __restrict__ coef,
+                                                                int d_in, int g, int r, const float* __restrict__ coef,
                                                                 const int* __restrict__ idx, float* __restrict__ gradT,
                                                                 int transpose_out, int groups_per_cta, const int32_t* status) {
   if (status && *status) return;
-  extern __shared__ float acc[];  // [k][64], then two tiles [64][g + 2]
-  const int tp = g + 2;
-  uint16_t* tile0 = (uint16_t*)(acc + (size_t)k * SC2_JS);
-  __shared__ float s_cf[2][256];
-  __shared__ int s_ix[2][256];
+  constexpr int RW = K / 8;  // rows of the block per warp
+  extern __shared__ __align__(16) uint16_t tiles[];  // two tiles [64][g + 4]
+  __shared__ float s_cf[2][K];
+  __shared__ int s_ix[2][K];
+  const int tp = g + 4;
   const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
   const int ng = d_in / g;
   const int Ga = blockIdx.z * groups_per_cta, Gb = min(ng, Ga + groups_per_cta);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int e = tid; e < k * SC2_JS; e += 256) acc[e] = 0.f;
-  const int half_g = g / 2;
+  const int qg = g / 4;  // 8-byte chunks per tile row
+  float a0[RW], a1[RW];
+#pragma unroll
+  for (int m = 0; m < RW; ++m) { a0[m] = 0.f; a1[m] = 0.f; }
   auto stage = [&](int G, int buf) {
-    uint16_t* tile = tile0 + (size_t)buf * SC2_JS * tp;
-    const uint16_t* src = W + ((long long)B * k + js) * ld + (long long)G * g;
-    for (int e = tid; e < SC2_JS * half_g; e += 256) {
-      const int jr = e / half_g, c2 = e - jr * half_g;
-      cp_async4(tile + jr * tp + 2 * c2, src + jr * ld + 2 * c2);
+    uint16_t* tile = tiles + (size_t)buf * SC2_JS * tp;
+    const uint16_t* src = W + ((long long)B * K + js) * ld + (long long)G * g;
+    for (int e = tid; e < SC2_JS * qg; e += 256) {
+      const int jr = e / qg, c4 = e - jr * qg;
+      cp_async8(tile + jr * tp + 4 * c4, src + jr * ld + 4 * c4);
     }
-    for (int i = tid; i < k; i += 256) {
-      const long long p = ((long long)B * k + i) * ng + G;
+    for (int i = tid; i < K; i += 256) {
+      const long long p = ((long long)B * K + i) * ng + G;
       cp_async4(&s_cf[buf][i], coef + p);
       cp_async4(&s_ix[buf][i], idx + p);
     }
@@ -679,23 +686,32 @@ __global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* 
       cp_async_wait<0>();
     }
     __syncthreads();
-    const uint16_t* tile = tile0 + (size_t)buf * SC2_JS * tp;
-    for (int i = warp; i < k; i += 8) {
-      const float cf = s_cf[buf][i];
-      if (cf == 0.f) continue;
-      const int c = s_ix[buf][i];
-      acc[i * SC2_JS + lane] = fmaf(cf, bf16_bits_to_float(tile[lane * tp + c]), acc[i * SC2_JS + lane]);
-      acc[i * SC2_JS + lane + 32] = fmaf(cf, bf16_bits_to_float(tile[(lane + 32) * tp + c]), acc[i * SC2_JS + lane + 32]);
+    const uint16_t* t0 = tiles + (size_t)buf * SC2_JS * tp + lane * tp;
+    const uint16_t* t1 = t0 + 32 * tp;
+    // lane m keeps the record of this warp's m-th row
+    const float cfl = (lane < RW) ? s_cf[buf][warp + 8 * lane] : 0.f;
+    const int ixl = (lane < RW) ? s_ix[buf][warp + 8 * lane] : 0;
+#pragma unroll
+    for (int m = 0; m < RW; ++m) {
+      const float cf = __shfl_sync(0xffffffffu, cfl, m);
+      const int c = __shfl_sync(0xffffffffu, ixl, m);
+      a0[m] = fmaf(cf, bf16_bits_to_float(t0[c]), a0[m]);
+      a1[m] = fmaf(cf, bf16_bits_to_float(t1[c]), a1[m]);
     }
     __syncthreads();
     buf ^= 1;
   }
-  __syncthreads();
-  float* out = gradT + (size_t)(B / r) * k * k;
-  for (int e = tid; e < k * SC2_JS; e += 256) {
-    const int i = e / SC2_JS, jj = js + (e - i * SC2_JS);
-    const float v = acc[e];
-    if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)jj * k + i] : &out[(size_t)i * k + jj], v);
+  float* out = gradT + (size_t)(B / r) * K * K;
+#pragma unroll
+  for (int m = 0; m < RW; ++m) {
+    const int i = warp + 8 * m;
+    if (!transpose_out) {
+      if (a0[m] != 0.f) atomicAdd(&out[(size_t)i * K + js + lane], a0[m]);
+      if (a1[m] != 0.f) atomicAdd(&out[(size_t)i * K + js + lane + 32], a1[m]);
+    } else {
+      if (a0[m] != 0.f) atomicAdd(&out[(size_t)(js + lane) * K + i], a0[m]);
+      if (a1[m] != 0.f) atomicAdd(&out[(size_t)(js + lane + 32) * K + i], a1[m]);
+    }
   }
 }
 
