@@ -394,6 +394,37 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
   int ti = kt_begin(2, st);
   const bool aligned = ((uintptr_t)W % 4 == 0) && (G.ld % 2 == 0);
   const int nG = (k >= G.g) ? k / G.g : 1;  // groups of one row inside one block (g | k or k | g on this path)
+  if (kk_fast(k) && G.axis == CAFEQ_AXIS_IN && (k % G.g == 0 || G.g % k == 0) && nG <= 8 && ((uintptr_t)W % 16 == 0) &&
+      (G.ld % 8 == 0)) {
+    const int strips = k / SC2_JS;
+    int rows_per = SCB_MAXP / nG;
+    if (rows_per > 2048) rows_per = 2048;
+    // enough CTAs to fill the machine twice over, but never more rows than the record buffer holds
+    int want = (148 * 4 + G.nbq * strips - 1) / (G.nbq * strips);
+    int rp2 = (G.d_out + want - 1) / want;
+    rp2 = ((rp2 + 31) / 32) * 32;
+    if (rp2 < rows_per) rows_per = rp2;
+    if (rows_per < 32) rows_per = 32;
+    const int splits = (G.d_out + rows_per - 1) / rows_per;
+    dim3 grid(G.nbq, strips, splits);
+    const size_t sh = (size_t)k * 65 * 4 + (size_t)SCB_MAXP * 6;
+    static bool attr = false;
+    if (!attr) {
+      cudaFuncSetAttribute(scatter_in_bucket_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 65 * 4 + SCB_MAXP * 6);
+      cudaFuncSetAttribute(scatter_in_bucket_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 65 * 4 + SCB_MAXP * 6);
+      cudaFuncSetAttribute(scatter_in_bucket_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 65 * 4 + SCB_MAXP * 6);
+      attr = true;
+    }
+#define SC_INB(KV)                                                                                                         \
+  CQ_LAUNCH(scatter_in_bucket_kernel<KV>, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, G.r, nG, coef, idx, gT, \
+            transpose_out, rows_per, status)
+    if (k == 64) SC_INB(64);
+    else if (k == 128) SC_INB(128);
+    else SC_INB(256);
+#undef SC_INB
+    kt_end(ti, st);
+    return;
+  }
   if (k % SC2_JS == 0 && k <= 256 && aligned && G.axis == CAFEQ_AXIS_IN && (k % G.g == 0 || G.g % k == 0) &&
       (nG == 1 || nG == 2 || nG == 4)) {
     static bool attr = false;

@@ -626,6 +626,123 @@ __global__ void __launch_bounds__(256, 3) scatter_in_strip_kernel(const uint16_t
   }
 }
 
+// axis IN, bucketed form (no floating-point atomics in shared memory): the CTA first sorts the (row, group)
+// records of its row range by target row i* (a counting sort in shared memory; integer atomics only), then
+// thread t owns target row t / TPB and a run of 64 / TPB strip columns with the accumulators in registers and
+// walks its bucket: every record adds coef * W[row, strip] (one 128-byte row segment, read with 16-byte loads).
+// The accumulators go through shared memory to a coalesced add into global memory.
+// K in {64, 128, 256}; rows_per_cta * NG <= SCB_MAXP; ld % 8 == 0 and W 16-byte aligned.
+constexpr int SCB_MAXP = 4096;
+
+template <int K>
+__global__ void __launch_bounds__(256, 2) scatter_in_bucket_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
+                                                                   int d_in, int g, int r, int NG, const float* __restrict__ coef,
+                                                                   const int* __restrict__ idx, float* __restrict__ gradT,
+                                                                   int transpose_out, int rows_per_cta, const int32_t* status) {
+  if (status && *status) return;
+  constexpr int TPB = 256 / K;   // threads per bucket
+  constexpr int CPT = 64 / TPB;  // strip columns per thread
+  constexpr int RPT = SCB_MAXP / 256;
+  extern __shared__ __align__(16) uint8_t sc_smem[];
+  float* stage = reinterpret_cast<float*>(sc_smem);                       // [K][65]
+  float* rec_cf = stage + K * 65;                                         // [SCB_MAXP]
+  uint16_t* rec_o = reinterpret_cast<uint16_t*>(rec_cf + SCB_MAXP);       // [SCB_MAXP]
+  __shared__ int cnt[K], start[K + 1], cursor[K], wsum[8];
+  const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
+  const int r0 = blockIdx.z * rows_per_cta, r1 = min(d_out, r0 + rows_per_cta);
+  const int R = r1 - r0;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ng = d_in / g;
+  const int G0 = (B * K) / g;
+  const int off = G0 * g - B * K;
+  for (int e = tid; e < K; e += 256) cnt[e] = 0;
+  __syncthreads();
+  // phase A: fetch this thread's records, count per target row
+  short bk[RPT];
+  float cfv[RPT];
+  const int np = R * NG;
+#pragma unroll
+  for (int u = 0; u < RPT; ++u) {
+    const int e = tid + u * 256;
+    bk[u] = -1;
+    cfv[u] = 0.f;
+    if (e < np) {
+      const int row = e / NG, q = e - row * NG;
+      const long long p = (long long)(r0 + row) * ng + G0 + q;
+      const float c = __ldg(coef + p);
+      const int col = q * g + __ldg(idx + p) + off;
+      if ((unsigned)col < (unsigned)K && c != 0.f) {
+        bk[u] = (short)col;
+        cfv[u] = c;
+        atomicAdd(&cnt[col], 1);
+      }
+    }
+  }
+  __syncthreads();
+  // exclusive scan of cnt -> start (K <= 256: one entry per thread)
+  {
+    int v = (tid < K) ? cnt[tid] : 0;
+    int x = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) wsum[warp] = x;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < warp; ++w) base += wsum[w];
+    if (tid < K) {
+      start[tid] = base + x - v;
+      cursor[tid] = base + x - v;
+    }
+    if (tid == K - 1) start[K] = base + x;
+  }
+  __syncthreads();
+  // phase B: place the records
+#pragma unroll
+  for (int u = 0; u < RPT; ++u) {
+    if (bk[u] >= 0) {
+      const int pos = atomicAdd(&cursor[bk[u]], 1);
+      const int e = tid + u * 256;
+      rec_o[pos] = (uint16_t)(e / NG);
+      rec_cf[pos] = cfv[u];
+    }
+  }
+  __syncthreads();
+  // phase C: every thread walks its bucket
+  const int b = tid / TPB, part = tid - b * TPB;
+  float acc[CPT];
+#pragma unroll
+  for (int c = 0; c < CPT; ++c) acc[c] = 0.f;
+  const uint16_t* Wb = W + (long long)r0 * ld + (long long)B * K + js + part * CPT;
+  const int p1 = start[b + 1];
+  for (int p = start[b]; p < p1; ++p) {
+    const float cf = rec_cf[p];
+    const uint4* src = reinterpret_cast<const uint4*>(Wb + (long long)rec_o[p] * ld);
+    uint4 w[CPT / 8];
+#pragma unroll
+    for (int v = 0; v < CPT / 8; ++v) w[v] = __ldg(src + v);
+#pragma unroll
+    for (int v = 0; v < CPT / 8; ++v) {
+      const uint32_t ww[4] = {w[v].x, w[v].y, w[v].z, w[v].w};
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        acc[v * 8 + 2 * h] = fmaf(cf, __uint_as_float(ww[h] << 16), acc[v * 8 + 2 * h]);
+        acc[v * 8 + 2 * h + 1] = fmaf(cf, __uint_as_float(ww[h] & 0xFFFF0000u), acc[v * 8 + 2 * h + 1]);
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < CPT; ++c) stage[b * 65 + part * CPT + c] = acc[c];
+  __syncthreads();
+  float* out = gradT + (size_t)(B / r) * K * K;
+  for (int e = tid; e < K * SC2_JS; e += 256) {
+    const int i = e / SC2_JS, c = e - i * SC2_JS;
+    const float v = stage[i * 65 + c];
+    if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)(js + c) * K + i] : &out[(size_t)i * K + js + c], v);
+  }
+}
+
 // axis OUT: pair (row B*k + i, group G) adds coef * W[B*k + j, G*g + idx] to gradT[i][j].  The CTA stages the
 // tile W[B*k + js .. +64, G*g .. +g] in shared memory; warp w owns the rows i = w, w+8, ... of the block and a
 // lane the strip columns lane and lane+32, with the K/8 x 2 accumulators in registers: every (i, j) has exactly
