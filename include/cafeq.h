@@ -161,7 +161,8 @@ int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, float* M, f
 
 /* P = W1 W2 of Section 4.2 in stored layout: W1 is stored [h, d1] (= W1^T), W2 is stored [d3, r*h]
  * (= W2^T), r = d2->replicas; P[x, y] = sum_j W1[(B/r)*k + j', x] W2[y, B*k + j'] over all blocks B of W2.
- * P is fp32 [d1, d3] row-major. */
+ * P is fp32 [d1, d3] row-major.  With a workspace (cafeq_workspace_size(d1, d2)) and every dimension a multiple
+ * of 64 the product runs on the tensor cores; otherwise (ws may be NULL) on a plain fp32 kernel. */
 int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
                        const void* W2, float* P, void* ws, size_t ws_bytes, void* stream);
 
@@ -186,8 +187,14 @@ int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, const cafeq
 
 /* Algorithm 1 (Section 5) on the transformed pair U = W1 M, V = M^-1 W2 with Q = the group quantiser of
  * each descriptor: codes1/scales1 for U (stored [h, d1]), codes2/scales2 for V (stored [d3, r*h]);
- * pqe_history: out fp32 [2*iters + 1], the product error after independent rounding and after every
- * half-iteration.  M = NULL rounds the untransformed pair. */
+ * pqe_history: out fp32 [2*iters + 1], the product error (Eq. 5, un-squared) after independent rounding and
+ * after every half-iteration.  M = NULL rounds the untransformed pair.  iters <= 15.
+ * The pseudo-inverses are computed by Newton-Schulz iteration on the tensor cores (three-term bf16 splits, fp32
+ * accumulate), not by an SVD.  With r replicas the second factor's update is expand(pinv(Uhat^T) P) / r (which
+ * equals the printed update when Uhat^T has full column rank) and the first factor's least-squares target is
+ * P pinv(fold(Vhat^T)); both reduce to the printed lines for r = 1.
+ * Every dimension (h, d1, d3) must be a multiple of 64 and the block size a multiple of 32, else
+ * CAFEQ_ERR_UNSUPPORTED. */
 int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
                          const void* W2, const float* M, int iters, int mode, int8_t* codes1, float* scales1,
                          int8_t* codes2, float* scales2, float* pqe_history, int32_t* status, void* ws,

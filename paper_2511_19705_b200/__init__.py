@@ -251,8 +251,9 @@ def _pair_descs(W1, W2, k, bits, group1, group2, replicas):
 def cafeq_pair_product(W1, W2, *, k, bits=4, group1=0, group2=0, replicas=1):
     d1, d2 = _pair_descs(W1, W2, k, bits, group1, group2, replicas)
     P = torch.empty((W1.shape[1], W2.shape[0]), dtype=torch.float32, device=W1.device)
-    rc = lib().cafeq_pair_product(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(P), _p(None),
-                                  ctypes.c_size_t(0), _stream())
+    ws = workspace(workspace_size(d1, d2), W1.device)
+    rc = lib().cafeq_pair_product(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(P), _p(ws),
+                                  ctypes.c_size_t(ws.numel()), _stream())
     _check(rc, "cafeq_pair_product")
     return P
 

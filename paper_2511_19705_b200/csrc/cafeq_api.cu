@@ -596,6 +596,8 @@ static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits
 
 }  // namespace cafeq
 
+#include "pair_dense.cuh"
+
 using namespace cafeq;
 
 // ------------------------------------------------------------------------------------------------
@@ -664,11 +666,11 @@ extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_mat
     rc = make_geo(d2, &G2, false);
     if (rc) return rc;
     b += matrix_scratch_bytes(G2);
-    // product-sized buffers: residual R and two pseudo-inverse work matrices of adaptive rounding
-    size_t d1n = (size_t)d1->d_in, d3n = (size_t)d2->d_out, H = (size_t)d2->d_in;
+    // product-sized buffers: the residual of Eq. 5 and the dense algebra of Algorithm 1
+    size_t d1n = (size_t)d1->d_in, d3n = (size_t)d2->d_out;
     b += (d1n * d3n * 4 + 256);
-    b += 6 * ((d1n > d3n ? d1n : d3n) * H * 4 + 256);
-    b += 4 * (H * H * 4 + 256);
+    const int rr = d2->replicas > 0 ? d2->replicas : 1;
+    b += dense_scratch_bytes(d1->d_out, d1->d_in, d2->d_out, rr, d1->tblock > 0 ? d1->tblock : d1->d_out, G1.ng, G2.ng);
   }
   *bytes = b;
   return CAFEQ_OK;
@@ -936,7 +938,13 @@ struct PairWS {
   float *Mc, *Minv, *Minv_c, *gMinv, *tmp, *RM, *amax, *R;
   double* acc;
   KkWS kk;
+  DenseWS dn;
+  bool dense;  // the product term runs on the tensor cores (every dimension a multiple of 64)
 };
+
+static bool dense_ok(const Geo& G1, const Geo& G2) {
+  return G1.d_out % 64 == 0 && G1.d_in % 64 == 0 && G2.d_out % 64 == 0 && G2.d_in % 64 == 0 && G1.k % 32 == 0;
+}
 
 static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool need_R) {
   carve_matrix(b, G1, &p->m1, true);
@@ -952,6 +960,8 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
   p->acc = b.take<double>(8);
   p->R = need_R ? b.take<float>((size_t)G1.d_in * G2.d_out) : nullptr;
   carve_kk(b, G1.nbT, G1.k, &p->kk);
+  p->dense = need_R && dense_ok(G1, G2);
+  if (p->dense) carve_dense(b, G1.d_out, G1.d_in, G2.d_out, G2.r, G1.k, G1.ng, G2.ng, &p->dn);
   return !b.overflow;
 }
 
@@ -999,7 +1009,10 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
     CQ_LAUNCH(sub_identity_kernel, grid_for(kk), 256, 0, st, p.tmp, k, kk);
     CQ_LAUNCH(sqsum_f32_kernel, grid_for(kk), 256, 0, st, p.tmp, kk, p.acc + 1);
   }
-  if (want_pqe) {
+  if (want_pqe && p.dense) {
+    // Eq. 5 on the tensor cores: || Uhat_exp^T Vhat^T - P ||_F^2 with three-term bf16 splits of the dequantised values
+    dense_pqe(st, p.m1.E, p.m2.E, P, p.dn, p.acc + 2, nullptr, status);
+  } else if (want_pqe) {
     launch_pair_product(st, p.m1.E, 0, G1.d_in, p.m2.E, 0, G2.d_in, G1, G2, p.R, status);
     CQ_LAUNCH(resid_sq_kernel, grid_for((long long)G1.d_in * G2.d_out), 256, 0, st, p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
                                                                              status);
@@ -1036,9 +1049,18 @@ extern "C" int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, c
   int rc = make_pair_geo(d1, d2, &G1, &G2);
   if (rc) return rc;
   if (!W1 || !W2 || !P) return CAFEQ_ERR_INVALID_ARG;
-  (void)ws;
-  (void)ws_bytes;
-  launch_pair_product((cudaStream_t)stream, W1, 1, G1.ld, W2, 1, G2.ld, G1, G2, P, nullptr);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (ws && !((uintptr_t)ws & 255) && dense_ok(G1, G2)) {
+    Bump b(ws, ws_bytes);
+    DenseWS w;
+    if (carve_dense(b, G1.d_out, G1.d_in, G2.d_out, G2.r, G1.k, G1.ng, G2.ng, &w)) {
+      CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G1.n), 256, 0, st, (const uint16_t*)W1, G1.ld, G1.d_out, G1.d_in, w.U);
+      CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G2.n), 256, 0, st, (const uint16_t*)W2, G2.ld, G2.d_out, G2.d_in, w.V);
+      dense_product(st, w.U, w.V, w, P, nullptr);
+      return last_launch();
+    }
+  }
+  launch_pair_product(st, W1, 1, G1.ld, W2, 1, G2.ld, G1, G2, P, nullptr);
   return last_launch();
 }
 
@@ -1109,9 +1131,35 @@ extern "C" int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1,
                                     const void* W2, const float* M, int iters, int mode, int8_t* codes1, float* scales1,
                                     int8_t* codes2, float* scales2, float* pqe_history, int32_t* status, void* ws,
                                     size_t ws_bytes, void* stream) {
-  (void)d1; (void)W1; (void)d2; (void)W2; (void)M; (void)iters; (void)mode; (void)codes1; (void)scales1;
-  (void)codes2; (void)scales2; (void)pqe_history; (void)status; (void)ws; (void)ws_bytes; (void)stream;
-  return CAFEQ_ERR_UNSUPPORTED;
+  Geo G1, G2;
+  int rc = make_pair_geo(d1, d2, &G1, &G2);
+  if (rc) return rc;
+  if (!W1 || !W2 || !codes1 || !scales1 || !codes2 || !scales2 || !pqe_history) return CAFEQ_ERR_INVALID_ARG;
+  if (mode != CAFEQ_ROUND_ALG1 || iters < 0 || iters > 15) return CAFEQ_ERR_INVALID_ARG;
+  if (!dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;  // every dimension a multiple of 64, block a multiple of 32
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  Bump b(ws, ws_bytes);
+  DenseWS w;
+  if (!carve_dense(b, G1.d_out, G1.d_in, G2.d_out, G2.r, G1.k, G1.ng, G2.ng, &w)) return CAFEQ_ERR_WORKSPACE;
+  const long long kk = (long long)G1.nbT * G1.k * G1.k;
+  float* Mc = b.take<float>(kk);
+  float* Minv = b.take<float>(kk);
+  float* Minv_c = b.take<float>(kk);
+  if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  if (M) {
+    // the transformed pair U = W1 M (operator bf16(M)^T on the stored rows), V = M^-1 W2 (operator bf16(inv(bf16(M))))
+    CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, Mc, kk, status);
+    launch_inverse(st, Mc, Minv, nullptr, G1.nbT, G1.k, status);
+    CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, Minv, Minv_c, kk, status);
+    launch_apply(st, W1, 1, G1.ld, G1, Mc, 1, w.U, G1.d_in, GEMM_STORE, nullptr, status);
+    launch_apply(st, W2, 1, G2.ld, G2, Minv_c, 0, w.V, G2.d_in, GEMM_STORE, nullptr, status);
+  } else {
+    CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G1.n), 256, 0, st, (const uint16_t*)W1, G1.ld, G1.d_out, G1.d_in, w.U);
+    CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G2.n), 256, 0, st, (const uint16_t*)W2, G2.ld, G2.d_out, G2.d_in, w.V);
+  }
+  alg1_run(st, d1->bits, G1.g, G2.g, iters, codes1, scales1, codes2, scales2, pqe_history, w, status);
+  return last_launch();
 }
 
 extern "C" int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed, void* stream) {

@@ -1,0 +1,134 @@
+// Dense-matrix helpers for the pairwise product term (Eq. 5) and Algorithm 1: bf16 split / transpose of
+// rectangular fp32 matrices (the operand layouts of the tensor-core product kernel), replica fold / expansion
+// of the inner dimension, and the small control kernels of the iterative pseudo-inverse.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels_generic.cuh"
+
+namespace cafeq {
+
+// X fp32 [R, C] (row pitch ld) times `scale` (or times 1 / *inv_scale when inv_scale is given) ->
+// bf16 hi / lo splits, row-major [R, C] and / or transposed [C, R]; optional fp32 copy Y of the scaled values
+// (row-major) and YT (transposed, holding hi + lo: used only as a starting guess).
+// One 32 x 32 tile per CTA (grid: ceil(C/32), ceil(R/32); block 32 x 8).
+__global__ void __launch_bounds__(256) split_rect_kernel(const float* __restrict__ X, int R, int C, long long ld, float scale,
+                                                         const double* __restrict__ inv_scale, float* __restrict__ Y,
+                                                         float* __restrict__ YT, uint16_t* __restrict__ hi, uint16_t* __restrict__ lo,
+                                                         uint16_t* __restrict__ thi, uint16_t* __restrict__ tlo,
+                                                         const int32_t* status) {
+  if (status && *status) return;
+  __shared__ uint32_t tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  float sc = scale;
+  if (inv_scale) sc = (float)((double)scale / fmax(*inv_scale, 1e-300));
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = r0 + ty + 8 * q, c = c0 + tx;
+    uint32_t packed = 0;
+    if (r < R && c < C) {
+      const float x = sc * X[(long long)r * ld + c];
+      const __nv_bfloat16 h = __float2bfloat16_rn(x);
+      const __nv_bfloat16 l = __float2bfloat16_rn(x - __bfloat162float(h));
+      const uint16_t hb = __bfloat16_as_ushort(h), lb = __bfloat16_as_ushort(l);
+      if (Y) Y[(long long)r * C + c] = x;
+      if (hi) hi[(long long)r * C + c] = hb;
+      if (lo) lo[(long long)r * C + c] = lb;
+      packed = (uint32_t)hb | ((uint32_t)lb << 16);
+    }
+    tile[ty + 8 * q][tx] = packed;
+  }
+  __syncthreads();
+  if (thi || tlo || YT) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = c0 + ty + 8 * q, r = r0 + tx;
+      if (r < R && c < C) {
+        const uint32_t v = tile[tx][ty + 8 * q];
+        if (thi) thi[(long long)c * R + r] = (uint16_t)(v & 0xFFFFu);
+        if (tlo) tlo[(long long)c * R + r] = (uint16_t)(v >> 16);
+        if (YT) YT[(long long)c * R + r] = __uint_as_float(v << 16) + __uint_as_float(v & 0xFFFF0000u);
+      }
+    }
+  }
+}
+
+// bf16 [R, C] (pitch ld) -> bf16 transposed [C, R]
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const uint16_t* __restrict__ X, int R, int C, long long ld,
+                                                             uint16_t* __restrict__ T) {
+  __shared__ uint16_t tile[32][34];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = r0 + ty + 8 * q, c = c0 + tx;
+    tile[ty + 8 * q][tx] = (r < R && c < C) ? X[(long long)r * ld + c] : (uint16_t)0;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int c = c0 + ty + 8 * q, r = r0 + tx;
+    if (r < R && c < C) T[(long long)c * R + r] = tile[tx][ty + 8 * q];
+  }
+}
+
+// Bf[B*k + j][y] = sum_rep V[y][(B*r + rep)*k + j]: fold the r replicas of every block of the inner dimension
+// and transpose (V fp32 [d3, r*h] -> Bf fp32 [h, d3]).  grid: ceil(d3/32), h/32 (k % 32 == 0); block 32 x 8.
+__global__ void __launch_bounds__(256) fold_transpose_kernel(const float* __restrict__ V, int d3, int h, int k, int r,
+                                                             float* __restrict__ Bf) {
+  __shared__ float tile[32][33];
+  const int y0 = blockIdx.x * 32, l0 = blockIdx.y * 32;  // l0 inside one block of k
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int B = l0 / k, j0 = l0 - B * k;
+  const long long ldv = (long long)r * h;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int y = y0 + ty + 8 * q;
+    float s = 0.f;
+    if (y < d3)
+      for (int rep = 0; rep < r; ++rep) s += V[(long long)y * ldv + (long long)(B * r + rep) * k + j0 + tx];
+    tile[ty + 8 * q][tx] = s;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int l = l0 + ty + 8 * q, y = y0 + tx;
+    if (y < d3) Bf[(long long)l * d3 + y] = tile[tx][ty + 8 * q];
+  }
+}
+
+// V[y][(B*r + rep)*k + j] = X[y][B*k + j] / r  (X fp32 [d3, h] -> V fp32 [d3, r*h])
+__global__ void expand_cols_kernel(const float* __restrict__ X, int d3, int h, int k, int r, float* __restrict__ V) {
+  const long long n = (long long)d3 * r * h;
+  const float inv = 1.f / (float)r;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const long long y = e / ((long long)r * h);
+    const int l = (int)(e - y * (long long)r * h);
+    const int Bq = l / k, j = l - Bq * k;
+    V[e] = inv * X[y * h + (long long)(Bq / r) * k + j];
+  }
+}
+
+// iteration control of the pseudo-inverse: keep running while the newest squared residual is above tol2 and
+// still falling (a rank-deficient matrix stalls at its rank defect); flag: 1 = run, 0 = skip
+__global__ void pinv_control_kernel(const double* __restrict__ sq, int it, double tol2, int* flag) {
+  if (*flag == 0) return;
+  const double cur = sq[it];
+  if (!(cur > tol2)) { *flag = 0; return; }
+  if (it >= 4) {
+    const double prev = sq[it - 1];
+    if (cur > prev * (1.0 - 1e-7) && cur < prev * (1.0 + 1e-7)) *flag = 0;  // stalled
+  }
+}
+
+__global__ void set_int_kernel(int* p, int v) { *p = v; }
+
+__global__ void sqrt_hist_kernel(const double* __restrict__ sq, float* __restrict__ out, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = (float)sqrt(fmax(sq[i], 0.0));
+}
+
+}  // namespace cafeq
