@@ -128,3 +128,20 @@ def test_pair_product_and_pqe_on_tensor_cores(cq):
     assert int(out["status"].item()) == 0
     L = out["losses"].cpu().numpy()
     assert abs(L[3] - f["pqe"] ** 2) <= 2e-3 * f["pqe"] ** 2
+
+
+def test_alg1_full_size_vo_pair(cq):
+    """The v-o pair of the 9B-shaped layer (v 2048 x 3584, o 3584 x 4096, two query heads per kv head, 3-bit,
+    group 128) through one iteration of Algorithm 1 after a rotation: the independent-rounding error against the
+    oracle's, and the reported final error against the error recomputed in float64 from the returned codes."""
+    k, r, bits, g = 256, 2, 3, 128
+    W1b, W2b = syn.make_weight(3, "v", 2048, 3584), syn.make_weight(3, "o", 3584, 4096)
+    M = syn.make_transform("v", 8, k)
+    out = cq.cafeq_adaptive_round(to_dev(W1b), to_dev(W2b), f32_dev(M), iters=1, bits=bits, group1=g, group2=g, replicas=r)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    hist = out["pqe"].cpu().numpy().astype(np.float64)
+    f = orc.pair_forward(w64(W1b), w64(W2b), M, bits, g, g, r, 5.0, 0.0, True)
+    assert abs(hist[0] - f["pqe"]) <= 2e-3 * f["pqe"], (hist, f["pqe"])
+    assert hist[1] < hist[0]                                   # the compensating update of the second factor helps
+    assert abs(hist[-1] - _recomputed_pqe(out, f["U"], f["V"], k, r, g, g)) <= 2e-3 * hist[-1]
