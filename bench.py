@@ -185,7 +185,9 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    spec, singles, pairs = host_layer(args.config, rank)
+    from paper_2511_19705_b200 import shard
+    my_layer = shard.layers_of_rank(world, world, rank)[0]     # weak scaling: one layer per rank, no data-path collective
+    spec, singles, pairs = host_layer(args.config, my_layer)
     bits, group = spec["bits"], spec["group"]
 
     def up_bf16(b):
@@ -274,10 +276,7 @@ def main():
         ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
     assert all(s == 0 for s in layer.statuses()), layer.statuses()
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = shard.max_over_ranks(ms, dev)
     ms_per_step = ms / args.steps
     value = world * args.steps / (ms * 1e-3)
     cfg_json.update(launch="cuda_graph_replay" if graph is not None else "eager",
