@@ -182,24 +182,26 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   static_assert(G == 64 || G == 128, "group size");
   if (p.status && *p.status) return;
 
-  const int major = blockIdx.x / p.ctas_per_major;
-  const int sub = blockIdx.x - major * p.ctas_per_major;
-  const int m_begin = (int)(((long long)sub * p.n_minor) / p.ctas_per_major);
-  const int m_end = (int)(((long long)(sub + 1) * p.n_minor) / p.ctas_per_major);
-  if (m_begin >= m_end) return;
+  // persistent CTA: a contiguous run of tiles in (major, minor) order; the operator block is reloaded when the
+  // run crosses into the next major
+  const int total_tiles = p.n_major * p.n_minor;
+  const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
+  const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
+  if (t_begin >= t_end) return;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sT = smem;
   uint8_t* sStage = smem + C::T_BYTES;
   uint64_t* bars = (uint64_t*)(sStage + C::NSTAGE * BD_STAGE_BYTES);
-  // barrier slots: full[NSTAGE], empty[NSTAGE], tfull, accf[2], acce[2]
+  // barrier slots: full[NSTAGE], empty[NSTAGE], tfull, accf[2], acce[2], tfree
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8 * C::NSTAGE;
   const uint32_t bar_tfull = bar_empty + 8 * C::NSTAGE;
   const uint32_t bar_accf = bar_tfull + 8;
   const uint32_t bar_acce = bar_accf + 16;
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 5);
+  const uint32_t bar_tfree = bar_acce + 16;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 6);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -212,6 +214,7 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       mbar_init(bar_empty + 8 * s, 1);
     }
     mbar_init(bar_tfull, 1);
+    mbar_init(bar_tfree, 1);
     mbar_init(bar_accf, 1);
     mbar_init(bar_accf + 8, 1);
     mbar_init(bar_acce, 8);
@@ -232,15 +235,23 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      mbar_expect_tx(bar_tfull, C::T_BYTES);
-      for (int bi = 0; bi < C::NBLK; ++bi) {
-        const int tb = (FORM == BD_IN) ? (major * C::NBLK + bi) / p.r : major / p.r;
-        for (int ci = 0; ci < K / 64; ++ci)
-          tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), &tmT, ci * 64, tb * K, bar_tfull);
-      }
-      uint32_t it = 0;
+      uint32_t it = 0, tloads = 0;
+      int cur_major = -1;
       bool ok = true;
-      for (int t = m_begin; t < m_end && ok; ++t) {
+      for (int tile = t_begin; tile < t_end && ok; ++tile) {
+        const int major = tile / p.n_minor, t = tile - major * p.n_minor;
+        if (major != cur_major) {
+          // the products of the previous major must have finished reading the operator block
+          if (tloads > 0 && !mbar_wait(bar_tfree, (tloads - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+          mbar_expect_tx(bar_tfull, C::T_BYTES);
+          for (int bi = 0; bi < C::NBLK; ++bi) {
+            const int tb = (FORM == BD_IN) ? (major * C::NBLK + bi) / p.r : major / p.r;
+            for (int ci = 0; ci < K / 64; ++ci)
+              tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), &tmT, ci * 64, tb * K, bar_tfull);
+          }
+          cur_major = major;
+          ++tloads;
+        }
         for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
           const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
@@ -261,13 +272,20 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      bool ok = mbar_wait(bar_tfull, 0, abort_flag, p.status);
-      tc_fence_after();
+      bool ok = true;
+      int cur_major = -1;
+      uint32_t tfulls = 0;
       constexpr uint32_t idesc_in = umma_idesc_bf16(128, K, 0, 0);
       constexpr uint32_t idesc_out = umma_idesc_bf16(128, 64, 0, 1);
       const uint32_t sT_u = smem_u32(sT), sSt_u = smem_u32(sStage);
       uint32_t it = 0, tl = 0;
-      for (int t = m_begin; t < m_end && ok; ++t, ++tl) {
+      for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
+        const int major = tile / p.n_minor;
+        if (major != cur_major) {
+          if (!mbar_wait(bar_tfull, tfulls & 1u, abort_flag, p.status)) { ok = false; break; }
+          ++tfulls;
+          cur_major = major;
+        }
         const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
         if (!mbar_wait(bar_acce + 8 * buf, aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
@@ -300,6 +318,8 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           tc_commit(bar_empty + 8 * s);
         }
         if (ok) tc_commit(bar_accf + 8 * buf);
+        // last tile of this major with more to come: signal when its products are done with the operator block
+        if (ok && tile + 1 < t_end && (tile + 1) / p.n_minor != major) tc_commit(bar_tfree);
       }
     }
   } else {
@@ -314,7 +334,8 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     bool bad = false;
     constexpr int NG = 128 / G;
     const int ng_row = p.d_in / G;
-    for (int t = m_begin; t < m_end && ok; ++t, ++tl) {
+    for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
+      const int major = tile / p.n_minor, t = tile - major * p.n_minor;
       const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
       ok = mbar_wait(bar_accf + 8 * buf, aph, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
@@ -338,20 +359,29 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       int bidx[NG];
 #pragma unroll
       for (int gi = 0; gi < NG; ++gi) { best[gi] = -1.f; bval[gi] = 0.f; bidx[gi] = 0; }
-      float sq = 0.f;
+      if (p.epi == EPI_SQSUM) {
+        // sum of squares only (second pass of the l2 proxy)
+        float sq = 0.f;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        tc_ld32(taddr + ch * 32, v);
-        const int gi = (G == 128) ? 0 : (ch >> 1);
-        const int e0 = (G == 128) ? ch * 32 : (ch & 1) * 32;
+        for (int ch = 0; ch < 4; ++ch) {
+          tc_ld32(taddr + ch * 32, v);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float av = fabsf(v[e]);
-          if (av > best[gi]) { best[gi] = av; bval[gi] = v[e]; bidx[gi] = e0 + e; }
-          sq = fmaf(v[e], v[e], sq);
+          for (int e = 0; e < 32; ++e) sq = fmaf(v[e], v[e], sq);
+        }
+        sq_local += valid ? (double)sq : 0.0;
+      } else {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          tc_ld32(taddr + ch * 32, v);
+          const int gi = (G == 128) ? 0 : (ch >> 1);
+          const int e0 = (G == 128) ? ch * 32 : (ch & 1) * 32;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float av = fabsf(v[e]);
+            if (av > best[gi]) { best[gi] = av; bval[gi] = v[e]; bidx[gi] = e0 + e; }
+          }
         }
       }
-      if (p.epi & EPI_SQSUM) sq_local += valid ? (double)sq : 0.0;
       if (p.epi & (EPI_ABSMAX | EPI_DELTA | EPI_CODES)) {
 #pragma unroll
         for (int gi = 0; gi < NG; ++gi)
@@ -367,6 +397,16 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
         if (p.epi & EPI_SURR) {
           float surf = 0.f;
+          if constexpr (FORM == BD_OUT) {
+            // the run of tiles moved on to another row block: hand over what this thread summed for its old row
+            if (valid && srow_row >= 0 && srow_row != row) {
+              if (srow != 0.f) {
+                const int Bq = srow_row / K;
+                atomicAdd(&p.Aacc[(Bq / p.r) * K + (srow_row - Bq * K)], (float)G * srow);
+              }
+              srow = 0.f;
+            }
+          }
 #pragma unroll
           for (int gi = 0; gi < NG; ++gi) {
             const int Gc = col0 / G + gi;
@@ -525,11 +565,10 @@ static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMa
     p.n_major = p.d_out / K;
     p.n_minor = (p.d_in + C::NC - 1) / C::NC;
   }
-  int cpm = 148 / p.n_major;
-  if (cpm < 1) cpm = 1;
-  if (cpm > p.n_minor) cpm = p.n_minor;
-  p.ctas_per_major = cpm;
-  bd_pass_kernel<FORM, K, G><<<p.n_major * cpm, BD_THREADS, C::SMEM, st>>>(tmX, tmT, p);
+  const long long total = (long long)p.n_major * p.n_minor;
+  const int grid = total < 148 ? (int)total : 148;  // one persistent CTA per SM
+  p.ctas_per_major = 0;
+  bd_pass_kernel<FORM, K, G><<<grid, BD_THREADS, C::SMEM, st>>>(tmX, tmT, p);
   return CAFEQ_OK;
 }
 
