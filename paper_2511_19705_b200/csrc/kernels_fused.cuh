@@ -142,6 +142,31 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// The same load without the wait, and a wait that names the destination registers so that no use of them can be
+// scheduled ahead of it: lets the load of the next 32 columns overlap the arithmetic on the current ones.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tc_ld_wait32(float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 bytes apart.
 // K-major operands step along K by moving the start address inside the swizzled row; MN-major operands
 // step along K by whole 8-row groups.
@@ -361,26 +386,57 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       for (int gi = 0; gi < NG; ++gi) { best[gi] = -1.f; bval[gi] = 0.f; bidx[gi] = 0; }
       if (p.epi == EPI_SQSUM) {
         // sum of squares only (second pass of the l2 proxy)
-        float sq = 0.f;
+        float sq4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           tc_ld32(taddr + ch * 32, v);
 #pragma unroll
-          for (int e = 0; e < 32; ++e) sq = fmaf(v[e], v[e], sq);
+          for (int e = 0; e < 32; ++e) sq4[e & 3] = fmaf(v[e], v[e], sq4[e & 3]);
         }
-        sq_local += valid ? (double)sq : 0.0;
+        sq_local += valid ? (double)((sq4[0] + sq4[1]) + (sq4[2] + sq4[3])) : 0.0;
       } else {
+        // group absmax with arg-max: four independent running candidates per group (columns e mod 4), merged at
+        // the end with the lowest index winning ties; the next 32 columns are in flight while these are compared
+        float v2[32];
+        float bv[NG][4], nz[4] = {0.f, 0.f, 0.f, 0.f};
+        int bi[NG][4];
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) { bv[gi][c] = 0.f; bi[gi][c] = 0; }
+        tc_ld32_issue(taddr, v);
+        tc_ld_wait32(v);
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
-          tc_ld32(taddr + ch * 32, v);
+          float* cur = (ch & 1) ? v2 : v;
+          float* nxt = (ch & 1) ? v : v2;
+          if (ch < 3) tc_ld32_issue(taddr + (ch + 1) * 32, nxt);
           const int gi = (G == 128) ? 0 : (ch >> 1);
           const int e0 = (G == 128) ? ch * 32 : (ch & 1) * 32;
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const float av = fabsf(v[e]);
-            if (av > best[gi]) { best[gi] = av; bval[gi] = v[e]; bidx[gi] = e0 + e; }
+            const int c = e & 3;
+            if (fabsf(cur[e]) > fabsf(bv[gi][c])) { bv[gi][c] = cur[e]; bi[gi][c] = e0 + e; }
+            nz[c] = fmaf(cur[e], 0.f, nz[c]);  // stays 0 unless a NaN or an infinity passes by
           }
+          if (ch < 3) tc_ld_wait32(nxt);
         }
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) {
+          float b = bv[gi][0];
+          int ix = bi[gi][0];
+#pragma unroll
+          for (int c = 1; c < 4; ++c) {
+            const float x = bv[gi][c];
+            const int jx = bi[gi][c];
+            const bool take = (fabsf(x) > fabsf(b)) || (fabsf(x) == fabsf(b) && jx < ix);
+            if (take) { b = x; ix = jx; }
+          }
+          best[gi] = fabsf(b);
+          bval[gi] = b;
+          bidx[gi] = ix;
+        }
+        if (valid && !((nz[0] + nz[1]) + (nz[2] + nz[3]) == 0.f)) bad = true;
       }
       if (p.epi & (EPI_ABSMAX | EPI_DELTA | EPI_CODES)) {
 #pragma unroll
