@@ -362,11 +362,6 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
       const int major = tile / p.n_minor, t = tile - major * p.n_minor;
       const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
-      ok = mbar_wait(bar_accf + 8 * buf, aph, abort_flag, p.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256u + hw * 128u;
       int row, col0;
       if constexpr (FORM == BD_IN) {
         row = t * 128 + L;
@@ -378,6 +373,20 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         row = major * 128 + L;
         col0 = t * 256 + hw * 128;
       }
+      // Eq. 4 weights of this thread's groups, requested before the wait for the accumulator so that the
+      // global-memory latency is hidden behind it
+      float wgt[NG];
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) wgt[gi] = 0.f;
+      if ((p.epi & EPI_SURR) && row < p.d_out && col0 < p.d_in) {
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) wgt[gi] = (FORM == BD_IN) ? __ldg(p.cw + col0 / G + gi) : __ldg(p.cw + row);
+      }
+      ok = mbar_wait(bar_accf + 8 * buf, aph, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256u + hw * 128u;
       const bool valid = (row < p.d_out) && (col0 < p.d_in);
       float v[32];
       float best[NG], bval[NG];
@@ -467,11 +476,10 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           for (int gi = 0; gi < NG; ++gi) {
             const int Gc = col0 / G + gi;
             const float av = valid ? best[gi] : 0.f;
-            const float wgt = valid ? ((FORM == BD_IN) ? p.cw[Gc] : p.cw[row]) : 0.f;
-            surf = fmaf(wgt * av, av, surf);
+            surf = fmaf(wgt[gi] * av, av, surf);
             if (valid && p.coef) {
               const float sg = (bval[gi] > 0.f) ? 1.f : ((bval[gi] < 0.f) ? -1.f : 0.f);
-              p.coef[(long long)row * ng_row + Gc] = 2.f * p.kappa * wgt * av * sg;
+              p.coef[(long long)row * ng_row + Gc] = 2.f * p.kappa * wgt[gi] * av * sg;
             }
             if constexpr (FORM == BD_IN) {
               float a2 = av * av;
