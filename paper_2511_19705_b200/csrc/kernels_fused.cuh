@@ -447,6 +447,15 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
         if (valid && !((nz[0] + nz[1]) + (nz[2] + nz[3]) == 0.f)) bad = true;
       }
+      // Without a second pass over the accumulator (codes / residual) everything still needed is in registers:
+      // hand the buffer back to the tensor cores now.  The arrive has release semantics, so issuing it after the
+      // global stores below would make every tile wait for those stores to land.
+      const bool early_release = (p.epi & (EPI_DELTA | EPI_CODES)) == 0;
+      if (early_release) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+      }
       if (p.epi & (EPI_ABSMAX | EPI_DELTA | EPI_CODES)) {
 #pragma unroll
         for (int gi = 0; gi < NG; ++gi)
@@ -532,9 +541,11 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+      if (!early_release) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+      }
     }
     if (p.epi & EPI_SQSUM) {
       for (int o = 16; o > 0; o >>= 1) sq_local += __shfl_xor_sync(0xffffffffu, sq_local, o);
