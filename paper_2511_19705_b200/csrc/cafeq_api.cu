@@ -388,8 +388,9 @@ static void launch_absmax(cudaStream_t st, const float* U, long long ld, const G
   CQ_LAUNCH(absmax_kernel, (unsigned)blocks, 256, 0, st, U, ld, G.d_out, G.ng, G.g, a, usel, idx, status);
 }
 
+// gm: the (row, group) records are group-major (written by the fused pass) instead of row-major
 static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const float* coef, const int* idx, float* gT,
-                           int transpose_out, const int32_t* status) {
+                           int transpose_out, const int32_t* status, int gm) {
   const int k = G.k;
   int ti = kt_begin(2, st);
   const bool aligned = ((uintptr_t)W % 4 == 0) && (G.ld % 2 == 0);
@@ -417,7 +418,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     }
 #define SC_INB(KV)                                                                                                         \
   CQ_LAUNCH(scatter_in_bucket_kernel<KV>, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, G.r, nG, coef, idx, gT, \
-            transpose_out, rows_per, status)
+            transpose_out, rows_per, status, gm)
     if (k == 64) SC_INB(64);
     else if (k == 128) SC_INB(128);
     else SC_INB(256);
@@ -444,7 +445,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     const size_t sh = (size_t)k * SC2_JS * 4;
 #define SC_IN(NGV)                                                                                                       \
   CQ_LAUNCH(scatter_in_strip_kernel<NGV>, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, \
-            gT, transpose_out, rows_per, status)
+            gT, transpose_out, rows_per, status, gm)
     if (nG == 1) SC_IN(1);
     else if (nG == 2) SC_IN(2);
     else SC_IN(4);
@@ -462,7 +463,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     const size_t sh = (size_t)2 * SC2_JS * (G.g + 4) * 2;
 #define SC_OUT(KV)                                                                                                      \
   CQ_LAUNCH(scatter_out_strip_kernel<KV>, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, G.r, coef, idx, gT, \
-            transpose_out, per, status)
+            transpose_out, per, status, gm)
     if (k == 64) SC_OUT(64);
     else if (k == 128) SC_OUT(128);
     else SC_OUT(256);
@@ -484,7 +485,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     splits = (G.d_out + rows_per - 1) / rows_per;
     dim3 grid(G.nbq, strips, splits);
     CQ_LAUNCH(scatter_in_kernel, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
-                                             transpose_out, rows_per, status);
+                                             transpose_out, rows_per, status, gm);
   } else {
     int want = (148 * 4) / (G.nbq * strips) + 1;
     int splits = want < 1 ? 1 : want;
@@ -493,7 +494,7 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     splits = (G.ng + per - 1) / per;
     dim3 grid(G.nbq, strips, splits);
     CQ_LAUNCH(scatter_out_kernel, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, k, G.r, coef, idx, gT,
-                                              transpose_out, per, status);
+                                              transpose_out, per, status, gm);
   }
   kt_end(ti, st);
 }
@@ -809,7 +810,7 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   CQ_LAUNCH(finalize_single_kernel, 1, 1, 0, st, s.acc, losses, hist, need_l2 ? 1 : 0);
   if (!want_grad) return;
   if (!ste) {
-    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
+    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status, fused ? 1 : 0);
     CQ_LAUNCH(gminv_kernel, grid_for(kk), 256, 0, st, s.Minv, s.A, in_r1 ? s.m.agrp : nullptr, G.g, 2.f * kappa, k, kk, s.gMinv);
   } else {
     // gMinv = 2 * sum_free E Delta^T ; gDelta = 2 Minv^T o E (overwrites Delta) ; scale path through arg-max
@@ -818,7 +819,7 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
     launch_apply(st, s.m.E, 0, G.d_in, G, s.Minv, 1, s.m.D, G.d_in, GEMM_STORE, nullptr, status, 2.f);
     CQ_LAUNCH(ste_scale_path_kernel, (unsigned)(((long long)G.d_out * G.ng * 32 + 255) / 256), 256, 0, st, 
         s.m.U, s.m.D, G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.usel, qm, offsets, off_kind, G.d_in, s.m.coef, status);
-    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status);
+    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status, 0);
   }
   // gradM -= Minv^T gMinv Minv^T
   if (tc) {
@@ -980,9 +981,9 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   else launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, p.Minv, p.Minv_c, kk, status);
   // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
-  forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
+  const bool f1 = forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
                 nullptr, status, !force_generic);
-  forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
+  const bool f2 = forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
                 nullptr, nullptr, status, !force_generic);
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
   CQ_LAUNCH(max_f32_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, status);
@@ -1026,9 +1027,9 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
   CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
   // U side: operator is M^T, so the block gradient is stored transposed
-  launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status);
+  launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status, f1 ? 1 : 0);
   // V side: gradient with respect to Minv, then through the inverse
-  launch_scatter(st, W2, G2, p.m2.coef, p.m2.idx, p.gMinv, 0, status);
+  launch_scatter(st, W2, G2, p.m2.coef, p.m2.idx, p.gMinv, 0, status, f2 ? 1 : 0);
   if (tc) {
     minv_path_tc(st, p.gMinv, gradM, G1.nbT, k, true, p.kk, status);
   } else {

@@ -32,7 +32,8 @@ struct BdParams {
   int ctas_per_major;
   int epi;
   float qmax;
-  float* a;            // [d_out, d_in / G] group absmax
+  // per (row, group) records are stored GROUP-MAJOR: index = group * d_out + row
+  float* a;            // [d_in / G, d_out] group absmax
   float* usel;         // signed value at the arg-max
   int* idx;            // arg-max position inside the group
   uint16_t* delta;     // bf16 [d_out, d_in], row stride d_in
@@ -42,8 +43,9 @@ struct BdParams {
   // EPI_SURR: Eq. 4 evaluated per entry inside the pass
   const float* cw;     // input axis: sum of c_t over each column group [d_in / G]; output axis: G * c_t per row [d_out]
   float kappa;
-  float* coef;         // [d_out, d_in / G] backward coefficient 2 kappa cw a sign(U at arg-max); may be null
+  float* coef;         // [d_in / G, d_out] (group-major) backward coefficient 2 kappa cw a sign(U at arg-max); may be null
   double* lossacc;     // += kappa * sum cw a^2
+  int a_always;        // write the maxima and their signed values even in EPI_SURR mode
   float* Aacc;         // input axis: [d_in / G] += a^2 per column group; output axis: [nbT * k] += G * sum_G a^2 per operator row
   int32_t* status;
 };
@@ -461,11 +463,17 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         for (int gi = 0; gi < NG; ++gi)
           if (valid && !(best[gi] <= 3.0e38f)) bad = true;
         if (valid && (p.epi & EPI_ABSMAX)) {
+          // with Eq. 4 evaluated right here nothing downstream reads the maxima or their signs: the backward only
+          // needs (arg-max index, coefficient).  Every scattered 4-byte store is a partial-sector write at L2.
+          const bool need_a = !(p.epi & EPI_SURR) || p.a_always;
 #pragma unroll
           for (int gi = 0; gi < NG; ++gi) {
-            const long long w = (long long)row * ng_row + (col0 / G + gi);
-            p.a[w] = best[gi];
-            p.usel[w] = bval[gi];
+            // group-major records: consecutive rows of one group are contiguous, so a warp's store is one line
+            const long long w = (long long)(col0 / G + gi) * p.d_out + row;
+            if (need_a) {
+              p.a[w] = best[gi];
+              p.usel[w] = bval[gi];
+            }
             p.idx[w] = bidx[gi];
           }
         }
@@ -488,7 +496,7 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             surf = fmaf(wgt[gi] * av, av, surf);
             if (valid && p.coef) {
               const float sg = (bval[gi] > 0.f) ? 1.f : ((bval[gi] < 0.f) ? -1.f : 0.f);
-              p.coef[(long long)row * ng_row + Gc] = 2.f * p.kappa * wgt[gi] * av * sg;
+              p.coef[(long long)Gc * p.d_out + row] = 2.f * p.kappa * wgt[gi] * av * sg;
             }
             if constexpr (FORM == BD_IN) {
               float a2 = av * av;

@@ -483,7 +483,7 @@ constexpr int SCATTER_JS = 32;
 __global__ void __launch_bounds__(256) scatter_in_kernel(const uint16_t* __restrict__ W, long long ld, int d_out, int d_in,
                                                          int g, int k, int r, const float* __restrict__ coef,
                                                          const int* __restrict__ idx, float* __restrict__ gradT,
-                                                         int transpose_out, int rows_per_cta, const int32_t* status) {
+                                                         int transpose_out, int rows_per_cta, const int32_t* status, int gm) {
   if (status && *status) return;
   extern __shared__ float acc[];  // [k][SCATTER_JS]
   const int B = blockIdx.x, js = blockIdx.y * SCATTER_JS;
@@ -498,7 +498,7 @@ __global__ void __launch_bounds__(256) scatter_in_kernel(const uint16_t* __restr
   for (int o = r0 + warp; o < r1; o += nw) {
     float w = (j < k) ? bf16_bits_to_float(W[o * ld + (long long)B * k + j]) : 0.f;
     for (int G = G0; G <= G1; ++G) {
-      long long p = (long long)o * ng + G;
+      long long p = gm ? (long long)G * d_out + o : (long long)o * ng + G;
       int col = G * g + idx[p];          // arg-max column of the group
       if (col < B * k || col >= B * k + k) continue;  // group larger than the block: arg-max in another block
       float cf = coef[p];
@@ -516,7 +516,7 @@ __global__ void __launch_bounds__(256) scatter_in_kernel(const uint16_t* __restr
 __global__ void __launch_bounds__(256) scatter_out_kernel(const uint16_t* __restrict__ W, long long ld, int d_out, int d_in,
                                                           int g, int k, int r, const float* __restrict__ coef,
                                                           const int* __restrict__ idx, float* __restrict__ gradT,
-                                                          int transpose_out, int groups_per_cta, const int32_t* status) {
+                                                          int transpose_out, int groups_per_cta, const int32_t* status, int gm) {
   if (status && *status) return;
   extern __shared__ float acc[];  // [k][SCATTER_JS]
   const int B = blockIdx.x, js = blockIdx.y * SCATTER_JS;
@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(256) scatter_out_kernel(const uint16_t* __rest
     float s = 0.f;
     long long row = (long long)B * k + i;
     for (int G = G0; G < G1; ++G) {
-      long long p = row * ng + G;
+      long long p = gm ? (long long)G * d_out + row : row * ng + G;
       float cf = coef[p];
       if (cf != 0.f) s = fmaf(cf, bf16_bits_to_float(W[((long long)B * k + j) * ld + (long long)G * g + idx[p]]), s);
     }
@@ -564,7 +564,7 @@ template <int NG>
 __global__ void __launch_bounds__(256, 3) scatter_in_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
                                                                   int d_in, int g, int k, int r, const float* __restrict__ coef,
                                                                   const int* __restrict__ idx, float* __restrict__ gradT,
-                                                                  int transpose_out, int rows_per_cta, const int32_t* status) {
+                                                                  int transpose_out, int rows_per_cta, const int32_t* status, int gm) {
   if (status && *status) return;
   extern __shared__ float acc[];  // [k][64]
   const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
@@ -584,11 +584,12 @@ __global__ void __launch_bounds__(256, 3) scatter_in_strip_kernel(const uint16_t
     {
       const int o = base + lane;
       const bool ok = o < r1;
-      const long long p = (long long)(ok ? o : r0) * ng + G0;
+      const int oo = ok ? o : r0;
 #pragma unroll
       for (int q = 0; q < NG; ++q) {
-        const int ix = __ldg(idx + p + q);
-        const float c = __ldg(coef + p + q);
+        const long long pq = gm ? (long long)(G0 + q) * d_out + oo : (long long)oo * ng + G0 + q;
+        const int ix = __ldg(idx + pq);
+        const float c = __ldg(coef + pq);
         const int col = q * g + ix + off;
         const bool in = ok && (unsigned)col < (unsigned)k;
         cf[q] = in ? c : 0.f;
@@ -638,7 +639,7 @@ template <int K>
 __global__ void __launch_bounds__(256, 2) scatter_in_bucket_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
                                                                    int d_in, int g, int r, int NG, const float* __restrict__ coef,
                                                                    const int* __restrict__ idx, float* __restrict__ gradT,
-                                                                   int transpose_out, int rows_per_cta, const int32_t* status) {
+                                                                   int transpose_out, int rows_per_cta, const int32_t* status, int gm) {
   if (status && *status) return;
   constexpr int TPB = 256 / K;   // threads per bucket
   constexpr int CPT = 64 / TPB;  // strip columns per thread
@@ -668,7 +669,7 @@ __global__ void __launch_bounds__(256, 2) scatter_in_bucket_kernel(const uint16_
     cfv[u] = 0.f;
     if (e < np) {
       const int row = e / NG, q = e - row * NG;
-      const long long p = (long long)(r0 + row) * ng + G0 + q;
+      const long long p = gm ? (long long)(G0 + q) * d_out + r0 + row : (long long)(r0 + row) * ng + G0 + q;
       const float c = __ldg(coef + p);
       const int col = q * g + __ldg(idx + p) + off;
       if ((unsigned)col < (unsigned)K && c != 0.f) {
@@ -764,7 +765,7 @@ template <int K>
 __global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
                                                                 int d_in, int g, int r, const float* __restrict__ coef,
                                                                 const int* __restrict__ idx, float* __restrict__ gradT,
-                                                                int transpose_out, int groups_per_cta, const int32_t* status) {
+                                                                int transpose_out, int groups_per_cta, const int32_t* status, int gm) {
   if (status && *status) return;
   constexpr int RW = K / 8;  // rows of the block per warp
   extern __shared__ __align__(16) uint16_t tiles[];  // two tiles [64][g + 4]
@@ -787,7 +788,7 @@ __global__ void __launch_bounds__(256) scatter_out_strip_kernel(const uint16_t* 
       cp_async8(tile + jr * tp + 4 * c4, src + jr * ld + 4 * c4);
     }
     for (int i = tid; i < K; i += 256) {
-      const long long p = ((long long)B * K + i) * ng + G;
+      const long long p = gm ? (long long)G * d_out + (long long)B * K + i : ((long long)B * K + i) * ng + G;
       cp_async4(&s_cf[buf][i], coef + p);
       cp_async4(&s_ix[buf][i], idx + p);
     }
