@@ -181,6 +181,17 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
   return d;
 }
 
+// Same, for an MN-major operand that spans several 64-element swizzle atoms along MN: `lbo_bytes` is the distance
+// between consecutive atoms.
+__device__ __forceinline__ uint64_t umma_desc_sw128_lbo(uint32_t saddr, uint32_t lbo_bytes) {
+  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
   return (1u << 4) /* fp32 accumulate */ | (1u << 7) /* A bf16 */ | (1u << 10) /* B bf16 */ |
          ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
@@ -196,7 +207,8 @@ struct BdCfg {
   static constexpr int T_BYTES = NBLK * K * K * 2;
   static constexpr int KH = (K >= 128) ? K / 128 : 1;                 // OUT: 128-row halves of the block
   static constexpr int NC = 256 / KH;                                 // OUT: d_in columns per tile
-  static constexpr int NSTAGE = (T_BYTES >= 131072) ? 5 : 6;
+  static constexpr int NCC = NC / 64;                                 // OUT: 64-column chunks per tile
+  static constexpr int NSTAGE = 6;                                    // even: the output-axis form consumes stages in pairs
   static constexpr int SMEM = 1024 + T_BYTES + NSTAGE * BD_STAGE_BYTES + 256;
 };
 
@@ -288,7 +300,7 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             x = major * 256 + sidx * 64;
             y = t * 128;
           } else {
-            const int nc = sidx / C::KH, kh = sidx % C::KH;
+            const int kh = sidx / C::NCC, nc = sidx % C::NCC;  // the chunks of one row half are consecutive stages
             x = t * C::NC + nc * 64;
             y = major * K + kh * 128;
           }
@@ -303,7 +315,7 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       int cur_major = -1;
       uint32_t tfulls = 0;
       constexpr uint32_t idesc_in = umma_idesc_bf16(128, K, 0, 0);
-      constexpr uint32_t idesc_out = umma_idesc_bf16(128, 64, 0, 1);
+      constexpr uint32_t idesc_out = umma_idesc_bf16(128, 128, 0, 1);
       const uint32_t sT_u = smem_u32(sT), sSt_u = smem_u32(sStage);
       uint32_t it = 0, tl = 0;
       for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
@@ -317,12 +329,12 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         if (!mbar_wait(bar_acce + 8 * buf, aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t dbase = tmem_base + buf * 256u;
-        for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
-          const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
-          if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
-          if constexpr (FORM == BD_IN) {
+        if constexpr (FORM == BD_IN) {
+          for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
+            const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
             const int bi = (sidx * 64) / K, ci = ((sidx * 64) % K) / 64;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
@@ -330,19 +342,30 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
               const uint64_t bd = umma_desc_sw128(sT_u + bi * K * K * 2 + ci * K * 128 + kk * 32);
               tc_mma_bf16(dbase + bi * K, ad, bd, idesc_in, (ci | kk) != 0 ? 1u : 0u);
             }
-          } else {
-            const int nc = sidx / C::KH, kh = sidx % C::KH;
+            tc_commit(bar_empty + 8 * s);
+          }
+        } else {
+          // two consecutive stages = two 64-column chunks of the same 128 weight rows: one N = 128 product, the
+          // second swizzle atom of the MN-major operand one stage further on
+          for (int sidx = 0; sidx < BD_STAGES_PER_TILE; sidx += 2, it += 2) {
+            const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait(bar_full + 8 * (s + 1), ph, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
+            const int kh = sidx / C::NCC, nc = sidx % C::NCC;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-              const uint64_t bd = umma_desc_sw128(stage + ks * 2048);
+              const uint64_t bd = umma_desc_sw128_lbo(stage + ks * 2048, BD_STAGE_BYTES);
 #pragma unroll
               for (int mh = 0; mh < C::KH; ++mh) {
                 const uint64_t ad = umma_desc_sw128(sT_u + (kh * 2 + ks / 4) * K * 128 + mh * 128 * 128 + (ks % 4) * 32);
                 tc_mma_bf16(dbase + mh * C::NC + nc * 64, ad, bd, idesc_out, (kh | ks) != 0 ? 1u : 0u);
               }
             }
+            tc_commit(bar_empty + 8 * s);
+            tc_commit(bar_empty + 8 * (s + 1));
           }
-          tc_commit(bar_empty + 8 * s);
         }
         if (ok) tc_commit(bar_accf + 8 * buf);
         // last tile of this major with more to come: signal when its products are done with the operator block
