@@ -397,10 +397,12 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
   const int nG = (k >= G.g) ? k / G.g : 1;  // groups of one row inside one block (g | k or k | g on this path)
   if (kk_fast(k) && G.axis == CAFEQ_AXIS_IN && (k % G.g == 0 || G.g % k == 0) && nG <= 8 && ((uintptr_t)W % 16 == 0) &&
       (G.ld % 8 == 0)) {
-    const int strips = k / SC2_JS;
+    // 8 strip columns per thread at least: strip 32 at k = 256 (one thread per target row), 64 otherwise
+    const int strip = (k == 256) ? 32 : 64;
+    const int strips = k / strip;
     int rows_per = SCB_MAXP / nG;
     if (rows_per > 2048) rows_per = 2048;
-    // enough CTAs to fill the machine twice over, but never more rows than the record buffer holds
+    // enough CTAs to fill the machine a few times over, but never more rows than the record buffer holds
     int want = (148 * 4 + G.nbq * strips - 1) / (G.nbq * strips);
     int rp2 = (G.d_out + want - 1) / want;
     rp2 = ((rp2 + 31) / 32) * 32;
@@ -408,20 +410,20 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     if (rows_per < 32) rows_per = 32;
     const int splits = (G.d_out + rows_per - 1) / rows_per;
     dim3 grid(G.nbq, strips, splits);
-    const size_t sh = (size_t)k * 65 * 4 + (size_t)SCB_MAXP * 6;
+    const size_t sh = (size_t)k * (strip + 1) * 4 + (size_t)SCB_MAXP * 6;
     static bool attr = false;
     if (!attr) {
-      cudaFuncSetAttribute(scatter_in_bucket_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 65 * 4 + SCB_MAXP * 6);
-      cudaFuncSetAttribute(scatter_in_bucket_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 65 * 4 + SCB_MAXP * 6);
-      cudaFuncSetAttribute(scatter_in_bucket_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 65 * 4 + SCB_MAXP * 6);
+      cudaFuncSetAttribute(scatter_in_bucket_kernel<256, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 33 * 4 + SCB_MAXP * 6);
+      cudaFuncSetAttribute(scatter_in_bucket_kernel<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 65 * 4 + SCB_MAXP * 6);
+      cudaFuncSetAttribute(scatter_in_bucket_kernel<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 65 * 4 + SCB_MAXP * 6);
       attr = true;
     }
-#define SC_INB(KV)                                                                                                         \
-  CQ_LAUNCH(scatter_in_bucket_kernel<KV>, grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, G.r, nG, coef, idx, gT, \
-            transpose_out, rows_per, status, gm)
-    if (k == 64) SC_INB(64);
-    else if (k == 128) SC_INB(128);
-    else SC_INB(256);
+#define SC_INB(KV, SV)                                                                                                   \
+  CQ_LAUNCH((scatter_in_bucket_kernel<KV, SV>), grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, G.r, nG, coef, \
+            idx, gT, transpose_out, rows_per, status, gm)
+    if (k == 64) SC_INB(64, 64);
+    else if (k == 128) SC_INB(128, 64);
+    else SC_INB(256, 32);
 #undef SC_INB
     kt_end(ti, st);
     return;
@@ -969,27 +971,43 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
 static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
                       const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
                       float* losses, float* hist, float* gradM, int32_t* status, PairWS& p, bool force_generic,
-                      bool warm = false) {
+                      bool warm = false, float* step_counter = nullptr) {
   const int k = G1.k;
   const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G1.nbT * k * k;
   const float sqrt_h = sqrtf((float)G1.d_out);
-  CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, p.acc, 8);
-  CQ_LAUNCH(fill_f32_kernel, 1, 32, 0, st, p.amax, 0.f, 1);
-  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, p.Mc, kk, status);
-  if (tc) ns_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, warm, p.kk, status);
-  else launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
+  if (tc) {
+    PrepArgs pa;
+    memset(&pa, 0, sizeof(pa));
+    pa.M = M; pa.Mc = p.Mc; pa.Ab = p.kk.Ab; pa.kk = kk;
+    pa.zero_f[0] = p.amax; pa.zero_fn[0] = 1;
+    if (gradM) {
+      pa.zero_f[1] = gradM; pa.zero_fn[1] = kk;
+      pa.zero_f[2] = p.gMinv; pa.zero_fn[2] = kk;
+    }
+    pa.zero_d[0] = p.acc; pa.zero_dn[0] = 8;
+    pa.zero_d[1] = p.kk.rn; pa.zero_dn[1] = NS_MAX_ITERS * G1.nbT;
+    pa.flag = p.kk.flag;
+    pa.step_counter = step_counter;
+    pa.status = status;
+    CQ_LAUNCH(step_prep_kernel, grid_for(kk), 256, 0, st, pa);
+    ns_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, warm, p.kk, status, true);
+  } else {
+    CQ_LAUNCH(zero_f64_kernel, 1, 32, 0, st, p.acc, 8);
+    CQ_LAUNCH(fill_f32_kernel, 1, 32, 0, st, p.amax, 0.f, 1);
+    CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, p.Mc, kk, status);
+    if (step_counter) CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, step_counter, status);
+    launch_inverse(st, p.Mc, p.Minv, nullptr, G1.nbT, k, status);
+  }
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, p.Minv, p.Minv_c, kk, status);
   // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
   const bool f1 = forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
                 nullptr, status, !force_generic);
   const bool f2 = forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
-                nullptr, nullptr, status, !force_generic);
+                nullptr, nullptr, status, !force_generic, nullptr, tc ? p.kk.Xh[p.kk.cur] : nullptr);  // Xh = bf16(Minv)
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
-  CQ_LAUNCH(max_f32_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, status);
-  CQ_LAUNCH(max_f32_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.amax, status);
-  CQ_LAUNCH(sumexp_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.amax, t, p.acc + 0, status);
-  CQ_LAUNCH(sumexp_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.amax, t, p.acc + 0, status);
+  CQ_LAUNCH(max2_f32_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, n1, p.m2.a, n2, p.amax, status);
+  CQ_LAUNCH(sumexp2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, n1, p.m2.a, n2, p.amax, t, p.acc + 0, status);
   // orthonormality penalty on the fp32 parameters: R = M M^T - I
   if (tc) {
     // R = M M^T - I (symmetric) with its bf16 splits, ||R||_F^2, and R M for the gradient
@@ -1020,12 +1038,12 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   }
   CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, want_pqe ? 1 : 0);
   if (!gradM) return;
-  CQ_LAUNCH(lse_coef_kernel, grid_for(n1), 256, 0, st, p.m1.a, p.m1.usel, n1, p.amax, t, p.acc + 0,
-                                                p.m1.coef, status);
-  CQ_LAUNCH(lse_coef_kernel, grid_for(n2), 256, 0, st, p.m2.a, p.m2.usel, n2, p.amax, t, p.acc + 0,
-                                                p.m2.coef, status);
-  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
-  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
+  CQ_LAUNCH(lse_coef2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, p.m1.usel, p.m1.coef, n1, p.m2.a, p.m2.usel, p.m2.coef, n2,
+            p.amax, t, p.acc + 0, status);
+  if (!tc) {
+    CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
+    CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
+  }
   // U side: operator is M^T, so the block gradient is stored transposed
   launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status, f1 ? 1 : 0);
   // V side: gradient with respect to Minv, then through the inverse
@@ -1109,22 +1127,20 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   const long long kk = (long long)G1.nbT * G1.k * G1.k;
   float* grad = b.take<float>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  // the inverse of the last step's transform lives in the optimiser state, so a resumed run refines it
   const bool resume = cfg->resume && opt_state;
-  if (resume) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, opt_state + 1 + 2 * kk, p.Minv, kk);
+  if (opt_state) p.Minv = opt_state + 1 + 2 * kk;
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = any_pqe && (it % cfg->eval_every == 0);
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
-              grad, status, p, false, resume || it > 0);
+              grad, status, p, false, resume || it > 0, opt_state);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
-      if (opt_state) CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
-      CQ_LAUNCH(adam_tick_kernel, 1, 1, 0, st, opt_state, status);
       CQ_LAUNCH(adam_update_kernel, grid_for(kk), 256, 0, st, M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,
                                                        status);
     }
   }
-  if (opt_state && cfg->steps > 0) CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, p.Minv, opt_state + 1 + 2 * kk, kk);
   return last_launch();
 }
 

@@ -635,21 +635,22 @@ __global__ void __launch_bounds__(256, 3) scatter_in_strip_kernel(const uint16_t
 // K in {64, 128, 256}; rows_per_cta * NG <= SCB_MAXP; ld % 8 == 0 and W 16-byte aligned.
 constexpr int SCB_MAXP = 4096;
 
-template <int K>
+template <int K, int STRIP>
 __global__ void __launch_bounds__(256, 2) scatter_in_bucket_kernel(const uint16_t* __restrict__ W, long long ld, int d_out,
                                                                    int d_in, int g, int r, int NG, const float* __restrict__ coef,
                                                                    const int* __restrict__ idx, float* __restrict__ gradT,
                                                                    int transpose_out, int rows_per_cta, const int32_t* status, int gm) {
   if (status && *status) return;
-  constexpr int TPB = 256 / K;   // threads per bucket
-  constexpr int CPT = 64 / TPB;  // strip columns per thread
+  constexpr int TPB = 256 / K;      // threads per bucket
+  constexpr int CPT = STRIP / TPB;  // strip columns per thread
+  constexpr int SP = STRIP + 1;     // padded row of the staging buffer
   constexpr int RPT = SCB_MAXP / 256;
   extern __shared__ __align__(16) uint8_t sc_smem[];
-  float* stage = reinterpret_cast<float*>(sc_smem);                       // [K][65]
-  float* rec_cf = stage + K * 65;                                         // [SCB_MAXP]
+  float* stage = reinterpret_cast<float*>(sc_smem);                       // [K][STRIP + 1]
+  float* rec_cf = stage + K * SP;                                         // [SCB_MAXP]
   uint16_t* rec_o = reinterpret_cast<uint16_t*>(rec_cf + SCB_MAXP);       // [SCB_MAXP]
   __shared__ int cnt[K], start[K + 1], cursor[K], wsum[8];
-  const int B = blockIdx.x, js = blockIdx.y * SC2_JS;
+  const int B = blockIdx.x, js = blockIdx.y * STRIP;
   const int r0 = blockIdx.z * rows_per_cta, r1 = min(d_out, r0 + rows_per_cta);
   const int R = r1 - r0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -717,14 +718,19 @@ __global__ void __launch_bounds__(256, 2) scatter_in_bucket_kernel(const uint16_
   for (int c = 0; c < CPT; ++c) acc[c] = 0.f;
   const uint16_t* Wb = W + (long long)r0 * ld + (long long)B * K + js + part * CPT;
   const int p1 = start[b + 1];
-  for (int p = start[b]; p < p1; ++p) {
-    const float cf = rec_cf[p];
+  // the row segment of the next record is requested before the current one is accumulated (two register sets)
+  constexpr int NV = CPT / 8;
+  uint4 wa[NV], wb[NV];
+  float cfa = 0.f, cfb = 0.f;
+  auto fetch = [&](int p, uint4* w, float& cf) {
+    cf = rec_cf[p];
     const uint4* src = reinterpret_cast<const uint4*>(Wb + (long long)rec_o[p] * ld);
-    uint4 w[CPT / 8];
 #pragma unroll
-    for (int v = 0; v < CPT / 8; ++v) w[v] = __ldg(src + v);
+    for (int v = 0; v < NV; ++v) w[v] = __ldg(src + v);
+  };
+  auto accumulate = [&](const uint4* w, float cf) {
 #pragma unroll
-    for (int v = 0; v < CPT / 8; ++v) {
+    for (int v = 0; v < NV; ++v) {
       const uint32_t ww[4] = {w[v].x, w[v].y, w[v].z, w[v].w};
 #pragma unroll
       for (int h = 0; h < 4; ++h) {
@@ -732,14 +738,24 @@ __global__ void __launch_bounds__(256, 2) scatter_in_bucket_kernel(const uint16_
         acc[v * 8 + 2 * h + 1] = fmaf(cf, __uint_as_float(ww[h] & 0xFFFF0000u), acc[v * 8 + 2 * h + 1]);
       }
     }
+  };
+  int p = start[b];
+  if (p < p1) fetch(p, wa, cfa);
+  while (p < p1) {
+    if (p + 1 < p1) fetch(p + 1, wb, cfb);
+    accumulate(wa, cfa);
+    if (++p >= p1) break;
+    if (p + 1 < p1) fetch(p + 1, wa, cfa);
+    accumulate(wb, cfb);
+    ++p;
   }
 #pragma unroll
-  for (int c = 0; c < CPT; ++c) stage[b * 65 + part * CPT + c] = acc[c];
+  for (int c = 0; c < CPT; ++c) stage[b * SP + part * CPT + c] = acc[c];
   __syncthreads();
   float* out = gradT + (size_t)(B / r) * K * K;
-  for (int e = tid; e < K * SC2_JS; e += 256) {
-    const int i = e / SC2_JS, c = e - i * SC2_JS;
-    const float v = stage[i * 65 + c];
+  for (int e = tid; e < K * STRIP; e += 256) {
+    const int i = e / STRIP, c = e - i * STRIP;
+    const float v = stage[i * SP + c];
     if (v != 0.f) atomicAdd(transpose_out ? &out[(size_t)(js + c) * K + i] : &out[(size_t)i * K + js + c], v);
   }
 }
@@ -1004,6 +1020,49 @@ __global__ void lse_coef_kernel(const float* __restrict__ a, const float* __rest
     float u = usel[w];
     float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
     coef[w] = expf(t * (a[w] - mx)) * zinv * sgn;
+  }
+}
+
+// two-array forms of the three LogSumExp kernels (the group maxima of U and of V in one launch each)
+__global__ void max2_f32_kernel(const float* __restrict__ a1, long long n1, const float* __restrict__ a2, long long n2,
+                                float* __restrict__ out_max, const int32_t* status) {
+  if (status && *status) return;
+  float m = 0.f;
+  const long long n = n1 + n2;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    m = fmaxf(m, i < n1 ? a1[i] : a2[i - n1]);
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) atomicMax((int*)out_max, __float_as_int(m));
+}
+
+__global__ void sumexp2_kernel(const float* __restrict__ a1, long long n1, const float* __restrict__ a2, long long n2,
+                               const float* __restrict__ amax, float t, double* __restrict__ acc, const int32_t* status) {
+  if (status && *status) return;
+  __shared__ double red[32];
+  const float mx = *amax;
+  double local = 0.0;
+  const long long n = n1 + n2;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    local += (double)expf(t * ((i < n1 ? a1[i] : a2[i - n1]) - mx));
+  double s = block_sum_double(local, red);
+  if (threadIdx.x == 0) atomicAdd(acc, s);
+}
+
+__global__ void lse_coef2_kernel(const float* __restrict__ a1, const float* __restrict__ u1, float* __restrict__ c1, long long n1,
+                                 const float* __restrict__ a2, const float* __restrict__ u2, float* __restrict__ c2, long long n2,
+                                 const float* __restrict__ amax, float t, const double* __restrict__ Z, const int32_t* status) {
+  if (status && *status) return;
+  const float mx = *amax;
+  const float zinv = (float)(1.0 / *Z);
+  const long long n = n1 + n2;
+  for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < n; w += (long long)gridDim.x * blockDim.x) {
+    const bool first = w < n1;
+    const long long i = first ? w : w - n1;
+    const float u = first ? u1[i] : u2[i];
+    const float av = first ? a1[i] : a2[i];
+    const float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
+    const float c = expf(t * (av - mx)) * zinv * sgn;
+    if (first) c1[i] = c; else c2[i] = c;
   }
 }
 
