@@ -154,25 +154,27 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
         const int nb0 = n0 + ch * 32;
         if (nb0 >= p.N) break;
         const bool inner = (nb0 + 32 <= p.N) && (m0 + 128 <= p.M);  // no edge in this chunk: no per-element checks
-        const bool full = rv && (nb0 + 32 <= p.N);
-        const float* c0p = p.C0 ? p.C0 + c0b + (long long)row * p.ldc0 + nb0 : nullptr;
-        const bool c0vec = full && c0p && ((p.ldc0 & 3) == 0) && (((uintptr_t)c0p & 15) == 0);
-        if (c0vec) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            const float4 c4 = *reinterpret_cast<const float4*>(c0p + e);
-            v[e] = fmaf(p.beta, c4.x, p.alpha * v[e]);
-            v[e + 1] = fmaf(p.beta, c4.y, p.alpha * v[e + 1]);
-            v[e + 2] = fmaf(p.beta, c4.z, p.alpha * v[e + 2]);
-            v[e + 3] = fmaf(p.beta, c4.w, p.alpha * v[e + 3]);
+        // Row-major global traffic goes through a per-warp 32 x 32 tile in shared memory (the stage buffers are
+        // free once the accumulator is complete): in the accumulator a lane owns a ROW, and 32 lanes reading or
+        // writing 32 different rows of a matrix whose pitch is a power of two all land on one cache set; with a
+        // lane per COLUMN every access is one contiguous line.
+        float* tile = reinterpret_cast<float*>(smem + (warp - 2) * 4352);  // [32][33]
+        const int rbase = m0 + q * 32;
+        const int ncol = nb0 + lane;
+        if (p.C0) {
+#pragma unroll 8
+          for (int r = 0; r < 32; ++r) {
+            float x = 0.f;
+            if (inner || (rbase + r < p.M && ncol < p.N)) x = p.C0[c0b + (long long)(rbase + r) * p.ldc0 + ncol];
+            tile[r * 33 + lane] = x;
           }
+          __syncwarp();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = fmaf(p.beta, tile[lane * 33 + e], p.alpha * v[e]);
+          __syncwarp();
         } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            float x = p.alpha * v[e];
-            if (c0p && rv && nb0 + e < p.N) x = fmaf(p.beta, c0p[e], x);
-            v[e] = x;
-          }
+          for (int e = 0; e < 32; ++e) v[e] = p.alpha * v[e];
         }
         if (p.gamma != 0.f && row >= nb0 && row < nb0 + 32) {
 #pragma unroll
@@ -191,68 +193,35 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
           }
           sq += (double)sqf;
         }
-        if (p.C && rv) {
-          float* dst = p.C + cb + (long long)row * p.ldc + nb0;
-          if (full && ((p.ldc & 3) == 0) && (((uintptr_t)dst & 15) == 0)) {
+        if (p.C || p.Chi) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-          } else {
-            for (int e = 0; e < 32; ++e)
-              if (nb0 + e < p.N) dst[e] = v[e];
+          for (int e = 0; e < 32; ++e) tile[lane * 33 + e] = v[e];
+          __syncwarp();
+#pragma unroll 8
+          for (int r = 0; r < 32; ++r) {
+            const float x = tile[r * 33 + lane];
+            if (inner || (rbase + r < p.M && ncol < p.N)) {
+              if (p.C) p.C[cb + (long long)(rbase + r) * p.ldc + ncol] = x;
+              if (p.Chi) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(x);
+                const long long o = sb_mn + (long long)(rbase + r) * p.N + ncol;
+                p.Chi[o] = __bfloat16_as_ushort(h);
+                if (p.Clo) p.Clo[o] = __bfloat16_as_ushort(__float2bfloat16_rn(x - __bfloat162float(h)));
+              }
+            }
           }
+          __syncwarp();
         }
-        if (p.Chi || p.Cthi) {
-          uint32_t hp[16], lp[16];
+        if (p.Cthi && rv) {
+          // transposed outputs: consecutive lanes are consecutive rows = consecutive addresses
+          uint16_t* cth = p.Cthi + sb_mn + (long long)nb0 * p.M + row;
+          uint16_t* ctl = p.Ctlo ? p.Ctlo + sb_mn + (long long)nb0 * p.M + row : nullptr;
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const __nv_bfloat16 h0 = __float2bfloat16_rn(v[e]), h1 = __float2bfloat16_rn(v[e + 1]);
-            const __nv_bfloat16 l0 = __float2bfloat16_rn(v[e] - __bfloat162float(h0));
-            const __nv_bfloat16 l1 = __float2bfloat16_rn(v[e + 1] - __bfloat162float(h1));
-            hp[e >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-            lp[e >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-          }
-          const long long ro = sb_mn + (long long)row * p.N + nb0;
-          const bool rvec = full && ((p.N & 7) == 0);
-          if (p.Chi && rv) {
-            if (rvec) {
-#pragma unroll
-              for (int w4 = 0; w4 < 4; ++w4)
-                *reinterpret_cast<uint4*>(p.Chi + ro + 8 * w4) = make_uint4(hp[4 * w4], hp[4 * w4 + 1], hp[4 * w4 + 2], hp[4 * w4 + 3]);
-            } else {
-              for (int e = 0; e < 32; ++e)
-                if (nb0 + e < p.N) p.Chi[ro + e] = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
-            }
-          }
-          if (p.Clo && rv) {
-            if (rvec) {
-#pragma unroll
-              for (int w4 = 0; w4 < 4; ++w4)
-                *reinterpret_cast<uint4*>(p.Clo + ro + 8 * w4) = make_uint4(lp[4 * w4], lp[4 * w4 + 1], lp[4 * w4 + 2], lp[4 * w4 + 3]);
-            } else {
-              for (int e = 0; e < 32; ++e)
-                if (nb0 + e < p.N) p.Clo[ro + e] = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
-            }
-          }
-          if (p.Cthi && rv) {
-            uint16_t* ct = p.Cthi + sb_mn + (long long)nb0 * p.M + row;
-            if (inner) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e, ct += p.M) *ct = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e, ct += p.M)
-                if (nb0 + e < p.N) *ct = (uint16_t)(hp[e >> 1] >> ((e & 1) * 16));
-            }
-          }
-          if (p.Ctlo && rv) {
-            uint16_t* ct = p.Ctlo + sb_mn + (long long)nb0 * p.M + row;
-            if (inner) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e, ct += p.M) *ct = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e, ct += p.M)
-                if (nb0 + e < p.N) *ct = (uint16_t)(lp[e >> 1] >> ((e & 1) * 16));
+          for (int e = 0; e < 32; ++e) {
+            if (inner || nb0 + e < p.N) {
+              const __nv_bfloat16 h = __float2bfloat16_rn(v[e]);
+              cth[(long long)e * p.M] = __bfloat16_as_ushort(h);
+              if (ctl) ctl[(long long)e * p.M] = __bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h)));
             }
           }
         }
