@@ -162,12 +162,14 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
         const int rbase = m0 + q * 32;
         const int ncol = nb0 + lane;
         if (p.C0) {
-#pragma unroll 8
-          for (int r = 0; r < 32; ++r) {
-            float x = 0.f;
-            if (inner || (rbase + r < p.M && ncol < p.N)) x = p.C0[c0b + (long long)(rbase + r) * p.ldc0 + ncol];
-            tile[r * 33 + lane] = x;
+          float c0v[32];
+#pragma unroll
+          for (int r = 0; r < 32; ++r) {  // all 32 row loads in flight together
+            c0v[r] = 0.f;
+            if (inner || (rbase + r < p.M && ncol < p.N)) c0v[r] = __ldg(p.C0 + c0b + (long long)(rbase + r) * p.ldc0 + ncol);
           }
+#pragma unroll
+          for (int r = 0; r < 32; ++r) tile[r * 33 + lane] = c0v[r];
           __syncwarp();
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = fmaf(p.beta, tile[lane * 33 + e], p.alpha * v[e]);
@@ -197,31 +199,73 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) tile[lane * 33 + e] = v[e];
           __syncwarp();
+          if (p.C) {
 #pragma unroll 8
-          for (int r = 0; r < 32; ++r) {
-            const float x = tile[r * 33 + lane];
-            if (inner || (rbase + r < p.M && ncol < p.N)) {
-              if (p.C) p.C[cb + (long long)(rbase + r) * p.ldc + ncol] = x;
-              if (p.Chi) {
-                const __nv_bfloat16 h = __float2bfloat16_rn(x);
-                const long long o = sb_mn + (long long)(rbase + r) * p.N + ncol;
-                p.Chi[o] = __bfloat16_as_ushort(h);
-                if (p.Clo) p.Clo[o] = __bfloat16_as_ushort(__float2bfloat16_rn(x - __bfloat162float(h)));
+            for (int r = 0; r < 32; ++r) {
+              const float x = tile[r * 33 + lane];
+              if (inner || (rbase + r < p.M && ncol < p.N)) p.C[cb + (long long)(rbase + r) * p.ldc + ncol] = x;
+            }
+          }
+          if (p.Chi) {
+            if (inner && (p.N & 1) == 0) {
+              // two rows per instruction, two columns per lane: 32-bit stores (2-byte stores serialise badly)
+#pragma unroll 4
+              for (int r2 = 0; r2 < 32; r2 += 2) {
+                const int rr = r2 + (lane >> 4), cc = (lane & 15) * 2;
+                const float x0 = tile[rr * 33 + cc], x1 = tile[rr * 33 + cc + 1];
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+                const long long o = sb_mn + (long long)(rbase + rr) * p.N + nb0 + cc;
+                *reinterpret_cast<uint32_t*>(p.Chi + o) = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                if (p.Clo) {
+                  const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+                  const __nv_bfloat16 l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+                  *reinterpret_cast<uint32_t*>(p.Clo + o) = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                }
+              }
+            } else {
+              for (int r = 0; r < 32; ++r) {
+                const float x = tile[r * 33 + lane];
+                if (rbase + r < p.M && ncol < p.N) {
+                  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+                  const long long o = sb_mn + (long long)(rbase + r) * p.N + ncol;
+                  p.Chi[o] = __bfloat16_as_ushort(h);
+                  if (p.Clo) p.Clo[o] = __bfloat16_as_ushort(__float2bfloat16_rn(x - __bfloat162float(h)));
+                }
               }
             }
           }
           __syncwarp();
         }
-        if (p.Cthi && rv) {
+        if (p.Cthi) {
           // transposed outputs: consecutive lanes are consecutive rows = consecutive addresses
-          uint16_t* cth = p.Cthi + sb_mn + (long long)nb0 * p.M + row;
-          uint16_t* ctl = p.Ctlo ? p.Ctlo + sb_mn + (long long)nb0 * p.M + row : nullptr;
+          if (inner && (p.M & 1) == 0) {
+            // neighbouring lanes trade one value so that every lane stores a 32-bit pair of rows: even lanes
+            // write column e, odd lanes column e + 1
+            const int odd = lane & 1;
+            const long long rowpair = row & ~1;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            if (inner || nb0 + e < p.N) {
-              const __nv_bfloat16 h = __float2bfloat16_rn(v[e]);
-              cth[(long long)e * p.M] = __bfloat16_as_ushort(h);
-              if (ctl) ctl[(long long)e * p.M] = __bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h)));
+            for (int e = 0; e < 32; e += 2) {
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(v[e]), h1 = __float2bfloat16_rn(v[e + 1]);
+              const uint32_t p0 = (uint32_t)__bfloat16_as_ushort(h0) |
+                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h0))) << 16);
+              const uint32_t p1 = (uint32_t)__bfloat16_as_ushort(h1) |
+                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e + 1] - __bfloat162float(h1))) << 16);
+              const uint32_t mine = odd ? p1 : p0;                       // (hi | lo << 16) of my row in the column I store
+              const uint32_t other = __shfl_xor_sync(0xffffffffu, odd ? p0 : p1, 1);  // the neighbour row's, same column
+              const uint32_t lo_row = odd ? other : mine, hi_row = odd ? mine : other;  // rows (2j, 2j + 1)
+              const long long o = sb_mn + (long long)(nb0 + e + odd) * p.M + rowpair;
+              *reinterpret_cast<uint32_t*>(p.Cthi + o) = (lo_row & 0xFFFFu) | (hi_row << 16);
+              if (p.Ctlo) *reinterpret_cast<uint32_t*>(p.Ctlo + o) = (lo_row >> 16) | (hi_row & 0xFFFF0000u);
+            }
+          } else if (rv) {
+            uint16_t* cth = p.Cthi + sb_mn + (long long)nb0 * p.M + row;
+            uint16_t* ctl = p.Ctlo ? p.Ctlo + sb_mn + (long long)nb0 * p.M + row : nullptr;
+            for (int e = 0; e < 32; ++e) {
+              if (nb0 + e < p.N) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(v[e]);
+                cth[(long long)e * p.M] = __bfloat16_as_ushort(h);
+                if (ctl) ctl[(long long)e * p.M] = __bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h)));
+              }
             }
           }
         }
