@@ -315,9 +315,13 @@ static int tg_launch_t(cudaStream_t st, const TgOperand* A, const TgOperand* B, 
 // K must be a multiple of 64; operands 16-byte aligned with pitches that are multiples of 8 elements.
 static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, const TgParams& p) {
   if (p.K % TG_BK || p.nterms < 1 || p.nterms > TG_MAX_TERMS) return CAFEQ_ERR_UNSUPPORTED;
-  if (p.N <= 64) return tg_launch_t<64>(st, A, B, p);
-  if (p.N <= 128 || (p.batch > 1 && p.N <= 256 && p.batch * ((p.M + 127) / 128) < 74)) return tg_launch_t<128>(st, A, B, p);
-  return tg_launch_t<256>(st, A, B, p);
+  // widest tile that still gives about one CTA per SM: these products are small, and a CTA's life is dominated
+  // by its epilogue (one accumulator row per thread), so more, narrower tiles finish sooner
+  const long long mt = (long long)p.batch * ((p.M + 127) / 128);
+  if (p.N > 128 && mt * ((p.N + 255) / 256) >= 96) return tg_launch_t<256>(st, A, B, p);
+  if (p.N > 64 && mt * ((p.N + 127) / 128) >= 96) return tg_launch_t<128>(st, A, B, p);
+  if (p.N <= 64 || mt * ((p.N + 127) / 128) < 96) return tg_launch_t<64>(st, A, B, p);
+  return tg_launch_t<128>(st, A, B, p);
 }
 
 // fp32 blocks [nb][k][k] -> bf16 hi / lo splits in row-major and transposed order; one 32 x 32 tile per CTA
