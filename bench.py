@@ -34,6 +34,22 @@ METRIC = "proxy-loss fwd+bwd steps/s (Gemma2-9B-shaped layer)"
 UNIT = "steps/s"
 
 
+def profiled_traffic():
+    """DRAM bytes per launch of the transform pass from the committed ncu summary, or None once the kernel source
+    differs from the one that was profiled."""
+    import hashlib
+    import re
+    try:
+        txt = open(os.path.join(ROOT, "profiles", "bd_pass_9b_layer.md")).read()
+        src = open(os.path.join(ROOT, "paper_2511_19705_b200", "csrc", "kernels_fused.cuh"), "rb").read()
+        sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]+)", txt).group(1)
+        if hashlib.sha256(src).hexdigest() != sha:
+            return None
+        return float(re.search(r"traffic_bytes_per_launch:\s*([0-9.e+]+)", txt).group(1))
+    except Exception:
+        return None
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -310,6 +326,10 @@ def main():
             ach = byts / t_pass / 1e9
             roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
                         traffic=None)
+        tb = profiled_traffic()
+        roof["traffic"] = tb
+        roof["traffic_note"] = "ncu dram bytes read+written per launch (mean over the 7 launches of a step)" if tb else None
+        roof["algorithmic_bytes_per_launch"] = byts / (len(tp) / args.steps)
         roof.update(kernel=names[tk], peak_source=peaks["source"] + (" sustained" if roof["bound"] == "tensor" else ""),
                     launches_per_step=len(tp) / args.steps, avg_launch_ms=sum(tp) / len(tp),
                     algorithmic_gb_per_step=byts / 1e9, algorithmic_tflop_per_step=flops / 1e12,
