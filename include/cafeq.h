@@ -172,7 +172,11 @@ int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, const cafeq_
  * M is [h/k, k, k].
  *   P       optional fp32 [d1, d3] from cafeq_pair_product; needed for PQE.
  *   losses  out fp32[4]: {LSE + lambda*orth, LSE, orth penalty, PQE^2 (Eq. 5 squared) or 0}.
- *   gradM   out [h/k, k, k]. */
+ *   gradM   out [h/k, k, k].
+ * loss_kind CAFEQ_LOSS_LSE is the surrogate of App. D.  CAFEQ_LOSS_PQE_STE differentiates Eq. 5 squared itself with
+ * the quantiser passed straight through (only the scale's dependence on its group's arg-max entry is kept): P is
+ * required, losses[0] = losses[3] = PQE^2, lambda_orth is ignored (losses[2] = 0), and every dimension must be
+ * a multiple of 64 with k a multiple of 32 (CAFEQ_ERR_UNSUPPORTED otherwise); its products run on the tensor cores. */
 int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
                             const void* W2, const float* M, const float* P, int loss_kind, float lse_t,
                             float lambda_orth, int flags, float* losses, float* gradM, int32_t* status,

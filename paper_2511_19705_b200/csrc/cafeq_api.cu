@@ -971,7 +971,7 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
 static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
                       const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
                       float* losses, float* hist, float* gradM, int32_t* status, PairWS& p, bool force_generic,
-                      bool warm = false, float* step_counter = nullptr) {
+                      bool warm = false, float* step_counter = nullptr, bool ste = false) {
   const int k = G1.k;
   const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G1.nbT * k * k;
@@ -1008,8 +1008,9 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
   CQ_LAUNCH(max2_f32_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, n1, p.m2.a, n2, p.amax, status);
   CQ_LAUNCH(sumexp2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, n1, p.m2.a, n2, p.amax, t, p.acc + 0, status);
-  // orthonormality penalty on the fp32 parameters: R = M M^T - I
-  if (tc) {
+  // orthonormality penalty on the fp32 parameters: R = M M^T - I (not part of the straight-through PQE loss)
+  if (ste) {
+  } else if (tc) {
     // R = M M^T - I (symmetric) with its bf16 splits, ||R||_F^2, and R M for the gradient
     KkWS& w = p.kk;
     launch_split(st, M, k, kk, w.Ph, w.Pl, w.Qh, w.Ql, nullptr, status);
@@ -1030,14 +1031,59 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   }
   if (want_pqe && p.dense) {
     // Eq. 5 on the tensor cores: || Uhat_exp^T Vhat^T - P ||_F^2 with three-term bf16 splits of the dequantised values
-    dense_pqe(st, p.m1.E, p.m2.E, P, p.dn, p.acc + 2, nullptr, status);
+    dense_pqe(st, p.m1.E, p.m2.E, P, p.dn, p.acc + 2, nullptr, status, ste);
   } else if (want_pqe) {
     launch_pair_product(st, p.m1.E, 0, G1.d_in, p.m2.E, 0, G2.d_in, G1, G2, p.R, status);
     CQ_LAUNCH(resid_sq_kernel, grid_for((long long)G1.d_in * G2.d_out), 256, 0, st, p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
                                                                              status);
   }
-  CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, want_pqe ? 1 : 0);
+  CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, ste ? 2 : (want_pqe ? 1 : 0));
   if (!gradM) return;
+  if (ste) {
+    // Straight-through gradient of ||Uhat_exp^T Vhat^T - P||_F^2 (Eq. 5 squared): the residual R [d1, d3] and
+    // its transpose are in p.dn.Ph/Pl/PTh/PTl; the quantiser passes gradients through except for its scale,
+    // whose dependence on the group's arg-max entry is kept.
+    DenseWS& w = p.dn;
+    {  // g Vhat' [d3, h] = 2 R^T Uhat^T, then one copy per replica of every inner block
+      launch_split_rect(st, p.m1.E, w.h, w.d1, w.d1, 1.f, nullptr, nullptr, nullptr, w.Awh, w.Awl, nullptr, nullptr, status);
+      const uint16_t* a[3] = {w.PTh, w.PTl, w.PTh};
+      const uint16_t* b[3] = {w.Awh, w.Awh, w.Awl};
+      DenseOut o;
+      o.C = w.X0T; o.ldc = w.h;
+      launch_dense_tc(st, 3, a, b, w.d3, w.h, w.d1, 2.f, 0.f, 0.f, o, status);
+      CQ_LAUNCH(expand_cols_kernel, grid_for((long long)w.d3 * w.rh), 256, 0, st, w.X0T, w.d3, w.h, w.k, w.r, 1.f, w.V);
+    }
+    {  // g Uhat [h, d1] = 2 fold(Vhat^T) R^T
+      dim3 grid((w.d3 + 31) / 32, w.h / 32);
+      CQ_LAUNCH(fold_transpose_kernel, grid, dim3(32, 8), 0, st, p.m2.E, w.d3, w.h, w.k, w.r, w.Bf);
+      launch_split_rect(st, w.Bf, w.h, w.d3, w.d3, 1.f, nullptr, nullptr, nullptr, w.Yh, w.Yl, nullptr, nullptr, status);
+      const uint16_t* a[3] = {w.Yh, w.Yl, w.Yh};
+      const uint16_t* b[3] = {w.Ph, w.Ph, w.Pl};
+      DenseOut o;
+      o.C = w.U; o.ldc = w.d1;
+      launch_dense_tc(st, 3, a, b, w.h, w.d1, w.d3, 2.f, 0.f, 0.f, o, status);
+    }
+    const long long n1w = (long long)G1.d_out * G1.ng, n2w = (long long)G2.d_out * G2.ng;
+    CQ_LAUNCH(ste_scale_path_kernel, (unsigned)((n1w * 32 + 255) / 256), 256, 0, st, p.m1.U, w.U, G1.d_in, G1.d_out, G1.ng, G1.g,
+              p.m1.a, p.m1.usel, qmax_of(d1->bits), nullptr, CAFEQ_OFFSETS_NONE, G1.d_in, p.m1.coef, status);
+    CQ_LAUNCH(add_argmax_kernel, grid_for(n1w), 256, 0, st, w.U, G1.d_in, G1.d_out, G1.ng, G1.g, p.m1.coef, p.m1.idx, status);
+    CQ_LAUNCH(ste_scale_path_kernel, (unsigned)((n2w * 32 + 255) / 256), 256, 0, st, p.m2.U, w.V, G2.d_in, G2.d_out, G2.ng, G2.g,
+              p.m2.a, p.m2.usel, qmax_of(d2->bits), nullptr, CAFEQ_OFFSETS_NONE, G2.d_in, p.m2.coef, status);
+    CQ_LAUNCH(add_argmax_kernel, grid_for(n2w), 256, 0, st, w.V, G2.d_in, G2.d_out, G2.ng, G2.g, p.m2.coef, p.m2.idx, status);
+    if (!tc) {
+      CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
+      CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
+    }
+    launch_opgrad(st, w.U, G1.d_in, W1, 1, G1.ld, G1, gradM, 1, 1.f, status);    // U side: operator M^T
+    launch_opgrad(st, w.V, G2.d_in, W2, 1, G2.ld, G2, p.gMinv, 0, 1.f, status);  // V side: operator Minv
+    if (tc) {
+      minv_path_tc(st, p.gMinv, gradM, G1.nbT, k, true, p.kk, status);
+    } else {
+      launch_kk(st, p.Minv, 1, p.gMinv, 0, p.RM, G1.nbT, k, 1.f, GEMM_STORE, status);
+      launch_kk(st, p.RM, 0, p.Minv, 1, gradM, G1.nbT, k, -1.f, GEMM_STORE | GEMM_ACCUM, status);
+    }
+    return;
+  }
   CQ_LAUNCH(lse_coef2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, p.m1.usel, p.m1.coef, n1, p.m2.a, p.m2.usel, p.m2.coef, n2,
             p.amax, t, p.acc + 0, status);
   if (!tc) {
@@ -1091,11 +1137,12 @@ extern "C" int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* 
   int rc = make_pair_geo(d1, d2, &G1, &G2);
   if (rc) return rc;
   if (!W1 || !W2 || !M || !losses) return CAFEQ_ERR_INVALID_ARG;
-  if (loss_kind == CAFEQ_LOSS_PQE_STE) return CAFEQ_ERR_UNSUPPORTED;
-  if (loss_kind != CAFEQ_LOSS_LSE) return CAFEQ_ERR_INVALID_ARG;
+  const bool ste = loss_kind == CAFEQ_LOSS_PQE_STE;
+  if (!ste && loss_kind != CAFEQ_LOSS_LSE) return CAFEQ_ERR_INVALID_ARG;
+  if (ste && !dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;
   if (!(lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
   const bool want_grad = !(flags & CAFEQ_FLAG_NO_GRAD);
-  const bool want_pqe = (flags & CAFEQ_FLAG_EXACT_LOSS) != 0;
+  const bool want_pqe = ste || (flags & CAFEQ_FLAG_EXACT_LOSS) != 0;
   if (want_grad && !gradM) return CAFEQ_ERR_INVALID_ARG;
   if (want_pqe && !P) return CAFEQ_ERR_INVALID_ARG;
   if ((rc = check_ws(ws, ws_bytes))) return rc;
@@ -1103,7 +1150,7 @@ extern "C" int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* 
   PairWS p;
   if (!carve_pair(b, G1, G2, &p, want_pqe)) return CAFEQ_ERR_WORKSPACE;
   pair_step((cudaStream_t)stream, d1, d2, G1, G2, W1, W2, M, P, lse_t, lambda_orth, want_pqe, losses, nullptr,
-            want_grad ? gradM : nullptr, status, p, (flags & CAFEQ_FLAG_GENERIC) != 0);
+            want_grad ? gradM : nullptr, status, p, (flags & CAFEQ_FLAG_GENERIC) != 0, false, nullptr, ste);
   return last_launch();
 }
 
@@ -1114,13 +1161,15 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   int rc = make_pair_geo(d1, d2, &G1, &G2);
   if (rc) return rc;
   if (!W1 || !W2 || !M || !cfg || cfg->struct_size != sizeof(cafeq_opt_cfg) || !loss_history) return CAFEQ_ERR_INVALID_ARG;
-  if (cfg->loss_kind == CAFEQ_LOSS_PQE_STE) return CAFEQ_ERR_UNSUPPORTED;
-  if (cfg->loss_kind != CAFEQ_LOSS_LSE || cfg->steps < 0 || !(cfg->lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
+  const bool ste = cfg->loss_kind == CAFEQ_LOSS_PQE_STE;
+  if ((!ste && cfg->loss_kind != CAFEQ_LOSS_LSE) || cfg->steps < 0 || !(cfg->lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
+  if (ste && !P) return CAFEQ_ERR_INVALID_ARG;
+  if (ste && !dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;
   if (cfg->optimizer == CAFEQ_OPT_ADAM && !opt_state) return CAFEQ_ERR_INVALID_ARG;
   if (cfg->optimizer != CAFEQ_OPT_ADAM && cfg->optimizer != CAFEQ_OPT_GD) return CAFEQ_ERR_INVALID_ARG;
   if ((rc = check_ws(ws, ws_bytes))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  const bool any_pqe = (P != nullptr) && cfg->eval_every > 0;
+  const bool any_pqe = ste || ((P != nullptr) && cfg->eval_every > 0);
   Bump b(ws, ws_bytes);
   PairWS p;
   if (!carve_pair(b, G1, G2, &p, any_pqe)) return CAFEQ_ERR_WORKSPACE;
@@ -1131,9 +1180,9 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   const bool resume = cfg->resume && opt_state;
   if (opt_state) p.Minv = opt_state + 1 + 2 * kk;
   for (int it = 0; it < cfg->steps; ++it) {
-    bool eval = any_pqe && (it % cfg->eval_every == 0);
+    bool eval = ste || (any_pqe && (it % cfg->eval_every == 0));
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
-              grad, status, p, false, resume || it > 0, opt_state);
+              grad, status, p, false, resume || it > 0, opt_state, ste);
     if (cfg->optimizer == CAFEQ_OPT_GD) {
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {

@@ -100,10 +100,10 @@ __global__ void __launch_bounds__(256) fold_transpose_kernel(const float* __rest
   }
 }
 
-// V[y][(B*r + rep)*k + j] = X[y][B*k + j] / r  (X fp32 [d3, h] -> V fp32 [d3, r*h])
-__global__ void expand_cols_kernel(const float* __restrict__ X, int d3, int h, int k, int r, float* __restrict__ V) {
+// V[y][(B*r + rep)*k + j] = scale * X[y][B*k + j]  (X fp32 [d3, h] -> V fp32 [d3, r*h])
+__global__ void expand_cols_kernel(const float* __restrict__ X, int d3, int h, int k, int r, float scale, float* __restrict__ V) {
   const long long n = (long long)d3 * r * h;
-  const float inv = 1.f / (float)r;
+  const float inv = scale;
   for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
     const long long y = e / ((long long)r * h);
     const int l = (int)(e - y * (long long)r * h);
@@ -125,6 +125,19 @@ __global__ void pinv_control_kernel(const double* __restrict__ sq, int it, doubl
 }
 
 __global__ void set_int_kernel(int* p, int v) { *p = v; }
+
+// gX[row][G*g + idx[row, G]] += coef[row, G]: the scale path of the straight-through quantiser lands on the
+// arg-max entry of its group (records row-major)
+__global__ void add_argmax_kernel(float* __restrict__ gX, long long ld, int rows, int ng, int g, const float* __restrict__ coef,
+                                  const int* __restrict__ idx, const int32_t* status) {
+  if (status && *status) return;
+  const long long n = (long long)rows * ng;
+  for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < n; w += (long long)gridDim.x * blockDim.x) {
+    const long long row = w / ng;
+    const int G = (int)(w - row * ng);
+    gX[row * ld + (long long)G * g + idx[w]] += coef[w];
+  }
+}
 
 __global__ void sqrt_hist_kernel(const double* __restrict__ sq, float* __restrict__ out, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;

@@ -1116,14 +1116,16 @@ __global__ void finalize_pair_kernel(const double* acc, const float* amax, float
                                      float* losses, float* hist, int want_pqe) {
   float lse = *amax + (float)(log(acc[0]) / (double)t);
   float orth = (float)(sqrt(acc[1]) / (double)sqrt_h);
+  // want_pqe == 2: the squared product error is the loss being minimised (straight-through mode)
+  const float loss = (want_pqe == 2) ? (float)acc[2] : lse + lambda * orth;
   if (losses) {
-    losses[0] = lse + lambda * orth;
+    losses[0] = loss;
     losses[1] = lse;
     losses[2] = orth;
     losses[3] = want_pqe ? (float)acc[2] : 0.f;
   }
   if (hist) {
-    hist[0] = lse + lambda * orth;
+    hist[0] = loss;
     hist[1] = want_pqe ? (float)acc[2] : nanf("");
   }
 }

@@ -181,13 +181,16 @@ static void dense_product(cudaStream_t st, const float* U, const float* V, Dense
 
 // *sq += || Uhat_exp^T Vhat^T - P ||_F^2 ; optionally stores the residual R [d1, d3]
 static void dense_pqe(cudaStream_t st, const float* Uhat, const float* Vhat, const float* P, DenseWS& w, double* sq, float* R,
-                      int32_t* status) {
+                      int32_t* status, bool keep_splits = false) {
   launch_split_rect(st, Uhat, w.h, w.d1, w.d1, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.UTh, w.UTl, status);
   launch_split_rect(st, Vhat, w.d3, w.rh, w.rh, 1.f, nullptr, nullptr, nullptr, w.Vh, w.Vl, nullptr, nullptr, status);
   const uint16_t* a[3] = {w.UTh, w.UTl, w.UTh};
   const uint16_t* b[3] = {w.Vh, w.Vh, w.Vl};
   DenseOut o;
   o.C0 = P; o.ldc0 = w.d3; o.C = R; o.ldc = w.d3; o.sq = sq;
+  if (keep_splits) {  // the residual and its transpose as operands of the backward products
+    o.Chi = w.Ph; o.Clo = w.Pl; o.Cthi = w.PTh; o.Ctlo = w.PTl;
+  }
   launch_dense_tc(st, 3, a, b, w.d1, w.d3, w.rh, 1.f, -1.f, 0.f, o, status, w.k, w.r);
 }
 
@@ -212,7 +215,7 @@ static void alg1_run(cudaStream_t st, int bits, int g1, int g2, int iters, int8_
       o.C = w.X0T; o.ldc = w.h;
       launch_dense_tc(st, 3, a, b, w.d3, w.h, w.d1, 1.f, 0.f, 0.f, o, status);
     }
-    CQ_LAUNCH(expand_cols_kernel, grid_for((long long)w.d3 * w.rh), 256, 0, st, w.X0T, w.d3, w.h, w.k, w.r, w.V);
+    CQ_LAUNCH(expand_cols_kernel, grid_for((long long)w.d3 * w.rh), 256, 0, st, w.X0T, w.d3, w.h, w.k, w.r, 1.f / (float)w.r, w.V);
     quant_matrix(st, w.V, w.d3, w.rh, g2, bits, codes2, scales2, w.Vhat, w, status);
     dense_pqe(st, w.Uhat, w.Vhat, w.P, w, w.sq + 2 * it + 1, nullptr, status);
     // U side: U' [h, d1] = pinv(Bf)^T P^T with Bf = fold(Vhat^T) [h, d3]
