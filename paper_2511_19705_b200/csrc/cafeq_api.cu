@@ -13,6 +13,7 @@
 #include "cafeq.h"
 #include "kernels_generic.cuh"
 #include "kernels_fused.cuh"
+#include "kernels_bwd.cuh"
 #include "kernels_gemm.cuh"
 
 namespace cafeq {
@@ -393,6 +394,21 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
                            int transpose_out, const int32_t* status, int gm) {
   const int k = G.k;
   int ti = kt_begin(2, st);
+  // block sizes 128 / 256: a dense product on the tensor cores whose left operand holds the routed coefficients
+  if (bw_supported(G.axis == CAFEQ_AXIS_IN, G.d_out, G.d_in, G.ld, k, G.g, W)) {
+    BwParams bp;
+    memset(&bp, 0, sizeof(bp));
+    bp.d_out = G.d_out; bp.d_in = G.d_in; bp.g = G.g; bp.ng = G.ng; bp.r = G.r;
+    bp.gm = gm; bp.transpose_out = transpose_out;
+    bp.coef = coef; bp.idx = idx; bp.gradT = gT;
+    bp.status = const_cast<int32_t*>(status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (bw_launch(st, G.axis == CAFEQ_AXIS_IN, k, W, G.ld, bp) == CAFEQ_OK) {
+      kt_end(ti, st);
+      return;
+    }
+    g_launches.fetch_sub(1, std::memory_order_relaxed);
+  }
   const bool aligned = ((uintptr_t)W % 4 == 0) && (G.ld % 2 == 0);
   const int nG = (k >= G.g) ? k / G.g : 1;  // groups of one row inside one block (g | k or k | g on this path)
   if (kk_fast(k) && G.axis == CAFEQ_AXIS_IN && (k % G.g == 0 || G.g % k == 0) && nG <= 8 && ((uintptr_t)W % 16 == 0) &&

@@ -1,0 +1,396 @@
+// Sparse backward of the transform pass on the tensor cores (tcgen05, sm_100a).
+//
+// Every (row, group) record of the forward pass carries a coefficient (dLoss / d group maximum, signed) and the
+// position of the group's arg-max entry.  The gradient with respect to an operator block is a sum of outer
+// products routed through those entries (Section 4.1: the group maximum is the only path from the transform
+// to Eq. 4; App. D: the same for the LogSumExp surrogate):
+//   input axis : gradT[B][i][j] = sum_o S[o][i] W[o, B k + j],   S[o][i] = coef(o, G) where i is the arg-max column of (o, G)
+//   output axis: gradT[B][i][j] = sum_c S[i][c] W[B k + j, c],   S[i][c] = coef(B k + i, G(c)) where c is its arg-max column
+// i.e. a dense k x k product whose left operand has one non-zero per (row, group).  The kernel streams the weight
+// tiles once with TMA, writes the few non-zeros of S as a two-term bf16 split (hi + lo: fp32-grade coefficients)
+// straight into shared memory in the swizzled operand layout, and accumulates the block gradient in tensor
+// memory over all tiles of the block that the CTA owns; one flush per block and CTA adds it to global memory.
+#pragma once
+
+#include "kernels_fused.cuh"
+
+namespace cafeq {
+
+struct BwParams {
+  int d_out, d_in;
+  int g, ng;           // group width, groups per row
+  int r;               // matrix blocks per operator block
+  int n_major;         // blocks (input axis: column blocks; output axis: row blocks)
+  int n_minor;         // tiles per block (input axis: 64-row tiles; output axis: 64-column tiles)
+  int NG;              // input axis: groups of one row examined per block, max(1, k / g)
+  int gm;              // records are group-major (index = group * d_out + row) instead of row-major
+  int transpose_out;   // store gradT[..][j][i]
+  const float* coef;
+  const int* idx;
+  float* gradT;        // [n_major / r, k, k], accumulated with atomic adds (caller zeroes it)
+  int32_t* status;
+};
+
+enum { BW_IN = 0, BW_OUT = 1 };
+constexpr int BW_THREADS = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: operand builders and flush
+constexpr int BW_NSTAGE = 3;
+constexpr uint32_t BW_NONE = 0xFFFFFFFFu;
+
+template <int K>
+struct BwCfg {
+  static constexpr int HALVES = K / 128;
+  static constexpr int STAGE_BYTES = K * 64 * 2;   // weight tile: 64 contraction entries x K
+  static constexpr int S_TERM_BYTES = K * 64 * 2;  // S tile: K targets x 64 contraction entries, K-major, one bf16 term
+  static constexpr int S_BUF_BYTES = 2 * S_TERM_BYTES;
+  static constexpr int TMEM_COLS = HALVES * K;     // 128 or 512
+  static constexpr int SMEM = 1024 + BW_NSTAGE * STAGE_BYTES + 2 * S_BUF_BYTES + 256;
+};
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// byte offset of S[target][kk] inside one term of the S tile (128-byte rows, 16-byte chunks XOR-swizzled by the
+// row index modulo 8, 128-target halves 16 KB apart)
+__device__ __forceinline__ uint32_t bw_s_offset(int target, int kk) {
+  const int half = target >> 7, il = target & 127;
+  return (uint32_t)(half * 16384 + (il >> 3) * 1024 + (il & 7) * 128 + ((((kk >> 3) ^ (il & 7)) & 7) << 4) + (kk & 7) * 2);
+}
+
+template <int FORM, int K>
+__global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_constant__ CUtensorMap tmW, const BwParams p) {
+  using C = BwCfg<K>;
+  static_assert(K == 128 || K == 256, "block size");
+  if (p.status && *p.status) return;
+  const int total_tiles = p.n_major * p.n_minor;
+  const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
+  const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
+  if (t_begin >= t_end) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sStage = smem;
+  uint8_t* sS = smem + BW_NSTAGE * C::STAGE_BYTES;
+  uint64_t* bars = (uint64_t*)(sS + 2 * C::S_BUF_BYTES);
+  // barrier slots: wfull[3], wempty[3], sfull[2], sempty[2], accf, acce, grp
+  const uint32_t bar_wfull = smem_u32(bars);
+  const uint32_t bar_wempty = bar_wfull + 8 * BW_NSTAGE;
+  const uint32_t bar_sfull = bar_wempty + 8 * BW_NSTAGE;
+  const uint32_t bar_sempty = bar_sfull + 16;
+  const uint32_t bar_accf = bar_sempty + 16;
+  const uint32_t bar_acce = bar_accf + 8;
+  const uint32_t bar_grp = bar_acce + 8;  // rendezvous of the 256 builder threads (bounded, unlike a named barrier)
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * BW_NSTAGE + 7);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmW);
+    for (int s = 0; s < BW_NSTAGE; ++s) {
+      mbar_init(bar_wfull + 8 * s, 1);
+      mbar_init(bar_wempty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_sfull + 8 * b, 256);
+      mbar_init(bar_sempty + 8 * b, 1);
+    }
+    mbar_init(bar_accf, 1);
+    mbar_init(bar_acce, 256);
+    mbar_init(bar_grp, 256);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // the S tiles start as zeros; afterwards the builders clear exactly what they wrote
+  {
+    uint4* z = reinterpret_cast<uint4*>(sS);
+    for (int e = threadIdx.x; e < 2 * C::S_BUF_BYTES / 16; e += BW_THREADS) z[e] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)C::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer: one weight tile per stage
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int tile = t_begin; tile < t_end; ++tile, ++it) {
+        const int major = tile / p.n_minor, t = tile - major * p.n_minor;
+        const uint32_t s = it % BW_NSTAGE, ph = (it / BW_NSTAGE) & 1u;
+        if (!mbar_wait(bar_wempty + 8 * s, ph ^ 1u, abort_flag, p.status)) break;
+        mbar_expect_tx(bar_wfull + 8 * s, C::STAGE_BYTES);
+        const uint32_t dst = smem_u32(sStage + s * C::STAGE_BYTES);
+        if constexpr (FORM == BW_IN) {
+          // 64 rows x K columns as K / 64 boxes of 64 x 64 (one swizzle atom of the MN-major operand each)
+          for (int n = 0; n < K / 64; ++n) tma_load_2d(dst + n * 8192, &tmW, major * K + n * 64, t * 64, bar_wfull + 8 * s);
+        } else {
+          // K rows x 64 columns: one box, K-major operand
+          tma_load_2d(dst, &tmW, t * 64, major * K, bar_wfull + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(128, K, 0, FORM == BW_IN ? 1 : 0);
+      const uint32_t sSt_u = smem_u32(sStage), sS_u = smem_u32(sS);
+      int cur_major = -1;
+      uint32_t run = 0, it = 0;
+      bool ok = true;
+      for (int tile = t_begin; tile < t_end && ok; ++tile, ++it) {
+        const int major = tile / p.n_minor;
+        const bool first = (major != cur_major);
+        if (first) {
+          // the flush of the previous block must have drained the accumulators
+          if (cur_major >= 0) {
+            if (!mbar_wait(bar_acce, (run - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+          }
+          cur_major = major;
+        }
+        const uint32_t s = it % BW_NSTAGE, ph = (it / BW_NSTAGE) & 1u;
+        const uint32_t b = it & 1u, sph = (it >> 1) & 1u;
+        if (!mbar_wait(bar_wfull + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar_sfull + 8 * b, sph, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t stage = sSt_u + s * C::STAGE_BYTES;
+#pragma unroll
+        for (int term = 0; term < 2; ++term) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t bd = (FORM == BW_IN) ? umma_desc_sw128_lbo(stage + ks * 2048, 8192) : umma_desc_sw128(stage + ks * 32);
+#pragma unroll
+            for (int h = 0; h < C::HALVES; ++h) {
+              const uint64_t ad = umma_desc_sw128(sS_u + b * C::S_BUF_BYTES + term * C::S_TERM_BYTES + h * 16384 + ks * 32);
+              tc_mma_bf16(tmem_base + h * K, ad, bd, idesc, (first && term == 0 && ks == 0) ? 0u : 1u);
+            }
+          }
+        }
+        tc_commit(bar_wempty + 8 * s);
+        tc_commit(bar_sempty + 8 * b);
+        const bool last = (tile + 1 == t_end) || ((tile + 1) / p.n_minor != major);
+        if (last) {
+          tc_commit(bar_accf);
+          ++run;
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- operand builders (one record per thread and tile) and flush
+    const int bt = threadIdx.x - 64;
+    const int q = warp & 3, hw = (warp - 2) >> 2;
+    float cfN = 0.f;
+    int tgN = -1, kkN = 0;
+    auto load_rec = [&](int tile) {
+      const int major = tile / p.n_minor, t = tile - major * p.n_minor;
+      cfN = 0.f;
+      tgN = -1;
+      kkN = 0;
+      if constexpr (FORM == BW_IN) {
+        const int rl = bt & 63, qq = bt >> 6;
+        const int row = t * 64 + rl;
+        const int G0 = (major * K) / p.g;
+        const int G = G0 + qq;
+        if (qq < p.NG && row < p.d_out && G < p.ng) {
+          const long long pi = p.gm ? (long long)G * p.d_out + row : (long long)row * p.ng + G;
+          const float c = __ldg(p.coef + pi);
+          const int col = qq * p.g + __ldg(p.idx + pi) + (G0 * p.g - major * K);
+          if (c != 0.f && (unsigned)col < (unsigned)K) {
+            cfN = c;
+            tgN = col;
+            kkN = rl;
+          }
+        }
+      } else {
+        if (bt < K) {
+          const int row = major * K + bt;
+          const int G = (t * 64) / p.g;
+          const long long pi = p.gm ? (long long)G * p.d_out + row : (long long)row * p.ng + G;
+          const float c = __ldg(p.coef + pi);
+          const int col = G * p.g + __ldg(p.idx + pi) - t * 64;
+          if (c != 0.f && (unsigned)col < 64u) {
+            cfN = c;
+            tgN = bt;
+            kkN = col;
+          }
+        }
+      }
+    };
+    // flush of one block: accumulators -> global memory (atomic adds; coalesced along the fastest output index)
+    auto flush = [&](int major, uint32_t run) -> bool {
+      bool ok = mbar_wait(bar_accf, run & 1u, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return false;
+      tc_fence_after();
+      float* out = p.gradT + (size_t)(major / p.r) * K * K;
+      float* stg = reinterpret_cast<float*>(sS) + (warp - 2) * (32 * 33);  // staging (S tiles are all-zero and idle here)
+      constexpr int CH = (K == 256) ? 8 : 2;  // 32-column chunks per thread
+      const int i0 = ((K == 256) ? hw * 128 : 0) + q * 32;
+      const int jbase = (K == 256) ? 0 : hw * 64;
+      const uint32_t tcol = (K == 256) ? (uint32_t)(hw * K) : (uint32_t)(hw * 64);
+      for (int ch = 0; ch < CH; ++ch) {
+        float v[32];
+        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + tcol + ch * 32, v);
+        const int j0 = jbase + ch * 32;
+        if (p.transpose_out) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (v[c] != 0.f) atomicAdd(&out[(size_t)(j0 + c) * K + i0 + lane], v[c]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) stg[lane * 33 + c] = v[c];
+          __syncwarp();
+#pragma unroll 8
+          for (int rr = 0; rr < 32; ++rr) {
+            const float x = stg[rr * 33 + lane];
+            if (x != 0.f) atomicAdd(&out[(size_t)(i0 + rr) * K + j0 + lane], x);
+          }
+          __syncwarp();
+        }
+      }
+      if (!p.transpose_out) {
+        for (int e = lane; e < 32 * 33; e += 32) stg[e] = 0.f;  // the staging area is operand memory again
+        fence_proxy_async_smem();
+      }
+      tc_fence_before();
+      mbar_arrive(bar_acce);
+      return true;
+    };
+
+    uint32_t prevA = BW_NONE, prevB = BW_NONE;  // offsets this thread wrote into S buffer 0 / 1
+    uint32_t gph = 0;
+    auto grp_sync = [&]() -> bool {
+      mbar_arrive(bar_grp);
+      const bool okw = mbar_wait(bar_grp, gph & 1u, abort_flag, p.status);
+      ++gph;
+      return __all_sync(0xffffffffu, okw);
+    };
+    // After the accumulator barrier of a block completes, every product that reads the S tiles is done: clear
+    // what this thread left in both buffers, meet the other builders, then flush through the (all-zero) S memory.
+    auto end_block = [&](int major, uint32_t run) -> bool {
+      bool okw = mbar_wait(bar_accf, run & 1u, abort_flag, p.status);
+      okw = __all_sync(0xffffffffu, okw);
+      if (!okw) return false;
+      if (prevA != BW_NONE) {
+        *reinterpret_cast<uint16_t*>(sS + prevA) = 0;
+        *reinterpret_cast<uint16_t*>(sS + C::S_TERM_BYTES + prevA) = 0;
+        prevA = BW_NONE;
+      }
+      if (prevB != BW_NONE) {
+        *reinterpret_cast<uint16_t*>(sS + C::S_BUF_BYTES + prevB) = 0;
+        *reinterpret_cast<uint16_t*>(sS + C::S_BUF_BYTES + C::S_TERM_BYTES + prevB) = 0;
+        prevB = BW_NONE;
+      }
+      if (!grp_sync()) return false;
+      if (!flush(major, run)) return false;
+      return grp_sync();
+    };
+    int cur_major = t_begin / p.n_minor;
+    uint32_t run = 0, tl = 0;
+    bool ok = true;
+    load_rec(t_begin);
+    for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
+      const int major = tile / p.n_minor;
+      const float cf = cfN;
+      const int tg = tgN, kk = kkN;
+      if (tile + 1 < t_end) load_rec(tile + 1);
+      const uint32_t b = tl & 1u, sph = (tl >> 1) & 1u;
+      if (major != cur_major) {
+        if (!end_block(cur_major, run)) { ok = false; break; }
+        ++run;
+        cur_major = major;
+      }
+      ok = mbar_wait(bar_sempty + 8 * b, sph ^ 1u, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      uint8_t* buf = sS + b * C::S_BUF_BYTES;
+      const uint32_t prev = b ? prevB : prevA;
+      if (prev != BW_NONE) {
+        *reinterpret_cast<uint16_t*>(buf + prev) = 0;
+        *reinterpret_cast<uint16_t*>(buf + C::S_TERM_BYTES + prev) = 0;
+      }
+      uint32_t now = BW_NONE;
+      if (tg >= 0) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(cf);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(cf - __bfloat162float(hi));
+        now = bw_s_offset(tg, kk);
+        *reinterpret_cast<uint16_t*>(buf + now) = __bfloat16_as_ushort(hi);
+        *reinterpret_cast<uint16_t*>(buf + C::S_TERM_BYTES + now) = __bfloat16_as_ushort(lo);
+      }
+      if (b) prevB = now; else prevA = now;
+      fence_proxy_async_smem();
+      mbar_arrive(bar_sfull + 8 * b);
+    }
+    if (ok) end_block(cur_major, run);
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+  }
+}
+
+// host side ------------------------------------------------------------------------------------------------
+static bool bw_supported(int axis_in, int d_out, int d_in, long long ld, int k, int g, const void* W) {
+  if (!(k == 128 || k == 256)) return false;
+  if ((ld % 8) || ((uintptr_t)W & 15)) return false;
+  if (axis_in) {
+    if (d_in % k) return false;
+    if (!(k % g == 0 || g % k == 0)) return false;
+    if (k / g > 4) return false;
+  } else {
+    if (d_out % k || d_in % 64 || g % 64 || d_in % g) return false;
+  }
+  return true;
+}
+
+template <int FORM, int K>
+static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& p) {
+  using C = BwCfg<K>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(bd_bwd_kernel<FORM, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+      return CAFEQ_ERR_CUDA;
+    attr_done = true;
+  }
+  // one persistent CTA per SM at most; small problems use fewer CTAs so that every CTA has several tiles per
+  // flush (a flush moves k * k floats whatever the number of tiles behind it)
+  const long long total = (long long)p.n_major * p.n_minor;
+  long long want = total / 6;
+  if (want < p.n_major) want = p.n_major;
+  if (want > total) want = total;
+  const int grid = want < 148 ? (int)want : 148;
+  bd_bwd_kernel<FORM, K><<<grid, BW_THREADS, C::SMEM, st>>>(tmW, p);
+  return CAFEQ_OK;
+}
+
+// W: bf16 [d_out, d_in] with pitch ld; records and gradT as in BwParams (n_major, n_minor, NG are filled here)
+static int bw_launch(cudaStream_t st, int axis_in, int k, const void* W, long long ld, BwParams p) {
+  CUtensorMap tmW;
+  if (!make_map_bf16(&tmW, W, p.d_in, p.d_out, ld, axis_in ? 64 : k)) return CAFEQ_ERR_UNSUPPORTED;
+  if (axis_in) {
+    p.n_major = p.d_in / k;
+    p.n_minor = (p.d_out + 63) / 64;
+    p.NG = (k >= p.g) ? k / p.g : 1;
+  } else {
+    p.n_major = p.d_out / k;
+    p.n_minor = p.d_in / 64;
+    p.NG = 1;
+  }
+  if (axis_in && k == 128) return bw_launch_t<BW_IN, 128>(st, tmW, p);
+  if (axis_in && k == 256) return bw_launch_t<BW_IN, 256>(st, tmW, p);
+  if (!axis_in && k == 128) return bw_launch_t<BW_OUT, 128>(st, tmW, p);
+  if (!axis_in && k == 256) return bw_launch_t<BW_OUT, 256>(st, tmW, p);
+  return CAFEQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace cafeq
