@@ -10,6 +10,8 @@
 // tiles once with TMA, writes the few non-zeros of S as a two-term bf16 split (hi + lo: fp32-grade coefficients)
 // straight into shared memory in the swizzled operand layout, and accumulates the block gradient in tensor
 // memory over all tiles of the block that the CTA owns; one flush per block and CTA adds it to global memory.
+// The product is issued in the orientation (S^T W or W^T S) whose accumulator rows run along the fastest index of
+// the requested output layout, so that the flush is coalesced atomic adds straight from registers.
 #pragma once
 
 #include "kernels_fused.cuh"
@@ -55,7 +57,9 @@ __device__ __forceinline__ uint32_t bw_s_offset(int target, int kk) {
   return (uint32_t)(half * 16384 + (il >> 3) * 1024 + (il & 7) * 128 + ((((kk >> 3) ^ (il & 7)) & 7) << 4) + (kk & 7) * 2);
 }
 
-template <int FORM, int K>
+// SWAP = 0: accumulator rows = targets i, columns = j (coalesced when the output is stored transposed);
+// SWAP = 1: rows = j, columns = i (coalesced for the plain layout).
+template <int FORM, int K, int SWAP>
 __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_constant__ CUtensorMap tmW, const BwParams p) {
   using C = BwCfg<K>;
   static_assert(K == 128 || K == 256, "block size");
@@ -70,15 +74,14 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
   uint8_t* sStage = smem;
   uint8_t* sS = smem + BW_NSTAGE * C::STAGE_BYTES;
   uint64_t* bars = (uint64_t*)(sS + 2 * C::S_BUF_BYTES);
-  // barrier slots: wfull[3], wempty[3], sfull[2], sempty[2], accf, acce, grp
+  // barrier slots: wfull[3], wempty[3], sfull[2], sempty[2], accf, acce
   const uint32_t bar_wfull = smem_u32(bars);
   const uint32_t bar_wempty = bar_wfull + 8 * BW_NSTAGE;
   const uint32_t bar_sfull = bar_wempty + 8 * BW_NSTAGE;
   const uint32_t bar_sempty = bar_sfull + 16;
   const uint32_t bar_accf = bar_sempty + 16;
   const uint32_t bar_acce = bar_accf + 8;
-  const uint32_t bar_grp = bar_acce + 8;  // rendezvous of the 256 builder threads (bounded, unlike a named barrier)
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * BW_NSTAGE + 7);
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * BW_NSTAGE + 6);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -94,7 +97,6 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
     }
     mbar_init(bar_accf, 1);
     mbar_init(bar_acce, 256);
-    mbar_init(bar_grp, 256);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -137,7 +139,8 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(128, K, 0, FORM == BW_IN ? 1 : 0);
+      // the weight tile is MN-major on the input axis (contraction over its rows), K-major on the output axis
+      constexpr uint32_t idesc = SWAP ? umma_idesc_bf16(128, K, FORM == BW_IN ? 1 : 0, 0) : umma_idesc_bf16(128, K, 0, FORM == BW_IN ? 1 : 0);
       const uint32_t sSt_u = smem_u32(sStage), sS_u = smem_u32(sS);
       int cur_major = -1;
       uint32_t run = 0, it = 0;
@@ -161,13 +164,23 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
         const uint32_t stage = sSt_u + s * C::STAGE_BYTES;
 #pragma unroll
         for (int term = 0; term < 2; ++term) {
+          const uint32_t sterm = sS_u + b * C::S_BUF_BYTES + term * C::S_TERM_BYTES;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t bd = (FORM == BW_IN) ? umma_desc_sw128_lbo(stage + ks * 2048, 8192) : umma_desc_sw128(stage + ks * 32);
+            const uint32_t acc = (first && term == 0 && ks == 0) ? 0u : 1u;
 #pragma unroll
             for (int h = 0; h < C::HALVES; ++h) {
-              const uint64_t ad = umma_desc_sw128(sS_u + b * C::S_BUF_BYTES + term * C::S_TERM_BYTES + h * 16384 + ks * 32);
-              tc_mma_bf16(tmem_base + h * K, ad, bd, idesc, (first && term == 0 && ks == 0) ? 0u : 1u);
+              uint64_t ad, bd;
+              if constexpr (SWAP == 0) {
+                ad = umma_desc_sw128(sterm + h * 16384 + ks * 32);
+                bd = (FORM == BW_IN) ? umma_desc_sw128_lbo(stage + ks * 2048, 8192) : umma_desc_sw128(stage + ks * 32);
+              } else {
+                // half h of the weight tile: 128 of its K columns (two swizzle atoms) or 128 of its K rows
+                ad = (FORM == BW_IN) ? umma_desc_sw128_lbo(stage + h * 16384 + ks * 2048, 8192)
+                                     : umma_desc_sw128(stage + h * 16384 + ks * 32);
+                bd = umma_desc_sw128(sterm + ks * 32);
+              }
+              tc_mma_bf16(tmem_base + h * K, ad, bd, idesc, acc);
             }
           }
         }
@@ -221,41 +234,25 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
         }
       }
     };
-    // flush of one block: accumulators -> global memory (atomic adds; coalesced along the fastest output index)
+    // flush of one block: accumulators -> global memory, coalesced atomic adds straight from the registers
+    // (accumulator row m = this thread's lane, 32 consecutive columns n per load)
     auto flush = [&](int major, uint32_t run) -> bool {
-      bool ok = mbar_wait(bar_accf, run & 1u, abort_flag, p.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) return false;
+      bool okw = mbar_wait(bar_accf, run & 1u, abort_flag, p.status);
+      okw = __all_sync(0xffffffffu, okw);
+      if (!okw) return false;
       tc_fence_after();
       float* out = p.gradT + (size_t)(major / p.r) * K * K;
-      float* stg = reinterpret_cast<float*>(sS) + (warp - 2) * (32 * 33);  // staging (S tiles are all-zero and idle here)
       constexpr int CH = (K == 256) ? 8 : 2;  // 32-column chunks per thread
-      const int i0 = ((K == 256) ? hw * 128 : 0) + q * 32;
-      const int jbase = (K == 256) ? 0 : hw * 64;
+      const int m = ((K == 256) ? hw * 128 : 0) + q * 32 + lane;
+      const int nbase = (K == 256) ? 0 : hw * 64;
       const uint32_t tcol = (K == 256) ? (uint32_t)(hw * K) : (uint32_t)(hw * 64);
       for (int ch = 0; ch < CH; ++ch) {
         float v[32];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + tcol + ch * 32, v);
-        const int j0 = jbase + ch * 32;
-        if (p.transpose_out) {
+        const int n0 = nbase + ch * 32;
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (v[c] != 0.f) atomicAdd(&out[(size_t)(j0 + c) * K + i0 + lane], v[c]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) stg[lane * 33 + c] = v[c];
-          __syncwarp();
-#pragma unroll 8
-          for (int rr = 0; rr < 32; ++rr) {
-            const float x = stg[rr * 33 + lane];
-            if (x != 0.f) atomicAdd(&out[(size_t)(i0 + rr) * K + j0 + lane], x);
-          }
-          __syncwarp();
-        }
-      }
-      if (!p.transpose_out) {
-        for (int e = lane; e < 32 * 33; e += 32) stg[e] = 0.f;  // the staging area is operand memory again
-        fence_proxy_async_smem();
+        for (int c = 0; c < 32; ++c)
+          if (v[c] != 0.f) atomicAdd(&out[(size_t)(n0 + c) * K + m], v[c]);
       }
       tc_fence_before();
       mbar_arrive(bar_acce);
@@ -263,33 +260,6 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
     };
 
     uint32_t prevA = BW_NONE, prevB = BW_NONE;  // offsets this thread wrote into S buffer 0 / 1
-    uint32_t gph = 0;
-    auto grp_sync = [&]() -> bool {
-      mbar_arrive(bar_grp);
-      const bool okw = mbar_wait(bar_grp, gph & 1u, abort_flag, p.status);
-      ++gph;
-      return __all_sync(0xffffffffu, okw);
-    };
-    // After the accumulator barrier of a block completes, every product that reads the S tiles is done: clear
-    // what this thread left in both buffers, meet the other builders, then flush through the (all-zero) S memory.
-    auto end_block = [&](int major, uint32_t run) -> bool {
-      bool okw = mbar_wait(bar_accf, run & 1u, abort_flag, p.status);
-      okw = __all_sync(0xffffffffu, okw);
-      if (!okw) return false;
-      if (prevA != BW_NONE) {
-        *reinterpret_cast<uint16_t*>(sS + prevA) = 0;
-        *reinterpret_cast<uint16_t*>(sS + C::S_TERM_BYTES + prevA) = 0;
-        prevA = BW_NONE;
-      }
-      if (prevB != BW_NONE) {
-        *reinterpret_cast<uint16_t*>(sS + C::S_BUF_BYTES + prevB) = 0;
-        *reinterpret_cast<uint16_t*>(sS + C::S_BUF_BYTES + C::S_TERM_BYTES + prevB) = 0;
-        prevB = BW_NONE;
-      }
-      if (!grp_sync()) return false;
-      if (!flush(major, run)) return false;
-      return grp_sync();
-    };
     int cur_major = t_begin / p.n_minor;
     uint32_t run = 0, tl = 0;
     bool ok = true;
@@ -301,7 +271,7 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
       if (tile + 1 < t_end) load_rec(tile + 1);
       const uint32_t b = tl & 1u, sph = (tl >> 1) & 1u;
       if (major != cur_major) {
-        if (!end_block(cur_major, run)) { ok = false; break; }
+        if (!flush(cur_major, run)) { ok = false; break; }
         ++run;
         cur_major = major;
       }
@@ -326,7 +296,7 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
       fence_proxy_async_smem();
       mbar_arrive(bar_sfull + 8 * b);
     }
-    if (ok) end_block(cur_major, run);
+    if (ok) flush(cur_major, run);
   }
 
   // ---------------------------------------------------------------- teardown
@@ -353,12 +323,12 @@ static bool bw_supported(int axis_in, int d_out, int d_in, long long ld, int k, 
   return true;
 }
 
-template <int FORM, int K>
+template <int FORM, int K, int SWAP>
 static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& p) {
   using C = BwCfg<K>;
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(bd_bwd_kernel<FORM, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+    if (cudaFuncSetAttribute(bd_bwd_kernel<FORM, K, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
       return CAFEQ_ERR_CUDA;
     attr_done = true;
   }
@@ -369,7 +339,7 @@ static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& 
   if (want < p.n_major) want = p.n_major;
   if (want > total) want = total;
   const int grid = want < 148 ? (int)want : 148;
-  bd_bwd_kernel<FORM, K><<<grid, BW_THREADS, C::SMEM, st>>>(tmW, p);
+  bd_bwd_kernel<FORM, K, SWAP><<<grid, BW_THREADS, C::SMEM, st>>>(tmW, p);
   return CAFEQ_OK;
 }
 
@@ -386,10 +356,18 @@ static int bw_launch(cudaStream_t st, int axis_in, int k, const void* W, long lo
     p.n_minor = p.d_in / 64;
     p.NG = 1;
   }
-  if (axis_in && k == 128) return bw_launch_t<BW_IN, 128>(st, tmW, p);
-  if (axis_in && k == 256) return bw_launch_t<BW_IN, 256>(st, tmW, p);
-  if (!axis_in && k == 128) return bw_launch_t<BW_OUT, 128>(st, tmW, p);
-  if (!axis_in && k == 256) return bw_launch_t<BW_OUT, 256>(st, tmW, p);
+  const int swap = p.transpose_out ? 0 : 1;  // accumulator rows along the fastest index of the output
+#define BW_CASE(AX, F, KK, SW) \
+  if ((axis_in != 0) == (AX) && k == KK && swap == SW) return bw_launch_t<F, KK, SW>(st, tmW, p);
+  BW_CASE(true, BW_IN, 128, 0)
+  BW_CASE(true, BW_IN, 128, 1)
+  BW_CASE(true, BW_IN, 256, 0)
+  BW_CASE(true, BW_IN, 256, 1)
+  BW_CASE(false, BW_OUT, 128, 0)
+  BW_CASE(false, BW_OUT, 128, 1)
+  BW_CASE(false, BW_OUT, 256, 0)
+  BW_CASE(false, BW_OUT, 256, 1)
+#undef BW_CASE
   return CAFEQ_ERR_UNSUPPORTED;
 }
 
