@@ -24,7 +24,8 @@ OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_debug_timer_begin", "cafeq_debug_timer_read", "cafeq_debug_launch_count",
+    "cafeq_pack", "cafeq_set_product_min_ctas", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
 
@@ -76,6 +77,12 @@ def status_string(code: int) -> str:
 
 def version() -> int:
     return lib().cafeq_version()
+
+
+def set_product_min_ctas(n: int) -> None:
+    """Process-wide tile-width rule of the k x k products: small n (default 28) favours throughput when several
+    problems run in different streams, 96 the latency of one problem running alone."""
+    _check(lib().cafeq_set_product_min_ctas(ctypes.c_int(int(n))), "cafeq_set_product_min_ctas")
 
 
 def launch_count() -> int:

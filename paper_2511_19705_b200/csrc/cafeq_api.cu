@@ -639,6 +639,12 @@ extern "C" int cafeq_version(void) { return 100; }
 
 extern "C" long long cafeq_debug_launch_count(void) { return g_launches.load(); }
 
+extern "C" int cafeq_set_product_min_ctas(int n) {
+  if (n < 1 || n > 4096) return CAFEQ_ERR_INVALID_ARG;
+  g_tg_min_ctas.store(n, std::memory_order_relaxed);
+  return CAFEQ_OK;
+}
+
 extern "C" int cafeq_debug_timer_begin(int capacity) {
   if (capacity < 0 || g_kt.on) return CAFEQ_ERR_INVALID_ARG;
   g_kt.a.resize(capacity);

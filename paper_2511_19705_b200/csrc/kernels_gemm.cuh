@@ -14,6 +14,8 @@
 // warps 2..9 = epilogue (one accumulator row and half of the tile's columns per thread).  Every mbarrier wait is bounded.
 #pragma once
 
+#include <atomic>
+
 #include "kernels_fused.cuh"
 
 namespace cafeq {
@@ -313,14 +315,17 @@ static int tg_launch_t(cudaStream_t st, const TgOperand* A, const TgOperand* B, 
 }
 
 // K must be a multiple of 64; operands 16-byte aligned with pitches that are multiples of 8 elements.
+// Tile-width rule of the small batched products: the widest tile that still gives at least this many CTAs.
+// A CTA's life is dominated by fixed latencies and its epilogue, so narrow tiles (many CTAs) finish one product
+// sooner, while wide tiles (few CTAs) cost far fewer SM-microseconds and leave room for the kernels of other
+// problems running in other streams.  Default: wide tiles (throughput); cafeq_set_product_min_ctas changes it.
+static std::atomic<int> g_tg_min_ctas{28};
 static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, const TgParams& p) {
   if (p.K % TG_BK || p.nterms < 1 || p.nterms > TG_MAX_TERMS) return CAFEQ_ERR_UNSUPPORTED;
-  // widest tile that still gives about one CTA per SM: these products are small, and a CTA's life is dominated
-  // by its epilogue (one accumulator row per thread), so more, narrower tiles finish sooner
   const long long mt = (long long)p.batch * ((p.M + 127) / 128);
-  if (p.N > 128 && mt * ((p.N + 255) / 256) >= 96) return tg_launch_t<256>(st, A, B, p);
-  if (p.N > 64 && mt * ((p.N + 127) / 128) >= 96) return tg_launch_t<128>(st, A, B, p);
-  if (p.N <= 64 || mt * ((p.N + 127) / 128) < 96) return tg_launch_t<64>(st, A, B, p);
+  if (p.N > 128 && mt * ((p.N + 255) / 256) >= g_tg_min_ctas.load(std::memory_order_relaxed)) return tg_launch_t<256>(st, A, B, p);
+  if (p.N > 64 && mt * ((p.N + 127) / 128) >= g_tg_min_ctas.load(std::memory_order_relaxed)) return tg_launch_t<128>(st, A, B, p);
+  if (p.N <= 64 || mt * ((p.N + 127) / 128) < g_tg_min_ctas.load(std::memory_order_relaxed)) return tg_launch_t<64>(st, A, B, p);
   return tg_launch_t<128>(st, A, B, p);
 }
 
