@@ -62,6 +62,7 @@ enum {
   CAFEQ_LOSS_PQE_STE = 3    /* pair: Eq. 5 squared, straight-through */
 };
 enum { CAFEQ_OPT_GD = 0, CAFEQ_OPT_ADAM = 1 };
+#define CAFEQ_OPT_STATE_HEADER 4 /* floats before the moment arrays of an optimiser state */
 /* flags for the forward/backward calls */
 enum {
   CAFEQ_FLAG_EXACT_LOSS = 1, /* also evaluate the quantised loss (l2 proxy / PQE) */
@@ -151,8 +152,9 @@ int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* W, const fl
 
 /* `cfg->steps` optimisation steps on a single matrix (Section 4.1: gradient descent on Eq. 4 from the
  * caller's initial M; Adam selectable).  M is updated in place (fp32 master parameters).
- * opt_state: fp32 [1 + 3*nb*k*k] = {step count, Adam first moments, Adam second moments, inverse of the last
- * step's transform}; required for Adam, optional for gradient descent.  Carrying it over between calls with
+ * opt_state: fp32 [CAFEQ_OPT_STATE_HEADER + 3*nb*k*k] = {step count, 3 reserved floats, Adam first moments, Adam
+ * second moments, inverse of the last step's transform}, 16-byte aligned (so that each array is: the kernels move
+ * them 16 bytes at a time); required for Adam, optional for gradient descent.  Carrying it over between calls with
  * cfg->resume = 1 resumes a run; the caller zeroes it before the first call.  loss_history: out fp32 [steps, 2] =
  * {surrogate, quantised loss or NaN when not evaluated at that step}. */
 int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, float* M, float* opt_state,

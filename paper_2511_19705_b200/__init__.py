@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcafeq.so")
 AXIS_IN, AXIS_OUT = 0, 1
 APPLY_T, APPLY_TT = 0, 1
 LOSS_SURROGATE, LOSS_L2_STE, LOSS_LSE, LOSS_PQE_STE = 0, 1, 2, 3
+OPT_STATE_HEADER = 4   # floats before the moment arrays of an optimiser state (CAFEQ_OPT_STATE_HEADER)
 OPT_GD, OPT_ADAM = 0, 1
 FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC, FLAG_WARM_MINV = 1, 2, 4, 8
 OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
@@ -239,7 +240,7 @@ def cafeq_optimize_single(W, M, cfg: OptCfg, *, bits, group, taxis=AXIS_IN, opt_
     hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W.device)
     status = torch.zeros(1, dtype=torch.int32, device=W.device)
     if cfg.optimizer == OPT_ADAM and opt_state is None:
-        opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W.device)
+        opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W.device)
     ws = workspace(workspace_size(d, None, cfg), W.device)
     rc = lib().cafeq_optimize_single(ctypes.byref(d), _p(W), _p(M), _p(opt_state), ctypes.byref(cfg), _p(hist),
                                      _p(status), _p(ws), ctypes.c_size_t(ws.numel()), _stream())
@@ -287,7 +288,7 @@ def cafeq_optimize_pair(W1, W2, M, cfg: OptCfg, *, bits, group1, group2, replica
     hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W1.device)
     status = torch.zeros(1, dtype=torch.int32, device=W1.device)
     if cfg.optimizer == OPT_ADAM and opt_state is None:
-        opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W1.device)
+        opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W1.device)
     ws = workspace(workspace_size(d1, d2, cfg), W1.device)
     rc = lib().cafeq_optimize_pair(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(M), _p(opt_state),
                                    _p(_f32(P, "P")), ctypes.byref(cfg), _p(hist), _p(status), _p(ws),

@@ -905,7 +905,7 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
   // the inverse of the last step's transform lives in the optimiser state, so a resumed run refines it
   const bool resume = cfg->resume && opt_state;
-  if (opt_state) s.Minv = opt_state + 1 + 2 * kk;
+  if (opt_state) s.Minv = opt_state + CAFEQ_OPT_STATE_HEADER + 2 * kk;
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = cfg->eval_every > 0 && (it % cfg->eval_every == 0);
     single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
@@ -1200,7 +1200,7 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
   // the inverse of the last step's transform lives in the optimiser state, so a resumed run refines it
   const bool resume = cfg->resume && opt_state;
-  if (opt_state) p.Minv = opt_state + 1 + 2 * kk;
+  if (opt_state) p.Minv = opt_state + CAFEQ_OPT_STATE_HEADER + 2 * kk;
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = ste || (any_pqe && (it % cfg->eval_every == 0));
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,

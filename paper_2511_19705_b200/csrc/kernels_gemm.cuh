@@ -149,32 +149,53 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
       const long long cb = (long long)b * p.sCb, c0b = (long long)b * p.sC0b;
       const long long sb_mn = (long long)b * p.M * p.N;
       constexpr int CH = BN / 64;  // 32-column chunks per warp
+      const bool vec_ok = ((p.N | p.ldc | p.ldc0 | p.sCb | p.sC0b | ((long long)p.M * p.N)) & 3) == 0 &&
+                          (((uintptr_t)p.C | (uintptr_t)p.C0) & 15) == 0 && (((uintptr_t)p.Chi | (uintptr_t)p.Clo) & 7) == 0;
+      // The kernel lives for microseconds and every CTA runs this code once or a few times, so its size counts
+      // (instruction fetch showed up as the top stall): one rolled loop over the chunks, one unrolled copy of
+      // each register <-> tile move shared by all paths, rolled loops on the edge paths.
+      float* tile = reinterpret_cast<float*>(smem + (warp - 2) * 4608);  // [32][36] per warp (stage buffers are free now)
+      const int rbase = m0 + q * 32;
+      const int r4 = lane >> 3, c4 = (lane & 7) * 4;
+#pragma unroll 1
       for (int ci = 0; ci < CH; ++ci) {
         const int ch = half * CH + ci;
-        float v[32];
-        tc_ld32(taddr + ch * 32, v);
         const int nb0 = n0 + ch * 32;
         if (nb0 >= p.N) break;
-        const bool inner = (nb0 + 32 <= p.N) && (m0 + 128 <= p.M);  // no edge in this chunk: no per-element checks
-        // Row-major global traffic goes through a per-warp 32 x 32 tile in shared memory (the stage buffers are
-        // free once the accumulator is complete): in the accumulator a lane owns a ROW, and 32 lanes reading or
-        // writing 32 different rows of a matrix whose pitch is a power of two all land on one cache set; with a
-        // lane per COLUMN every access is one contiguous line.
-        float* tile = reinterpret_cast<float*>(smem + (warp - 2) * 4352);  // [32][33]
-        const int rbase = m0 + q * 32;
+        float v[32];
+        tc_ld32(taddr + ch * 32, v);
+        const bool inner = (nb0 + 32 <= p.N) && (m0 + 128 <= p.M);  // no edge in this chunk
+        // Vector path (no edge, every pitch a multiple of 4 elements, aligned bases): a lane moves 16 bytes per
+        // shared-memory access (pitch 36 floats: conflict-free by quarter warps) and a warp instruction covers
+        // 4 rows x 128 bytes of global memory.  In the accumulator a lane owns a ROW; global traffic wants a
+        // lane per COLUMN (32 lanes on 32 rows of a power-of-two pitch serialise in the memory pipe).
+        const bool vec = inner && vec_ok;
         const int ncol = nb0 + lane;
         if (p.C0) {
-          float c0v[32];
+          if (vec) {
+            float4 cv[8];
 #pragma unroll
-          for (int r = 0; r < 32; ++r) {  // all 32 row loads in flight together
-            c0v[r] = 0.f;
-            if (inner || (rbase + r < p.M && ncol < p.N)) c0v[r] = __ldg(p.C0 + c0b + (long long)(rbase + r) * p.ldc0 + ncol);
+            for (int i = 0; i < 8; ++i)
+              cv[i] = __ldg(reinterpret_cast<const float4*>(p.C0 + c0b + (long long)(rbase + i * 4 + r4) * p.ldc0 + nb0 + c4));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(tile + (i * 4 + r4) * 36 + c4) = cv[i];
+          } else {
+#pragma unroll 1
+            for (int r = 0; r < 32; ++r) {
+              float x = 0.f;
+              if (rbase + r < p.M && ncol < p.N) x = __ldg(p.C0 + c0b + (long long)(rbase + r) * p.ldc0 + ncol);
+              tile[r * 36 + lane] = x;
+            }
           }
-#pragma unroll
-          for (int r = 0; r < 32; ++r) tile[r * 33 + lane] = c0v[r];
           __syncwarp();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = fmaf(p.beta, tile[lane * 33 + e], p.alpha * v[e]);
+          for (int j = 0; j < 8; ++j) {
+            const float4 x = *reinterpret_cast<const float4*>(tile + lane * 36 + 4 * j);
+            v[4 * j] = fmaf(p.beta, x.x, p.alpha * v[4 * j]);
+            v[4 * j + 1] = fmaf(p.beta, x.y, p.alpha * v[4 * j + 1]);
+            v[4 * j + 2] = fmaf(p.beta, x.z, p.alpha * v[4 * j + 2]);
+            v[4 * j + 3] = fmaf(p.beta, x.w, p.alpha * v[4 * j + 3]);
+          }
           __syncwarp();
         } else {
 #pragma unroll
@@ -186,48 +207,50 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
             if (nb0 + e == row) v[e] += p.gamma;
         }
         if (p.sq) {
+          const int nv = rv ? min(32, p.N - nb0) : 0;
           float sqf = 0.f;
-          if (inner) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) sqf = fmaf(v[e], v[e], sqf);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (rv && nb0 + e < p.N) sqf = fmaf(v[e], v[e], sqf);
-          }
+          for (int e = 0; e < 32; ++e)
+            if (e < nv) sqf = fmaf(v[e], v[e], sqf);
           sq += (double)sqf;
         }
-        if (p.C || p.Chi) {
+        if (p.C || p.Chi || (p.Cthi && !(inner && (p.M & 1) == 0))) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) tile[lane * 33 + e] = v[e];
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4*>(tile + lane * 36 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
           __syncwarp();
-          if (p.C) {
-#pragma unroll 8
-            for (int r = 0; r < 32; ++r) {
-              const float x = tile[r * 33 + lane];
-              if (inner || (rbase + r < p.M && ncol < p.N)) p.C[cb + (long long)(rbase + r) * p.ldc + ncol] = x;
-            }
-          }
-          if (p.Chi) {
-            if (inner && (p.N & 1) == 0) {
-              // two rows per instruction, two columns per lane: 32-bit stores (2-byte stores serialise badly)
-#pragma unroll 4
-              for (int r2 = 0; r2 < 32; r2 += 2) {
-                const int rr = r2 + (lane >> 4), cc = (lane & 15) * 2;
-                const float x0 = tile[rr * 33 + cc], x1 = tile[rr * 33 + cc + 1];
-                const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
-                const long long o = sb_mn + (long long)(rbase + rr) * p.N + nb0 + cc;
-                *reinterpret_cast<uint32_t*>(p.Chi + o) = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          if (vec) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int rr = i * 4 + r4;
+              const float4 x = *reinterpret_cast<const float4*>(tile + rr * 36 + c4);
+              if (p.C) *reinterpret_cast<float4*>(p.C + cb + (long long)(rbase + rr) * p.ldc + nb0 + c4) = x;
+              if (p.Chi) {
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(x.x), h1 = __float2bfloat16_rn(x.y);
+                const __nv_bfloat16 h2 = __float2bfloat16_rn(x.z), h3 = __float2bfloat16_rn(x.w);
+                const long long o = sb_mn + (long long)(rbase + rr) * p.N + nb0 + c4;
+                *reinterpret_cast<uint2*>(p.Chi + o) =
+                    make_uint2((uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16),
+                               (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16));
                 if (p.Clo) {
-                  const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0));
-                  const __nv_bfloat16 l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
-                  *reinterpret_cast<uint32_t*>(p.Clo + o) = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                  const __nv_bfloat16 l0 = __float2bfloat16_rn(x.x - __bfloat162float(h0));
+                  const __nv_bfloat16 l1 = __float2bfloat16_rn(x.y - __bfloat162float(h1));
+                  const __nv_bfloat16 l2 = __float2bfloat16_rn(x.z - __bfloat162float(h2));
+                  const __nv_bfloat16 l3 = __float2bfloat16_rn(x.w - __bfloat162float(h3));
+                  *reinterpret_cast<uint2*>(p.Clo + o) =
+                      make_uint2((uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16),
+                                 (uint32_t)__bfloat16_as_ushort(l2) | ((uint32_t)__bfloat16_as_ushort(l3) << 16));
                 }
               }
-            } else {
-              for (int r = 0; r < 32; ++r) {
-                const float x = tile[r * 33 + lane];
-                if (rbase + r < p.M && ncol < p.N) {
+            }
+          } else {
+            // edge chunk or odd pitches: one element per lane and row, everything guarded
+#pragma unroll 1
+            for (int r = 0; r < 32; ++r) {
+              if (rbase + r < p.M && ncol < p.N) {
+                const float x = tile[r * 36 + lane];
+                if (p.C) p.C[cb + (long long)(rbase + r) * p.ldc + ncol] = x;
+                if (p.Chi) {
                   const __nv_bfloat16 h = __float2bfloat16_rn(x);
                   const long long o = sb_mn + (long long)(rbase + r) * p.N + ncol;
                   p.Chi[o] = __bfloat16_as_ushort(h);
@@ -236,39 +259,41 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
               }
             }
           }
-          __syncwarp();
-        }
-        if (p.Cthi) {
-          // transposed outputs: consecutive lanes are consecutive rows = consecutive addresses
-          if (inner && (p.M & 1) == 0) {
-            // neighbouring lanes trade one value so that every lane stores a 32-bit pair of rows: even lanes
-            // write column e, odd lanes column e + 1
-            const int odd = lane & 1;
-            const long long rowpair = row & ~1;
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              const __nv_bfloat16 h0 = __float2bfloat16_rn(v[e]), h1 = __float2bfloat16_rn(v[e + 1]);
-              const uint32_t p0 = (uint32_t)__bfloat16_as_ushort(h0) |
-                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h0))) << 16);
-              const uint32_t p1 = (uint32_t)__bfloat16_as_ushort(h1) |
-                                  ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e + 1] - __bfloat162float(h1))) << 16);
-              const uint32_t mine = odd ? p1 : p0;                       // (hi | lo << 16) of my row in the column I store
-              const uint32_t other = __shfl_xor_sync(0xffffffffu, odd ? p0 : p1, 1);  // the neighbour row's, same column
-              const uint32_t lo_row = odd ? other : mine, hi_row = odd ? mine : other;  // rows (2j, 2j + 1)
-              const long long o = sb_mn + (long long)(nb0 + e + odd) * p.M + rowpair;
-              *reinterpret_cast<uint32_t*>(p.Cthi + o) = (lo_row & 0xFFFFu) | (hi_row << 16);
-              if (p.Ctlo) *reinterpret_cast<uint32_t*>(p.Ctlo + o) = (lo_row >> 16) | (hi_row & 0xFFFF0000u);
-            }
-          } else if (rv) {
+          if (p.Cthi && !(inner && (p.M & 1) == 0) && rv) {
+            // transposed outputs on an edge: this lane's row, one column at a time (read back from its tile row)
             uint16_t* cth = p.Cthi + sb_mn + (long long)nb0 * p.M + row;
             uint16_t* ctl = p.Ctlo ? p.Ctlo + sb_mn + (long long)nb0 * p.M + row : nullptr;
+#pragma unroll 1
             for (int e = 0; e < 32; ++e) {
               if (nb0 + e < p.N) {
-                const __nv_bfloat16 h = __float2bfloat16_rn(v[e]);
+                const float x = tile[lane * 36 + e];
+                const __nv_bfloat16 h = __float2bfloat16_rn(x);
                 cth[(long long)e * p.M] = __bfloat16_as_ushort(h);
-                if (ctl) ctl[(long long)e * p.M] = __bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h)));
+                if (ctl) ctl[(long long)e * p.M] = __bfloat16_as_ushort(__float2bfloat16_rn(x - __bfloat162float(h)));
               }
             }
+          }
+          __syncwarp();
+        }
+        if (p.Cthi && inner && (p.M & 1) == 0) {
+          // transposed outputs: consecutive lanes are consecutive rows = consecutive addresses.  Neighbouring
+          // lanes trade one value so that every lane stores a 32-bit pair of rows: even lanes write column e,
+          // odd lanes column e + 1.
+          const int odd = lane & 1;
+          const long long rowpair = row & ~1;
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(v[e]), h1 = __float2bfloat16_rn(v[e + 1]);
+            const uint32_t p0 = (uint32_t)__bfloat16_as_ushort(h0) |
+                                ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(h0))) << 16);
+            const uint32_t p1 = (uint32_t)__bfloat16_as_ushort(h1) |
+                                ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e + 1] - __bfloat162float(h1))) << 16);
+            const uint32_t mine = odd ? p1 : p0;                       // (hi | lo << 16) of my row in the column I store
+            const uint32_t other = __shfl_xor_sync(0xffffffffu, odd ? p0 : p1, 1);  // the neighbour row's, same column
+            const uint32_t lo_row = odd ? other : mine, hi_row = odd ? mine : other;  // rows (2j, 2j + 1)
+            const long long o = sb_mn + (long long)(nb0 + e + odd) * p.M + rowpair;
+            *reinterpret_cast<uint32_t*>(p.Cthi + o) = (lo_row & 0xFFFFu) | (hi_row << 16);
+            if (p.Ctlo) *reinterpret_cast<uint32_t*>(p.Ctlo + o) = (lo_row >> 16) | (hi_row & 0xFFFF0000u);
           }
         }
       }

@@ -953,8 +953,8 @@ __global__ void adam_update_kernel(float* __restrict__ M, const float* __restric
   if (status && *status) return;
   const float step = state[0];
   const float c1 = 1.f - powf(b1, step), c2 = 1.f - powf(b2, step);
-  float* m = state + 1;
-  float* v = state + 1 + n;
+  float* m = state + CAFEQ_OPT_STATE_HEADER;
+  float* v = state + CAFEQ_OPT_STATE_HEADER + n;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     float gi = g[i];
     float mi = b1 * m[i] + (1.f - b1) * gi;

@@ -16,7 +16,7 @@ import ctypes
 
 import torch
 
-from . import (AXIS_IN, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, OPT_ADAM, OPT_GD, _check, _p,
+from . import (AXIS_IN, OPT_STATE_HEADER, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, OPT_ADAM, OPT_GD, _check, _p,
                _pair_descs, _stream, lib, make_cfg, make_desc, set_product_min_ctas, workspace_size)
 
 
@@ -30,7 +30,7 @@ class SingleProblem:
         self.status = torch.zeros(1, dtype=torch.int32, device=W.device)
         self.ws_bytes = workspace_size(self.desc)
         self.weights = W.numel()
-        self.opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W.device)
+        self.opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W.device)
         self.hist = torch.zeros((1, 2), dtype=torch.float32, device=W.device)
         self.cfg = make_cfg(loss_kind=LOSS_SURROGATE, optimizer=OPT_GD, lr=lr, steps=1, eval_every=0, resume=0)
 
@@ -61,7 +61,7 @@ class PairProblem:
         self.lse_t, self.lambda_orth = lse_t, lambda_orth
         self.weights = W1.numel() + W2.numel()
         self.P = None
-        self.opt_state = torch.zeros(1 + 3 * M.numel(), dtype=torch.float32, device=W1.device)
+        self.opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W1.device)
         self.hist = torch.zeros((1, 2), dtype=torch.float32, device=W1.device)
         self.cfg = make_cfg(loss_kind=LOSS_LSE, optimizer=OPT_ADAM, lr=lr, beta1=0.1, beta2=0.999, eps=1e-8,
                             lambda_orth=lambda_orth, lse_t=lse_t, steps=1, eval_every=0, resume=0)
