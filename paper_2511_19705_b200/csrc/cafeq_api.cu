@@ -339,7 +339,7 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   }
   if (!warm) CQ_LAUNCH(transpose_blocks_kernel, grid_for(kk), 256, 0, st, Mc, X, k, kk);
   int cur = 0;
-  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
+  launch_split(st, X, k, kk, w.Xh[cur], iters > 0 ? nullptr : w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
   for (int it = 0; it < iters; ++it) {
     // R = I - A X needs X to full precision (the product cancels against I): two terms over the split of X.
     const uint16_t* a1[2] = {w.Ab, w.Ab};
@@ -350,8 +350,9 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
     // (the error it leaves is 2^-8 |R| relative, below 4e-5 for every accepted residual).
     const uint16_t* a2[1] = {w.Xh[cur]};
     const uint16_t* b2[1] = {w.RTh};
-    launch_kk_tc(st, 1, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], w.Xl[cur ^ 1], w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr,
-                 nullptr, status);
+    // (the row-major low half is only read after the last iteration, by the M^-1 path of the gradient)
+    launch_kk_tc(st, 1, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], (it == iters - 1) ? w.Xl[cur ^ 1] : nullptr,
+                 w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr, nullptr, status);
     cur ^= 1;
   }
   w.cur = cur;

@@ -20,7 +20,8 @@
 
 namespace cafeq {
 
-constexpr int TG_THREADS = 320;
+constexpr int TG_EPI_PARTS = 4;                       // epilogue warps per 32-lane quarter of the accumulator
+constexpr int TG_THREADS = 64 + 128 * TG_EPI_PARTS;  // warp 0: TMA, warp 1: MMA, then the epilogue warps
 constexpr int TG_BK = 64;
 constexpr int TG_MAX_TERMS = 3;
 
@@ -136,8 +137,10 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
       if (ok) tc_commit(bar_acc);
     }
   } else {
-    // eight epilogue warps: two per 32-lane quarter of the accumulator, each taking half of the columns
-    const int q = warp & 3, half = (warp - 2) >> 2;
+    // a warp reads the accumulator lanes of its quarter (warp index modulo 4); the warps of one quarter share
+    // its 32-column chunks round-robin: with two warps per scheduler the dependent chains of the epilogue
+    // (shuffles, conversions, stores) left the issue slots empty
+    const int q = warp & 3, part = (warp - 2) >> 2;
     const int row = m0 + q * 32 + lane;
     bool ok = mbar_wait(bar_acc, 0, abort_flag, p.status);
     ok = __all_sync(0xffffffffu, ok);
@@ -148,7 +151,6 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
       double sq = 0.0;
       const long long cb = (long long)b * p.sCb, c0b = (long long)b * p.sC0b;
       const long long sb_mn = (long long)b * p.M * p.N;
-      constexpr int CH = BN / 64;  // 32-column chunks per warp
       const bool vec_ok = ((p.N | p.ldc | p.ldc0 | p.sCb | p.sC0b | ((long long)p.M * p.N)) & 3) == 0 &&
                           (((uintptr_t)p.C | (uintptr_t)p.C0) & 15) == 0 && (((uintptr_t)p.Chi | (uintptr_t)p.Clo) & 7) == 0;
       // The kernel lives for microseconds and every CTA runs this code once or a few times, so its size counts
@@ -158,8 +160,7 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
       const int rbase = m0 + q * 32;
       const int r4 = lane >> 3, c4 = (lane & 7) * 4;
 #pragma unroll 1
-      for (int ci = 0; ci < CH; ++ci) {
-        const int ch = half * CH + ci;
+      for (int ch = part; ch < BN / 32; ch += TG_EPI_PARTS) {
         const int nb0 = n0 + ch * 32;
         if (nb0 >= p.N) break;
         float v[32];
