@@ -309,6 +309,13 @@ def main():
              5: "transform_pass_tcgen05"}
     kernel_ms = {names.get(kd, str(kd)): dict(launches_per_step=len(v) / args.steps, ms_per_step=sum(v) / args.steps)
                  for kd, v in by_kind.items()}
+    if "sparse_backward" in kernel_ms and k in (128, 256):
+        # the backward is a second tensor-core product over the same weights: 2k flop per weight of algorithmic
+        # work, issued twice (the routed coefficients are a two-term bf16 split)
+        sb = kernel_ms["sparse_backward"]
+        sb["algorithmic_tflops"] = 2.0 * k * layer.weights / (sb["ms_per_step"] * 1e-3) / 1e12
+        sb["issued_tflops"] = 2.0 * sb["algorithmic_tflops"]
+        sb["kernel"] = "bd_bwd_kernel (tcgen05)"
     roof = None
     tk = max((kd for kd in (1, 5) if kd in by_kind), key=lambda kd: sum(by_kind[kd]), default=None)
     if tk is not None:
