@@ -16,13 +16,14 @@ import ctypes
 
 import torch
 
-from . import (AXIS_IN, OPT_STATE_HEADER, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, OPT_ADAM, OPT_GD, _check, _p,
+from . import (AXIS_IN, LOSS_PQE_STE, OPT_STATE_HEADER, cafeq_pair_product, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, OPT_ADAM, OPT_GD, _check, _p,
                _pair_descs, _stream, lib, make_cfg, make_desc, set_product_min_ctas, workspace_size)
 
 
 class SingleProblem:
-    def __init__(self, name, W, M, bits, group, taxis=AXIS_IN, lr=1e-3):
+    def __init__(self, name, W, M, bits, group, taxis=AXIS_IN, lr=1e-3, loss_kind=LOSS_SURROGATE):
         self.name, self.W, self.M = name, W, M
+        self.loss_kind = loss_kind
         d_out, d_in = W.shape
         self.desc = make_desc(d_out, d_in, bits, group, M.shape[-1], taxis, 0, 1, W.stride(0))
         self.losses = torch.zeros(4, dtype=torch.float32, device=W.device)
@@ -32,9 +33,10 @@ class SingleProblem:
         self.weights = W.numel()
         self.opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W.device)
         self.hist = torch.zeros((1, 2), dtype=torch.float32, device=W.device)
-        self.cfg = make_cfg(loss_kind=LOSS_SURROGATE, optimizer=OPT_GD, lr=lr, steps=1, eval_every=0, resume=0)
+        self.cfg = make_cfg(loss_kind=loss_kind, optimizer=OPT_GD, lr=lr, steps=1, eval_every=0, resume=0)
 
-    def step(self, ws, flags=0, loss_kind=LOSS_SURROGATE):
+    def step(self, ws, flags=0, loss_kind=None):
+        loss_kind = self.loss_kind if loss_kind is None else loss_kind
         rc = lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(self.desc), _p(self.W), _p(self.M), _p(None), _p(None),
                                             ctypes.c_int(OFFSETS_NONE), ctypes.c_int(loss_kind), ctypes.c_float(0.0),
                                             ctypes.c_int(flags), _p(self.losses), _p(self.grad), _p(self.status),
@@ -51,8 +53,10 @@ class SingleProblem:
 
 
 class PairProblem:
-    def __init__(self, name, W1, W2, M, bits, group1, group2, replicas, lse_t=5.0, lambda_orth=0.1, lr=1e-4):
+    def __init__(self, name, W1, W2, M, bits, group1, group2, replicas, lse_t=5.0, lambda_orth=0.1, lr=1e-4,
+                 loss_kind=LOSS_LSE):
         self.name, self.W1, self.W2, self.M = name, W1, W2, M
+        self.loss_kind = loss_kind
         self.d1, self.d2 = _pair_descs(W1, W2, M.shape[-1], bits, group1, group2, replicas)
         self.losses = torch.zeros(4, dtype=torch.float32, device=W1.device)
         self.grad = torch.empty_like(M)
@@ -61,15 +65,18 @@ class PairProblem:
         self.lse_t, self.lambda_orth = lse_t, lambda_orth
         self.weights = W1.numel() + W2.numel()
         self.P = None
+        if loss_kind == LOSS_PQE_STE:  # the product term is the objective itself: W1 W2 is needed every step
+            self.P = cafeq_pair_product(W1, W2, k=M.shape[-1], replicas=replicas)
         self.opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W1.device)
         self.hist = torch.zeros((1, 2), dtype=torch.float32, device=W1.device)
-        self.cfg = make_cfg(loss_kind=LOSS_LSE, optimizer=OPT_ADAM, lr=lr, beta1=0.1, beta2=0.999, eps=1e-8,
+        self.cfg = make_cfg(loss_kind=loss_kind, optimizer=OPT_ADAM, lr=lr, beta1=0.1, beta2=0.999, eps=1e-8,
                             lambda_orth=lambda_orth, lse_t=lse_t, steps=1, eval_every=0, resume=0)
 
     def step(self, ws, flags=0):
         rc = lib().cafeq_pair_loss_fwd_bwd(ctypes.byref(self.d1), _p(self.W1), ctypes.byref(self.d2), _p(self.W2),
-                                           _p(self.M), _p(self.P if (flags & FLAG_EXACT_LOSS) else None),
-                                           ctypes.c_int(LOSS_LSE), ctypes.c_float(self.lse_t),
+                                           _p(self.M),
+                                           _p(self.P if ((flags & FLAG_EXACT_LOSS) or self.loss_kind == LOSS_PQE_STE) else None),
+                                           ctypes.c_int(self.loss_kind), ctypes.c_float(self.lse_t),
                                            ctypes.c_float(self.lambda_orth), ctypes.c_int(flags), _p(self.losses),
                                            _p(self.grad), _p(self.status), _p(ws), ctypes.c_size_t(ws.numel()),
                                            _stream())
@@ -78,7 +85,8 @@ class PairProblem:
     def opt_step(self, ws, eval_exact=False):
         self.cfg.eval_every = 1 if (eval_exact and self.P is not None) else 0
         rc = lib().cafeq_optimize_pair(ctypes.byref(self.d1), _p(self.W1), ctypes.byref(self.d2), _p(self.W2),
-                                       _p(self.M), _p(self.opt_state), _p(self.P if self.cfg.eval_every else None),
+                                       _p(self.M), _p(self.opt_state),
+                                       _p(self.P if (self.cfg.eval_every or self.loss_kind == LOSS_PQE_STE) else None),
                                        ctypes.byref(self.cfg), _p(self.hist), _p(self.status), _p(ws),
                                        ctypes.c_size_t(ws.numel()), _stream())
         _check(rc, "cafeq_optimize_pair")
