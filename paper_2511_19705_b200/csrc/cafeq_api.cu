@@ -115,7 +115,7 @@ static int make_geo(const cafeq_matrix_desc* d, Geo* o, bool need_transform) {
 static size_t kk_scratch_bytes(int nbT, int k);
 
 // scratch that one matrix needs in any call
-static size_t matrix_scratch_bytes(const Geo& G) {
+static size_t matrix_scratch_bytes(const Geo& G, bool with_backward = true) {
   size_t kk = (size_t)(G.nbT > 0 ? G.nbT : 1) * (size_t)(G.k > 0 ? G.k : 1) * (size_t)(G.k > 0 ? G.k : 1);
   size_t rows_ng = (size_t)G.d_out * G.ng;
   size_t b = 0;
@@ -127,6 +127,7 @@ static size_t matrix_scratch_bytes(const Geo& G) {
   b += 4 * ((size_t)(G.nbT + 1) * (G.k + 1) * 4 + 256);  // c, A
   b += 4096;                                          // accumulators
   b += kk_scratch_bytes(G.nbT, G.k);                  // bf16 splits of the k x k algebra
+  if (with_backward) b += 3 * ((size_t)G.n * 2 + 256) + kk * 4 + 256;  // straight-through path on the tensor cores
   return b;
 }
 
@@ -741,6 +742,9 @@ struct SingleWS {
   float *Mc, *Minv, *gMinv, *tmp, *c, *A;
   double* acc;
   KkWS kk;
+  // tensor-core straight-through path: second bf16 term of the residual, both terms transposed, N = Minv^T Minv
+  uint16_t *Dlo, *DTh, *DTl;
+  float* Nf;
 };
 
 static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
@@ -754,6 +758,10 @@ static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
   s->A = b.take<float>((size_t)G.nbT * G.k);
   s->acc = b.take<double>(8);
   carve_kk(b, G.nbT, G.k, &s->kk);
+  s->Dlo = b.take<uint16_t>(G.n);
+  s->DTh = b.take<uint16_t>(G.n);
+  s->DTl = b.take<uint16_t>(G.n);
+  s->Nf = b.take<float>(kk);
   return !b.overflow;
 }
 
@@ -770,6 +778,9 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   const bool need_l2 = want_exact || ste;
   const bool want_grad = (gradM != nullptr);
   const bool in_r1 = (G.axis == CAFEQ_AXIS_IN && G.r == 1);
+  // straight-through mode on the tensor cores: input axis, no rounding offsets, shapes the fused pass covers
+  const bool ste_tc = ste && tc && in_r1 && off_kind == CAFEQ_OFFSETS_NONE && G.d_out % 64 == 0 &&
+                      bd_supported(BD_IN, G.d_out, G.d_in, G.ld, k, G.g, W);
   if (tc) {
     PrepArgs pa;
     memset(&pa, 0, sizeof(pa));
@@ -810,8 +821,86 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   sp.coef = (want_grad && !ste) ? s.m.coef : nullptr;
   sp.lossacc = s.acc + 0;
   sp.Aacc = (G.axis == CAFEQ_AXIS_IN) ? s.m.agrp : s.A;
+  if (ste_tc) {
+    sp.delta_lo = s.Dlo;
+    sp.a_always = 1;
+  }
   const bool fused = forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, nullptr,
-                                   status, !ste && !force_generic, &sp, tc ? s.kk.Ab : nullptr);
+                                   status, (!ste || ste_tc) && !force_generic, &sp, tc ? s.kk.Ab : nullptr);
+  if (ste_tc && fused) {
+    // Nothing below needs E = Minv o Delta itself.  With Gram_B = sum_o Delta[o, B]^T Delta[o, B] (k x k per block) and
+    // N = Minv^T Minv:  L2 = <N, Gram>,  dL/dMinv = 2 Minv Gram,  gDelta = 2 N o Delta (one more block-diagonal
+    // apply), and the scale path needs sum_e gDelta_e Delta_e per group.  Every product runs on the tensor cores
+    // with the residual as a two-term bf16 split (three-term products: fp32-grade).
+    KkWS& w = s.kk;
+    const int c = w.cur;
+    {
+      dim3 tg((G.d_in + 31) / 32, (G.d_out + 31) / 32);
+      CQ_LAUNCH(transpose_bf16_kernel, tg, dim3(32, 8), 0, st, s.m.Dbf, G.d_out, G.d_in, (long long)G.d_in, s.DTh);
+      CQ_LAUNCH(transpose_bf16_kernel, tg, dim3(32, 8), 0, st, s.Dlo, G.d_out, G.d_in, (long long)G.d_in, s.DTl);
+    }
+    {  // Gram (fp32 in s.tmp, splits in w.Ph / w.Pl): contraction over the d_out rows
+      TgOperand oa[3], ob[3];
+      const uint16_t* at[3] = {s.DTh, s.DTl, s.DTh};
+      const uint16_t* bt[3] = {s.DTh, s.DTh, s.DTl};
+      for (int t = 0; t < 3; ++t) {
+        oa[t] = TgOperand{at[t], G.d_in, G.d_out, G.d_out};
+        ob[t] = TgOperand{bt[t], G.d_in, G.d_out, G.d_out};
+      }
+      TgParams p;
+      memset(&p, 0, sizeof(p));
+      p.M = p.N = k; p.K = G.d_out; p.batch = G.nbT; p.nterms = 3;
+      p.rowsA_per_batch = p.rowsB_per_batch = k;
+      p.divA = 1; p.a_rep_k = G.d_out; p.a_rep_r = 1;
+      p.alpha = 1.f;
+      p.C = s.tmp; p.ldc = k; p.sCb = (long long)k * k;
+      p.Chi = w.Ph; p.Clo = w.Pl;
+      p.min_ctas = 148;  // a long contraction: as many CTAs as the tile shapes give
+      p.status = status;
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      tg_launch(st, oa, ob, p);
+    }
+    {  // N = Minv^T Minv (fp32 in s.Nf, splits in w.Qh / w.Ql)
+      const uint16_t* a1[3] = {w.XTh[c], w.XTl[c], w.XTh[c]};
+      const uint16_t* b1[3] = {w.XTh[c], w.XTh[c], w.XTl[c]};
+      launch_kk_tc(st, 3, a1, b1, G.nbT, k, 1.f, 0.f, 0.f, nullptr, s.Nf, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status);
+    }
+    CQ_LAUNCH(dot_f32_kernel, grid_for(kk), 256, 0, st, s.Nf, s.tmp, kk, s.acc + 1);
+    CQ_LAUNCH(sqsum_bf16_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);
+    CQ_LAUNCH(finalize_single_kernel, 1, 1, 0, st, s.acc, losses, hist, 1);
+    if (!want_grad) return;
+    {  // dL/dMinv = 2 Minv Gram (Gram is symmetric: its rows serve as the contraction-major second operand)
+      const uint16_t* a2[3] = {w.Xh[c], w.Xl[c], w.Xh[c]};
+      const uint16_t* b2[3] = {w.Ph, w.Ph, w.Pl};
+      launch_kk_tc(st, 3, a2, b2, G.nbT, k, 2.f, 0.f, 0.f, nullptr, s.gMinv, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                   status);
+    }
+    {  // gDelta[o, B k + j] = 2 sum_l N_B[j][l] Delta[o, B k + l]  -> s.m.D (fp32 [d_out, d_in])
+      TgOperand oa[3], ob[3];
+      const uint16_t* at[3] = {s.m.Dbf, s.Dlo, s.m.Dbf};
+      const uint16_t* bt[3] = {w.Qh, w.Qh, w.Ql};
+      for (int t = 0; t < 3; ++t) {
+        oa[t] = TgOperand{at[t], G.d_out, G.d_in, G.d_in};
+        ob[t] = TgOperand{bt[t], (long long)G.nbT * k, k, k};
+      }
+      TgParams p;
+      memset(&p, 0, sizeof(p));
+      p.M = G.d_out; p.N = k; p.K = k; p.batch = G.nbT; p.nterms = 3;
+      p.rowsA_per_batch = 0; p.colsA_per_batch = k; p.rowsB_per_batch = k;
+      p.divA = 1; p.a_rep_k = k; p.a_rep_r = 1;
+      p.alpha = 2.f;
+      p.C = s.m.D; p.ldc = G.d_in; p.sCb = k;  // batch b writes the columns [b k, b k + k)
+      p.status = status;
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      tg_launch(st, oa, ob, p);
+    }
+    const long long nrec = (long long)G.d_out * G.ng;
+    CQ_LAUNCH(ste_scale_coef_kernel, (unsigned)((nrec * 32 + 255) / 256), 256, 0, st, s.m.D, (long long)G.d_in, s.m.Dbf, s.Dlo,
+              (long long)G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.usel, 1, s.m.coef, status);
+    launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status, 1);
+    minv_path_tc(st, s.gMinv, gradM, G.nbT, k, true, s.kk, status);
+    return;
+  }
   if (need_l2) {
     // E = Minv o Delta, L2 = sum E^2
     bool done = false;
@@ -1273,9 +1362,10 @@ static std::mutex g_noalloc_mu;
 
 extern "C" int cafeq_rtn_noalloc(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
                                  void* stream) {
-  size_t need = 0;
-  int rc = cafeq_workspace_size(d, nullptr, nullptr, &need);
+  Geo Gq;
+  int rc = make_geo(d, &Gq, false);
   if (rc) return rc;
+  const size_t need = matrix_scratch_bytes(Gq, false);  // quantisation only: none of the backward scratch
   if (need > (size_t)CAFEQ_NOALLOC_SCRATCH_BYTES) return CAFEQ_ERR_TOO_LARGE;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return CAFEQ_ERR_CUDA;

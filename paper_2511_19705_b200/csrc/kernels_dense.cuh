@@ -139,6 +139,44 @@ __global__ void add_argmax_kernel(float* __restrict__ gX, long long ld, int rows
   }
 }
 
+// Scale path of the straight-through quantiser from the residual itself: with Uhat = s q and Delta = Uhat - U the
+// derivative of Uhat with respect to the scale is q - U / s = Delta / s, and s = a / qmax, so the coefficient routed
+// to the group's arg-max entry is sign(U at arg-max) / qmax * sum_e gDelta_e Delta_e / s = sign * sum_e gDelta_e Delta_e / a.
+// Delta comes as a two-term bf16 split (row pitch ldd); records are group-major when gm is set.  One warp per record.
+__global__ void ste_scale_coef_kernel(const float* __restrict__ gD, long long ldg, const uint16_t* __restrict__ Dh,
+                                      const uint16_t* __restrict__ Dl, long long ldd, int rows, int ng, int g,
+                                      const float* __restrict__ a, const float* __restrict__ usel, int gm,
+                                      float* __restrict__ coef, const int32_t* status) {
+  if (status && *status) return;
+  const long long w = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= (long long)rows * ng) return;
+  // consecutive warps take consecutive groups of one row (the rows of gD and Delta are read contiguously)
+  const int row = (int)(w / ng), G = (int)(w - (long long)row * ng);
+  float sum = 0.f;
+  for (int e = lane; e < g; e += 32) {
+    const long long col = (long long)G * g + e;
+    const float d = bf16_bits_to_float(Dh[row * ldd + col]) + bf16_bits_to_float(Dl[row * ldd + col]);
+    sum = fmaf(gD[row * ldg + col], d, sum);
+  }
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) {
+    const long long pi = gm ? (long long)G * rows + row : w;
+    const float av = a[pi], u = usel[pi];
+    const float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
+    coef[pi] = (av > 0.f) ? sgn * sum / av : 0.f;
+  }
+}
+
+// acc += sum x[i] y[i]
+__global__ void dot_f32_kernel(const float* __restrict__ x, const float* __restrict__ y, long long n, double* acc) {
+  double s = 0.0;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x)
+    s += (double)x[e] * (double)y[e];
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x & 31) == 0 && s != 0.0) atomicAdd(acc, s);
+}
+
 __global__ void sqrt_hist_kernel(const double* __restrict__ sq, float* __restrict__ out, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = (float)sqrt(fmax(sq[i], 0.0));

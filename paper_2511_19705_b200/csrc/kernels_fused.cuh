@@ -37,6 +37,7 @@ struct BdParams {
   float* usel;         // signed value at the arg-max
   int* idx;            // arg-max position inside the group
   uint16_t* delta;     // bf16 [d_out, d_in], row stride d_in
+  uint16_t* delta_lo;  // optional second bf16 term of the residual (delta + delta_lo carries 16 mantissa bits)
   int8_t* codes;       // [d_out, d_in]
   float* scales;       // [d_out, d_in / G]
   double* sqacc;
@@ -543,7 +544,7 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           for (int ch = 0; ch < 4; ++ch) {
             tc_ld32(taddr + ch * 32, v);
             const float s = sc[(G == 128) ? 0 : (ch >> 1)];
-            uint32_t dpk[16];
+            uint32_t dpk[16], lpk[16];
             uint32_t cpk[8];
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
@@ -552,9 +553,10 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
               q0 = fminf(fmaxf(q0, -p.qmax), p.qmax);
               q1 = fminf(fmaxf(q1, -p.qmax), p.qmax);
               const float d0 = s * q0 - v[e], d1 = s * q1 - v[e + 1];
-              const uint32_t lo = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d0));
-              const uint32_t hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d1));
-              dpk[e >> 1] = lo | (hi << 16);
+              const __nv_bfloat16 b0 = __float2bfloat16_rn(d0), b1 = __float2bfloat16_rn(d1);
+              dpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+              lpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d0 - __bfloat162float(b0))) |
+                            ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d1 - __bfloat162float(b1))) << 16);
               const uint32_t c0 = (uint32_t)((int)q0) & 0xFFu, c1 = (uint32_t)((int)q1) & 0xFFu;
               if ((e & 2) == 0) cpk[e >> 2] = c0 | (c1 << 8);
               else cpk[e >> 2] |= (c0 << 16) | (c1 << 24);
@@ -563,6 +565,11 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
               uint4* dst = reinterpret_cast<uint4*>(p.delta + (long long)row * p.d_in + col0 + ch * 32);
 #pragma unroll
               for (int w4 = 0; w4 < 4; ++w4) dst[w4] = make_uint4(dpk[4 * w4], dpk[4 * w4 + 1], dpk[4 * w4 + 2], dpk[4 * w4 + 3]);
+              if (p.delta_lo) {
+                uint4* dl = reinterpret_cast<uint4*>(p.delta_lo + (long long)row * p.d_in + col0 + ch * 32);
+#pragma unroll
+                for (int w4 = 0; w4 < 4; ++w4) dl[w4] = make_uint4(lpk[4 * w4], lpk[4 * w4 + 1], lpk[4 * w4 + 2], lpk[4 * w4 + 3]);
+              }
             }
             if (valid && (p.epi & EPI_CODES)) {
               uint4* dst = reinterpret_cast<uint4*>(p.codes + (long long)row * p.d_in + col0 + ch * 32);

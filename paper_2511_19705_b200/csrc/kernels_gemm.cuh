@@ -34,6 +34,9 @@ struct TgParams {
   int M, N, K, batch, nterms;
   int rowsA_per_batch, rowsB_per_batch;  // row offset of batch b in the 2-D operand views (0 for a shared operand)
   int divA;                              // batch b reads A rows of batch b / divA
+  int colsA_per_batch;                   // column offset of batch b in the A view (block-diagonal operands: batch b
+                                         // multiplies columns [b * k, b * k + k) of a wide matrix); 0 otherwise
+  int min_ctas;                          // > 0: overrides the process-wide tile-width rule for this launch
   int a_rep_k, a_rep_r;                  // replicated contraction blocks of A: chunk at l reads columns ((l / k) / r) * k + l % k
   float alpha, beta, gamma;
   const float* C0;
@@ -115,6 +118,7 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
         const int l0 = c * TG_BK;
         int xa = l0;
         if (p.a_rep_r > 1) xa = ((l0 / p.a_rep_k) / p.a_rep_r) * p.a_rep_k + (l0 % p.a_rep_k);
+        xa += (b / p.divA) * p.colsA_per_batch;
         uint8_t* st = smem + s * C::STAGE;
         tma_load_2d(smem_u32(st), &maps.a[t], xa, ya, bar_full + 8 * s);
         tma_load_2d(smem_u32(st + C::A_BYTES), &maps.b[t], l0, yb, bar_full + 8 * s);
@@ -348,10 +352,11 @@ static int tg_launch_t(cudaStream_t st, const TgOperand* A, const TgOperand* B, 
 static std::atomic<int> g_tg_min_ctas{28};
 static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, const TgParams& p) {
   if (p.K % TG_BK || p.nterms < 1 || p.nterms > TG_MAX_TERMS) return CAFEQ_ERR_UNSUPPORTED;
+  const int min_ctas = p.min_ctas > 0 ? p.min_ctas : g_tg_min_ctas.load(std::memory_order_relaxed);
   const long long mt = (long long)p.batch * ((p.M + 127) / 128);
-  if (p.N > 128 && mt * ((p.N + 255) / 256) >= g_tg_min_ctas.load(std::memory_order_relaxed)) return tg_launch_t<256>(st, A, B, p);
-  if (p.N > 64 && mt * ((p.N + 127) / 128) >= g_tg_min_ctas.load(std::memory_order_relaxed)) return tg_launch_t<128>(st, A, B, p);
-  if (p.N <= 64 || mt * ((p.N + 127) / 128) < g_tg_min_ctas.load(std::memory_order_relaxed)) return tg_launch_t<64>(st, A, B, p);
+  if (p.N > 128 && mt * ((p.N + 255) / 256) >= min_ctas) return tg_launch_t<256>(st, A, B, p);
+  if (p.N > 64 && mt * ((p.N + 127) / 128) >= min_ctas) return tg_launch_t<128>(st, A, B, p);
+  if (p.N <= 64 || mt * ((p.N + 127) / 128) < min_ctas) return tg_launch_t<64>(st, A, B, p);
   return tg_launch_t<128>(st, A, B, p);
 }
 

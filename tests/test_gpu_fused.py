@@ -149,3 +149,39 @@ def test_fused_full_size_v_matrix_output_axis(cq):
                                  trole=cq.APPLY_TT)
     U = orc.apply_blocks(w64(Wb), np.transpose(orc.round_bf16(M), (0, 2, 1)), "out")
     assert_codes_tie_aware(codes.cpu().numpy(), scales.cpu().numpy(), orc.quant_sym(U, 3, 128), U, 128)
+
+
+# ------------------------------------------------------------------ straight-through mode on the tensor cores
+# input axis, d_in % 256 == 0, d_out % 64 == 0: the residual leaves the pass as a two-term bf16 split and every
+# product of the backward (Gram matrix of the residual, Minv^T Minv, the apply of that to the residual) is a
+# three-term tensor-core product; compared with the float64 oracle like the shape-agnostic path
+STE_SHAPES = [(64, 64, 4, (128, 256)), (128, 128, 3, (320, 512)), (256, 128, 3, (576, 768)), (256, 64, 4, (192, 512)),
+              (128, 64, 4, (1088, 256))]
+
+
+@pytest.mark.parametrize("k,group,bits,shape", STE_SHAPES)
+def test_fused_single_ste_matches_oracle(cq, k, group, bits, shape):
+    d_out, d_in = shape
+    Wb = syn.weight_student_t(d_out, d_in, seed=77, n_outlier_channels=2, mult=10.0)
+    nb = d_in // k
+    M = syn.perturbed_blocks(nb, k, 19, 0.1)
+    out = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=bits, group=group, loss_kind=cq.LOSS_L2_STE)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    W = w64(Wb)
+    f = orc.single_forward(W, M, bits, group, "in")
+    g = orc.single_grad_ste(W, f, bits, group, "in")
+    L = out["losses"].cpu().numpy()
+    assert abs(L[0] - f["surrogate"]) <= TOL * f["surrogate"]
+    assert abs(L[1] - f["L2"]) <= TOL * f["L2"]
+    assert abs(L[2] - f["normW2"]) <= 1e-5 * f["normW2"]
+    gg = out["gradM"].cpu().numpy()
+    assert np.isfinite(gg).all()
+    # near-tie code flips change single terms of the scale path: compare over all blocks together too
+    assert rel_err(gg, g) <= 2 * TOL
+    for b in range(nb):
+        assert rel_err(gg[b], g[b]) <= 5 * TOL, f"block {b}"
+    # the shape-agnostic path of the same call agrees as well
+    ref = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=bits, group=group, loss_kind=cq.LOSS_L2_STE,
+                                      flags=cq.FLAG_GENERIC)
+    assert rel_err(gg, ref["gradM"].cpu().numpy()) <= 2 * TOL
