@@ -698,6 +698,7 @@ extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_mat
     b += (d1n * d3n * 4 + 256);
     const int rr = d2->replicas > 0 ? d2->replicas : 1;
     b += dense_scratch_bytes(d1->d_out, d1->d_in, d2->d_out, rr, d1->tblock > 0 ? d1->tblock : d1->d_out, G1.ng, G2.ng);
+    b += 3 * ((size_t)G2.n * 2 + 256);  // transposed second factor and its gradient split (straight-through pair mode)
   }
   *bytes = b;
   return CAFEQ_OK;
@@ -1055,7 +1056,36 @@ struct PairWS {
   KkWS kk;
   DenseWS dn;
   bool dense;  // the product term runs on the tensor cores (every dimension a multiple of 64)
+  uint16_t *W2T, *gVTh, *gVTl;  // [r h, d3]: transposed second factor and transposed split of its gradient
 };
+
+// Operator gradient of a block-diagonal apply as batched k x k tensor-core products with a two-term split of the
+// fp32 factor: out[b][m][n] (+)= sum_l A[(b r + rep) k + m][l] * (Bh + Bl)[(b r + rep) k + n][l], summed over rep.
+// A bf16 [nb r k, K] (pitch lda), Bh / Bl bf16 [nb r k, K] (pitch K).
+static void opgrad_tc(cudaStream_t st, const uint16_t* A, long long lda, const uint16_t* Bh, const uint16_t* Bl, int nb, int r,
+                      int k, int K, float* out, bool a_is_split_side, int32_t* status) {
+  (void)a_is_split_side;
+  for (int rep = 0; rep < r; ++rep) {
+    TgOperand oa[2], ob[2];
+    const long long rows = (long long)nb * r * k - (long long)rep * k;
+    oa[0] = oa[1] = TgOperand{A + (long long)rep * k * lda, rows, K, lda};
+    ob[0] = TgOperand{Bh + (long long)rep * k * K, rows, K, K};
+    ob[1] = TgOperand{Bl + (long long)rep * k * K, rows, K, K};
+    TgParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = p.N = k; p.K = K; p.batch = nb; p.nterms = 2;
+    p.rowsA_per_batch = p.rowsB_per_batch = r * k;
+    p.divA = 1; p.a_rep_k = K; p.a_rep_r = 1;
+    p.alpha = 1.f;
+    p.beta = rep ? 1.f : 0.f;
+    p.C0 = rep ? out : nullptr; p.ldc0 = k; p.sC0b = (long long)k * k;
+    p.C = out; p.ldc = k; p.sCb = (long long)k * k;
+    p.min_ctas = 148;  // long contraction, few output tiles: the narrowest tile
+    p.status = status;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    tg_launch(st, oa, ob, p);
+  }
+}
 
 static bool dense_ok(const Geo& G1, const Geo& G2) {
   return G1.d_out % 64 == 0 && G1.d_in % 64 == 0 && G2.d_out % 64 == 0 && G2.d_in % 64 == 0 && G1.k % 32 == 0;
@@ -1077,6 +1107,12 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
   carve_kk(b, G1.nbT, G1.k, &p->kk);
   p->dense = need_R && dense_ok(G1, G2);
   if (p->dense) carve_dense(b, G1.d_out, G1.d_in, G2.d_out, G2.r, G1.k, G1.ng, G2.ng, &p->dn);
+  p->W2T = p->gVTh = p->gVTl = nullptr;
+  if (p->dense) {
+    p->W2T = b.take<uint16_t>(G2.n);
+    p->gVTh = b.take<uint16_t>(G2.n);
+    p->gVTl = b.take<uint16_t>(G2.n);
+  }
   return !b.overflow;
 }
 
@@ -1186,8 +1222,26 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
       CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
       CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
     }
-    launch_opgrad(st, w.U, G1.d_in, W1, 1, G1.ld, G1, gradM, 1, 1.f, status);    // U side: operator M^T
-    launch_opgrad(st, w.V, G2.d_in, W2, 1, G2.ld, G2, p.gMinv, 0, 1.f, status);  // V side: operator Minv
+    const bool og_tc = tc && ((uintptr_t)W1 % 16 == 0) && (G1.ld % 8 == 0) && ((uintptr_t)W2 % 4 == 0) && G1.r == 1;
+    if (og_tc) {
+      // U side (operator M^T): gradM[b][m][n] = sum_c W1[b k + m][c] gU[b k + n][c], contraction along the rows' own
+      // direction: both operands as they are stored
+      launch_split_rect(st, w.U, w.h, w.d1, w.d1, 1.f, nullptr, nullptr, nullptr, w.Awh, w.Awl, nullptr, nullptr, status);
+      opgrad_tc(st, (const uint16_t*)W1, G1.ld, w.Awh, w.Awl, G1.nbT, 1, k, G1.d_in, gradM, false, status);
+      // V side (operator Minv): gMinv[b][i][j] = sum over replicas and rows o of gV[o][.. + i] W2[o][.. + j]: the
+      // contraction runs down the columns, so both factors are transposed first
+      {
+        dim3 tg((G2.d_in + 31) / 32, (G2.d_out + 31) / 32);
+        CQ_LAUNCH(transpose_bf16_kernel, tg, dim3(32, 8), 0, st, (const uint16_t*)W2, G2.d_out, G2.d_in, G2.ld, p.W2T);
+      }
+      launch_split_rect(st, w.V, w.d3, w.rh, w.rh, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, p.gVTh, p.gVTl, status);
+      opgrad_tc(st, p.W2T, G2.d_out, p.gVTh, p.gVTl, G1.nbT, G2.r, k, G2.d_out, p.RM, true, status);
+      // (W2^T as the first factor gives the transpose: RM[b][j][i]; put it back as gMinv[b][i][j])
+      CQ_LAUNCH(transpose_blocks_kernel, grid_for(kk), 256, 0, st, p.RM, p.gMinv, k, kk);
+    } else {
+      launch_opgrad(st, w.U, G1.d_in, W1, 1, G1.ld, G1, gradM, 1, 1.f, status);    // U side: operator M^T
+      launch_opgrad(st, w.V, G2.d_in, W2, 1, G2.ld, G2, p.gMinv, 0, 1.f, status);  // V side: operator Minv
+    }
     if (tc) {
       minv_path_tc(st, p.gMinv, gradM, G1.nbT, k, true, p.kk, status);
     } else {
