@@ -78,3 +78,25 @@ def test_chunked_pair_run_with_resume_matches_one_call(cq):
     # same arithmetic in the same order up to the floating-point atomics of the reductions
     assert rel_err(Mb.cpu().numpy() - M0, Ma.cpu().numpy() - M0) <= 1e-3
     assert abs(float(hb[0, 0].item()) - float(ha[2, 0].item())) <= 1e-4 * abs(float(ha[2, 0].item()))
+
+
+def test_product_tile_rule_does_not_change_results(cq):
+    """The process-wide tile-width knob of the k x k products is a tuning parameter only: forward + backward of a
+    single matrix give the same losses and (to accumulation order) the same gradient with narrow and wide tiles."""
+    k, d_out, d_in = 256, 192, 768
+    Wb = syn.weight_student_t(d_out, d_in, seed=5, n_outlier_channels=2, mult=10.0)
+    M = f32_dev(syn.perturbed_blocks(d_in // k, k, 9, 0.1))
+    outs = []
+    try:
+        for n in (96, 1):
+            cq.set_product_min_ctas(n)
+            o = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), M, bits=3, group=128, flags=cq.FLAG_EXACT_LOSS)
+            torch.cuda.synchronize()
+            assert int(o["status"].item()) == 0
+            outs.append((o["losses"].cpu().numpy().copy(), o["gradM"].cpu().numpy().copy()))
+        with pytest.raises(RuntimeError):
+            cq.set_product_min_ctas(0)
+    finally:
+        cq.set_product_min_ctas(28)
+    assert np.allclose(outs[0][0], outs[1][0], rtol=1e-6)
+    assert rel_err(outs[0][1], outs[1][1]) <= 1e-5
