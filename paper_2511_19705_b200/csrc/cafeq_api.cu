@@ -15,6 +15,7 @@
 #include "kernels_fused.cuh"
 #include "kernels_bwd.cuh"
 #include "kernels_gemm.cuh"
+#include "kernels_dense.cuh"
 
 namespace cafeq {
 
@@ -587,12 +588,47 @@ static bool fused_pass(cudaStream_t st, const void* X, long long ldx, const Geo&
   return rc == CAFEQ_OK;
 }
 
+// U = T o W in fp32 as one-term batched products on the tensor cores (bf16 x bf16 products are exact, fp32
+// accumulation: the same arithmetic as the fused pass).  Tb: bf16 operator blocks in applied orientation
+// [nbT k, k].  Output axis: the contraction runs down the rows of W, so its transpose goes through WT first.
+static bool apply_tc(cudaStream_t st, const void* W, const Geo& G, const uint16_t* Tb, float* U, uint16_t* WT, int32_t* status) {
+  const int k = G.k;
+  if (!kk_fast(k) || ((uintptr_t)W & 15) || (G.ld % 8) || (G.d_in % 4)) return false;
+  TgOperand oa[1], ob[1];
+  TgParams p;
+  memset(&p, 0, sizeof(p));
+  p.nterms = 1; p.K = k; p.batch = G.nbq; p.alpha = 1.f;
+  p.a_rep_k = k; p.a_rep_r = 1; p.divA = 1;
+  p.C = U; p.ldc = G.d_in;
+  p.status = status;
+  if (G.axis == CAFEQ_AXIS_IN) {
+    oa[0] = TgOperand{W, G.d_out, G.d_in, G.ld};
+    ob[0] = TgOperand{Tb, (long long)G.nbT * k, k, k};
+    p.M = G.d_out; p.N = k;
+    p.rowsA_per_batch = 0; p.colsA_per_batch = k;
+    p.rowsB_per_batch = k; p.divB = G.r;
+    p.sCb = k;
+  } else {
+    if (!WT || (G.d_out % 8)) return false;
+    dim3 tg((G.d_in + 31) / 32, (G.d_out + 31) / 32);
+    CQ_LAUNCH(transpose_bf16_kernel, tg, dim3(32, 8), 0, st, (const uint16_t*)W, G.d_out, G.d_in, G.ld, WT);
+    oa[0] = TgOperand{Tb, (long long)G.nbT * k, k, k};
+    ob[0] = TgOperand{WT, G.d_in, G.d_out, G.d_out};
+    p.M = k; p.N = G.d_in;
+    p.rowsA_per_batch = k; p.divA = G.r;
+    p.rowsB_per_batch = 0; p.colsB_per_batch = k;
+    p.sCb = (long long)k * G.d_in;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return tg_launch(st, oa, ob, p) == CAFEQ_OK;
+}
+
 // U = T o W, group absmax / arg-max, and (optionally) the quantiser outputs.  Returns true when the fused
 // tensor-core pass ran (then the residual is in w.Dbf as bf16 instead of w.D as fp32, and U is not stored).
 static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits, const float* Tc, int transposed,
                           const MatWS& w, const void* offsets, int off_kind, bool want_delta, float* Uhat, int8_t* codes,
                           float* scales, int32_t* status, bool allow_fused, const BdParams* surr = nullptr,
-                          const uint16_t* Tb_ready = nullptr) {
+                          const uint16_t* Tb_ready = nullptr, uint16_t* WT_scratch = nullptr) {
   if (Tc && allow_fused && off_kind == CAFEQ_OFFSETS_NONE && !Uhat) {
     BdParams p;
     memset(&p, 0, sizeof(p));
@@ -603,7 +639,15 @@ static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits
     p.delta = w.Dbf; p.codes = codes; p.scales = scales;
     if (fused_pass(st, W, G.ld, G, Tc, transposed, w.Tb, p, status, Tb_ready)) return true;
   }
-  if (Tc) launch_apply(st, W, 1, G.ld, G, Tc, transposed, w.U, G.d_in, GEMM_STORE, nullptr, status);
+  bool applied = false;
+  if (Tc && allow_fused) {  // (allow_fused is off when the caller asked for the shape-agnostic kernels)
+    const uint16_t* Tb = (Tb_ready && !transposed) ? Tb_ready : w.Tb;
+    const long long kk = (long long)G.nbT * G.k * G.k;
+    if (Tb == w.Tb && kk_fast(G.k)) CQ_LAUNCH(operator_to_bf16_kernel, grid_for(kk), 256, 0, st, Tc, w.Tb, G.k, kk, transposed, status);
+    applied = apply_tc(st, W, G, Tb, w.U, WT_scratch, status);
+  }
+  if (applied) {
+  } else if (Tc) launch_apply(st, W, 1, G.ld, G, Tc, transposed, w.U, G.d_in, GEMM_STORE, nullptr, status);
   else CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, w.U);
   launch_absmax(st, w.U, G.d_in, G, w.a, w.usel, w.idx, status);
   if (want_delta || Uhat || codes)
@@ -699,6 +743,7 @@ extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_mat
     const int rr = d2->replicas > 0 ? d2->replicas : 1;
     b += dense_scratch_bytes(d1->d_out, d1->d_in, d2->d_out, rr, d1->tblock > 0 ? d1->tblock : d1->d_out, G1.ng, G2.ng);
     b += 3 * ((size_t)G2.n * 2 + 256);  // transposed second factor and its gradient split (straight-through pair mode)
+    b += (size_t)G1.n * 2 + 256;        // transposed first factor
   }
   *bytes = b;
   return CAFEQ_OK;
@@ -1057,6 +1102,7 @@ struct PairWS {
   DenseWS dn;
   bool dense;  // the product term runs on the tensor cores (every dimension a multiple of 64)
   uint16_t *W2T, *gVTh, *gVTl;  // [r h, d3]: transposed second factor and transposed split of its gradient
+  uint16_t* W1T;                // [d1, h]: transposed first factor (its apply contracts down the rows)
 };
 
 // Operator gradient of a block-diagonal apply as batched k x k tensor-core products with a two-term split of the
@@ -1107,8 +1153,9 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
   carve_kk(b, G1.nbT, G1.k, &p->kk);
   p->dense = need_R && dense_ok(G1, G2);
   if (p->dense) carve_dense(b, G1.d_out, G1.d_in, G2.d_out, G2.r, G1.k, G1.ng, G2.ng, &p->dn);
-  p->W2T = p->gVTh = p->gVTl = nullptr;
+  p->W2T = p->gVTh = p->gVTl = p->W1T = nullptr;
   if (p->dense) {
+    p->W1T = b.take<uint16_t>(G1.n);
     p->W2T = b.take<uint16_t>(G2.n);
     p->gVTh = b.take<uint16_t>(G2.n);
     p->gVTl = b.take<uint16_t>(G2.n);
@@ -1150,7 +1197,7 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, p.Minv, p.Minv_c, kk, status);
   // U = M_c^T o W1 (axis OUT), V = Minv_c o W2 (axis IN); Uhat kept in the E buffers when PQE is wanted
   const bool f1 = forward_quant(st, W1, G1, d1->bits, p.Mc, 1, p.m1, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m1.E : nullptr, nullptr,
-                nullptr, status, !force_generic);
+                nullptr, status, !force_generic, nullptr, nullptr, p.W1T);
   const bool f2 = forward_quant(st, W2, G2, d2->bits, p.Minv_c, 0, p.m2, nullptr, CAFEQ_OFFSETS_NONE, false, want_pqe ? p.m2.E : nullptr,
                 nullptr, nullptr, status, !force_generic, nullptr, tc ? p.kk.Xh[p.kk.cur] : nullptr);  // Xh = bf16(Minv)
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;

@@ -36,6 +36,7 @@ struct TgParams {
   int divA;                              // batch b reads A rows of batch b / divA
   int colsA_per_batch;                   // column offset of batch b in the A view (block-diagonal operands: batch b
                                          // multiplies columns [b * k, b * k + k) of a wide matrix); 0 otherwise
+  int divB, colsB_per_batch;             // the same for B (divB = 0 means 1)
   int min_ctas;                          // > 0: overrides the process-wide tile-width rule for this launch
   int a_rep_k, a_rep_r;                  // replicated contraction blocks of A: chunk at l reads columns ((l / k) / r) * k + l % k
   float alpha, beta, gamma;
@@ -109,7 +110,8 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
   if (warp == 0) {
     if (lane == 0) {
       const int ya = (b / p.divA) * p.rowsA_per_batch + m0;
-      const int yb = b * p.rowsB_per_batch + n0;
+      const int bb = p.divB > 1 ? b / p.divB : b;
+      const int yb = bb * p.rowsB_per_batch + n0;
       for (int it = 0; it < total; ++it) {
         const int t = it / kchunks, c = it - t * kchunks;
         const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
@@ -121,7 +123,7 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
         xa += (b / p.divA) * p.colsA_per_batch;
         uint8_t* st = smem + s * C::STAGE;
         tma_load_2d(smem_u32(st), &maps.a[t], xa, ya, bar_full + 8 * s);
-        tma_load_2d(smem_u32(st + C::A_BYTES), &maps.b[t], l0, yb, bar_full + 8 * s);
+        tma_load_2d(smem_u32(st + C::A_BYTES), &maps.b[t], l0 + bb * p.colsB_per_batch, yb, bar_full + 8 * s);
       }
     }
   } else if (warp == 1) {
