@@ -137,6 +137,20 @@ def pow2_diag_blocks(nb: int, k: int, seed: int, emin: int = -3, emax: int = 3) 
     return out
 
 
+def hadamard_blocks(nb: int, k: int, seed: int) -> np.ndarray:
+    """Randomised Hadamard blocks H diag(+-1) / sqrt(k) (k a power of two; Sylvester construction): the fixed,
+    data-independent rotation used as the random baseline.  For k = 4^m every entry is +-2^-m, exact in bf16."""
+    assert k > 0 and (k & (k - 1)) == 0
+    h = np.ones((1, 1))
+    while h.shape[0] < k:
+        h = np.block([[h, h], [h, -h]])
+    rng = _rng(seed, 8)
+    out = np.empty((nb, k, k), dtype=np.float64)
+    for b in range(nb):
+        out[b] = h * rng.choice([-1.0, 1.0], size=k)[None, :] / np.sqrt(k)
+    return out.astype(np.float32)
+
+
 # --------------------------------------------------------------------------
 # workload tables (shapes of the benchmark configurations)
 # --------------------------------------------------------------------------

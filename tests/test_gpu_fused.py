@@ -185,3 +185,37 @@ def test_fused_single_ste_matches_oracle(cq, k, group, bits, shape):
     ref = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=bits, group=group, loss_kind=cq.LOSS_L2_STE,
                                       flags=cq.FLAG_GENERIC)
     assert rel_err(gg, ref["gradM"].cpu().numpy()) <= 2 * TOL
+
+
+# ------------------------------------------------------------------ the random baseline through the same kernels
+def test_randomised_hadamard_baseline_and_learning(cq):
+    """Heavy-tailed weights with outlier input channels, 3-bit, g = 128, k = 256: a randomised Hadamard block transform
+    (the fixed rotation baseline, Section 5) goes through the fused pass like any other operator - codes tie-aware
+    against the oracle - and lowers the relative l2 error of plain round-to-nearest; gradient descent on Eq. 4
+    started from it lowers it further (Table 1's ordering: learned < random rotation < none)."""
+    k, d_out, d_in, bits, group = 256, 512, 1024, 3, 128
+    Wb = syn.weight_student_t(d_out, d_in, seed=2025, n_outlier_channels=4, mult=15.0)
+    Wd, W = to_dev(Wb), w64(Wb)
+    H = syn.hadamard_blocks(d_in // k, k, 31)
+    assert np.array_equal(orc.round_bf16(H), H.astype(np.float64))          # +-1/16: exact in bf16
+    codes, scales = cq.cafeq_rtn(Wd, f32_dev(H), bits=bits, group=group, tblock=k)
+    U = orc.apply_blocks(W, H.astype(np.float64), "in")
+    assert_codes_tie_aware(codes.cpu().numpy(), scales.cpu().numpy(), orc.quant_sym(U, bits, group), U, group)
+
+    def rel_l2(M):
+        o = cq.cafeq_proxy_loss_fwd_bwd(Wd, f32_dev(M), bits=bits, group=group, flags=cq.FLAG_EXACT_LOSS | cq.FLAG_NO_GRAD)
+        L = o["losses"].cpu().numpy()
+        return float(np.sqrt(L[1] / L[2]))
+
+    e_id, e_h = rel_l2(syn.identity_blocks(d_in // k, k)), rel_l2(H)
+    f = orc.single_forward(W, H, bits, group, "in")
+    assert abs(e_h - np.sqrt(f["L2"] / f["normW2"])) <= 1e-3 * e_h
+    assert e_h < 0.9 * e_id
+    M = f32_dev(H)
+    g0 = cq.cafeq_proxy_loss_fwd_bwd(Wd, M, bits=bits, group=group)["gradM"]
+    cfg = cq.make_cfg(loss_kind=cq.LOSS_SURROGATE, optimizer=cq.OPT_GD, lr=float(2e-3 / g0.abs().max().item()), steps=150)
+    _, status, _ = cq.cafeq_optimize_single(Wd, M, cfg, bits=bits, group=group)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    e_learned = rel_l2(M.cpu().numpy())
+    assert e_learned < e_h
