@@ -214,13 +214,13 @@ int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed,
 
 const char* cafeq_status_string(int status);
 int cafeq_version(void);
-/* Tuning knob, process-wide (the paper has no counterpart): the k x k products of the block algebra (Newton-Schulz
- * inverse, M^-1 path of the gradient, orthonormality term) pick the widest output tile that still yields at
- * least n CTAs.  Small n (default 28: always the widest tile at k = 256) minimises SM time per product, which is
- * what counts when several problems run concurrently in different streams; n = 96 minimises the latency of a
- * single product chain when one problem runs alone.  Results do not depend on it.  Returns
- * CAFEQ_ERR_INVALID_ARG outside 1..4096. */
-int cafeq_set_product_min_ctas(int n);
+/* Tuning knob, process-wide (the paper has no counterpart).  overlapped = 1 (default): the caller runs several
+ * problems concurrently in different streams (the matrices and pairs of a layer are independent), so kernels
+ * should cost few SM-microseconds rather than finish one chain as early as possible: the k x k products of the
+ * block algebra take the widest output tile (fewest CTAs), and the transform pass gives a small matrix fewer CTAs
+ * (at least 6 tiles each).  overlapped = 0: one problem runs alone: narrow product tiles (about one CTA per SM)
+ * and every SM on every pass.  Results do not depend on it.  CAFEQ_ERR_INVALID_ARG unless 0 or 1. */
+int cafeq_set_overlap_mode(int overlapped);
 
 /* Number of kernels this library has launched in the calling process so far (host counter, for
  * benchmarks that must state how many of the library's kernels ran inside a timed region). */

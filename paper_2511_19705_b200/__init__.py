@@ -25,7 +25,7 @@ OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_set_product_min_ctas", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_pack", "cafeq_set_overlap_mode", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
     "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
@@ -80,10 +80,10 @@ def version() -> int:
     return lib().cafeq_version()
 
 
-def set_product_min_ctas(n: int) -> None:
-    """Process-wide tile-width rule of the k x k products: small n (default 28) favours throughput when several
-    problems run in different streams, 96 the latency of one problem running alone."""
-    _check(lib().cafeq_set_product_min_ctas(ctypes.c_int(int(n))), "cafeq_set_product_min_ctas")
+def set_overlap_mode(overlapped: bool) -> None:
+    """Process-wide launch-shape rule: True (default) when several problems run concurrently in different streams
+    (kernels then take fewer CTAs: fewer SM-microseconds each), False when one problem runs alone (lowest latency)."""
+    _check(lib().cafeq_set_overlap_mode(ctypes.c_int(1 if overlapped else 0)), "cafeq_set_overlap_mode")
 
 
 def launch_count() -> int:

@@ -685,9 +685,10 @@ extern "C" int cafeq_version(void) { return 100; }
 
 extern "C" long long cafeq_debug_launch_count(void) { return g_launches.load(); }
 
-extern "C" int cafeq_set_product_min_ctas(int n) {
-  if (n < 1 || n > 4096) return CAFEQ_ERR_INVALID_ARG;
-  g_tg_min_ctas.store(n, std::memory_order_relaxed);
+extern "C" int cafeq_set_overlap_mode(int overlapped) {
+  if (overlapped != 0 && overlapped != 1) return CAFEQ_ERR_INVALID_ARG;
+  g_tg_min_ctas.store(overlapped ? 28 : 96, std::memory_order_relaxed);
+  g_bd_min_tiles.store(overlapped ? 6 : 1, std::memory_order_relaxed);
   return CAFEQ_OK;
 }
 

@@ -12,6 +12,8 @@
 // word, all roles leave their loops, tensor memory is released and the kernel returns.
 #pragma once
 
+#include <atomic>
+
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -662,6 +664,8 @@ static bool bd_supported(int form, int d_out, int d_in, long long ld, int k, int
   return true;
 }
 
+static std::atomic<int> g_bd_min_tiles{6};
+
 template <int FORM, int K, int G>
 static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmT, BdParams p) {
   using C = BdCfg<FORM, K, G>;
@@ -679,7 +683,12 @@ static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMa
     p.n_minor = (p.d_in + C::NC - 1) / C::NC;
   }
   const long long total = (long long)p.n_major * p.n_minor;
-  const int grid = total < 148 ? (int)total : 148;  // one persistent CTA per SM
+  // one persistent CTA per SM at most; when several problems overlap in streams, small matrices take fewer CTAs
+  // (at least g_bd_min_tiles tiles each): the fixed cost of a CTA is spread over more tiles and the SMs left over
+  // run another problem's kernel
+  long long want = total / g_bd_min_tiles.load(std::memory_order_relaxed);
+  if (want < 1) want = 1;
+  const int grid = want < 148 ? (int)want : 148;
   p.ctas_per_major = 0;
   bd_pass_kernel<FORM, K, G><<<grid, BD_THREADS, C::SMEM, st>>>(tmX, tmT, p);
   return CAFEQ_OK;

@@ -17,7 +17,7 @@ import ctypes
 import torch
 
 from . import (AXIS_IN, LOSS_PQE_STE, OPT_STATE_HEADER, cafeq_pair_product, FLAG_EXACT_LOSS, LOSS_LSE, LOSS_SURROGATE, OFFSETS_NONE, OPT_ADAM, OPT_GD, _check, _p,
-               _pair_descs, _stream, lib, make_cfg, make_desc, set_product_min_ctas, workspace_size)
+               _pair_descs, _stream, lib, make_cfg, make_desc, set_overlap_mode, workspace_size)
 
 
 class SingleProblem:
@@ -125,9 +125,9 @@ class LayerStep:
 
     def opt_step(self, eval_exact=False):
         probs = self.singles + self.pairs
-        # wide product tiles when the problems overlap (fewer SM-microseconds each), narrow ones when a single
-        # chain of kernels runs alone (lower latency)
-        set_product_min_ctas(28 if self.parallel else 96)
+        # launch shapes for overlapping problems (fewer SM-microseconds per kernel) or for a single chain of kernels
+        # running alone (lowest latency)
+        set_overlap_mode(self.parallel)
         if not self.parallel:
             for p in probs:
                 p.opt_step(p.ws, eval_exact)

