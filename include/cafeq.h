@@ -218,7 +218,7 @@ int cafeq_version(void);
  * problems concurrently in different streams (the matrices and pairs of a layer are independent), so kernels
  * should cost few SM-microseconds rather than finish one chain as early as possible: the k x k products of the
  * block algebra take the widest output tile (fewest CTAs), and the transform pass gives a small matrix fewer CTAs
- * (at least 6 tiles each).  overlapped = 0: one problem runs alone: narrow product tiles (about one CTA per SM)
+ * (at least 14 tiles each; the sparse backward likewise).  overlapped = 0: one problem runs alone: narrow product tiles (about one CTA per SM)
  * and every SM on every pass.  Results do not depend on it.  CAFEQ_ERR_INVALID_ARG unless 0 or 1. */
 int cafeq_set_overlap_mode(int overlapped);
 

@@ -688,7 +688,8 @@ extern "C" long long cafeq_debug_launch_count(void) { return g_launches.load(); 
 extern "C" int cafeq_set_overlap_mode(int overlapped) {
   if (overlapped != 0 && overlapped != 1) return CAFEQ_ERR_INVALID_ARG;
   g_tg_min_ctas.store(overlapped ? 28 : 96, std::memory_order_relaxed);
-  g_bd_min_tiles.store(overlapped ? 6 : 1, std::memory_order_relaxed);
+  g_bd_min_tiles.store(overlapped ? 14 : 1, std::memory_order_relaxed);
+  g_bw_min_tiles.store(overlapped ? 14 : 6, std::memory_order_relaxed);
   return CAFEQ_OK;
 }
 

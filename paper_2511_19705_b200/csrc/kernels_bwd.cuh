@@ -323,6 +323,8 @@ static bool bw_supported(int axis_in, int d_out, int d_in, long long ld, int k, 
   return true;
 }
 
+static std::atomic<int> g_bw_min_tiles{14};  // tiles per CTA at least (more when problems overlap: see cafeq_set_overlap_mode)
+
 template <int FORM, int K, int SWAP>
 static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& p) {
   using C = BwCfg<K>;
@@ -335,7 +337,7 @@ static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& 
   // one persistent CTA per SM at most; small problems use fewer CTAs so that every CTA has several tiles per
   // flush (a flush moves k * k floats whatever the number of tiles behind it)
   const long long total = (long long)p.n_major * p.n_minor;
-  long long want = total / 6;
+  long long want = total / g_bw_min_tiles.load(std::memory_order_relaxed);
   if (want < p.n_major) want = p.n_major;
   if (want > total) want = total;
   const int grid = want < 148 ? (int)want : 148;
