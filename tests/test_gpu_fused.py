@@ -219,3 +219,24 @@ def test_randomised_hadamard_baseline_and_learning(cq):
     assert int(status.item()) == 0
     e_learned = rel_l2(M.cpu().numpy())
     assert e_learned < e_h
+
+
+def test_fused_full_size_k_matrix_straight_through(cq):
+    """k of the 9B-shaped layer (2048 x 3584, k = 256, 3-bit, g = 128) in the straight-through mode, on the launch
+    configuration the benchmark's `--loss ste` run times: losses and the whole gradient against the oracle."""
+    name, d_out, d_in = "k", 2048, 3584
+    Wb = syn.make_weight(3, name, d_out, d_in)
+    M = syn.make_transform(name, d_in // 256, 256)
+    out = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=3, group=128, loss_kind=cq.LOSS_L2_STE)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    W = w64(Wb)
+    f = orc.single_forward(W, M, 3, 128, "in")
+    g = orc.single_grad_ste(W, f, 3, 128, "in")
+    L = out["losses"].cpu().numpy()
+    assert abs(L[1] - f["L2"]) <= TOL * f["L2"]
+    assert abs(L[2] - f["normW2"]) <= 1e-5 * f["normW2"]
+    gg = out["gradM"].cpu().numpy()
+    assert rel_err(gg, g) <= 2 * TOL
+    for b in range(d_in // 256):
+        assert rel_err(gg[b], g[b]) <= 5 * TOL, f"block {b}"
