@@ -168,13 +168,15 @@ __global__ void ste_scale_coef_kernel(const float* __restrict__ gD, long long ld
   }
 }
 
-// acc += sum x[i] y[i]
-__global__ void dot_f32_kernel(const float* __restrict__ x, const float* __restrict__ y, long long n, double* acc) {
+// acc += sum x[i] y[i]  (fp32 products summed in double; one atomic per block)
+__global__ void __launch_bounds__(256) dot_f32_kernel(const float* __restrict__ x, const float* __restrict__ y, long long n,
+                                                      double* acc) {
+  __shared__ double red[32];
   double s = 0.0;
   for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x)
-    s += (double)x[e] * (double)y[e];
-  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if ((threadIdx.x & 31) == 0 && s != 0.0) atomicAdd(acc, s);
+    s += (double)(x[e] * y[e]);
+  s = block_sum_double(s, red);
+  if (threadIdx.x == 0 && s != 0.0) atomicAdd(acc, s);
 }
 
 __global__ void sqrt_hist_kernel(const double* __restrict__ sq, float* __restrict__ out, int n) {

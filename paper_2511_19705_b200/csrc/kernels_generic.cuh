@@ -973,11 +973,31 @@ __global__ void sqsum_bf16_kernel(const uint16_t* __restrict__ W, long long ld, 
   if (status && *status) return;
   __shared__ double red[32];
   double local = 0.0;
-  const long long n = (long long)rows * cols;
-  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
-    int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
-    float v = bf16_bits_to_float(W[row * ld + col]);
-    local += (double)v * v;
+  if ((cols % 8) == 0 && (ld % 8) == 0 && ((uintptr_t)W % 16) == 0) {
+    // eight values per 16-byte load, fp32 inside the chunk (double arithmetic is scarce), double across chunks
+    const int cpr = cols / 8;
+    const long long nch = (long long)rows * cpr;
+    for (long long c = blockIdx.x * (long long)blockDim.x + threadIdx.x; c < nch; c += (long long)gridDim.x * blockDim.x) {
+      const long long row = c / cpr;
+      const int cc = (int)(c - row * cpr);
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(W + row * ld) + cc);
+      const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+      float s = 0.f;
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const float lo = __uint_as_float(w4[h] << 16), hi = __uint_as_float(w4[h] & 0xFFFF0000u);
+        s = fmaf(lo, lo, s);
+        s = fmaf(hi, hi, s);
+      }
+      local += (double)s;
+    }
+  } else {
+    const long long n = (long long)rows * cols;
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+      int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
+      float v = bf16_bits_to_float(W[row * ld + col]);
+      local += (double)v * v;
+    }
   }
   double s = block_sum_double(local, red);
   if (threadIdx.x == 0) atomicAdd(acc, s);
