@@ -179,6 +179,66 @@ __global__ void __launch_bounds__(256) dot_f32_kernel(const float* __restrict__ 
   if (threadIdx.x == 0 && s != 0.0) atomicAdd(acc, s);
 }
 
+// Power iteration for the largest singular value of S [R, C] (fp32, row-major), used to scale the starting guess
+// of the pseudo-inverse iteration.  v [C], u [R] scratch; three small kernels per round:
+//   u = S v (one warp per row);  v2 = S^T u (one thread per column), nrm += |v2|^2;  v = v2 / |v2|.
+// After the last round *sig2 = safety * |S^T S v| (v of unit norm): a Rayleigh-type estimate from below of sigma_max^2.
+__global__ void pw_init_kernel(float* __restrict__ v, int C, double* nrm) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < C) {
+    uint32_t h = (uint32_t)j * 2654435761u;
+    h ^= h >> 15;
+    v[j] = ((h & 1u) ? 1.f : -1.f) * rsqrtf((float)C);  // fixed +-1 pattern of unit norm
+  }
+  if (j == 0) *nrm = 0.0;
+}
+__global__ void pw_rows_kernel(const float* __restrict__ S, const float* __restrict__ v, int R, int C, float* __restrict__ u) {
+  const long long w = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= R) return;
+  float s = 0.f;
+  for (int j = lane; j < C; j += 32) s = fmaf(S[w * C + j], v[j], s);
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) u[w] = s;
+}
+// grid: (ceil(C / 256), row slices); partial sums are added atomically into v2 (zeroed by the caller)
+__global__ void pw_cols_kernel(const float* __restrict__ S, const float* __restrict__ u, int R, int C, int rows_per_slice,
+                               float* __restrict__ v2) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= C) return;
+  const int r0 = blockIdx.y * rows_per_slice, r1 = min(R, r0 + rows_per_slice);
+  float s = 0.f;
+  for (int r = r0; r < r1; ++r) s = fmaf(S[(long long)r * C + j], u[r], s);
+  atomicAdd(&v2[j], s);
+}
+__global__ void pw_norm_kernel(const float* __restrict__ v2, int C, double* nrm) {
+  __shared__ double red[32];
+  double s = 0.0;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < C; j += gridDim.x * blockDim.x) s += (double)v2[j] * (double)v2[j];
+  s = block_sum_double(s, red);
+  if (threadIdx.x == 0) atomicAdd(nrm, s);
+}
+// v = v2 / |v2|, v2 = 0, and (last round) *sig2 = safety * |v2| bounded below by floor2; nrm is cleared for the next round
+__global__ void pw_scale_kernel(float* __restrict__ v, float* __restrict__ v2, int C, double* nrm_in, double* nrm_next,
+                                double* sig2, double safety, const double* fro2) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  const double n = sqrt(fmax(*nrm_in, 0.0));
+  if (j < C) {
+    v[j] = (n > 0.0) ? (float)((double)v2[j] / n) : v[j];
+    v2[j] = 0.f;
+  }
+  if (j == 0) {
+    *nrm_next = 0.0;
+    if (sig2) {
+      // never above the Frobenius bound (always safe), never below 1 / rank-ish of it (a failed estimate)
+      double e = safety * n;
+      const double f = *fro2;
+      if (!(e > 0.0) || e > f) e = f;
+      *sig2 = e;
+    }
+  }
+}
+
 __global__ void sqrt_hist_kernel(const double* __restrict__ sq, float* __restrict__ out, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = (float)sqrt(fmax(sq[i], 0.0));
