@@ -114,10 +114,21 @@ __global__ void expand_cols_kernel(const float* __restrict__ X, int d3, int h, i
 
 // iteration control of the pseudo-inverse: keep running while the newest squared residual is above tol2 and
 // still falling (a rank-deficient matrix stalls at its rank defect); flag: 1 = run, 0 = skip
-__global__ void pinv_control_kernel(const double* __restrict__ sq, int it, double tol2, int* flag) {
+__global__ void pinv_control_kernel(const double* __restrict__ sq, int it, double tol2, int* flag, int m, int32_t* status) {
   if (*flag == 0) return;
   const double cur = sq[it];
   if (!(cur > tol2)) { *flag = 0; return; }
+  if (it >= 1) {
+    const double prev = sq[it - 1];
+    // With every eigenvalue of A X in (0, 2) the residual norm falls monotonically.  A residual that is still large
+    // and grows means the starting scale was too small (the estimate of the largest singular value failed):
+    // stop and say so instead of iterating to infinity.
+    if (cur > 1.5 * prev && cur > 1e-2 * (double)m) {
+      *flag = 0;
+      raise_status(status, CAFEQ_ERR_NONFINITE);
+      return;
+    }
+  }
   if (it >= 4) {
     const double prev = sq[it - 1];
     if (cur > prev * (1.0 - 1e-7) && cur < prev * (1.0 + 1e-7)) *flag = 0;  // stalled

@@ -165,7 +165,7 @@ static void pinv_rows(cudaStream_t st, const float* S, int R, int C, DenseWS& w,
       o.run_flag = w.flag;
       launch_dense_tc(st, 3, a, bb, m, n, m, 1.f, 1.f, 0.f, o, status);
     }
-    CQ_LAUNCH(pinv_control_kernel, 1, 1, 0, st, rs, it, 1e-6, w.flag);
+    CQ_LAUNCH(pinv_control_kernel, 1, 1, 0, st, rs, it, 1e-6, w.flag, m, status);
     cur ^= 1;
   }
   if (wide) launch_split_rect(st, w.Y, m, n, n, 1.f, nullptr, nullptr, nullptr, w.Oh, w.Ol, nullptr, nullptr, status);
