@@ -1449,6 +1449,21 @@ extern "C" int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8
   if (rc) return rc;
   if (!codes || !packed) return CAFEQ_ERR_INVALID_ARG;
   if (G.d_in % 8) return CAFEQ_ERR_UNSUPPORTED;
+  if (G.d_in % 32 == 0 && ((uintptr_t)codes % 16) == 0 && ((uintptr_t)packed % 4) == 0 && d->bits >= 2 && d->bits <= 8) {
+    cudaStream_t ps = (cudaStream_t)stream;
+    const unsigned pg = grid_for(G.n / 32);
+    uint32_t* pw = reinterpret_cast<uint32_t*>(packed);
+    switch (d->bits) {
+      case 2: CQ_LAUNCH(pack32_kernel<2>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+      case 3: CQ_LAUNCH(pack32_kernel<3>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+      case 4: CQ_LAUNCH(pack32_kernel<4>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+      case 5: CQ_LAUNCH(pack32_kernel<5>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+      case 6: CQ_LAUNCH(pack32_kernel<6>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+      case 7: CQ_LAUNCH(pack32_kernel<7>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+      default: CQ_LAUNCH(pack32_kernel<8>, pg, 256, 0, ps, codes, pw, G.d_out, G.d_in); break;
+    }
+    return last_launch();
+  }
   CQ_LAUNCH(pack_kernel, grid_for(G.n / 8), 256, 0, (cudaStream_t)stream, codes, packed, G.d_out, G.d_in, d->bits);
   return last_launch();
 }

@@ -548,20 +548,47 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             const float s = sc[(G == 128) ? 0 : (ch >> 1)];
             uint32_t dpk[16], lpk[16];
             uint32_t cpk[8];
+            // the flags are uniform over the launch: only the outputs that were asked for are formed
+            const bool want_d = (p.epi & EPI_DELTA) != 0, want_dl = want_d && p.delta_lo != nullptr;
+            const bool want_c = (p.epi & EPI_CODES) != 0;
+            // code = rne(fl32(u / s)).  The IEEE division is a long dependent sequence with a slow-path branch per
+            // element; u * (1 / s) differs from the exact quotient by less than 1.5 ulp, and from fl32(u / s) by
+            // less than 2 ulp, i.e. by less than (qmax + 1) * 2.4e-7, so it rounds to the same integer unless the
+            // quotient lies within that distance of a half-integer.  Those (rare) chunks are redone with the division.
+            float qv[32];
+            {
+              const float rs = (s > 0.f) ? __frcp_rn(s) : 0.f;
+              const float win = 0.5f - (p.qmax + 1.f) * 1.0e-6f;
+              bool near_half = !(rs < 3.0e38f);  // a scale so small that its reciprocal overflows: take the division
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                const float x = v[e] * rs;
+                const float q = rintf(x);
+                near_half |= fabsf(x - q) > win;
+                qv[e] = q;
+              }
+              if (near_half) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) qv[e] = (s > 0.f) ? rintf(__fdiv_rn(v[e], s)) : 0.f;
+              }
+            }
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
-              float q0 = (s > 0.f) ? rintf(__fdiv_rn(v[e], s)) : 0.f;
-              float q1 = (s > 0.f) ? rintf(__fdiv_rn(v[e + 1], s)) : 0.f;
-              q0 = fminf(fmaxf(q0, -p.qmax), p.qmax);
-              q1 = fminf(fmaxf(q1, -p.qmax), p.qmax);
-              const float d0 = s * q0 - v[e], d1 = s * q1 - v[e + 1];
-              const __nv_bfloat16 b0 = __float2bfloat16_rn(d0), b1 = __float2bfloat16_rn(d1);
-              dpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
-              lpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d0 - __bfloat162float(b0))) |
-                            ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d1 - __bfloat162float(b1))) << 16);
-              const uint32_t c0 = (uint32_t)((int)q0) & 0xFFu, c1 = (uint32_t)((int)q1) & 0xFFu;
-              if ((e & 2) == 0) cpk[e >> 2] = c0 | (c1 << 8);
-              else cpk[e >> 2] |= (c0 << 16) | (c1 << 24);
+              const float q0 = fminf(fmaxf(qv[e], -p.qmax), p.qmax);
+              const float q1 = fminf(fmaxf(qv[e + 1], -p.qmax), p.qmax);
+              if (want_d) {
+                const float d0 = s * q0 - v[e], d1 = s * q1 - v[e + 1];
+                const __nv_bfloat16 b0 = __float2bfloat16_rn(d0), b1 = __float2bfloat16_rn(d1);
+                dpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+                if (want_dl)
+                  lpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d0 - __bfloat162float(b0))) |
+                                ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d1 - __bfloat162float(b1))) << 16);
+              }
+              if (want_c) {
+                const uint32_t c0 = (uint32_t)((int)q0) & 0xFFu, c1 = (uint32_t)((int)q1) & 0xFFu;
+                if ((e & 2) == 0) cpk[e >> 2] = c0 | (c1 << 8);
+                else cpk[e >> 2] |= (c0 << 16) | (c1 << 24);
+              }
             }
             if (valid && (p.epi & EPI_DELTA)) {
               uint4* dst = reinterpret_cast<uint4*>(p.delta + (long long)row * p.d_in + col0 + ch * 32);

@@ -1169,4 +1169,34 @@ __global__ void pack_kernel(const int8_t* __restrict__ codes, uint8_t* __restric
   }
 }
 
+// The same stream, 32 codes per thread: 32 b-bit fields are exactly b 32-bit words, so a thread reads two 16-byte
+// vectors of codes and writes whole words (cols % 32 == 0, codes 16-byte aligned, packed 4-byte aligned).
+template <int BITS>
+__global__ void __launch_bounds__(256) pack32_kernel(const int8_t* __restrict__ codes, uint32_t* __restrict__ packed, int rows,
+                                                     int cols) {
+  const long long chunks_per_row = cols / 32;
+  const long long n = (long long)rows * chunks_per_row;
+  constexpr int qmax = (1 << (BITS - 1)) - 1;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  for (long long c = blockIdx.x * (long long)blockDim.x + threadIdx.x; c < n; c += (long long)gridDim.x * blockDim.x) {
+    const uint4* src = reinterpret_cast<const uint4*>(codes) + 2 * c;  // rows are contiguous: chunk c starts at 32 c
+    const uint4 q0 = __ldg(src), q1 = __ldg(src + 1);
+    const uint32_t w8[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+    uint32_t out[BITS];
+#pragma unroll
+    for (int b = 0; b < BITS; ++b) out[b] = 0u;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int8_t q = (int8_t)((w8[i >> 2] >> (8 * (i & 3))) & 0xFFu);
+      const uint32_t u = (uint32_t)(q + qmax) & mask;
+      const int bit = BITS * i;  // compile-time after unrolling
+      out[bit >> 5] |= u << (bit & 31);
+      if ((bit & 31) + BITS > 32) out[(bit >> 5) + 1] |= u >> (32 - (bit & 31));
+    }
+    uint32_t* dst = packed + c * BITS;
+#pragma unroll
+    for (int b = 0; b < BITS; ++b) dst[b] = out[b];
+  }
+}
+
 }  // namespace cafeq
