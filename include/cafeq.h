@@ -214,12 +214,13 @@ int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed,
 
 const char* cafeq_status_string(int status);
 int cafeq_version(void);
-/* Tuning knob, process-wide (the paper has no counterpart).  overlapped = 1 (default): the caller runs several
- * problems concurrently in different streams (the matrices and pairs of a layer are independent), so kernels
- * should cost few SM-microseconds rather than finish one chain as early as possible: the k x k products of the
- * block algebra take the widest output tile (fewest CTAs), and the transform pass gives a small matrix fewer CTAs
- * (at least 14 tiles each; the sparse backward likewise).  overlapped = 0: one problem runs alone: narrow product tiles (about one CTA per SM)
- * and every SM on every pass.  Results do not depend on it.  CAFEQ_ERR_INVALID_ARG unless 0 or 1. */
+/* Tuning knob, process-wide (the paper has no counterpart).  overlapped = 0 (default): one problem runs alone:
+ * narrow product tiles (about one CTA per SM) and every SM on every pass, for the lowest latency of a single chain
+ * of kernels.  overlapped = 1: the caller runs several problems concurrently in different streams (the matrices
+ * and pairs of a layer are independent), so a kernel should cost few SM-microseconds rather than finish early:
+ * the k x k products of the block algebra take the widest output tile (fewest CTAs), and the transform pass and
+ * the sparse backward give a small matrix fewer CTAs (at least 14 tiles each).  Results do not depend on it.
+ * Returns CAFEQ_ERR_INVALID_ARG unless 0 or 1. */
 int cafeq_set_overlap_mode(int overlapped);
 
 /* Number of kernels this library has launched in the calling process so far (host counter, for

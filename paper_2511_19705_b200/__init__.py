@@ -81,8 +81,8 @@ def version() -> int:
 
 
 def set_overlap_mode(overlapped: bool) -> None:
-    """Process-wide launch-shape rule: True (default) when several problems run concurrently in different streams
-    (kernels then take fewer CTAs: fewer SM-microseconds each), False when one problem runs alone (lowest latency)."""
+    """Process-wide launch-shape rule: True when several problems run concurrently in different streams (kernels
+    then take fewer CTAs: fewer SM-microseconds each), False (default) when one problem runs alone (lowest latency)."""
     _check(lib().cafeq_set_overlap_mode(ctypes.c_int(1 if overlapped else 0)), "cafeq_set_overlap_mode")
 
 

@@ -323,7 +323,7 @@ static bool bw_supported(int axis_in, int d_out, int d_in, long long ld, int k, 
   return true;
 }
 
-static std::atomic<int> g_bw_min_tiles{14};  // tiles per CTA at least (more when problems overlap: see cafeq_set_overlap_mode)
+static std::atomic<int> g_bw_min_tiles{6};  // tiles per CTA at least (more when problems overlap: see cafeq_set_overlap_mode)
 
 template <int FORM, int K, int SWAP>
 static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& p) {

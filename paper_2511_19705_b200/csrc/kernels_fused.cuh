@@ -691,7 +691,7 @@ static bool bd_supported(int form, int d_out, int d_in, long long ld, int k, int
   return true;
 }
 
-static std::atomic<int> g_bd_min_tiles{14};
+static std::atomic<int> g_bd_min_tiles{1};
 
 template <int FORM, int K, int G>
 static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmT, BdParams p) {

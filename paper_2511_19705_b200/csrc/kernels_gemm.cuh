@@ -350,8 +350,8 @@ static int tg_launch_t(cudaStream_t st, const TgOperand* A, const TgOperand* B, 
 // Tile-width rule of the small batched products: the widest tile that still gives at least this many CTAs.
 // A CTA's life is dominated by fixed latencies and its epilogue, so narrow tiles (many CTAs) finish one product
 // sooner, while wide tiles (few CTAs) cost far fewer SM-microseconds and leave room for the kernels of other
-// problems running in other streams.  Default: wide tiles (throughput); cafeq_set_overlap_mode changes it.
-static std::atomic<int> g_tg_min_ctas{28};
+// problems running in other streams.  Default: narrow tiles (one chain alone); cafeq_set_overlap_mode changes it.
+static std::atomic<int> g_tg_min_ctas{96};
 static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, const TgParams& p) {
   if (p.K % TG_BK || p.nterms < 1 || p.nterms > TG_MAX_TERMS) return CAFEQ_ERR_UNSUPPORTED;
   const int min_ctas = p.min_ctas > 0 ? p.min_ctas : g_tg_min_ctas.load(std::memory_order_relaxed);

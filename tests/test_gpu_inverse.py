@@ -103,6 +103,6 @@ def test_overlap_mode_does_not_change_results(cq):
         with pytest.raises(RuntimeError):
             cq._check(cq.lib().cafeq_set_overlap_mode(7), "cafeq_set_overlap_mode")
     finally:
-        cq.set_overlap_mode(True)
+        cq.set_overlap_mode(False)
     assert np.allclose(outs[0][0], outs[1][0], rtol=1e-6)
     assert rel_err(outs[0][1], outs[1][1]) <= 1e-5
