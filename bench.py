@@ -356,6 +356,13 @@ def main():
                     launches_per_step=len(tp) / args.steps, avg_launch_ms=sum(tp) / len(tp),
                     algorithmic_gb_per_step=byts / 1e9, algorithmic_tflop_per_step=flops / 1e12,
                     hbm_gbs_achieved=byts / t_pass / 1e9)
+        sbk = kernel_ms.get("sparse_backward")
+        if sbk:
+            # forward pass + sparse backward taken together against the same algorithmic work (one 2k-flop-per-weight
+            # transform and one read of the weights per step): what a single fused kernel would be held to
+            t_fb = t_pass + sbk["ms_per_step"] * 1e-3
+            roof["fwd_plus_bwd"] = dict(ms_per_step=t_fb * 1e3, achieved=flops / t_fb / 1e12, unit="TFLOP/s",
+                                        frac=flops / t_fb / 1e12 / tc_peak)
 
     # ---- end to end through the C ABI with host buffers (pinned): H2D of every weight and transform, the step,
     #      D2H of the loss histories and the updated transforms, every step
