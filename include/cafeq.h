@@ -212,6 +212,51 @@ int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1, const cafe
  * library's.  d_in*bits must be a multiple of 8. */
 int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed, void* stream);
 
+/* ---- one decoder layer at a time --------------------------------------------------------------------------
+ * Section 6 quantises a model layer by layer; within a layer every matrix (block-diagonal transform, Section 4.1)
+ * and every coupled pair (Section 4.2) is an independent optimisation problem.  The calls below advance all
+ * problems of a layer together.  Each step computes exactly what cafeq_optimize_single (loss CAFEQ_LOSS_SURROGATE,
+ * Eq. 4) and cafeq_optimize_pair (loss CAFEQ_LOSS_LSE, Appendix D) compute for that problem; only the launch
+ * structure differs: the k x k algebra runs once over the operator blocks of all problems, and the transform pass
+ * and the backward take all matrices of a form in one launch each.
+ *
+ * One problem.  pair = 0: d1 / W1 describe the matrix, d2 / W2 are ignored.  pair = 1: d1 / W1 and d2 / W2 as in
+ * cafeq_optimize_pair.  M [nb,k,k] is updated in place; opt_state as in the per-problem calls (required for Adam;
+ * its stored-inverse slot is not used here); loss_history fp32 [steps, 2] = {loss, NaN}.  cfg: loss_kind must be
+ * CAFEQ_LOSS_SURROGATE (single) or CAFEQ_LOSS_LSE (pair), eval_every 0 (the quantised losses are evaluated by the
+ * per-problem calls); cfg.steps and cfg.resume are ignored.
+ * Limits: at most 8 problems; one block size (128 or 256) and one group size (64 or 128) for the whole layer;
+ * every matrix must be a shape the tensor-core pass covers (d_in a multiple of 256 on the input axis; d_out a
+ * multiple of k and d_in of 128 on the output axis; 16-byte aligned rows).  Otherwise CAFEQ_ERR_UNSUPPORTED and the
+ * per-problem calls apply.  M and opt_state must be 16-byte aligned. */
+typedef struct {
+  uint32_t struct_size; /* sizeof(cafeq_layer_problem) */
+  int32_t pair;
+  cafeq_matrix_desc d1, d2;
+  const void* W1;
+  const void* W2;
+  float* M;
+  float* opt_state;
+  float* loss_history;
+  cafeq_opt_cfg cfg;
+} cafeq_layer_problem;
+
+/* Scratch bytes for the layer calls on these problems (`probs` and `bytes` are host pointers; the device pointers
+ * inside the problems are not read).  Includes an fp16 copy of every weight (2 bytes per weight). */
+int cafeq_layer_workspace_size(const cafeq_layer_problem* probs, int n, size_t* bytes);
+
+/* Once per layer, before the first cafeq_optimize_layer on `ws`: makes the fp16 copies of the weights that the
+ * backward reads (scaled by a power of two per matrix; exact for every bf16 value within 2^-38 of the matrix
+ * maximum) and inverts the initial transforms.  The workspace then carries that state (copies, last inverse)
+ * between cafeq_optimize_layer calls: pass the same problems and the same `ws`, and let nothing else write it. */
+int cafeq_layer_prepare(const cafeq_layer_problem* probs, int n, int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* `steps` optimisation steps of every problem (forward, backward, parameter update), enqueued on `stream`.
+ * Step i writes row i of every loss_history.  Every step refines the inverse of the previous step's transforms
+ * (Newton-Schulz, checked on the device, recomputed by elimination when it did not converge). */
+int cafeq_optimize_layer(const cafeq_layer_problem* probs, int n, int steps, int32_t* status, void* ws, size_t ws_bytes,
+                         void* stream);
+
 const char* cafeq_status_string(int status);
 int cafeq_version(void);
 /* Tuning knob, process-wide (the paper has no counterpart).  overlapped = 0 (default): one problem runs alone:

@@ -25,7 +25,7 @@ OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_set_overlap_mode", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_set_overlap_mode", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
     "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
@@ -44,6 +44,12 @@ class OptCfg(ctypes.Structure):
                 ("eps", ctypes.c_float), ("lambda_orth", ctypes.c_float), ("lse_t", ctypes.c_float),
                 ("kappa", ctypes.c_float), ("steps", ctypes.c_int32), ("eval_every", ctypes.c_int32),
                 ("resume", ctypes.c_int32)]
+
+
+class LayerProblem(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("pair", ctypes.c_int32), ("d1", MatrixDesc), ("d2", MatrixDesc),
+                ("W1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("M", ctypes.c_void_p),
+                ("opt_state", ctypes.c_void_p), ("loss_history", ctypes.c_void_p), ("cfg", OptCfg)]
 
 
 class CafeqError(RuntimeError):
@@ -326,3 +332,69 @@ def cafeq_pack(codes, *, bits):
     rc = lib().cafeq_pack(ctypes.byref(d), _p(codes), _p(packed), _stream())
     _check(rc, "cafeq_pack")
     return packed
+
+
+# ----------------------------------------------------------------------------- one layer at a time
+class LayerOptimizer:
+    """All single matrices and coupled pairs of one layer behind cafeq_layer_prepare / cafeq_optimize_layer.
+
+    singles: list of dict(W=bf16 [d_out,d_in], M=fp32 [nb,k,k], bits, group, taxis=AXIS_IN, cfg=OptCfg)
+    pairs:   list of dict(W1, W2, M, bits, group1, group2, replicas, cfg=OptCfg)
+    Marshalling only: builds the descriptor array, owns the workspace, the optimiser states and the loss histories."""
+
+    def __init__(self, singles, pairs, max_steps=1):
+        probs = []
+        self.keep = []
+        dev = (singles[0]["W"] if singles else pairs[0]["W1"]).device
+        self.max_steps = max_steps
+        self.hist, self.state, self.M = [], [], []
+        for s in singles:
+            W, M = _bits_tensor(s["W"]), _f32(s["M"], "M")
+            d = make_desc(W.shape[0], W.shape[1], s["bits"], s["group"], M.shape[-1], s.get("taxis", AXIS_IN), APPLY_T, 1,
+                          W.stride(0))
+            probs.append((0, d, d, W, None, M, s["cfg"]))
+        for q in pairs:
+            M = _f32(q["M"], "M")
+            d1, d2 = _pair_descs(q["W1"], q["W2"], M.shape[-1], q["bits"], q["group1"], q["group2"], q.get("replicas", 1))
+            probs.append((1, d1, d2, q["W1"], q["W2"], M, q["cfg"]))
+        self.n = len(probs)
+        self.arr = (LayerProblem * self.n)()
+        for i, (pair, d1, d2, W1, W2, M, cfg) in enumerate(probs):
+            hist = torch.zeros((max_steps, 2), dtype=torch.float32, device=dev)
+            state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=dev)
+            self.hist.append(hist)
+            self.state.append(state)
+            self.M.append(M)
+            self.keep += [W1, W2]
+            a = self.arr[i]
+            a.struct_size = ctypes.sizeof(LayerProblem)
+            a.pair = pair
+            a.d1, a.d2 = d1, d2
+            a.W1 = W1.data_ptr()
+            a.W2 = W2.data_ptr() if W2 is not None else None
+            a.M = M.data_ptr()
+            a.opt_state = state.data_ptr()
+            a.loss_history = hist.data_ptr()
+            a.cfg = cfg
+        n = ctypes.c_size_t(0)
+        _check(lib().cafeq_layer_workspace_size(self.arr, ctypes.c_int(self.n), ctypes.byref(n)), "cafeq_layer_workspace_size")
+        self.ws_bytes = int(n.value)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.prepared = False
+
+    def set_lr(self, i, lr):
+        self.arr[i].cfg.lr = lr
+
+    def prepare(self):
+        _check(lib().cafeq_layer_prepare(self.arr, ctypes.c_int(self.n), _p(self.status), _p(self.ws),
+                                         ctypes.c_size_t(self.ws_bytes), _stream()), "cafeq_layer_prepare")
+        self.prepared = True
+
+    def step(self, steps=1):
+        if not self.prepared:
+            self.prepare()
+        if steps > self.max_steps:
+            raise ValueError("steps exceeds the loss-history rows this object allocated")
+        _check(lib().cafeq_optimize_layer(self.arr, ctypes.c_int(self.n), ctypes.c_int(steps), _p(self.status), _p(self.ws),
+                                          ctypes.c_size_t(self.ws_bytes), _stream()), "cafeq_optimize_layer")

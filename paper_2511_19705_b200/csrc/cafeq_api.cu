@@ -430,12 +430,10 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
     const int splits = (G.d_out + rows_per - 1) / rows_per;
     dim3 grid(G.nbq, strips, splits);
     const size_t sh = (size_t)k * (strip + 1) * 4 + (size_t)SCB_MAXP * 6;
-    static bool attr = false;
-    if (!attr) {
+    {  // the attribute is per device: set it on every call (cheap)
       cudaFuncSetAttribute(scatter_in_bucket_kernel<256, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 33 * 4 + SCB_MAXP * 6);
       cudaFuncSetAttribute(scatter_in_bucket_kernel<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 65 * 4 + SCB_MAXP * 6);
       cudaFuncSetAttribute(scatter_in_bucket_kernel<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 65 * 4 + SCB_MAXP * 6);
-      attr = true;
     }
 #define SC_INB(KV, SV)                                                                                                   \
   CQ_LAUNCH((scatter_in_bucket_kernel<KV, SV>), grid, 256, sh, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, G.g, G.r, nG, coef, \
@@ -449,12 +447,10 @@ static void launch_scatter(cudaStream_t st, const void* W, const Geo& G, const f
   }
   if (k % SC2_JS == 0 && k <= 256 && aligned && G.axis == CAFEQ_AXIS_IN && (k % G.g == 0 || G.g % k == 0) &&
       (nG == 1 || nG == 2 || nG == 4)) {
-    static bool attr = false;
-    if (!attr) {
+    {
       cudaFuncSetAttribute(scatter_in_strip_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4);
       cudaFuncSetAttribute(scatter_in_strip_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4);
       cudaFuncSetAttribute(scatter_in_strip_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * SC2_JS * 4);
-      attr = true;
     }
     const int strips = k / SC2_JS;
     int splits = (148 * 3 + G.nbq * strips - 1) / (G.nbq * strips);
@@ -1467,6 +1463,8 @@ extern "C" int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8
   CQ_LAUNCH(pack_kernel, grid_for(G.n / 8), 256, 0, (cudaStream_t)stream, codes, packed, G.d_out, G.d_in, d->bits);
   return last_launch();
 }
+
+#include "layer_step.cuh"
 
 // ------------------------------------------------------------------------------------------------
 // cafeq_rtn without a caller workspace: scratch lives in the library image

@@ -12,7 +12,17 @@
 // memory over all tiles of the block that the CTA owns; one flush per block and CTA adds it to global memory.
 // The product is issued in the orientation (S^T W or W^T S) whose accumulator rows run along the fastest index of
 // the requested output layout, so that the flush is coalesced atomic adds straight from registers.
+//
+// F16 form: when the caller holds an fp16 copy of the weights (W * 2^e, exact for every bf16 value that matters:
+// fp16 keeps 11 significand bits against bf16's 8) the coefficients are written as ONE fp16 term (relative error
+// 2^-12, scaled by a power of two so that the largest lands near 2^14) and the product is issued once instead of
+// twice; the flush undoes both power-of-two scales.
+//
+// Several matrices can share one launch (see BwMulti): the tiles of all sub-problems form one list and every
+// persistent CTA takes a contiguous run of it.
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "kernels_fused.cuh"
 
@@ -30,7 +40,20 @@ struct BwParams {
   const float* coef;
   const int* idx;
   float* gradT;        // [n_major / r, k, k], accumulated with atomic adds (caller zeroes it)
+  const float* coefmax;      // F16 form: device word holding max |coef| of this matrix (sets the coefficient scale)
+  const float* w_inv_scale;  // F16 form: device word holding 2^-e of the fp16 weight copy
+  const double* out_div;     // optional device word: the flushed gradient is divided by it (LogSumExp normaliser)
   int32_t* status;
+};
+
+constexpr int BW_MAX_SUB = 8;
+struct BwMaps {
+  CUtensorMap w[BW_MAX_SUB];
+};
+struct BwMulti {
+  int n;
+  int tile_end[BW_MAX_SUB];
+  BwParams p[BW_MAX_SUB];  // all share one status word
 };
 
 enum { BW_IN = 0, BW_OUT = 1 };
@@ -38,15 +61,35 @@ constexpr int BW_THREADS = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: operand
 constexpr int BW_NSTAGE = 3;
 constexpr uint32_t BW_NONE = 0xFFFFFFFFu;
 
-template <int K>
+template <int K, int F16>
 struct BwCfg {
   static constexpr int HALVES = K / 128;
+  static constexpr int TERMS = F16 ? 1 : 2;
+  static constexpr int NSTAGE = F16 ? 4 : BW_NSTAGE;
   static constexpr int STAGE_BYTES = K * 64 * 2;   // weight tile: 64 contraction entries x K
-  static constexpr int S_TERM_BYTES = K * 64 * 2;  // S tile: K targets x 64 contraction entries, K-major, one bf16 term
-  static constexpr int S_BUF_BYTES = 2 * S_TERM_BYTES;
+  static constexpr int S_TERM_BYTES = K * 64 * 2;  // S tile: K targets x 64 contraction entries, K-major, one 16-bit term
+  static constexpr int S_BUF_BYTES = TERMS * S_TERM_BYTES;
   static constexpr int TMEM_COLS = HALVES * K;     // 128 or 512
-  static constexpr int SMEM = 1024 + BW_NSTAGE * STAGE_BYTES + 2 * S_BUF_BYTES + 256;
+  static constexpr int SMEM = 1024 + NSTAGE * STAGE_BYTES + 2 * S_BUF_BYTES + 256;
 };
+
+// instruction descriptor for fp16 operands (format field 0), fp32 accumulation
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+
+// power of two that brings max |coef| just below 2^14 (fp16 holds up to 65504); 1 when there is nothing to scale
+__device__ __forceinline__ float bw_coef_scale(const float* coefmax) {
+  const float m = coefmax ? __ldg(coefmax) : 0.f;
+  if (!(m > 0.f) || !(m < 3.0e38f)) return 1.f;
+  int e;
+  frexpf(m, &e);  // m = f * 2^e, f in [0.5, 1)
+  int sh = 14 - e;
+  if (sh > 120) sh = 120;
+  if (sh < -120) sh = -120;
+  return exp2f((float)sh);
+}
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -59,35 +102,38 @@ __device__ __forceinline__ uint32_t bw_s_offset(int target, int kk) {
 
 // SWAP = 0: accumulator rows = targets i, columns = j (coalesced when the output is stored transposed);
 // SWAP = 1: rows = j, columns = i (coalesced for the plain layout).
-template <int FORM, int K, int SWAP>
-__global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_constant__ CUtensorMap tmW, const BwParams p) {
-  using C = BwCfg<K>;
+template <int FORM, int K, int SWAP, int F16>
+__global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_constant__ BwMaps maps, const __grid_constant__ BwMulti mp) {
+  using C = BwCfg<K, F16>;
   static_assert(K == 128 || K == 256, "block size");
-  if (p.status && *p.status) return;
-  const int total_tiles = p.n_major * p.n_minor;
+  int32_t* const status = mp.p[0].status;
+  if (status && *status) return;
+  const int total_tiles = mp.tile_end[mp.n - 1];
   const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
   const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
   if (t_begin >= t_end) return;
+  int s_first = 0;
+  while (mp.tile_end[s_first] <= t_begin) ++s_first;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sStage = smem;
-  uint8_t* sS = smem + BW_NSTAGE * C::STAGE_BYTES;
+  uint8_t* sS = smem + C::NSTAGE * C::STAGE_BYTES;
   uint64_t* bars = (uint64_t*)(sS + 2 * C::S_BUF_BYTES);
-  // barrier slots: wfull[3], wempty[3], sfull[2], sempty[2], accf, acce
+  // barrier slots: wfull[NSTAGE], wempty[NSTAGE], sfull[2], sempty[2], accf, acce
   const uint32_t bar_wfull = smem_u32(bars);
-  const uint32_t bar_wempty = bar_wfull + 8 * BW_NSTAGE;
-  const uint32_t bar_sfull = bar_wempty + 8 * BW_NSTAGE;
+  const uint32_t bar_wempty = bar_wfull + 8 * C::NSTAGE;
+  const uint32_t bar_sfull = bar_wempty + 8 * C::NSTAGE;
   const uint32_t bar_sempty = bar_sfull + 16;
   const uint32_t bar_accf = bar_sempty + 16;
   const uint32_t bar_acce = bar_accf + 8;
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * BW_NSTAGE + 6);
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 6);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    tma_prefetch_desc(&tmW);
-    for (int s = 0; s < BW_NSTAGE; ++s) {
+    tma_prefetch_desc(&maps.w[s_first]);
+    for (int s = 0; s < C::NSTAGE; ++s) {
       mbar_init(bar_wfull + 8 * s, 1);
       mbar_init(bar_wempty + 8 * s, 1);
     }
@@ -121,18 +167,23 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
     // ---------------------------------------------------------------- TMA producer: one weight tile per stage
     if (lane == 0) {
       uint32_t it = 0;
-      for (int tile = t_begin; tile < t_end; ++tile, ++it) {
-        const int major = tile / p.n_minor, t = tile - major * p.n_minor;
-        const uint32_t s = it % BW_NSTAGE, ph = (it / BW_NSTAGE) & 1u;
-        if (!mbar_wait(bar_wempty + 8 * s, ph ^ 1u, abort_flag, p.status)) break;
+      int sub = s_first;
+      for (int gt = t_begin; gt < t_end; ++gt, ++it) {
+        while (gt >= mp.tile_end[sub]) ++sub;
+        const int tile = gt - (sub ? mp.tile_end[sub - 1] : 0);
+        const int n_minor = mp.p[sub].n_minor;
+        const CUtensorMap* tmW = &maps.w[sub];
+        const int major = tile / n_minor, t = tile - major * n_minor;
+        const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+        if (!mbar_wait(bar_wempty + 8 * s, ph ^ 1u, abort_flag, status)) break;
         mbar_expect_tx(bar_wfull + 8 * s, C::STAGE_BYTES);
         const uint32_t dst = smem_u32(sStage + s * C::STAGE_BYTES);
         if constexpr (FORM == BW_IN) {
           // 64 rows x K columns as K / 64 boxes of 64 x 64 (one swizzle atom of the MN-major operand each)
-          for (int n = 0; n < K / 64; ++n) tma_load_2d(dst + n * 8192, &tmW, major * K + n * 64, t * 64, bar_wfull + 8 * s);
+          for (int n = 0; n < K / 64; ++n) tma_load_2d(dst + n * 8192, tmW, major * K + n * 64, t * 64, bar_wfull + 8 * s);
         } else {
           // K rows x 64 columns: one box, K-major operand
-          tma_load_2d(dst, &tmW, t * 64, major * K, bar_wfull + 8 * s);
+          tma_load_2d(dst, tmW, t * 64, major * K, bar_wfull + 8 * s);
         }
       }
     }
@@ -140,30 +191,35 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       // the weight tile is MN-major on the input axis (contraction over its rows), K-major on the output axis
-      constexpr uint32_t idesc = SWAP ? umma_idesc_bf16(128, K, FORM == BW_IN ? 1 : 0, 0) : umma_idesc_bf16(128, K, 0, FORM == BW_IN ? 1 : 0);
+      constexpr int WMN = (FORM == BW_IN) ? 1 : 0;
+      constexpr uint32_t idesc = F16 ? (SWAP ? umma_idesc_f16(128, K, WMN, 0) : umma_idesc_f16(128, K, 0, WMN))
+                                     : (SWAP ? umma_idesc_bf16(128, K, WMN, 0) : umma_idesc_bf16(128, K, 0, WMN));
       const uint32_t sSt_u = smem_u32(sStage), sS_u = smem_u32(sS);
-      int cur_major = -1;
+      int cur_id = -1, sub = s_first;
       uint32_t run = 0, it = 0;
       bool ok = true;
-      for (int tile = t_begin; tile < t_end && ok; ++tile, ++it) {
-        const int major = tile / p.n_minor;
-        const bool first = (major != cur_major);
+      for (int gt = t_begin; gt < t_end && ok; ++gt, ++it) {
+        while (gt >= mp.tile_end[sub]) ++sub;
+        const int tile = gt - (sub ? mp.tile_end[sub - 1] : 0);
+        const int n_minor = mp.p[sub].n_minor;
+        const int id = (sub << 24) | (tile / n_minor);
+        const bool first = (id != cur_id);
         if (first) {
           // the flush of the previous block must have drained the accumulators
-          if (cur_major >= 0) {
-            if (!mbar_wait(bar_acce, (run - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+          if (cur_id >= 0) {
+            if (!mbar_wait(bar_acce, (run - 1) & 1u, abort_flag, status)) { ok = false; break; }
             tc_fence_after();
           }
-          cur_major = major;
+          cur_id = id;
         }
-        const uint32_t s = it % BW_NSTAGE, ph = (it / BW_NSTAGE) & 1u;
+        const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
         const uint32_t b = it & 1u, sph = (it >> 1) & 1u;
-        if (!mbar_wait(bar_wfull + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-        if (!mbar_wait(bar_sfull + 8 * b, sph, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar_wfull + 8 * s, ph, abort_flag, status)) { ok = false; break; }
+        if (!mbar_wait(bar_sfull + 8 * b, sph, abort_flag, status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t stage = sSt_u + s * C::STAGE_BYTES;
 #pragma unroll
-        for (int term = 0; term < 2; ++term) {
+        for (int term = 0; term < C::TERMS; ++term) {
           const uint32_t sterm = sS_u + b * C::S_BUF_BYTES + term * C::S_TERM_BYTES;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
@@ -186,7 +242,9 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
         }
         tc_commit(bar_wempty + 8 * s);
         tc_commit(bar_sempty + 8 * b);
-        const bool last = (tile + 1 == t_end) || ((tile + 1) / p.n_minor != major);
+        // last tile of this block in this CTA's run: hand the accumulators to the flush
+        bool last = (gt + 1 == t_end) || (gt + 1 >= mp.tile_end[sub]);
+        if (!last) last = ((tile + 1) / n_minor != tile / n_minor);
         if (last) {
           tc_commit(bar_accf);
           ++run;
@@ -199,7 +257,8 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
     const int q = warp & 3, hw = (warp - 2) >> 2;
     float cfN = 0.f;
     int tgN = -1, kkN = 0;
-    auto load_rec = [&](int tile) {
+    auto load_rec = [&](int sub, int tile) {
+      const BwParams& p = mp.p[sub];
       const int major = tile / p.n_minor, t = tile - major * p.n_minor;
       cfN = 0.f;
       tgN = -1;
@@ -233,14 +292,19 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
           }
         }
       }
+      if constexpr (F16) cfN *= bw_coef_scale(p.coefmax);
     };
     // flush of one block: accumulators -> global memory, coalesced atomic adds straight from the registers
     // (accumulator row m = this thread's lane, 32 consecutive columns n per load)
-    auto flush = [&](int major, uint32_t run) -> bool {
-      bool okw = mbar_wait(bar_accf, run & 1u, abort_flag, p.status);
+    auto flush = [&](int sub, int major, uint32_t run) -> bool {
+      const BwParams& p = mp.p[sub];
+      bool okw = mbar_wait(bar_accf, run & 1u, abort_flag, status);
       okw = __all_sync(0xffffffffu, okw);
       if (!okw) return false;
       tc_fence_after();
+      float mul = 1.f;
+      if constexpr (F16) mul = (p.w_inv_scale ? __ldg(p.w_inv_scale) : 1.f) / bw_coef_scale(p.coefmax);
+      if (p.out_div) mul = (float)((double)mul / *p.out_div);
       float* out = p.gradT + (size_t)(major / p.r) * K * K;
       constexpr int CH = (K == 256) ? 8 : 2;  // 32-column chunks per thread
       const int m = ((K == 256) ? hw * 128 : 0) + q * 32 + lane;
@@ -252,7 +316,7 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
         const int n0 = nbase + ch * 32;
 #pragma unroll
         for (int c = 0; c < 32; ++c)
-          if (v[c] != 0.f) atomicAdd(&out[(size_t)(n0 + c) * K + m], v[c]);
+          if (v[c] != 0.f) atomicAdd(&out[(size_t)(n0 + c) * K + m], v[c] * mul);
       }
       tc_fence_before();
       mbar_arrive(bar_acce);
@@ -260,43 +324,55 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
     };
 
     uint32_t prevA = BW_NONE, prevB = BW_NONE;  // offsets this thread wrote into S buffer 0 / 1
-    int cur_major = t_begin / p.n_minor;
+    int sub = s_first;
+    int cur_sub = s_first, cur_major = (t_begin - (s_first ? mp.tile_end[s_first - 1] : 0)) / mp.p[s_first].n_minor;
     uint32_t run = 0, tl = 0;
     bool ok = true;
-    load_rec(t_begin);
-    for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
-      const int major = tile / p.n_minor;
+    load_rec(sub, t_begin - (sub ? mp.tile_end[sub - 1] : 0));
+    for (int gt = t_begin; gt < t_end && ok; ++gt, ++tl) {
+      while (gt >= mp.tile_end[sub]) ++sub;
+      const int tile = gt - (sub ? mp.tile_end[sub - 1] : 0);
+      const int major = tile / mp.p[sub].n_minor;
       const float cf = cfN;
       const int tg = tgN, kk = kkN;
-      if (tile + 1 < t_end) load_rec(tile + 1);
+      if (gt + 1 < t_end) {
+        int sn = sub;
+        while (gt + 1 >= mp.tile_end[sn]) ++sn;
+        load_rec(sn, gt + 1 - (sn ? mp.tile_end[sn - 1] : 0));
+      }
       const uint32_t b = tl & 1u, sph = (tl >> 1) & 1u;
-      if (major != cur_major) {
-        if (!flush(cur_major, run)) { ok = false; break; }
+      if (major != cur_major || sub != cur_sub) {
+        if (!flush(cur_sub, cur_major, run)) { ok = false; break; }
         ++run;
         cur_major = major;
+        cur_sub = sub;
       }
-      ok = mbar_wait(bar_sempty + 8 * b, sph ^ 1u, abort_flag, p.status);
+      ok = mbar_wait(bar_sempty + 8 * b, sph ^ 1u, abort_flag, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       uint8_t* buf = sS + b * C::S_BUF_BYTES;
       const uint32_t prev = b ? prevB : prevA;
       if (prev != BW_NONE) {
         *reinterpret_cast<uint16_t*>(buf + prev) = 0;
-        *reinterpret_cast<uint16_t*>(buf + C::S_TERM_BYTES + prev) = 0;
+        if constexpr (!F16) *reinterpret_cast<uint16_t*>(buf + C::S_TERM_BYTES + prev) = 0;
       }
       uint32_t now = BW_NONE;
       if (tg >= 0) {
-        const __nv_bfloat16 hi = __float2bfloat16_rn(cf);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(cf - __bfloat162float(hi));
         now = bw_s_offset(tg, kk);
-        *reinterpret_cast<uint16_t*>(buf + now) = __bfloat16_as_ushort(hi);
-        *reinterpret_cast<uint16_t*>(buf + C::S_TERM_BYTES + now) = __bfloat16_as_ushort(lo);
+        if constexpr (F16) {
+          *reinterpret_cast<uint16_t*>(buf + now) = __half_as_ushort(__float2half_rn(cf));
+        } else {
+          const __nv_bfloat16 hi = __float2bfloat16_rn(cf);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(cf - __bfloat162float(hi));
+          *reinterpret_cast<uint16_t*>(buf + now) = __bfloat16_as_ushort(hi);
+          *reinterpret_cast<uint16_t*>(buf + C::S_TERM_BYTES + now) = __bfloat16_as_ushort(lo);
+        }
       }
       if (b) prevB = now; else prevA = now;
       fence_proxy_async_smem();
       mbar_arrive(bar_sfull + 8 * b);
     }
-    if (ok) flush(cur_major, run);
+    if (ok) flush(cur_sub, cur_major, run);
   }
 
   // ---------------------------------------------------------------- teardown
@@ -325,30 +401,7 @@ static bool bw_supported(int axis_in, int d_out, int d_in, long long ld, int k, 
 
 static std::atomic<int> g_bw_min_tiles{6};  // tiles per CTA at least (more when problems overlap: see cafeq_set_overlap_mode)
 
-template <int FORM, int K, int SWAP>
-static int bw_launch_t(cudaStream_t st, const CUtensorMap& tmW, const BwParams& p) {
-  using C = BwCfg<K>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(bd_bwd_kernel<FORM, K, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
-      return CAFEQ_ERR_CUDA;
-    attr_done = true;
-  }
-  // one persistent CTA per SM at most; small problems use fewer CTAs so that every CTA has several tiles per
-  // flush (a flush moves k * k floats whatever the number of tiles behind it)
-  const long long total = (long long)p.n_major * p.n_minor;
-  long long want = total / g_bw_min_tiles.load(std::memory_order_relaxed);
-  if (want < p.n_major) want = p.n_major;
-  if (want > total) want = total;
-  const int grid = want < 148 ? (int)want : 148;
-  bd_bwd_kernel<FORM, K, SWAP><<<grid, BW_THREADS, C::SMEM, st>>>(tmW, p);
-  return CAFEQ_OK;
-}
-
-// W: bf16 [d_out, d_in] with pitch ld; records and gradT as in BwParams (n_major, n_minor, NG are filled here)
-static int bw_launch(cudaStream_t st, int axis_in, int k, const void* W, long long ld, BwParams p) {
-  CUtensorMap tmW;
-  if (!make_map_bf16(&tmW, W, p.d_in, p.d_out, ld, axis_in ? 64 : k)) return CAFEQ_ERR_UNSUPPORTED;
+static void bw_fill_tiles(BwParams& p, int axis_in, int k) {
   if (axis_in) {
     p.n_major = p.d_in / k;
     p.n_minor = (p.d_out + 63) / 64;
@@ -358,19 +411,88 @@ static int bw_launch(cudaStream_t st, int axis_in, int k, const void* W, long lo
     p.n_minor = p.d_in / 64;
     p.NG = 1;
   }
-  const int swap = p.transpose_out ? 0 : 1;  // accumulator rows along the fastest index of the output
-#define BW_CASE(AX, F, KK, SW) \
-  if ((axis_in != 0) == (AX) && k == KK && swap == SW) return bw_launch_t<F, KK, SW>(st, tmW, p);
-  BW_CASE(true, BW_IN, 128, 0)
-  BW_CASE(true, BW_IN, 128, 1)
-  BW_CASE(true, BW_IN, 256, 0)
-  BW_CASE(true, BW_IN, 256, 1)
-  BW_CASE(false, BW_OUT, 128, 0)
-  BW_CASE(false, BW_OUT, 128, 1)
-  BW_CASE(false, BW_OUT, 256, 0)
-  BW_CASE(false, BW_OUT, 256, 1)
+}
+
+template <int FORM, int K, int SWAP, int F16>
+static int bw_launch_t(cudaStream_t st, const BwMaps& maps, BwMulti mp, int min_tiles) {
+  using C = BwCfg<K, F16>;
+  static std::atomic<unsigned long long> done{0};
+  if (!opt_in_smem(bd_bwd_kernel<FORM, K, SWAP, F16>, C::SMEM, done)) return CAFEQ_ERR_CUDA;
+  // one persistent CTA per SM at most; small problems use fewer CTAs so that every CTA has several tiles per
+  // flush (a flush moves k * k floats whatever the number of tiles behind it)
+  long long total = 0, majors = 0;
+  for (int s = 0; s < mp.n; ++s) {
+    bw_fill_tiles(mp.p[s], FORM == BW_IN, K);
+    total += (long long)mp.p[s].n_major * mp.p[s].n_minor;
+    majors += mp.p[s].n_major;
+    mp.tile_end[s] = (int)total;
+  }
+  for (int s = mp.n; s < BW_MAX_SUB; ++s) mp.tile_end[s] = (int)total;
+  long long want = total / (min_tiles > 0 ? min_tiles : 1);
+  if (want < majors) want = majors;
+  if (want > total) want = total;
+  const int grid = want < 148 ? (int)want : 148;
+  bd_bwd_kernel<FORM, K, SWAP, F16><<<grid, BW_THREADS, C::SMEM, st>>>(maps, mp);
+  return CAFEQ_OK;
+}
+
+static int bw_dispatch(cudaStream_t st, int axis_in, int k, int swap, int f16, const BwMaps& maps, const BwMulti& mp, int min_tiles) {
+#define BW_CASE(AX, F, KK, SW, HF) \
+  if ((axis_in != 0) == (AX) && k == KK && swap == SW && f16 == HF) return bw_launch_t<F, KK, SW, HF>(st, maps, mp, min_tiles);
+  BW_CASE(true, BW_IN, 128, 0, 0)
+  BW_CASE(true, BW_IN, 128, 1, 0)
+  BW_CASE(true, BW_IN, 256, 0, 0)
+  BW_CASE(true, BW_IN, 256, 1, 0)
+  BW_CASE(false, BW_OUT, 128, 0, 0)
+  BW_CASE(false, BW_OUT, 128, 1, 0)
+  BW_CASE(false, BW_OUT, 256, 0, 0)
+  BW_CASE(false, BW_OUT, 256, 1, 0)
+  BW_CASE(true, BW_IN, 128, 0, 1)
+  BW_CASE(true, BW_IN, 128, 1, 1)
+  BW_CASE(true, BW_IN, 256, 0, 1)
+  BW_CASE(true, BW_IN, 256, 1, 1)
+  BW_CASE(false, BW_OUT, 128, 0, 1)
+  BW_CASE(false, BW_OUT, 128, 1, 1)
+  BW_CASE(false, BW_OUT, 256, 0, 1)
+  BW_CASE(false, BW_OUT, 256, 1, 1)
 #undef BW_CASE
   return CAFEQ_ERR_UNSUPPORTED;
+}
+
+// W: bf16 [d_out, d_in] with pitch ld; records and gradT as in BwParams (n_major, n_minor, NG are filled here)
+static int bw_launch(cudaStream_t st, int axis_in, int k, const void* W, long long ld, BwParams p) {
+  BwMaps maps;
+  BwMulti mp;
+  memset(&mp, 0, sizeof(mp));
+  if (!make_map_bf16(&maps.w[0], W, p.d_in, p.d_out, ld, axis_in ? 64 : k)) return CAFEQ_ERR_UNSUPPORTED;
+  for (int s = 1; s < BW_MAX_SUB; ++s) maps.w[s] = maps.w[0];
+  mp.n = 1;
+  mp.p[0] = p;
+  const int swap = p.transpose_out ? 0 : 1;  // accumulator rows along the fastest index of the output
+  return bw_dispatch(st, axis_in, k, swap, 0, maps, mp, g_bw_min_tiles.load(std::memory_order_relaxed));
+}
+
+// One sub-problem of a multi-matrix launch; W16 is the matrix in 16-bit storage (bf16, or the scaled fp16 copy of the
+// F16 form) with pitch ld.  All sub-problems of a launch share axis, block size, output orientation and form.
+struct BwSub {
+  const void* W16;
+  long long ld;
+  BwParams p;
+};
+
+static int bw_launch_many(cudaStream_t st, int axis_in, int k, int transpose_out, int f16, const BwSub* subs, int n) {
+  if (n < 1 || n > BW_MAX_SUB) return CAFEQ_ERR_INVALID_ARG;
+  BwMaps maps;
+  BwMulti mp;
+  memset(&mp, 0, sizeof(mp));
+  for (int s = 0; s < n; ++s) {
+    if (!make_map_bf16(&maps.w[s], subs[s].W16, subs[s].p.d_in, subs[s].p.d_out, subs[s].ld, axis_in ? 64 : k)) return CAFEQ_ERR_UNSUPPORTED;
+    mp.p[s] = subs[s].p;
+    mp.p[s].transpose_out = transpose_out;
+  }
+  for (int s = n; s < BW_MAX_SUB; ++s) maps.w[s] = maps.w[0];
+  mp.n = n;
+  return bw_dispatch(st, axis_in, k, transpose_out ? 0 : 1, f16, maps, mp, 6);
 }
 
 }  // namespace cafeq

@@ -13,6 +13,8 @@
 #pragma once
 
 #include <atomic>
+#include <mutex>
+#include <string.h>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -50,7 +52,22 @@ struct BdParams {
   double* lossacc;     // += kappa * sum cw a^2
   int a_always;        // write the maxima and their signed values even in EPI_SURR mode
   float* Aacc;         // input axis: [d_in / G] += a^2 per column group; output axis: [nbT * k] += G * sum_G a^2 per operator row
+  float* vmax;         // optional: atomic maximum (bit pattern of a non-negative float) of |coef| when coefficients are
+                       // written, of the group maxima otherwise
   int32_t* status;
+};
+
+// Several matrices in one launch (the problems of a layer are independent): the tiles of all sub-problems form one
+// list, sub-problem s owning [tile_end[s-1], tile_end[s]), and every persistent CTA takes a contiguous run of it.
+constexpr int BD_MAX_SUB = 8;
+struct BdMaps {
+  CUtensorMap x[BD_MAX_SUB];  // the matrices
+  CUtensorMap t[BD_MAX_SUB];  // their operator blocks
+};
+struct BdMulti {
+  int n;
+  int tile_end[BD_MAX_SUB];
+  BdParams p[BD_MAX_SUB];     // all share one status word
 };
 
 constexpr int BD_THREADS = 320;
@@ -217,19 +234,22 @@ struct BdCfg {
 
 template <int FORM, int K, int G>
 __global__ void __launch_bounds__(BD_THREADS, 1)
-bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmT, const BdParams p) {
+bd_pass_kernel(const __grid_constant__ BdMaps maps, const __grid_constant__ BdMulti mp) {
   using C = BdCfg<FORM, K, G>;
   static_assert(K == 64 || K == 128 || K == 256, "block size");
   static_assert(FORM == BD_IN || K >= 128, "output-axis form needs k >= 128");
   static_assert(G == 64 || G == 128, "group size");
-  if (p.status && *p.status) return;
+  int32_t* const status = mp.p[0].status;
+  if (status && *status) return;
 
-  // persistent CTA: a contiguous run of tiles in (major, minor) order; the operator block is reloaded when the
-  // run crosses into the next major
-  const int total_tiles = p.n_major * p.n_minor;
+  // persistent CTA: a contiguous run of tiles in (sub-problem, major, minor) order; the operator block is reloaded
+  // when the run crosses into the next major or the next sub-problem
+  const int total_tiles = mp.tile_end[mp.n - 1];
   const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
   const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
   if (t_begin >= t_end) return;
+  int s_first = 0;
+  while (mp.tile_end[s_first] <= t_begin) ++s_first;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -249,8 +269,8 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    tma_prefetch_desc(&tmX);
-    tma_prefetch_desc(&tmT);
+    tma_prefetch_desc(&maps.x[s_first]);
+    tma_prefetch_desc(&maps.t[s_first]);
     for (int s = 0; s < C::NSTAGE; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
@@ -278,36 +298,45 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       uint32_t it = 0, tloads = 0;
-      int cur_major = -1;
       bool ok = true;
-      for (int tile = t_begin; tile < t_end && ok; ++tile) {
-        const int major = tile / p.n_minor, t = tile - major * p.n_minor;
-        if (major != cur_major) {
-          // the products of the previous major must have finished reading the operator block
-          if (tloads > 0 && !mbar_wait(bar_tfree, (tloads - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-          mbar_expect_tx(bar_tfull, C::T_BYTES);
-          for (int bi = 0; bi < C::NBLK; ++bi) {
-            const int tb = (FORM == BD_IN) ? (major * C::NBLK + bi) / p.r : major / p.r;
-            for (int ci = 0; ci < K / 64; ++ci)
-              tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), &tmT, ci * 64, tb * K, bar_tfull);
+      for (int sub = s_first; sub < mp.n && ok; ++sub) {
+        const int base = sub ? mp.tile_end[sub - 1] : 0;
+        if (base >= t_end) break;
+        const BdParams& p = mp.p[sub];
+        const CUtensorMap* tmX = &maps.x[sub];
+        const CUtensorMap* tmT = &maps.t[sub];
+        const int lo = (t_begin > base ? t_begin : base) - base;
+        const int hi = (t_end < mp.tile_end[sub] ? t_end : mp.tile_end[sub]) - base;
+        int cur_major = -1;
+        for (int tile = lo; tile < hi && ok; ++tile) {
+          const int major = tile / p.n_minor, t = tile - major * p.n_minor;
+          if (major != cur_major) {
+            // the products of the previous operator block must have finished reading it
+            if (tloads > 0 && !mbar_wait(bar_tfree, (tloads - 1) & 1u, abort_flag, status)) { ok = false; break; }
+            mbar_expect_tx(bar_tfull, C::T_BYTES);
+            for (int bi = 0; bi < C::NBLK; ++bi) {
+              const int tb = (FORM == BD_IN) ? (major * C::NBLK + bi) / p.r : major / p.r;
+              for (int ci = 0; ci < K / 64; ++ci)
+                tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), tmT, ci * 64, tb * K, bar_tfull);
+            }
+            cur_major = major;
+            ++tloads;
           }
-          cur_major = major;
-          ++tloads;
-        }
-        for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
-          const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
-          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-          mbar_expect_tx(bar_full + 8 * s, BD_STAGE_BYTES);
-          int x, y;
-          if constexpr (FORM == BD_IN) {
-            x = major * 256 + sidx * 64;
-            y = t * 128;
-          } else {
-            const int kh = sidx / C::NCC, nc = sidx % C::NCC;  // the chunks of one row half are consecutive stages
-            x = t * C::NC + nc * 64;
-            y = major * K + kh * 128;
+          for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
+            const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+            if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, status)) { ok = false; break; }
+            mbar_expect_tx(bar_full + 8 * s, BD_STAGE_BYTES);
+            int x, y;
+            if constexpr (FORM == BD_IN) {
+              x = major * 256 + sidx * 64;
+              y = t * 128;
+            } else {
+              const int kh = sidx / C::NCC, nc = sidx % C::NCC;  // the chunks of one row half are consecutive stages
+              x = t * C::NC + nc * 64;
+              y = major * K + kh * 128;
+            }
+            tma_load_2d(smem_u32(sStage + s * BD_STAGE_BYTES), tmX, x, y, bar_full + 8 * s);
           }
-          tma_load_2d(smem_u32(sStage + s * BD_STAGE_BYTES), &tmX, x, y, bar_full + 8 * s);
         }
       }
     }
@@ -315,64 +344,71 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       bool ok = true;
-      int cur_major = -1;
       uint32_t tfulls = 0;
       constexpr uint32_t idesc_in = umma_idesc_bf16(128, K, 0, 0);
       constexpr uint32_t idesc_out = umma_idesc_bf16(128, 128, 0, 1);
       const uint32_t sT_u = smem_u32(sT), sSt_u = smem_u32(sStage);
       uint32_t it = 0, tl = 0;
-      for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
-        const int major = tile / p.n_minor;
-        if (major != cur_major) {
-          if (!mbar_wait(bar_tfull, tfulls & 1u, abort_flag, p.status)) { ok = false; break; }
-          ++tfulls;
-          cur_major = major;
-        }
-        const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
-        if (!mbar_wait(bar_acce + 8 * buf, aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t dbase = tmem_base + buf * 256u;
-        if constexpr (FORM == BD_IN) {
-          for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
-            const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
-            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
-            const int bi = (sidx * 64) / K, ci = ((sidx * 64) % K) / 64;
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const uint64_t ad = umma_desc_sw128(stage + kk * 32);
-              const uint64_t bd = umma_desc_sw128(sT_u + bi * K * K * 2 + ci * K * 128 + kk * 32);
-              tc_mma_bf16(dbase + bi * K, ad, bd, idesc_in, (ci | kk) != 0 ? 1u : 0u);
-            }
-            tc_commit(bar_empty + 8 * s);
+      for (int sub = s_first; sub < mp.n && ok; ++sub) {
+        const int base = sub ? mp.tile_end[sub - 1] : 0;
+        if (base >= t_end) break;
+        const int n_minor = mp.p[sub].n_minor;
+        const int lo = (t_begin > base ? t_begin : base) - base;
+        const int hi = (t_end < mp.tile_end[sub] ? t_end : mp.tile_end[sub]) - base;
+        int cur_major = -1;
+        for (int tile = lo; tile < hi && ok; ++tile, ++tl) {
+          const int major = tile / n_minor;
+          if (major != cur_major) {
+            if (!mbar_wait(bar_tfull, tfulls & 1u, abort_flag, status)) { ok = false; break; }
+            ++tfulls;
+            cur_major = major;
           }
-        } else {
-          // two consecutive stages = two 64-column chunks of the same 128 weight rows: one N = 128 product, the
-          // second swizzle atom of the MN-major operand one stage further on
-          for (int sidx = 0; sidx < BD_STAGES_PER_TILE; sidx += 2, it += 2) {
-            const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
-            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-            if (!mbar_wait(bar_full + 8 * (s + 1), ph, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
-            const int kh = sidx / C::NCC, nc = sidx % C::NCC;
+          const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
+          if (!mbar_wait(bar_acce + 8 * buf, aph ^ 1u, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t dbase = tmem_base + buf * 256u;
+          if constexpr (FORM == BD_IN) {
+            for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
+              const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+              if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, status)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
+              const int bi = (sidx * 64) / K, ci = ((sidx * 64) % K) / 64;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              const uint64_t bd = umma_desc_sw128_lbo(stage + ks * 2048, BD_STAGE_BYTES);
-#pragma unroll
-              for (int mh = 0; mh < C::KH; ++mh) {
-                const uint64_t ad = umma_desc_sw128(sT_u + (kh * 2 + ks / 4) * K * 128 + mh * 128 * 128 + (ks % 4) * 32);
-                tc_mma_bf16(dbase + mh * C::NC + nc * 64, ad, bd, idesc_out, (kh | ks) != 0 ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t ad = umma_desc_sw128(stage + kk * 32);
+                const uint64_t bd = umma_desc_sw128(sT_u + bi * K * K * 2 + ci * K * 128 + kk * 32);
+                tc_mma_bf16(dbase + bi * K, ad, bd, idesc_in, (ci | kk) != 0 ? 1u : 0u);
               }
+              tc_commit(bar_empty + 8 * s);
             }
-            tc_commit(bar_empty + 8 * s);
-            tc_commit(bar_empty + 8 * (s + 1));
+          } else {
+            // two consecutive stages = two 64-column chunks of the same 128 weight rows: one N = 128 product, the
+            // second swizzle atom of the MN-major operand one stage further on
+            for (int sidx = 0; sidx < BD_STAGES_PER_TILE; sidx += 2, it += 2) {
+              const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
+              if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, status)) { ok = false; break; }
+              if (!mbar_wait(bar_full + 8 * (s + 1), ph, abort_flag, status)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
+              const int kh = sidx / C::NCC, nc = sidx % C::NCC;
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t bd = umma_desc_sw128_lbo(stage + ks * 2048, BD_STAGE_BYTES);
+#pragma unroll
+                for (int mh = 0; mh < C::KH; ++mh) {
+                  const uint64_t ad = umma_desc_sw128(sT_u + (kh * 2 + ks / 4) * K * 128 + mh * 128 * 128 + (ks % 4) * 32);
+                  tc_mma_bf16(dbase + mh * C::NC + nc * 64, ad, bd, idesc_out, (kh | ks) != 0 ? 1u : 0u);
+                }
+              }
+              tc_commit(bar_empty + 8 * s);
+              tc_commit(bar_empty + 8 * (s + 1));
+            }
           }
+          if (ok) tc_commit(bar_accf + 8 * buf);
+          // last tile of this operator block with more to come: signal when its products are done with the block
+          if (ok && base + tile + 1 < t_end && (tile + 1 == hi || (tile + 1) / n_minor != major)) tc_commit(bar_tfree);
         }
-        if (ok) tc_commit(bar_accf + 8 * buf);
-        // last tile of this major with more to come: signal when its products are done with the operator block
-        if (ok && tile + 1 < t_end && (tile + 1) / p.n_minor != major) tc_commit(bar_tfree);
       }
     }
   } else {
@@ -381,13 +417,19 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     const int L = q * 32 + lane;
     uint32_t tl = 0;
     bool ok = true;
+    constexpr int NG = 128 / G;
+    for (int sub = s_first; sub < mp.n && ok; ++sub) {
+    const int base = sub ? mp.tile_end[sub - 1] : 0;
+    if (base >= t_end) break;
+    const BdParams& p = mp.p[sub];
+    const int lo = (t_begin > base ? t_begin : base) - base;
+    const int hi = (t_end < mp.tile_end[sub] ? t_end : mp.tile_end[sub]) - base;
     double sq_local = 0.0, sur_local = 0.0;
-    float srow = 0.f;
+    float srow = 0.f, vm = 0.f;
     int srow_row = -1;
     bool bad = false;
-    constexpr int NG = 128 / G;
     const int ng_row = p.d_in / G;
-    for (int tile = t_begin; tile < t_end && ok; ++tile, ++tl) {
+    for (int tile = lo; tile < hi && ok; ++tile, ++tl) {
       const int major = tile / p.n_minor, t = tile - major * p.n_minor;
       const uint32_t buf = tl & 1u, aph = (tl >> 1) & 1u;
       int row, col0;
@@ -410,7 +452,7 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
         for (int gi = 0; gi < NG; ++gi) wgt[gi] = (FORM == BD_IN) ? __ldg(p.cw + col0 / G + gi) : __ldg(p.cw + row);
       }
-      ok = mbar_wait(bar_accf + 8 * buf, aph, abort_flag, p.status);
+      ok = mbar_wait(bar_accf + 8 * buf, aph, abort_flag, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -488,6 +530,10 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
         for (int gi = 0; gi < NG; ++gi)
           if (valid && !(best[gi] <= 3.0e38f)) bad = true;
+        if (valid && p.vmax && !((p.epi & EPI_SURR) && p.coef)) {
+#pragma unroll
+          for (int gi = 0; gi < NG; ++gi) vm = fmaxf(vm, best[gi]);
+        }
         if (valid && (p.epi & EPI_ABSMAX)) {
           // with Eq. 4 evaluated right here nothing downstream reads the maxima or their signs: the backward only
           // needs (arg-max index, coefficient).  Every scattered 4-byte store is a partial-sector write at L2.
@@ -522,7 +568,9 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             surf = fmaf(wgt[gi] * av, av, surf);
             if (valid && p.coef) {
               const float sg = (bval[gi] > 0.f) ? 1.f : ((bval[gi] < 0.f) ? -1.f : 0.f);
-              p.coef[(long long)Gc * p.d_out + row] = 2.f * p.kappa * wgt[gi] * av * sg;
+              const float cf = 2.f * p.kappa * wgt[gi] * av;
+              p.coef[(long long)Gc * p.d_out + row] = cf * sg;
+              vm = fmaxf(vm, cf);
             }
             if constexpr (FORM == BD_IN) {
               float a2 = av * av;
@@ -628,7 +676,12 @@ bd_pass_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
       }
     }
-    if (__any_sync(0xffffffffu, bad) && lane == 0) raise_status(p.status, CAFEQ_ERR_NONFINITE);
+    if (p.vmax) {
+      for (int o = 16; o > 0; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
+      if (lane == 0 && vm > 0.f) atomicMax(reinterpret_cast<int*>(p.vmax), __float_as_int(vm));
+    }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) raise_status(status, CAFEQ_ERR_NONFINITE);
+    }  // sub-problems
   }
 
   // ---------------------------------------------------------------- teardown
@@ -650,15 +703,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 static EncodeTiledFn get_encode_tiled() {
   static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static std::once_flag once;
+  std::call_once(once, [] {
     void* ptr = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
       fn = (EncodeTiledFn)ptr;
-  }
+  });
   return fn;
 }
 
@@ -693,15 +745,22 @@ static bool bd_supported(int form, int d_out, int d_in, long long ld, int k, int
 
 static std::atomic<int> g_bd_min_tiles{1};
 
+// opt the kernel into its dynamic shared memory once per device (the attribute is per device and per function)
+template <typename KernelT>
+static bool opt_in_smem(KernelT kernel, int bytes, std::atomic<unsigned long long>& done_mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done_mask.load(std::memory_order_acquire) & bit) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  done_mask.fetch_or(bit, std::memory_order_release);
+  return true;
+}
+
+// tile geometry of one sub-problem
 template <int FORM, int K, int G>
-static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmT, BdParams p) {
+static void bd_fill_tiles(BdParams& p) {
   using C = BdCfg<FORM, K, G>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(bd_pass_kernel<FORM, K, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
-      return CAFEQ_ERR_CUDA;
-    attr_done = true;
-  }
   if (FORM == BD_IN) {
     p.n_major = p.d_in / 256;
     p.n_minor = (p.d_out + 127) / 128;
@@ -709,25 +768,34 @@ static int bd_launch_t(cudaStream_t st, const CUtensorMap& tmX, const CUtensorMa
     p.n_major = p.d_out / K;
     p.n_minor = (p.d_in + C::NC - 1) / C::NC;
   }
-  const long long total = (long long)p.n_major * p.n_minor;
+  p.ctas_per_major = 0;
+}
+
+template <int FORM, int K, int G>
+static int bd_launch_multi_t(cudaStream_t st, const BdMaps& maps, BdMulti mp, int min_tiles) {
+  using C = BdCfg<FORM, K, G>;
+  static std::atomic<unsigned long long> done{0};
+  if (!opt_in_smem(bd_pass_kernel<FORM, K, G>, C::SMEM, done)) return CAFEQ_ERR_CUDA;
+  long long total = 0;
+  for (int s = 0; s < mp.n; ++s) {
+    bd_fill_tiles<FORM, K, G>(mp.p[s]);
+    total += (long long)mp.p[s].n_major * mp.p[s].n_minor;
+    mp.tile_end[s] = (int)total;
+  }
+  for (int s = mp.n; s < BD_MAX_SUB; ++s) mp.tile_end[s] = (int)total;
   // one persistent CTA per SM at most; when several problems overlap in streams, small matrices take fewer CTAs
-  // (at least g_bd_min_tiles tiles each): the fixed cost of a CTA is spread over more tiles and the SMs left over
+  // (at least min_tiles tiles each): the fixed cost of a CTA is spread over more tiles and the SMs left over
   // run another problem's kernel
-  long long want = total / g_bd_min_tiles.load(std::memory_order_relaxed);
+  long long want = total / (min_tiles > 0 ? min_tiles : 1);
   if (want < 1) want = 1;
   const int grid = want < 148 ? (int)want : 148;
-  p.ctas_per_major = 0;
-  bd_pass_kernel<FORM, K, G><<<grid, BD_THREADS, C::SMEM, st>>>(tmX, tmT, p);
+  bd_pass_kernel<FORM, K, G><<<grid, BD_THREADS, C::SMEM, st>>>(maps, mp);
   return CAFEQ_OK;
 }
 
-// X: bf16 [d_out, d_in] with pitch ld; Tb: bf16 operator blocks [nbT * k, k] in applied orientation.
-static int bd_launch(cudaStream_t st, int form, int k, int g, const void* X, long long ld, const void* Tb, int nbT, BdParams p) {
-  CUtensorMap tmX, tmT;
-  if (!make_map_bf16(&tmX, X, p.d_in, p.d_out, ld, 128)) return CAFEQ_ERR_UNSUPPORTED;
-  if (!make_map_bf16(&tmT, Tb, k, (long long)nbT * k, k, k)) return CAFEQ_ERR_UNSUPPORTED;
+static int bd_dispatch(cudaStream_t st, int form, int k, int g, const BdMaps& maps, const BdMulti& mp, int min_tiles) {
 #define BD_CASE(F, KK, GG) \
-  if (form == F && k == KK && g == GG) return bd_launch_t<F, KK, GG>(st, tmX, tmT, p);
+  if (form == F && k == KK && g == GG) return bd_launch_multi_t<F, KK, GG>(st, maps, mp, min_tiles);
   BD_CASE(BD_IN, 64, 64)
   BD_CASE(BD_IN, 64, 128)
   BD_CASE(BD_IN, 128, 64)
@@ -740,6 +808,45 @@ static int bd_launch(cudaStream_t st, int form, int k, int g, const void* X, lon
   BD_CASE(BD_OUT, 256, 128)
 #undef BD_CASE
   return CAFEQ_ERR_UNSUPPORTED;
+}
+
+// X: bf16 [d_out, d_in] with pitch ld; Tb: bf16 operator blocks [nbT * k, k] in applied orientation.
+static int bd_launch(cudaStream_t st, int form, int k, int g, const void* X, long long ld, const void* Tb, int nbT, BdParams p) {
+  BdMaps maps;
+  BdMulti mp;
+  memset(&mp, 0, sizeof(mp));
+  if (!make_map_bf16(&maps.x[0], X, p.d_in, p.d_out, ld, 128)) return CAFEQ_ERR_UNSUPPORTED;
+  if (!make_map_bf16(&maps.t[0], Tb, k, (long long)nbT * k, k, k)) return CAFEQ_ERR_UNSUPPORTED;
+  for (int s = 1; s < BD_MAX_SUB; ++s) { maps.x[s] = maps.x[0]; maps.t[s] = maps.t[0]; }
+  mp.n = 1;
+  mp.p[0] = p;
+  return bd_dispatch(st, form, k, g, maps, mp, g_bd_min_tiles.load(std::memory_order_relaxed));
+}
+
+// One sub-problem of a multi-matrix launch: the matrix, its operator blocks (bf16, applied orientation) and its
+// epilogue parameters (d_out, d_in, r, epi, ... filled by the caller).
+struct BdSub {
+  const void* X;
+  long long ld;
+  const void* Tb;
+  int nbT;
+  BdParams p;
+};
+
+// Up to BD_MAX_SUB matrices of the same form, block size and group size in one persistent launch.
+static int bd_launch_many(cudaStream_t st, int form, int k, int g, const BdSub* subs, int n) {
+  if (n < 1 || n > BD_MAX_SUB) return CAFEQ_ERR_INVALID_ARG;
+  BdMaps maps;
+  BdMulti mp;
+  memset(&mp, 0, sizeof(mp));
+  for (int s = 0; s < n; ++s) {
+    if (!make_map_bf16(&maps.x[s], subs[s].X, subs[s].p.d_in, subs[s].p.d_out, subs[s].ld, 128)) return CAFEQ_ERR_UNSUPPORTED;
+    if (!make_map_bf16(&maps.t[s], subs[s].Tb, k, (long long)subs[s].nbT * k, k, k)) return CAFEQ_ERR_UNSUPPORTED;
+    mp.p[s] = subs[s].p;
+  }
+  for (int s = n; s < BD_MAX_SUB; ++s) { maps.x[s] = maps.x[0]; maps.t[s] = maps.t[0]; }
+  mp.n = n;
+  return bd_dispatch(st, form, k, g, maps, mp, 1);
 }
 
 // fp32 operator blocks -> bf16 in applied orientation (transposed when the role asks for T^T)

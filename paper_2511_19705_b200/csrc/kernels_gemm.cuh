@@ -329,12 +329,8 @@ struct TgOperand {
 template <int BN>
 static int tg_launch_t(cudaStream_t st, const TgOperand* A, const TgOperand* B, TgParams p) {
   using C = TgCfg<BN>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
-      return CAFEQ_ERR_CUDA;
-    attr_done = true;
-  }
+  static std::atomic<unsigned long long> done{0};
+  if (!opt_in_smem(tc_gemm_kernel<BN>, C::SMEM, done)) return CAFEQ_ERR_CUDA;
   TgMaps maps;
   memset(&maps, 0, sizeof(maps));
   for (int t = 0; t < p.nterms; ++t) {
