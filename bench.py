@@ -170,6 +170,10 @@ def main():
     ap.add_argument("--serial", action="store_true", help="one stream and one shared workspace for the whole layer")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
     ap.add_argument("--sample-frac", type=int, default=32)
+    ap.add_argument("--min-seconds", type=float, default=2.0, help="repeat the block of --steps steps until the timed region lasts this long")
+    ap.add_argument("--lr-frac", type=float, default=1e-3, help="step of the single matrices = this / max|first gradient|")
+    ap.add_argument("--pair-lr", type=float, default=1e-4)
+    ap.add_argument("--per-problem", action="store_true", help="time the per-problem calls on one stream each instead of the layer call")
     ap.add_argument("--loss", default="surrogate", choices=["surrogate", "ste"],
                     help="surrogate: Eq. 4 (singles) + LogSumExp (pairs), the paper's objectives; ste: straight-through "
                          "gradients of the quantised losses themselves (Eq. 3 singles, Eq. 5 pairs)")
@@ -204,7 +208,6 @@ def main():
 
     import torch
     import paper_2511_19705_b200 as cq
-    from paper_2511_19705_b200.layer import LayerStep, PairProblem, SingleProblem
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -216,22 +219,14 @@ def main():
     from paper_2511_19705_b200 import shard
     my_layer = shard.layers_of_rank(world, world, rank)[0]     # weak scaling: one layer per rank, no data-path collective
     spec, singles, pairs = host_layer(args.config, my_layer)
-    bits, group = spec["bits"], spec["group"]
+    bits, group, k = spec["bits"], spec["group"], spec["k"]
 
     def up_bf16(b):
         return torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
 
     ste = args.loss == "ste"
-    sp = [SingleProblem(n, up_bf16(W), torch.from_numpy(M).to(dev), bits, group,
-                        loss_kind=cq.LOSS_L2_STE if ste else cq.LOSS_SURROGATE) for n, W, M in singles]
-    pp = [PairProblem(n, up_bf16(W1), up_bf16(W2), torch.from_numpy(M).to(dev), bits, group, group, r, lr=1e-4,
-                      loss_kind=cq.LOSS_PQE_STE if ste else cq.LOSS_LSE) for n, W1, W2, M, r in pairs]
-
-    if args.exact:
-        for p in pp:
-            p.P = cq.cafeq_pair_product(p.W1, p.W2, k=p.M.shape[-1], replicas=p.d2.replicas)
-    layer = LayerStep(sp, pp, parallel=not args.serial)
-    cfg_json.update(weights_per_step=int(layer.weights), bits=bits, group=group, block=spec["k"])
+    weights = sum(w.size for _, w, _ in singles) + sum(a.size + b.size for _, a, b, _, _ in pairs)
+    cfg_json.update(weights_per_step=int(weights), bits=bits, group=group, block=k)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -239,25 +234,73 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    # gradient-descent step size of the single matrices: a small fixed fraction of the first gradient's largest
-    # entry, so that the transforms move every step (the block inverse has real work) without leaving the
-    # neighbourhood of the initial rotations during the run
-    layer.step(0)
-    torch.cuda.synchronize()
-    for p in sp:
-        p.cfg.lr = float(1e-3 / max(float(p.grad.abs().max().item()), 1e-30))
+    # device copies of the layer
+    devS = [(n, up_bf16(W), torch.from_numpy(M).to(dev)) for n, W, M in singles]
+    devP = [(n, up_bf16(W1), up_bf16(W2), torch.from_numpy(M).to(dev), r) for n, W1, W2, M, r in pairs]
 
-    def one_step():
-        layer.opt_step(eval_exact=args.exact)
+    # gradient-descent step size of the single matrices: a fixed fraction (--lr-frac) of the first gradient's largest
+    # entry, so that the transforms move every step and the warm-started block inverse has real work
+    lr_single = {}
+    for n, W, M in devS:
+        out = cq.cafeq_proxy_loss_fwd_bwd(W, M, bits=bits, group=group)
+        lr_single[n] = float(args.lr_frac / max(float(out["gradM"].abs().max().item()), 1e-30))
+    torch.cuda.synchronize()
+
+    use_layer = (not ste) and (not args.exact) and (not args.per_problem)
+    if use_layer:
+        opt = cq.LayerOptimizer(
+            [dict(W=W, M=M, bits=bits, group=group,
+                  cfg=cq.make_cfg(loss_kind=cq.LOSS_SURROGATE, optimizer=cq.OPT_GD, lr=lr_single[n])) for n, W, M in devS],
+            [dict(W1=W1, W2=W2, M=M, bits=bits, group1=group, group2=group, replicas=r,
+                  cfg=cq.make_cfg(loss_kind=cq.LOSS_LSE, optimizer=cq.OPT_ADAM, lr=args.pair_lr, beta1=0.1, beta2=0.999, eps=1e-8,
+                                  lambda_orth=0.1, lse_t=5.0)) for n, W1, W2, M, r in devP], max_steps=1)
+        opt.prepare()
+
+        def one_step():
+            opt.step(1)
+
+        def statuses():
+            return [int(opt.status.item())]
+
+        def set_serial(flag):
+            pass
+
+        step_tensors_in = [t for _, W, M in devS for t in (W, M)] + [t for _, W1, W2, M, _ in devP for t in (W1, W2, M)]
+        step_tensors_out = list(opt.hist) + list(opt.M)
+        n_streams = 1
+        step_desc = "cafeq_optimize_layer: fwd+bwd+update of all 5 problems (GD singles, Adam pairs), warm-started block inverse"
+    else:
+        from paper_2511_19705_b200.layer import LayerStep, PairProblem, SingleProblem
+        sp = [SingleProblem(n, W, M, bits, group, lr=lr_single[n],
+                            loss_kind=cq.LOSS_L2_STE if ste else cq.LOSS_SURROGATE) for n, W, M in devS]
+        pp = [PairProblem(n, W1, W2, M, bits, group, group, r, lr=args.pair_lr,
+                          loss_kind=cq.LOSS_PQE_STE if ste else cq.LOSS_LSE) for n, W1, W2, M, r in devP]
+        if args.exact:
+            for p in pp:
+                p.P = cq.cafeq_pair_product(p.W1, p.W2, k=p.M.shape[-1], replicas=p.d2.replicas)
+        layer = LayerStep(sp, pp, parallel=not args.serial)
+
+        def one_step():
+            layer.opt_step(eval_exact=args.exact)
+
+        def statuses():
+            return layer.statuses()
+
+        def set_serial(flag):
+            layer.parallel = (not flag) and (not args.serial)
+
+        step_tensors_in = [t for p in sp for t in (p.W, p.M)] + [t for p in pp for t in (p.W1, p.W2, p.M)]
+        step_tensors_out = [t for p in sp + pp for t in (p.hist, p.M)]
+        n_streams = len(layer.streams) if layer.parallel else 1
+        step_desc = "per-problem calls: fwd+bwd+update (GD singles, Adam pairs), warm-started block inverse"
 
     for _ in range(max(args.warmup, 3)):
         one_step()
     sync_all()
-    assert all(s == 0 for s in layer.statuses()), layer.statuses()
+    assert all(s == 0 for s in statuses()), statuses()
 
     # ---- pass 1: eager launches on one stream with the library's in-stream event pairs around its main kernels
-    par = layer.parallel
-    layer.parallel = False
+    set_serial(True)
     n_timed = 64 * args.steps
     cq.timer_begin(n_timed)
     l0 = cq.launch_count()
@@ -268,12 +311,14 @@ def main():
         one_step()
     e1.record()
     sync_all()
-    launches = cq.launch_count() - l0
+    launches_per_step = (cq.launch_count() - l0) / args.steps
     ms_eager = e0.elapsed_time(e1)
     kms, kinds = cq.timer_read(n_timed)
-    layer.parallel = par
+    set_serial(False)
 
-    # ---- pass 2 (the reported value): the same step captured once into a CUDA graph and replayed
+    # ---- pass 2 (the reported value): the same step captured once into a CUDA graph and replayed.  `--steps` steps
+    #      form one block; blocks are repeated until the timed region lasts --min-seconds, so that the clock sampler
+    #      sees the run and the clocks are the sustained ones.
     graph = None
     if not args.no_graph:
         try:
@@ -284,39 +329,46 @@ def main():
             print(f"graph capture failed: {exc}", file=sys.stderr)
             graph = None
             torch.cuda.synchronize()
+    run_step = graph.replay if graph is not None else one_step
+    for _ in range(3):
+        run_step()
+    sync_all()
+    e0.record()
+    for _ in range(args.steps):
+        run_step()
+    e1.record()
+    sync_all()
+    est = max(e0.elapsed_time(e1), 1e-3)
+    reps = max(1, int(np.ceil(args.min_seconds * 1e3 / est)))
+    if dist is not None:
+        t = torch.tensor([reps], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        reps = int(t.item())
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    if graph is not None:
-        for _ in range(3):
-            graph.replay()
-        sync_all()
-        e0.record()
-        for _ in range(args.steps):
-            graph.replay()
-        e1.record()
-        sync_all()
-        ms = e0.elapsed_time(e1)
-    else:
-        sync_all()
-        e0.record()
-        for _ in range(args.steps):
-            one_step()
-        e1.record()
-        sync_all()
-        ms = e0.elapsed_time(e1)
+    sync_all()
+    e0.record()
+    for _ in range(reps * args.steps):
+        run_step()
+    e1.record()
+    sync_all()
+    ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
-    assert all(s == 0 for s in layer.statuses()), layer.statuses()
+    assert all(s == 0 for s in statuses()), statuses()
     ms = shard.max_over_ranks(ms, dev)
-    ms_per_step = ms / args.steps
-    value = world * args.steps / (ms * 1e-3)
-    cfg_json.update(launch="cuda_graph_replay" if graph is not None else "eager",
-                    streams=len(layer.streams) if layer.parallel else 1, eager_ms_per_step=ms_eager / args.steps,
-                    step="fwd+bwd+update (GD singles, Adam pairs), warm-started block inverse")
+    timed_steps = reps * args.steps
+    ms_per_step = ms / timed_steps
+    value = world * timed_steps / (ms * 1e-3)
+    launches = int(round(launches_per_step * timed_steps))
+    cfg_json.update(launch="cuda_graph_replay" if graph is not None else "eager", streams=n_streams,
+                    eager_ms_per_step=ms_eager / args.steps, step=step_desc, timed_steps=timed_steps,
+                    timed_region_s=ms * 1e-3, single_lr="%g / max|grad0|" % args.lr_frac, pair_lr=args.pair_lr)
 
-    # ---- roofline of the dominant kernel (the block-diagonal transform pass), from the in-stream event pairs
+    # ---- roofline of the weight-touching kernels (transform pass + sparse backward), from the in-stream event pairs.
+    #      Bound: what ONE fused forward+backward kernel would need: every weight read once (2 B) and one 2k-flop
+    #      transform per weight; the larger of the two times at the measured peaks.
     peaks = load_peaks()
-    k = spec["k"]
     by_kind = {}
     for d, kd in zip(kms, kinds):
         by_kind.setdefault(kd, []).append(d)
@@ -324,54 +376,45 @@ def main():
              5: "transform_pass_tcgen05"}
     kernel_ms = {names.get(kd, str(kd)): dict(launches_per_step=len(v) / args.steps, ms_per_step=sum(v) / args.steps)
                  for kd, v in by_kind.items()}
-    if "sparse_backward" in kernel_ms and k in (128, 256):
-        # the backward is a second tensor-core product over the same weights: 2k flop per weight of algorithmic
-        # work, issued twice (the routed coefficients are a two-term bf16 split)
-        sb = kernel_ms["sparse_backward"]
-        sb["algorithmic_tflops"] = 2.0 * k * layer.weights / (sb["ms_per_step"] * 1e-3) / 1e12
-        sb["issued_tflops"] = 2.0 * sb["algorithmic_tflops"]
-        sb["kernel"] = "bd_bwd_kernel (tcgen05)"
     roof = None
     tk = max((kd for kd in (1, 5) if kd in by_kind), key=lambda kd: sum(by_kind[kd]), default=None)
-    if tk is not None:
-        tp = by_kind[tk]
-        t_pass = sum(tp) / args.steps * 1e-3                    # seconds of transform passes per step
-        passes = len(tp) / args.steps / 7.0                     # passes over the layer per step
-        flops = 2.0 * k * layer.weights * passes                # 2k flop per weight per pass
-        byts = 2.0 * layer.weights * passes                     # bf16 weights read once per pass
-        tc_peak = peaks["bf16_sus"] or peaks["bf16_tflops"]
-        t_hbm, t_tc = byts / (peaks["hbm_gbs"] * 1e9), flops / (tc_peak * 1e12)
-        if t_tc >= t_hbm:
-            ach = flops / t_pass / 1e12
-            roof = dict(bound="tensor", achieved=ach, peak=tc_peak, unit="TFLOP/s", frac=ach / tc_peak, traffic=None)
+    if tk is not None and not ste:
+        t_pass = sum(by_kind[tk]) / args.steps * 1e-3
+        t_bwd = sum(by_kind.get(2, [])) / args.steps * 1e-3
+        t_fb = t_pass + t_bwd
+        flops = 2.0 * k * weights
+        byts = 2.0 * weights
+        sus = peaks["bf16_sus"] or peaks["bf16_tflops"]
+        bound_is_tensor = flops / (sus * 1e12) >= byts / (peaks["hbm_gbs"] * 1e9)
+        n_launch = (len(by_kind[tk]) + len(by_kind.get(2, []))) / args.steps
+        if bound_is_tensor:
+            ach = flops / t_fb / 1e12
+            roof = dict(bound="tensor", achieved=ach, peak=sus, unit="TFLOP/s", frac=ach / sus,
+                        frac_of_burst_peak=ach / peaks["bf16_tflops"])
         else:
-            ach = byts / t_pass / 1e9
-            roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
-                        traffic=None)
-        tb = profiled_traffic() if tk == 5 else None  # the committed ncu capture is of the tcgen05 pass
-        roof["traffic"] = tb
-        roof["traffic_note"] = "ncu dram bytes read+written per launch (mean over the 7 launches of a step)" if tb else None
-        roof["algorithmic_bytes_per_launch"] = byts / (len(tp) / args.steps)
-        roof.update(kernel=names[tk], peak_source=peaks["source"] + (" sustained" if roof["bound"] == "tensor" else ""),
-                    launches_per_step=len(tp) / args.steps, avg_launch_ms=sum(tp) / len(tp),
-                    algorithmic_gb_per_step=byts / 1e9, algorithmic_tflop_per_step=flops / 1e12,
-                    hbm_gbs_achieved=byts / t_pass / 1e9)
-        sbk = kernel_ms.get("sparse_backward")
-        if sbk:
-            # forward pass + sparse backward taken together against the same algorithmic work (one 2k-flop-per-weight
-            # transform and one read of the weights per step): what a single fused kernel would be held to
-            t_fb = t_pass + sbk["ms_per_step"] * 1e-3
-            roof["fwd_plus_bwd"] = dict(ms_per_step=t_fb * 1e3, achieved=flops / t_fb / 1e12, unit="TFLOP/s",
-                                        frac=flops / t_fb / 1e12 / tc_peak)
+            ach = byts / t_fb / 1e9
+            roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+        roof.update(traffic=profiled_traffic(),
+                    kernel="transform pass + sparse backward (bd_pass_kernel + bd_bwd_kernel), the forward+backward of one step",
+                    peak_source=peaks["source"] + (" sustained (timed inside a seconds-long run)" if bound_is_tensor else ""),
+                    launches_per_step=n_launch, ms_per_step=t_fb * 1e3,
+                    algorithmic_bytes_per_step=byts, algorithmic_flop_per_step=flops,
+                    hbm_gbs_achieved=byts / t_fb / 1e9,
+                    forward_only=dict(ms_per_step=t_pass * 1e3, tflops=flops / t_pass / 1e12, frac=flops / t_pass / 1e12 / sus,
+                                      hbm_gbs=byts / t_pass / 1e9),
+                    backward_only=dict(ms_per_step=t_bwd * 1e3, hbm_gbs=byts / t_bwd / 1e9 if t_bwd > 0 else None,
+                                       issued_tflops=(flops if use_layer else 2 * flops) / t_bwd / 1e12 if t_bwd > 0 else None,
+                                       form="one fp16 term" if use_layer else "two bf16 terms"),
+                    whole_step_frac=(flops / (ms_per_step * 1e-3) / 1e12 / sus) if bound_is_tensor else
+                                    (byts / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]))
 
     # ---- end to end through the C ABI with host buffers (pinned): H2D of every weight and transform, the step,
     #      D2H of the loss histories and the updated transforms, every step
     e2e = None
     if not args.no_e2e and rank == 0:
-        hostW = [t.cpu().pin_memory() for p in sp for t in (p.W, p.M)] + \
-                [t.cpu().pin_memory() for p in pp for t in (p.W1, p.W2, p.M)]
-        devW = [t for p in sp for t in (p.W, p.M)] + [t for p in pp for t in (p.W1, p.W2, p.M)]
-        outs = [t for p in sp + pp for t in (p.hist, p.M)]
+        hostW = [t.cpu().pin_memory() for t in step_tensors_in]
+        devW = step_tensors_in
+        outs = step_tensors_out
         hostO = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
         h2d = sum(t.numel() * t.element_size() for t in hostW)
         d2h = sum(t.numel() * t.element_size() for t in outs)
@@ -407,8 +450,8 @@ def main():
                    ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                    data="synthetic", config=cfg_json, clocks=clocks, e2e=e2e, gpu_launches=int(launches),
                    roofline=roof, cpu_baseline=cpu_base, kernels=kernel_ms,
-                   gb_per_s_algorithmic=2.0 * layer.weights * world / (ms_per_step * 1e-3) / 1e9,
-                   tflops_algorithmic=2.0 * k * layer.weights * world / (ms_per_step * 1e-3) / 1e12)
+                   gb_per_s_algorithmic=2.0 * weights * world / (ms_per_step * 1e-3) / 1e9,
+                   tflops_algorithmic=2.0 * k * weights * world / (ms_per_step * 1e-3) / 1e12)
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()

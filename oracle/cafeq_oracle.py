@@ -335,7 +335,7 @@ def orth_penalty(M):
 
 
 def pair_forward(W1s, W2s, M, bits: int, group1: int, group2: int, r: int = 1,
-                 t: float = 5.0, lam: float = 0.0, want_pqe: bool = True, prec: str = "bf16"):
+                 t: float = 5.0, lam: float = 0.0, want_pqe: bool = True, prec: str = "bf16", Minv_c=None):
     """Forward for a coupled pair.
 
     Stored W1s is [h, d1] (the paper's W1 transposed), stored W2s is [d3, r*h].
@@ -343,13 +343,20 @@ def pair_forward(W1s, W2s, M, bits: int, group1: int, group2: int, r: int = 1,
     the d_in axis with Minv_c = bf16(inv(M_c)).  LSE = (1/t) log(sum_G e^{t a_G}) over the
     group maxima of both (the quantiser's own groups), plus lam * orth_penalty(M).
     PQE = ||Uhat Vhat - W1 W2||_F, relative to ||W1 W2||_F.
+    Minv_c: optional, the second factor's operator given from outside (an inverse rounded to bf16 elsewhere:
+    which way an entry of an inverse rounds to bf16 depends on its last bits, so two computations of
+    bf16(inv(M_c)) can differ in single entries by one bf16 step; a caller that compares integer codes
+    passes the operator that was actually applied).  Gradients still differentiate through inv(M_c).
     """
     W1s = np.asarray(W1s, dtype=np.float64)
     W2s = np.asarray(W2s, dtype=np.float64)
     Mc = round_bf16(M) if prec == "bf16" else np.asarray(M, dtype=np.float64)
     k = Mc.shape[1]
     Minv = block_inverse(Mc)
-    Minv_c = round_bf16(Minv) if prec == "bf16" else Minv
+    if Minv_c is not None:
+        Minv_c = np.asarray(Minv_c, dtype=np.float64)
+    else:
+        Minv_c = round_bf16(Minv) if prec == "bf16" else Minv
     McT = np.transpose(Mc, (0, 2, 1))
     U = apply_blocks(W1s, McT, "out", 1)
     V = apply_blocks(W2s, Minv_c, "in", r)

@@ -264,7 +264,8 @@ static size_t kk_scratch_bytes(int nbT, int k) {
 // C[b] = alpha * sum_t A_t[b] B_t[b]^T + beta * C0[b] + gamma * I for nb blocks of k x k; operands bf16 [nb*k, k]
 static int launch_kk_tc(cudaStream_t st, int nterms, const uint16_t* const* A, const uint16_t* const* B, int nb, int k,
                         float alpha, float beta, float gamma, const float* C0, float* C, uint16_t* Chi, uint16_t* Clo,
-                        uint16_t* Cthi, uint16_t* Ctlo, double* sq, const int* run_flag, int32_t* status, int sq_stride = 1) {
+                        uint16_t* Cthi, uint16_t* Ctlo, double* sq, const int* run_flag, int32_t* status, int sq_stride = 1,
+                        const double* gate = nullptr, double gate_tol = 0.0) {
   TgOperand oa[TG_MAX_TERMS], ob[TG_MAX_TERMS];
   for (int t = 0; t < nterms; ++t) {
     oa[t] = TgOperand{A[t], (long long)nb * k, k, k};
@@ -285,6 +286,8 @@ static int launch_kk_tc(cudaStream_t st, int nterms, const uint16_t* const* A, c
   p.Chi = Chi; p.Clo = Clo; p.Cthi = Cthi; p.Ctlo = Ctlo;
   p.sq = sq; p.sq_stride = sq_stride;
   p.run_flag = run_flag;
+  p.gate = gate;
+  p.gate_tol = gate_tol;
   p.status = status;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return tg_launch(st, oa, ob, p);
@@ -320,9 +323,10 @@ __global__ void colnorm_kernel(const float* __restrict__ X, int k, int nb, float
 }
 
 static void launch_split(cudaStream_t st, const float* X, int k, long long n, uint16_t* hi, uint16_t* lo, uint16_t* thi,
-                         uint16_t* tlo, const int* run_flag, const int32_t* status) {
+                         uint16_t* tlo, const int* run_flag, const int32_t* status, const double* gate = nullptr,
+                         double gate_tol = 0.0) {
   dim3 grid(k / 32, k / 32, (unsigned)(n / ((long long)k * k)));
-  CQ_LAUNCH(split_bf16_kernel, grid, dim3(32, 8), 0, st, X, k, hi, lo, thi, tlo, run_flag, status);
+  CQ_LAUNCH(split_bf16_kernel, grid, dim3(32, 8), 0, st, X, k, hi, lo, thi, tlo, run_flag, status, gate, gate_tol);
 }
 
 // Minv = inv(bf16(M)) by Newton-Schulz iteration X <- X + X (I - A X) on the tensor cores, from X0 = A^T
@@ -331,9 +335,12 @@ static void launch_split(cudaStream_t st, const float* X, int k, long long n, ui
 // recomputes everything.  Leaves fp32 Minv in X, its bf16 splits in w.Xh/Xl/XTh/XTl[w.cur], and c = column
 // square norms of Minv (optional).
 static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm, int nb, int k, bool warm, KkWS& w,
-                       int32_t* status, bool prepped = false) {
+                       int32_t* status, bool prepped = false, bool splits_kept = false) {
   const long long kk = (long long)nb * k * k;
   const int iters = warm ? NS_WARM_ITERS : NS_COLD_ITERS;
+  // A warm start that is already close needs one iteration: a block whose residual ||I - A X||_F was below
+  // NS_GATE before an update (below NS_GATE^2 after it) skips the iterations that follow.
+  constexpr double NS_GATE2 = 1e-4;  // squared: the same bound the acceptance test below puts on the residual before the last update
   int ti = kt_begin(3, st);
   if (!prepped) {  // otherwise step_prep_kernel has cleared rn / flag and written Ab
     CQ_LAUNCH(zero_ns_kernel, (NS_MAX_ITERS * nb + 127) / 128, 128, 0, st, w.rn, NS_MAX_ITERS * nb, w.flag);
@@ -341,26 +348,33 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   }
   if (!warm) CQ_LAUNCH(transpose_blocks_kernel, grid_for(kk), 256, 0, st, Mc, X, k, kk);
   int cur = 0;
-  launch_split(st, X, k, kk, w.Xh[cur], iters > 0 ? nullptr : w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
+  // (splits_kept: the splits of X that the previous call left in set 0 are still there)
+  if (!(warm && splits_kept))
+    launch_split(st, X, k, kk, w.Xh[cur], iters > 0 ? nullptr : w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
   for (int it = 0; it < iters; ++it) {
+    const double* gate = (warm && it > 0) ? w.rn + (size_t)(it - 1) * nb : nullptr;
     // R = I - A X needs X to full precision (the product cancels against I): two terms over the split of X.
     const uint16_t* a1[2] = {w.Ab, w.Ab};
     const uint16_t* b1[2] = {w.XTh[cur], w.XTl[cur]};
     launch_kk_tc(st, 2, a1, b1, nb, k, -1.f, 0.f, 1.f, nullptr, nullptr, nullptr, nullptr, w.RTh, nullptr, w.rn + (size_t)it * nb,
-                 nullptr, status);
+                 nullptr, status, 1, gate, NS_GATE2);
     // X += X R: the correction is small and the iteration corrects its own errors, so one bf16 term is enough
     // (the error it leaves is 2^-8 |R| relative, below 4e-5 for every accepted residual).
     const uint16_t* a2[1] = {w.Xh[cur]};
     const uint16_t* b2[1] = {w.RTh};
     // (the row-major low half is only read after the last iteration, by the M^-1 path of the gradient)
     launch_kk_tc(st, 1, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], (it == iters - 1) ? w.Xl[cur ^ 1] : nullptr,
-                 w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr, nullptr, status);
+                 w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr, nullptr, status, 1, gate, NS_GATE2);
     cur ^= 1;
   }
   w.cur = cur;
-  // accept when ||I - A X||_F before the last update was below 1e-2 (the update squares it: <= 1e-4 after)
+  // accept when ||I - A X||_F before the last update was below 1e-2 (the update squares it: <= 1e-4 after); a block
+  // that skipped the last iteration has a zero there and was accepted by the gate
   launch_inverse(st, Mc, X, nullptr, nb, k, status, w.rn + (size_t)(iters - 1) * nb, 1e-4, w.flag);
-  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], w.flag, status);
+  // final splits: written by the last iteration's epilogue, except for blocks that skipped it (and for everything
+  // when the elimination recomputed a block)
+  const double* last_gate = (warm && iters > 1) ? w.rn + (size_t)(iters - 2) * nb : nullptr;
+  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], w.flag, status, last_gate, NS_GATE2);
   if (cnorm) {
     dim3 grid((k + 127) / 128, nb);
     CQ_LAUNCH(colnorm_kernel, grid, 128, 0, st, X, k, nb, cnorm);

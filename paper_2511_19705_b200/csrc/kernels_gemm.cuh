@@ -49,6 +49,8 @@ struct TgParams {
   double* sq;             // sum of C^2: sq[b * sq_stride]
   int sq_stride;
   const int* run_flag;    // optional: skip the whole launch when *run_flag == 0
+  const double* gate;     // optional: batch b is skipped when gate[b] <= gate_tol (its iteration has converged)
+  double gate_tol;
   int32_t* status;
 };
 
@@ -68,6 +70,7 @@ tc_gemm_kernel(const __grid_constant__ TgMaps maps, const TgParams p) {
   using C = TgCfg<BN>;
   if (p.status && *p.status) return;
   if (p.run_flag && *p.run_flag == 0) return;
+  if (p.gate && p.gate[blockIdx.z] <= p.gate_tol) return;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -362,9 +365,15 @@ static int tg_launch(cudaStream_t st, const TgOperand* A, const TgOperand* B, co
 // (grid: k/32, k/32, nb; block 32 x 8), transposed outputs staged through shared memory.  k % 32 == 0.
 __global__ void __launch_bounds__(256) split_bf16_kernel(const float* __restrict__ X, int k, uint16_t* __restrict__ hi,
                                                          uint16_t* __restrict__ lo, uint16_t* __restrict__ thi,
-                                                         uint16_t* __restrict__ tlo, const int* run_flag, const int32_t* status) {
+                                                         uint16_t* __restrict__ tlo, const int* run_flag, const int32_t* status,
+                                                         const double* gate = nullptr, double gate_tol = 0.0) {
+  // runs for every block by default; with run_flag and / or gate: only when *run_flag != 0, or for the blocks
+  // with gate[block] <= gate_tol
   if (status && *status) return;
-  if (run_flag && *run_flag == 0) return;
+  if (run_flag || gate) {
+    const bool run = (run_flag && *run_flag != 0) || (gate && gate[blockIdx.z] <= gate_tol);
+    if (!run) return;
+  }
   __shared__ uint32_t tile[32][33];
   const size_t base = (size_t)blockIdx.z * k * k;
   const int j0 = blockIdx.x * 32, i0 = blockIdx.y * 32;

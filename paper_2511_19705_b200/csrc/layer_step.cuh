@@ -42,24 +42,27 @@ struct LyPrepArgs {
   const int32_t* status;
 };
 
-__global__ void layer_prep_kernel(const LyPrepArgs a) {
+__global__ void __launch_bounds__(256) layer_prep_kernel(const LyPrepArgs a) {
   if (a.status && *a.status) return;
   const long long stride = (long long)gridDim.x * blockDim.x, t0 = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   const long long kk = (long long)a.k * a.k;
-  const long long total = (long long)a.blk0[a.n] * kk;
+  const long long total4 = (long long)a.blk0[a.n] * kk / 4;   // k is a multiple of 64 and every pointer 16-byte aligned
   const long long pair0 = (long long)a.pair_blk0 * kk;
-  for (long long e = t0; e < total; e += stride) {
+  for (long long q = t0; q < total4; q += stride) {
+    const long long e = q * 4;
     const int b = (int)(e / kk);
     int p = 0;
     while (b >= a.blk0[p + 1]) ++p;
-    const float m = a.M[p][e - (long long)a.blk0[p] * kk];
-    const __nv_bfloat16 h = __float2bfloat16_rn(m);
-    a.Mc[e] = __bfloat162float(h);
-    a.Ab[e] = __bfloat16_as_ushort(h);
-    a.grad[e] = 0.f;
+    const float4 m = *reinterpret_cast<const float4*>(a.M[p] + (e - (long long)a.blk0[p] * kk));
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(m.x), h1 = __float2bfloat16_rn(m.y);
+    const __nv_bfloat16 h2 = __float2bfloat16_rn(m.z), h3 = __float2bfloat16_rn(m.w);
+    *reinterpret_cast<float4*>(a.Mc + e) = make_float4(__bfloat162float(h0), __bfloat162float(h1), __bfloat162float(h2), __bfloat162float(h3));
+    *reinterpret_cast<uint2*>(a.Ab + e) = make_uint2((uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16),
+                                                     (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16));
+    *reinterpret_cast<float4*>(a.grad + e) = make_float4(0.f, 0.f, 0.f, 0.f);
     if (e >= pair0) {
-      a.Mf[e - pair0] = m;
-      a.gMinv[e] = 0.f;
+      *reinterpret_cast<float4*>(a.Mf + (e - pair0)) = m;
+      *reinterpret_cast<float4*>(a.gMinv + e) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
   for (long long e = t0; e < a.zone_n16; e += stride) a.zone[e] = make_uint4(0u, 0u, 0u, 0u);
@@ -68,6 +71,78 @@ __global__ void layer_prep_kernel(const LyPrepArgs a) {
     *a.flag = 0;
     for (int p = 0; p < a.n; ++p)
       if (a.step_counter[p]) *a.step_counter[p] += 1.f;
+  }
+}
+
+// Column square norms of the inverse for the single matrices' blocks (blockIdx.y = block, all singles in one launch):
+// c[b][t] = sum_i Minv[b][i][t]^2 and, for an input-axis matrix with one block per operator block, the group weights
+// of Eq. 4: cw[G] += sum_{t in G} c[t].
+struct LyColArgs {
+  int n, k;
+  int blk0[LY_MAX_PROBS + 1];   // block ranges of the singles (they come first)
+  float* cw[LY_MAX_PROBS];      // null: only c is written
+  int g[LY_MAX_PROBS];
+};
+
+__global__ void __launch_bounds__(256) layer_colnorm_kernel(const float* __restrict__ X, float* __restrict__ c, const LyColArgs a) {
+  __shared__ float part[8][33];
+  const int b = blockIdx.y, t = blockIdx.x * 32 + threadIdx.x, k = a.k;
+  int p = 0;
+  while (b >= a.blk0[p + 1]) ++p;
+  const float* Xb = X + (size_t)b * k * k;
+  float s = 0.f;
+  for (int i = threadIdx.y; i < k; i += 8) {
+    const float v = Xb[(size_t)i * k + t];
+    s = fmaf(v, v, s);
+  }
+  part[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) tot += part[q][threadIdx.x];
+    c[(size_t)b * k + t] = tot;
+    float* cw = a.cw[p];
+    if (cw) {
+      const int g = a.g[p];
+      const int col = (b - a.blk0[p]) * k + t;  // position along the transformed axis of that matrix
+      if (g >= 32) {
+        for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+        if (threadIdx.x == 0) atomicAdd(&cw[col / g], tot);
+      } else {
+        atomicAdd(&cw[col / g], tot);
+      }
+    }
+  }
+}
+
+// dL/dMinv of Eq. 4 for all single matrices: out[b][i][t] = scale_p * Minv[b][i][t] * A_t, A_t from the matrix's
+// group sums (input axis, one block per operator block) or from its per-row sums.
+struct LyGminvArgs {
+  int n, k;
+  int blk0[LY_MAX_PROBS + 1];
+  const float* A[LY_MAX_PROBS];
+  const float* Agrp[LY_MAX_PROBS];
+  int g[LY_MAX_PROBS];
+  float scale[LY_MAX_PROBS];
+};
+
+__global__ void __launch_bounds__(256) layer_gminv_kernel(const float* __restrict__ Minv, float* __restrict__ out, const LyGminvArgs a) {
+  const long long kk = (long long)a.k * a.k;
+  const long long total4 = (long long)a.blk0[a.n] * kk / 4;
+  for (long long q = blockIdx.x * (long long)blockDim.x + threadIdx.x; q < total4; q += (long long)gridDim.x * blockDim.x) {
+    const long long e = q * 4;
+    const int b = (int)(e / kk);
+    int p = 0;
+    while (b >= a.blk0[p + 1]) ++p;
+    const int t = (int)(e % a.k);
+    const int bl = b - a.blk0[p];
+    float At[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) At[j] = a.Agrp[p] ? a.Agrp[p][(bl * a.k + t + j) / a.g[p]] : a.A[p][bl * a.k + t + j];
+    const float4 x = *reinterpret_cast<const float4*>(Minv + e);
+    const float sc = a.scale[p];
+    *reinterpret_cast<float4*>(out + e) = make_float4(sc * x.x * At[0], sc * x.y * At[1], sc * x.z * At[2], sc * x.w * At[3]);
   }
 }
 
@@ -151,32 +226,49 @@ __global__ void __launch_bounds__(256) layer_finish_kernel(const LyFinishArgs f)
     f.hist[p][0] = loss;
     f.hist[p][1] = nanf("");
   }
-  float* M = f.M[p];
-  const float* g = f.grad + off;
-  const float* RM = f.pair[p] ? f.RM + (off - (long long)f.pair_blk0 * kk) : nullptr;
+  float4* M4 = reinterpret_cast<float4*>(f.M[p]);
+  const float4* g4 = reinterpret_cast<const float4*>(f.grad + off);
+  const float4* RM4 = f.pair[p] ? reinterpret_cast<const float4*>(f.RM + (off - (long long)f.pair_blk0 * kk)) : nullptr;
   const float lr = f.lr[p];
-  if (f.optimizer[p] == CAFEQ_OPT_GD) {
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-      float gi = g[i];
-      if (orth_f != 0.f) gi = fmaf(orth_f, RM[i], gi);
-      M[i] = M[i] - lr * gi;
-    }
-  } else {
+  const long long n4 = n / 4;
+  const bool adam = f.optimizer[p] != CAFEQ_OPT_GD;
+  float b1 = 0.f, b2 = 0.f, eps = 0.f, c1 = 1.f, c2 = 1.f;
+  float4 *m4 = nullptr, *v4 = nullptr;
+  if (adam) {
     float* state = f.state[p];
     const float step = state[0];
-    const float b1 = f.b1[p], b2 = f.b2[p], eps = f.eps[p];
-    const float c1 = 1.f - powf(b1, step), c2 = 1.f - powf(b2, step);
-    float* m = state + CAFEQ_OPT_STATE_HEADER;
-    float* v = state + CAFEQ_OPT_STATE_HEADER + n;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-      float gi = g[i];
-      if (orth_f != 0.f) gi = fmaf(orth_f, RM[i], gi);
-      const float mi = b1 * m[i] + (1.f - b1) * gi;
-      const float vi = b2 * v[i] + (1.f - b2) * gi * gi;
-      m[i] = mi;
-      v[i] = vi;
-      M[i] = M[i] - lr * (mi / c1) / (sqrtf(vi / c2) + eps);
+    b1 = f.b1[p]; b2 = f.b2[p]; eps = f.eps[p];
+    c1 = 1.f - powf(b1, step);
+    c2 = 1.f - powf(b2, step);
+    m4 = reinterpret_cast<float4*>(state + CAFEQ_OPT_STATE_HEADER);
+    v4 = reinterpret_cast<float4*>(state + CAFEQ_OPT_STATE_HEADER + n);
+  }
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
+    float4 gq = g4[i];
+    float gi[4] = {gq.x, gq.y, gq.z, gq.w};
+    if (orth_f != 0.f) {
+      const float4 r = RM4[i];
+      gi[0] = fmaf(orth_f, r.x, gi[0]); gi[1] = fmaf(orth_f, r.y, gi[1]);
+      gi[2] = fmaf(orth_f, r.z, gi[2]); gi[3] = fmaf(orth_f, r.w, gi[3]);
     }
+    const float4 mq = M4[i];
+    float mv[4] = {mq.x, mq.y, mq.z, mq.w};
+    if (!adam) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) mv[j] = mv[j] - lr * gi[j];
+    } else {
+      const float4 ma = m4[i], va = v4[i];
+      float mm[4] = {ma.x, ma.y, ma.z, ma.w}, vv[4] = {va.x, va.y, va.z, va.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        mm[j] = b1 * mm[j] + (1.f - b1) * gi[j];
+        vv[j] = b2 * vv[j] + (1.f - b2) * gi[j] * gi[j];
+        mv[j] = mv[j] - lr * (mm[j] / c1) / (sqrtf(vv[j] / c2) + eps);
+      }
+      m4[i] = make_float4(mm[0], mm[1], mm[2], mm[3]);
+      v4[i] = make_float4(vv[0], vv[1], vv[2], vv[3]);
+    }
+    M4[i] = make_float4(mv[0], mv[1], mv[2], mv[3]);
   }
 }
 
@@ -426,7 +518,7 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
     a.zone = reinterpret_cast<uint4*>(L.zone); a.zone_n16 = (long long)(L.zone_bytes / 16);
     a.rn = w.rn; a.rn_n = NS_MAX_ITERS * NB; a.flag = w.flag;
     a.status = status;
-    CQ_LAUNCH(layer_prep_kernel, grid_for(kk), 256, 0, st, a);
+    CQ_LAUNCH(layer_prep_kernel, grid_for(kk / 4), 256, 0, st, a);
   }
   bool any_lambda = false;
   for (int q = 0; q < L.n; ++q) any_lambda |= (L.p[q].pair && L.p[q].cfg.lambda_orth != 0.f);
@@ -444,18 +536,31 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
       launch_kk_tc(st, 3, a2, b2, nbP, k, 1.f, 0.f, 0.f, nullptr, L.RM, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, status);
     }
   }
-  ns_inverse(st, L.Mc, L.Minv, nullptr, NB, k, true, w, status, true);
-  // Eq. 4 weights of the single matrices
-  for (int q = 0; q < L.n; ++q) {
-    const LyProb& P = L.p[q];
-    if (P.pair) continue;
-    const LyMat& Mt = L.m[P.m0];
-    const Geo& G = Mt.G;
-    const bool in_r1 = (G.axis == CAFEQ_AXIS_IN && G.r == 1);
-    const long long off = (long long)P.blk0 * kk1;
-    dim3 cg(k / 32, P.nb);
-    CQ_LAUNCH(colnorm_cw_kernel, cg, dim3(32, 8), 0, st, L.Minv + off, k, L.c + (size_t)P.blk0 * k, in_r1 ? Mt.cw : nullptr, G.g);
-    if (!in_r1) {
+  ns_inverse(st, L.Mc, L.Minv, nullptr, NB, k, true, w, status, true, true);
+  // Eq. 4 weights of the single matrices (they own the first pair_blk0 blocks)
+  if (L.pair_blk0 > 0) {
+    LyColArgs ca;
+    memset(&ca, 0, sizeof(ca));
+    ca.k = k;
+    int ns = 0;
+    for (int q = 0; q < L.n; ++q) {
+      const LyProb& P = L.p[q];
+      if (P.pair) continue;
+      const Geo& G = L.m[P.m0].G;
+      ca.blk0[ns] = P.blk0;
+      ca.cw[ns] = (G.axis == CAFEQ_AXIS_IN && G.r == 1) ? L.m[P.m0].cw : nullptr;
+      ca.g[ns] = G.g;
+      ++ns;
+    }
+    ca.blk0[ns] = L.pair_blk0;
+    ca.n = ns;
+    CQ_LAUNCH(layer_colnorm_kernel, dim3(k / 32, L.pair_blk0), dim3(32, 8), 0, st, L.Minv, L.c, ca);
+    for (int q = 0; q < L.n; ++q) {
+      const LyProb& P = L.p[q];
+      if (P.pair) continue;
+      const LyMat& Mt = L.m[P.m0];
+      const Geo& G = Mt.G;
+      if (G.axis == CAFEQ_AXIS_IN && G.r == 1) continue;
       if (G.axis == CAFEQ_AXIS_IN) CQ_LAUNCH(cw_in_kernel, (G.ng + 127) / 128, 128, 0, st, L.c + (size_t)P.blk0 * k, G.d_in, G.g, k, G.r, Mt.cw);
       else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, L.c + (size_t)P.blk0 * k, G.d_out, G.g, k, G.r, Mt.cw);
     }
@@ -561,15 +666,28 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
       }
     }
   // dL/dMinv of Eq. 4 for the singles, then grad -= Minv^T (dL/dMinv) Minv^T over all blocks
-  for (int q = 0; q < L.n; ++q) {
-    const LyProb& P = L.p[q];
-    if (P.pair) continue;
-    const LyMat& Mt = L.m[P.m0];
-    const Geo& G = Mt.G;
-    const bool in_r1 = (G.axis == CAFEQ_AXIS_IN && G.r == 1);
-    const long long off = (long long)P.blk0 * kk1, kkp = (long long)P.nb * kk1;
-    if (G.axis == CAFEQ_AXIS_IN && !in_r1) CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, Mt.agrp, G.d_in, G.g, k, G.r, Mt.A);
-    CQ_LAUNCH(gminv_kernel, grid_for(kkp), 256, 0, st, L.Minv + off, Mt.A, in_r1 ? Mt.agrp : nullptr, G.g, 2.f * P.kappa, k, kkp, L.gMinv + off);
+  if (L.pair_blk0 > 0) {
+    LyGminvArgs ga;
+    memset(&ga, 0, sizeof(ga));
+    ga.k = k;
+    int ns = 0;
+    for (int q = 0; q < L.n; ++q) {
+      const LyProb& P = L.p[q];
+      if (P.pair) continue;
+      const LyMat& Mt = L.m[P.m0];
+      const Geo& G = Mt.G;
+      const bool in_r1 = (G.axis == CAFEQ_AXIS_IN && G.r == 1);
+      if (G.axis == CAFEQ_AXIS_IN && !in_r1) CQ_LAUNCH(expand_agrp_kernel, (G.d_in + 127) / 128, 128, 0, st, Mt.agrp, G.d_in, G.g, k, G.r, Mt.A);
+      ga.blk0[ns] = P.blk0;
+      ga.A[ns] = Mt.A;
+      ga.Agrp[ns] = in_r1 ? Mt.agrp : nullptr;
+      ga.g[ns] = G.g;
+      ga.scale[ns] = 2.f * P.kappa;
+      ++ns;
+    }
+    ga.blk0[ns] = L.pair_blk0;
+    ga.n = ns;
+    CQ_LAUNCH(layer_gminv_kernel, grid_for((long long)L.pair_blk0 * kk1 / 4), 256, 0, st, L.Minv, L.gMinv, ga);
   }
   minv_path_tc(st, L.gMinv, L.grad, NB, k, true, w, status);
   {
@@ -593,7 +711,7 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
     f.orth_sq = L.orth_sq; f.pair_blk0 = L.pair_blk0;
     f.grad = L.grad; f.RM = L.RM;
     f.status = status;
-    CQ_LAUNCH(layer_finish_kernel, dim3(grid_for(nmax, 256, 148 * 2), L.n), 256, 0, st, f);
+    CQ_LAUNCH(layer_finish_kernel, dim3(grid_for(nmax / 4, 256, 148 * 4), L.n), 256, 0, st, f);
   }
   return CAFEQ_OK;
 }
@@ -640,7 +758,7 @@ extern "C" int cafeq_layer_prepare(const cafeq_layer_problem* probs, int n, int3
     a.zone = reinterpret_cast<uint4*>(L.zone); a.zone_n16 = (long long)(L.zone_bytes / 16);
     a.rn = L.kk.rn; a.rn_n = NS_MAX_ITERS * L.NB; a.flag = L.kk.flag;
     a.status = status;
-    CQ_LAUNCH(layer_prep_kernel, grid_for(kk), 256, 0, st, a);
+    CQ_LAUNCH(layer_prep_kernel, grid_for(kk / 4), 256, 0, st, a);
   }
   ns_inverse(st, L.Mc, L.Minv, nullptr, L.NB, L.k, false, L.kk, status, true);
   return last_launch();

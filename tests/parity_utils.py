@@ -53,3 +53,58 @@ def assert_codes_tie_aware(q_gpu, s_gpu, Q, U64, group, window=2e-4, max_frac=2e
         assert np.all(dist[bad] <= window * np.maximum(1.0, np.abs(x[bad]))), "code differs away from a tie"
     assert frac <= max_frac, f"too many near-tie mismatches: {frac}"
     return float(frac)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# inputs without rounding ties
+# ---------------------------------------------------------------------------------------------------------
+def near_tie_mask(U64, bits, group, window):
+    """Entries of a transformed matrix whose quotient U/s lies within `window` * max(1, |x|) of a rounding boundary,
+    and groups whose two largest magnitudes are within 1e-5 relative of each other (either would let fp32 and
+    float64 arithmetic disagree about an integer decision).  Returns a boolean [d_out, d_in] mask."""
+    from oracle import cafeq_oracle as orc
+    Q = orc.quant_sym(U64, bits, group)
+    d_out, d_in = U64.shape
+    g = d_in if group == 0 else group
+    s_e = np.repeat(Q["s"].astype(np.float64), g, axis=1)
+    x = np.where(s_e > 0, U64 / np.where(s_e > 0, s_e, 1.0), 0.0)
+    dist = np.abs(np.abs(x - np.floor(x)) - 0.5)
+    bad = dist <= window * np.maximum(1.0, np.abs(x))
+    A = np.sort(np.abs(U64).reshape(d_out, d_in // g, g), axis=2)
+    close = (A[..., -1] - A[..., -2]) <= 1e-5 * A[..., -1]
+    return bad | np.repeat(close, g, axis=1)
+
+
+def tie_free_weight(draw, transform, bits, group, redraw, window=2e-4, max_iter=200):
+    """A seeded weight (bf16 bit patterns) none of whose transformed entries is a near-tie.
+
+    draw(i) -> uint16 [d_out, d_in] bit patterns of the i-th independent draw; transform(W64) -> U64;
+    redraw = "rows" when a transformed entry depends only on its own row of W (input-axis transform), "cols" when
+    it depends only on its own column (output-axis transform).  Rows / columns holding a near-tie are replaced from
+    the next draw until none is left.  Comparing the device with the oracle on such inputs removes the one
+    difference that is not an error: an fp32 quotient and a float64 quotient landing on opposite sides of a
+    half-integer."""
+    Wb = draw(0).copy()
+    for it in range(1, max_iter + 1):
+        mask = near_tie_mask(transform(w64(Wb)), bits, group, window)
+        lines = mask.any(axis=1) if redraw == "rows" else mask.any(axis=0)
+        if not lines.any():
+            return Wb
+        fresh = draw(it)
+        if redraw == "rows":
+            Wb[lines] = fresh[lines]
+        else:
+            Wb[:, lines] = fresh[:, lines]
+    raise AssertionError("could not draw a tie-free weight")
+
+
+def device_inverse(cq, M):
+    """inv(bf16(M)) as the device computes it from a cold start (float32 numpy [nb,k,k]); the pair calls apply
+    bf16 of exactly this to the second factor."""
+    import torch
+    nb, k, _ = M.shape
+    Wd = torch.zeros((64, nb * k), dtype=torch.bfloat16, device="cuda")
+    out = cq.cafeq_proxy_loss_fwd_bwd(Wd, f32_dev(M), bits=4, group=0, flags=cq.FLAG_NO_GRAD, want_minv=True)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    return out["Minv"].cpu().numpy()
