@@ -5,7 +5,7 @@ import pytest
 
 import cafeq_synth as syn
 from oracle import cafeq_oracle as orc
-from parity_utils import assert_codes_tie_aware, f32_dev, rel_err, to_dev, w64
+from parity_utils import assert_codes_tie_aware, f32_dev, rel_err, tie_free_weight, to_dev, w64
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -162,9 +162,11 @@ STE_SHAPES = [(64, 64, 4, (128, 256)), (128, 128, 3, (320, 512)), (256, 128, 3, 
 @pytest.mark.parametrize("k,group,bits,shape", STE_SHAPES)
 def test_fused_single_ste_matches_oracle(cq, k, group, bits, shape):
     d_out, d_in = shape
-    Wb = syn.weight_student_t(d_out, d_in, seed=77, n_outlier_channels=2, mult=10.0)
     nb = d_in // k
     M = syn.perturbed_blocks(nb, k, 19, 0.1)
+    # inputs without rounding ties: the straight-through gradient is compared at codes both sides agree on
+    Wb = tie_free_weight(lambda i: syn.weight_student_t(d_out, d_in, seed=77 + 1000 * i, n_outlier_channels=2, mult=10.0),
+                         lambda W: orc.apply_blocks(W, orc.round_bf16(M), "in"), bits, group, "rows")
     out = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=bits, group=group, loss_kind=cq.LOSS_L2_STE)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
@@ -177,14 +179,16 @@ def test_fused_single_ste_matches_oracle(cq, k, group, bits, shape):
     assert abs(L[2] - f["normW2"]) <= 1e-5 * f["normW2"]
     gg = out["gradM"].cpu().numpy()
     assert np.isfinite(gg).all()
-    # near-tie code flips change single terms of the scale path: compare over all blocks together too
-    assert rel_err(gg, g) <= 2 * TOL
+    assert rel_err(gg, g) <= TOL
     for b in range(nb):
-        assert rel_err(gg[b], g[b]) <= 5 * TOL, f"block {b}"
-    # the shape-agnostic path of the same call agrees as well
+        assert rel_err(gg[b], g[b]) <= TOL, f"block {b}"
+    # the shape-agnostic path of the same call against the oracle as well
     ref = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=bits, group=group, loss_kind=cq.LOSS_L2_STE,
                                       flags=cq.FLAG_GENERIC)
-    assert rel_err(gg, ref["gradM"].cpu().numpy()) <= 2 * TOL
+    gr = ref["gradM"].cpu().numpy()
+    assert rel_err(gr, g) <= TOL
+    for b in range(nb):
+        assert rel_err(gr[b], g[b]) <= TOL, f"generic path, block {b}"
 
 
 # ------------------------------------------------------------------ the random baseline through the same kernels
@@ -225,8 +229,11 @@ def test_fused_full_size_k_matrix_straight_through(cq):
     """k of the 9B-shaped layer (2048 x 3584, k = 256, 3-bit, g = 128) in the straight-through mode, on the launch
     configuration the benchmark's `--loss ste` run times: losses and the whole gradient against the oracle."""
     name, d_out, d_in = "k", 2048, 3584
-    Wb = syn.make_weight(3, name, d_out, d_in)
     M = syn.make_transform(name, d_in // 256, 256)
+    # the benchmark's seeded weight with the rows that hold a rounding tie under this transform re-drawn from the
+    # following layers' seeds
+    Wb = tie_free_weight(lambda i: syn.make_weight(3, name, d_out, d_in, i),
+                         lambda W: orc.apply_blocks(W, orc.round_bf16(M), "in"), 3, 128, "rows", window=1e-4)
     out = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=3, group=128, loss_kind=cq.LOSS_L2_STE)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
@@ -237,6 +244,6 @@ def test_fused_full_size_k_matrix_straight_through(cq):
     assert abs(L[1] - f["L2"]) <= TOL * f["L2"]
     assert abs(L[2] - f["normW2"]) <= 1e-5 * f["normW2"]
     gg = out["gradM"].cpu().numpy()
-    assert rel_err(gg, g) <= 2 * TOL
+    assert rel_err(gg, g) <= TOL
     for b in range(d_in // 256):
-        assert rel_err(gg[b], g[b]) <= 5 * TOL, f"block {b}"
+        assert rel_err(gg[b], g[b]) <= TOL, f"block {b}"

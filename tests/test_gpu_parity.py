@@ -8,7 +8,7 @@ import pytest
 
 import cafeq_synth as syn
 from oracle import cafeq_oracle as orc
-from parity_utils import assert_codes_tie_aware, f32_dev, rel_err, to_dev, w64
+from parity_utils import assert_codes_tie_aware, device_inverse, f32_dev, rel_err, tie_free_weight, to_dev, w64
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -114,9 +114,12 @@ def test_single_surrogate_fwd_bwd(cq, axis, k, bits, group, shape):
 
 @pytest.mark.parametrize("axis,k,bits,group,shape", CASES_SINGLE[:5])
 def test_single_ste_fwd_bwd(cq, axis, k, bits, group, shape):
-    Wb = syn.weight_student_t(*shape, seed=43, n_outlier_channels=2, mult=10.0)
     nb = (shape[1] if axis == "in" else shape[0]) // k
     M = syn.perturbed_blocks(nb, k, 15, 0.1)
+    # inputs without rounding ties: the straight-through gradient is compared at codes both sides agree on
+    Wb = tie_free_weight(lambda i: syn.weight_student_t(*shape, seed=43 + 1000 * i, n_outlier_channels=2, mult=10.0),
+                         lambda W: orc.apply_blocks(W, orc.round_bf16(M), axis), bits, group,
+                         "rows" if axis == "in" else "cols")
     out = cq.cafeq_proxy_loss_fwd_bwd(to_dev(Wb), f32_dev(M), bits=bits, group=group, taxis=_axis(axis, cq),
                                       loss_kind=cq.LOSS_L2_STE)
     W = w64(Wb)
@@ -125,10 +128,9 @@ def test_single_ste_fwd_bwd(cq, axis, k, bits, group, shape):
     L = out["losses"].cpu().numpy()
     assert abs(L[1] - f["L2"]) <= TOL * f["L2"]
     gg = out["gradM"].cpu().numpy()
-    # near-tie code flips change single terms of the scale path: compare over all blocks together too
-    assert rel_err(gg, g) <= 2 * TOL
+    assert rel_err(gg, g) <= TOL
     for b in range(nb):
-        assert rel_err(gg[b], g[b]) <= 5 * TOL, f"block {b}"
+        assert rel_err(gg[b], g[b]) <= TOL, f"block {b}"
 
 
 def test_offsets_exhaustive_tiny(cq):
@@ -247,14 +249,20 @@ PAIR_CASES = [(32, 1, 0, 32, (64, 96, 80)), (64, 2, 128, 64, (128, 256, 192)), (
 @pytest.mark.parametrize("k,r,g1,g2,dims", PAIR_CASES)
 def test_pair_lse_pqe_fwd_bwd(cq, k, r, g1, g2, dims):
     h, d1, d3 = dims
-    W1b = syn.weight_student_t(h, d1, 51, 2, 10.0)
-    W2b = syn.weight_student_t(d3, r * h, 52, 2, 10.0)
     M = syn.perturbed_blocks(h // k, k, 17, 0.1)
     bits, lam, t = 4, 0.1, 5.0
+    # the second factor's operator is bf16 of the inverse as the device computes it (single entries of an inverse
+    # round to bf16 differently in fp32 and float64); weights without rounding ties under both operators
+    Minv_c = orc.round_bf16(device_inverse(cq, M))
+    McT = np.transpose(orc.round_bf16(M), (0, 2, 1))
+    W1b = tie_free_weight(lambda i: syn.weight_student_t(h, d1, 51 + 1000 * i, 2, 10.0),
+                          lambda W: orc.apply_blocks(W, McT, "out", 1), bits, g1, "cols")
+    W2b = tie_free_weight(lambda i: syn.weight_student_t(d3, r * h, 52 + 1000 * i, 2, 10.0),
+                          lambda W: orc.apply_blocks(W, Minv_c, "in", r), bits, g2, "rows")
     W1d, W2d, Md = to_dev(W1b), to_dev(W2b), f32_dev(M)
     P = cq.cafeq_pair_product(W1d, W2d, k=k, replicas=r)
     W1, W2 = w64(W1b), w64(W2b)
-    f = orc.pair_forward(W1, W2, M, bits, g1, g2, r, t, lam, True)
+    f = orc.pair_forward(W1, W2, M, bits, g1, g2, r, t, lam, True, Minv_c=Minv_c)
     assert rel_err(P.cpu().numpy(), f["P"]) <= 1e-5
     out = cq.cafeq_pair_loss_fwd_bwd(W1d, W2d, Md, bits=bits, group1=g1, group2=g2, replicas=r, P=P, lse_t=t,
                                      lambda_orth=lam, flags=cq.FLAG_EXACT_LOSS)
@@ -264,7 +272,7 @@ def test_pair_lse_pqe_fwd_bwd(cq, k, r, g1, g2, dims):
     assert abs(L[0] - f["loss"]) <= TOL * abs(f["loss"])
     assert abs(L[1] - f["lse"]) <= TOL * abs(f["lse"])
     assert abs(L[2] - f["orth"]) <= TOL * f["orth"]
-    assert abs(L[3] - f["pqe"] ** 2) <= 2 * TOL * f["pqe"] ** 2
+    assert abs(L[3] - f["pqe"] ** 2) <= TOL * f["pqe"] ** 2
     g = orc.pair_grad_lse(W1, W2, f, g1, g2)
     gg = out["gradM"].cpu().numpy()
     # the LSE gradient is dominated by a handful of arg-max entries: compare the whole parameter
