@@ -102,8 +102,14 @@ typedef struct {
                          inverse is refined instead of inverting from scratch) */
 } cafeq_opt_cfg;
 
-/* Scratch bytes needed by any call on d1 (and d2 for pair calls; NULL otherwise).  cfg may be NULL.
- * `bytes` is a host pointer.  The same size serves every entry point below for these descriptors. */
+/* Scratch bytes needed by the calls on d1 (and d2 for pair calls; NULL otherwise).  `bytes` is a host pointer.
+ * cfg = NULL: the size that serves every entry point and every mode for these descriptors (matrix-sized fp32 and
+ * bf16 buffers: about 30 bytes per weight).
+ * cfg given: the size cafeq_optimize_single / cafeq_optimize_pair need for exactly that configuration.  For the
+ * paper's objectives (CAFEQ_LOSS_SURROGATE / CAFEQ_LOSS_LSE) with eval_every = 0, block size 64 / 128 / 256 and a
+ * shape the tensor-core pass covers, nothing matrix-sized is needed: the per-(row, group) records (16 bytes per
+ * group) and the k x k scratch.  The size assumes 16-byte aligned weight rows; a call whose weights do not qualify
+ * then returns CAFEQ_ERR_WORKSPACE. */
 int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
                          size_t* bytes);
 
@@ -114,6 +120,12 @@ int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d
 int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
               void* ws, size_t ws_bytes, void* stream);
 
+/* Scratch bytes cafeq_rtn takes from its workspace for this descriptor (host out), with (has_transform != 0) or
+ * without an operator, for 16-byte aligned W and 8-byte aligned codes: 0 without a transform when the group is
+ * 32 / 64 / 128 / 256 (one streaming kernel, ws may then be NULL); the per-group records when the tensor-core pass
+ * covers the transformed call; matrix-sized buffers otherwise.  Never more than cafeq_workspace_size(d, NULL, NULL). */
+int cafeq_rtn_workspace_size(const cafeq_matrix_desc* d, int has_transform, size_t* bytes);
+
 /* cafeq_rtn for callers that cannot allocate device memory and therefore have no workspace to hand
  * over: code running inside a memory-pool or allocator callback, between the driver calls of another
  * library that forbids allocation, in a process whose memory budget is already fixed, or anywhere a
@@ -123,7 +135,7 @@ int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t*
  *     that loads the library holds it from then until the process exits.  Inputs and outputs are still
  *     the caller's.  Neither this call nor anything under it calls cudaMalloc, cudaFree or an
  *     allocating library routine.
- *   - A descriptor whose cafeq_workspace_size exceeds CAFEQ_NOALLOC_SCRATCH_BYTES is refused with
+ *   - A call whose scratch need (cafeq_rtn_workspace_size) exceeds CAFEQ_NOALLOC_SCRATCH_BYTES is refused with
  *     CAFEQ_ERR_TOO_LARGE before anything is launched (use cafeq_rtn with your own workspace then).
  *   - The first call on each device looks up the buffer's device address (with that device current);
  *     make that first call outside any stream capture.  Later calls only enqueue kernels.
@@ -279,6 +291,14 @@ long long cafeq_debug_launch_count(void);
  * Not thread-safe; launches beyond the capacity are simply not timed. */
 int cafeq_debug_timer_begin(int capacity);
 int cafeq_debug_timer_read(float* ms, int* kinds, int* count);
+
+/* Self-test of the kernels' bounded waits (the paper has no counterpart).  Every wait inside the kernels of this
+ * library is limited (2 s); when one runs out the kernel raises CAFEQ_ERR_TIMEOUT in the status word, its roles
+ * leave their loops and it returns.  This call runs that wait helper in a one-thread kernel on a barrier that nothing
+ * completes, with the limit given here (nanoseconds), then lets the thread complete the barrier itself and wait
+ * again.  Device outputs: `status` receives CAFEQ_ERR_TIMEOUT (if it was 0), result[0] = 1 when the first wait gave
+ * up, result[1] = 1 when the second succeeded.  Nothing in it can hang: no other thread is waited for. */
+int cafeq_debug_wait_probe(unsigned long long limit_ns, int32_t* status, int* result, void* stream);
 
 #ifdef __cplusplus
 }

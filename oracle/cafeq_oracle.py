@@ -322,15 +322,16 @@ def pair_product(A1s, A2s, k: int, r: int):
 def orth_penalty(M):
     """||M M^T - I||_F / sqrt(d) on the whole block-diagonal M, and its gradient.
 
-    The norm is not squared, so its gradient has no limit at M M^T = I; below 1e-5 (the noise floor
-    of an fp32 product of a rotation stored in fp32) the gradient is taken as zero."""
+    The norm is not squared, so its gradient has no limit at M M^T = I; exactly there (norm 0) the
+    sub-gradient 0 is taken.  (A device that forms M M^T in fp32 cannot tell a rotation from its
+    rounding noise; that floor belongs to the device and to the inputs a parity test chooses, not here.)"""
     M = np.asarray(M, dtype=np.float64)
     nb, k, _ = M.shape
     R = M @ np.transpose(M, (0, 2, 1)) - np.eye(k)
     nrm = np.sqrt(np.sum(R * R))
     d = nb * k
-    if nrm / np.sqrt(d) < 1e-5:
-        return float(nrm / np.sqrt(d)), np.zeros_like(M)
+    if nrm == 0.0:
+        return 0.0, np.zeros_like(M)
     return float(nrm / np.sqrt(d)), (2.0 * R @ M) / (nrm * np.sqrt(d))
 
 
@@ -554,10 +555,42 @@ def brute_force_single(W, M, bits: int, group: int, axis: str = "in"):
 
 
 def pqe_with_offsets(U1s, V2s, bits, group1, group2, k, r, off1, off2):
+    """Eq. 5 for a transformed pair (stored layouts) with both factors rounded by given floor/ceil offsets at
+    their round-to-nearest scales: || Q_off1(U) Q_off2(V) - U V ||_F."""
     P = pair_product(U1s, V2s, k, r)
     Q1 = quant_sym(U1s, bits, group1, off1)
     Q2 = quant_sym(V2s, bits, group2, off2)
     return float(np.linalg.norm(pair_product(Q1["Uhat"], Q2["Uhat"], k, r) - P))
+
+
+def brute_force_pair(U1s, V2s, bits: int, group1: int, group2: int, k: int, r: int):
+    """All 2^(n1+n2) floor/ceil choices of both factors at their round-to-nearest scales (n1 + n2 <= 16):
+    returns (best PQE, best offsets of the first factor, of the second, all PQE values in enumeration order)."""
+    U1s = np.asarray(U1s, dtype=np.float64)
+    V2s = np.asarray(V2s, dtype=np.float64)
+    n1, n2 = U1s.size, V2s.size
+    if n1 + n2 > 16:
+        raise ValueError("brute force is for n1 + n2 <= 16")
+    best, b1, b2, allv = np.inf, None, None, []
+    for bitsv in itertools.product((0.0, 1.0), repeat=n1 + n2):
+        o1 = np.array(bitsv[:n1]).reshape(U1s.shape)
+        o2 = np.array(bitsv[n1:]).reshape(V2s.shape)
+        v = pqe_with_offsets(U1s, V2s, bits, group1, group2, k, r, o1, o2)
+        allv.append(v)
+        if v < best:
+            best, b1, b2 = v, o1, o2
+    return best, b1, b2, np.array(allv)
+
+
+def rtn_offsets(U, bits: int, group: int):
+    """The floor/ceil offsets that reproduce round-to-nearest: offset = rne(x) - floor(x) for x = U/s."""
+    Q = quant_sym(U, bits, group)
+    g = _groups(np.asarray(U).shape[1], group)
+    s_e = np.repeat(Q["s"], g, axis=1)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        x = (np.asarray(U, dtype=np.float64).astype(F32) / s_e).astype(F32)
+    x = np.where(s_e > 0, x, F32(0))
+    return (np.rint(x) - np.floor(x)).astype(np.float64)
 
 
 # ---------------------------------------------------------------------------

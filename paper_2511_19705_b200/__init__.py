@@ -23,9 +23,9 @@ FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC, FLAG_WARM_MINV = 1, 2, 4, 8
 OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 
 EXPORTS = [
-    "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
+    "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_workspace_size", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_set_overlap_mode", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
     "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
@@ -143,6 +143,13 @@ def workspace_size(d1: MatrixDesc, d2: MatrixDesc | None = None, cfg: OptCfg | N
     rc = lib().cafeq_workspace_size(ctypes.byref(d1), ctypes.byref(d2) if d2 is not None else None,
                                     ctypes.byref(cfg) if cfg is not None else None, ctypes.byref(n))
     _check(rc, "cafeq_workspace_size")
+    return int(n.value)
+
+
+def rtn_workspace_size(d: MatrixDesc, has_transform: bool) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().cafeq_rtn_workspace_size(ctypes.byref(d), ctypes.c_int(1 if has_transform else 0), ctypes.byref(n)),
+           "cafeq_rtn_workspace_size")
     return int(n.value)
 
 

@@ -16,6 +16,7 @@
 #include "kernels_bwd.cuh"
 #include "kernels_gemm.cuh"
 #include "kernels_dense.cuh"
+#include "kernels_rtn.cuh"
 
 namespace cafeq {
 
@@ -57,10 +58,11 @@ struct Bump {
   size_t cap, used;
   bool overflow;
   Bump(void* b, size_t c) : base((char*)b), cap(c), used(0), overflow(false) {}
+  // (base == nullptr: nothing is handed out, `used` still adds up -- the size queries run the same carving code)
   template <typename T>
   T* take(size_t count) {
     size_t bytes = (count * sizeof(T) + 255) & ~(size_t)255;
-    if (used + bytes > cap) { overflow = true; used += bytes; return nullptr; }
+    if (!base || used + bytes > cap) { overflow = true; used += bytes; return nullptr; }
     T* p = (T*)(base + used);
     used += bytes;
     return p;
@@ -111,25 +113,6 @@ static int make_geo(const cafeq_matrix_desc* d, Geo* o, bool need_transform) {
     return CAFEQ_ERR_INVALID_ARG;
   }
   return CAFEQ_OK;
-}
-
-static size_t kk_scratch_bytes(int nbT, int k);
-
-// scratch that one matrix needs in any call
-static size_t matrix_scratch_bytes(const Geo& G, bool with_backward = true) {
-  size_t kk = (size_t)(G.nbT > 0 ? G.nbT : 1) * (size_t)(G.k > 0 ? G.k : 1) * (size_t)(G.k > 0 ? G.k : 1);
-  size_t rows_ng = (size_t)G.d_out * G.ng;
-  size_t b = 0;
-  b += 3 * ((size_t)G.n * 4 + 256);                   // U, Delta / gDelta, E / Uhat
-  b += (size_t)G.n * 2 + 256;                         // bf16 residual of the fused pass
-  b += 4 * (rows_ng * 4 + 256);                       // a, usel, idx, coef
-  b += ((size_t)G.ng + G.d_out + G.d_in) * 4 + 1024;  // cw, Agrp
-  b += 8 * (kk * 4 + 256);                            // Mc, Minv, Minv_c, gMinv, tmp, RM, ...
-  b += 4 * ((size_t)(G.nbT + 1) * (G.k + 1) * 4 + 256);  // c, A
-  b += 4096;                                          // accumulators
-  b += kk_scratch_bytes(G.nbT, G.k);                  // bf16 splits of the k x k algebra
-  if (with_backward) b += 3 * ((size_t)G.n * 2 + 256) + kk * 4 + 256;  // straight-through path on the tensor cores
-  return b;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -255,10 +238,6 @@ static void carve_kk(Bump& b, int nbT, int k, KkWS* w) {
   w->rn = b.take<double>((size_t)NS_MAX_ITERS * nbT);
   w->flag = b.take<int>(64);
   w->cur = 0;
-}
-static size_t kk_scratch_bytes(int nbT, int k) {
-  const size_t kk = (size_t)(nbT > 0 ? nbT : 1) * (k > 0 ? k : 1) * (k > 0 ? k : 1);
-  return 15 * (kk * 2 + 256) + (size_t)NS_MAX_ITERS * (nbT + 1) * 8 + 1024;
 }
 
 // C[b] = alpha * sum_t A_t[b] B_t[b]^T + beta * C0[b] + gamma * I for nb blocks of k x k; operands bf16 [nb*k, k]
@@ -564,12 +543,14 @@ struct MatWS {
   int* idx;
 };
 
-static void carve_matrix(Bump& b, const Geo& G, MatWS* w, bool need_E) {
+// lean: the matrix goes through the fused tensor-core pass and nothing but the per-group records leaves it (Eq. 4 /
+// LogSumExp steps without the quantised loss): no matrix-sized scratch at all.
+static void carve_matrix(Bump& b, const Geo& G, MatWS* w, bool need_E, bool lean = false) {
   w->Tb = b.take<uint16_t>((size_t)(G.nbT > 0 ? G.nbT : 1) * (G.k > 0 ? G.k : 1) * (G.k > 0 ? G.k : 1));
-  w->Dbf = b.take<uint16_t>(G.n);
-  w->U = b.take<float>(G.n);
-  w->D = b.take<float>(G.n);
-  w->E = need_E ? b.take<float>(G.n) : nullptr;
+  w->Dbf = lean ? nullptr : b.take<uint16_t>(G.n);
+  w->U = lean ? nullptr : b.take<float>(G.n);
+  w->D = lean ? nullptr : b.take<float>(G.n);
+  w->E = (need_E && !lean) ? b.take<float>(G.n) : nullptr;
   size_t rows_ng = (size_t)G.d_out * G.ng;
   w->a = b.take<float>(rows_ng);
   w->usel = b.take<float>(rows_ng);
@@ -649,6 +630,7 @@ static bool forward_quant(cudaStream_t st, const void* W, const Geo& G, int bits
     p.delta = w.Dbf; p.codes = codes; p.scales = scales;
     if (fused_pass(st, W, G.ld, G, Tc, transposed, w.Tb, p, status, Tb_ready)) return true;
   }
+  if (!w.U) return false;  // lean workspace: there is no scratch for the shape-agnostic kernels (callers check first)
   bool applied = false;
   if (Tc && allow_fused) {  // (allow_fused is off when the caller asked for the shape-agnostic kernels)
     const uint16_t* Tb = (Tb_ready && !transposed) ? Tb_ready : w.Tb;
@@ -703,6 +685,12 @@ extern "C" int cafeq_set_overlap_mode(int overlapped) {
   return CAFEQ_OK;
 }
 
+extern "C" int cafeq_debug_wait_probe(unsigned long long limit_ns, int32_t* status, int* result, void* stream) {
+  if (!status || !result) return CAFEQ_ERR_INVALID_ARG;
+  CQ_LAUNCH(wait_probe_kernel, 1, 32, 0, (cudaStream_t)stream, (uint64_t)limit_ns, status, result);
+  return cudaGetLastError() == cudaSuccess ? CAFEQ_OK : CAFEQ_ERR_CUDA;
+}
+
 extern "C" int cafeq_debug_timer_begin(int capacity) {
   if (capacity < 0 || g_kt.on) return CAFEQ_ERR_INVALID_ARG;
   g_kt.a.resize(capacity);
@@ -737,30 +725,6 @@ extern "C" int cafeq_debug_timer_read(float* ms, int* kinds, int* count) {
   return rc;
 }
 
-extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
-                                    size_t* bytes) {
-  (void)cfg;
-  if (!bytes) return CAFEQ_ERR_INVALID_ARG;
-  Geo G1, G2;
-  int rc = make_geo(d1, &G1, false);
-  if (rc) return rc;
-  size_t b = matrix_scratch_bytes(G1);
-  if (d2) {
-    rc = make_geo(d2, &G2, false);
-    if (rc) return rc;
-    b += matrix_scratch_bytes(G2);
-    // product-sized buffers: the residual of Eq. 5 and the dense algebra of Algorithm 1
-    size_t d1n = (size_t)d1->d_in, d3n = (size_t)d2->d_out;
-    b += (d1n * d3n * 4 + 256);
-    const int rr = d2->replicas > 0 ? d2->replicas : 1;
-    b += dense_scratch_bytes(d1->d_out, d1->d_in, d2->d_out, rr, d1->tblock > 0 ? d1->tblock : d1->d_out, G1.ng, G2.ng);
-    b += 3 * ((size_t)G2.n * 2 + 256);  // transposed second factor and its gradient split (straight-through pair mode)
-    b += (size_t)G1.n * 2 + 256;        // transposed first factor
-  }
-  *bytes = b;
-  return CAFEQ_OK;
-}
-
 static int check_ws(void* ws, size_t ws_bytes) {
   if (!ws || ((uintptr_t)ws & 255)) return CAFEQ_ERR_WORKSPACE;
   (void)ws_bytes;
@@ -770,19 +734,53 @@ static int check_ws(void* ws, size_t ws_bytes) {
 static int last_launch() { return cudaGetLastError() == cudaSuccess ? CAFEQ_OK : CAFEQ_ERR_CUDA; }
 
 // ------------------------------------------------------------------------------------------------
+// What cafeq_rtn needs from its workspace: nothing when the streaming kernel covers the call (no transform, group 32 /
+// 64 / 128 / 256, aligned rows), the per-group records and the rounded operator when the fused tensor-core pass
+// covers it, matrix-sized fp32 buffers otherwise.  W / codes may be null (a size query): aligned pointers are assumed.
+static size_t rtn_scratch(const Geo& G, bool has_T, const void* W, const int8_t* codes, Bump* carve, MatWS* w, float** Tc) {
+  Bump count(nullptr, 0);
+  Bump& b = carve ? *carve : count;
+  MatWS tmp;
+  MatWS& m = w ? *w : tmp;
+  if (!has_T && (G.g == 32 || G.g == 64 || G.g == 128 || G.g == 256) && !((uintptr_t)W & 15) && !(G.ld % 8) &&
+      !((uintptr_t)codes & 7))
+    return 0;
+  const bool lean = has_T && kk_fast(G.k) &&
+                    bd_supported(G.axis == CAFEQ_AXIS_IN ? BD_IN : BD_OUT, G.d_out, G.d_in, G.ld, G.k, G.g, W);
+  carve_matrix(b, G, &m, false, lean);
+  float* t = has_T ? b.take<float>((size_t)G.nbT * G.k * G.k) : nullptr;
+  if (Tc) *Tc = t;
+  return b.used;
+}
+
+extern "C" int cafeq_rtn_workspace_size(const cafeq_matrix_desc* d, int has_transform, size_t* bytes) {
+  Geo G;
+  int rc = make_geo(d, &G, false);
+  if (rc) return rc;
+  if (!bytes) return CAFEQ_ERR_INVALID_ARG;
+  *bytes = rtn_scratch(G, has_transform != 0 && G.k > 0, nullptr, nullptr, nullptr, nullptr, nullptr);
+  return CAFEQ_OK;
+}
+
 extern "C" int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float* T, int8_t* codes, float* scales,
                          void* ws, size_t ws_bytes, void* stream) {
   Geo G;
   int rc = make_geo(d, &G, false);
   if (rc) return rc;
   if (!W || !codes || !scales) return CAFEQ_ERR_INVALID_ARG;
-  if ((rc = check_ws(ws, ws_bytes))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const bool has_T = (T != nullptr && G.k > 0);
+  if (!has_T) {
+    // no transform: one streaming kernel, no scratch (the workspace may be null)
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (rtn_stream_launch(st, W, G.ld, G.d_out, G.d_in, G.g, qmax_of(d->bits), codes, scales)) return last_launch();
+    g_launches.fetch_sub(1, std::memory_order_relaxed);
+  }
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
   Bump b(ws, ws_bytes);
   MatWS w;
-  carve_matrix(b, G, &w, false);
-  float* Tc = has_T ? b.take<float>((size_t)G.nbT * G.k * G.k) : nullptr;
+  float* Tc = nullptr;
+  rtn_scratch(G, has_T, W, codes, &b, &w, &Tc);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
   if (has_T) CQ_LAUNCH(round_bf16_kernel, grid_for((long long)G.nbT * G.k * G.k), 256, 0, st, T, Tc, (long long)G.nbT * G.k * G.k, nullptr);
   forward_quant(st, W, G, d->bits, Tc, d->trole == CAFEQ_APPLY_TT, w, nullptr, CAFEQ_OFFSETS_NONE, false, nullptr, codes,
@@ -803,10 +801,14 @@ struct SingleWS {
   // tensor-core straight-through path: second bf16 term of the residual, both terms transposed, N = Minv^T Minv
   uint16_t *Dlo, *DTh, *DTl;
   float* Nf;
+  bool lean;  // carved without matrix-sized scratch: only the fused surrogate path may run
+  int err;    // host-side error found while enqueuing a step
 };
 
-static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
-  carve_matrix(b, G, &s->m, need_E);
+static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E, bool lean = false) {
+  s->lean = lean;
+  s->err = CAFEQ_OK;
+  carve_matrix(b, G, &s->m, need_E, lean);
   size_t kk = (size_t)G.nbT * G.k * G.k;
   s->Mc = b.take<float>(kk);
   s->Minv = b.take<float>(kk);
@@ -816,13 +818,20 @@ static bool carve_single(Bump& b, const Geo& G, SingleWS* s, bool need_E) {
   s->A = b.take<float>((size_t)G.nbT * G.k);
   s->acc = b.take<double>(8);
   carve_kk(b, G.nbT, G.k, &s->kk);
-  s->Dlo = b.take<uint16_t>(G.n);
-  s->DTh = b.take<uint16_t>(G.n);
-  s->DTl = b.take<uint16_t>(G.n);
+  s->Dlo = lean ? nullptr : b.take<uint16_t>(G.n);
+  s->DTh = lean ? nullptr : b.take<uint16_t>(G.n);
+  s->DTl = lean ? nullptr : b.take<uint16_t>(G.n);
   s->Nf = b.take<float>(kk);
   return !b.overflow;
 }
 
+// Lean workspaces: a step of Eq. 4 / LogSumExp without the quantised loss on shapes the fused pass covers leaves
+// nothing matrix-sized in scratch.  (W itself is not known to the size query: 16-byte aligned rows are assumed; a
+// call whose weights turn out not to qualify returns CAFEQ_ERR_WORKSPACE.)
+static bool lean_single_ok(const Geo& G, const cafeq_opt_cfg* cfg, const void* W) {
+  if (!cfg || cfg->loss_kind != CAFEQ_LOSS_SURROGATE || cfg->eval_every != 0) return false;
+  return kk_fast(G.k) && bd_supported(G.axis == CAFEQ_AXIS_IN ? BD_IN : BD_OUT, G.d_out, G.d_in, G.ld, G.k, G.g, W);
+}
 // Enqueue one forward(+backward) for a single matrix; gradM may be null.  hist is an optional [2] slot.
 static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& G, const void* W, const float* M,
                         float* Minv_out, const void* offsets, int off_kind, int loss_kind, float kappa, bool want_exact,
@@ -882,6 +891,11 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
   if (ste_tc) {
     sp.delta_lo = s.Dlo;
     sp.a_always = 1;
+  }
+  if (s.lean && (ste || need_l2 || !tc || force_generic || off_kind != CAFEQ_OFFSETS_NONE ||
+                 !bd_supported(G.axis == CAFEQ_AXIS_IN ? BD_IN : BD_OUT, G.d_out, G.d_in, G.ld, k, G.g, W))) {
+    s.err = CAFEQ_ERR_WORKSPACE;  // this mode needs the matrix-sized scratch the workspace was sized without
+    return;
   }
   const bool fused = forward_quant(st, W, G, d->bits, s.Mc, 0, s.m, offsets, off_kind, need_l2, nullptr, nullptr, nullptr,
                                    status, (!ste || ste_tc) && !force_generic, &sp, tc ? s.kk.Ab : nullptr);
@@ -1047,7 +1061,7 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
   cudaStream_t st = (cudaStream_t)stream;
   Bump b(ws, ws_bytes);
   SingleWS s;
-  if (!carve_single(b, G, &s, true)) return CAFEQ_ERR_WORKSPACE;
+  if (!carve_single(b, G, &s, true, lean_single_ok(G, cfg, W))) return CAFEQ_ERR_WORKSPACE;
   const long long kk = (long long)G.nbT * G.k * G.k;
   float* grad = b.take<float>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
@@ -1058,6 +1072,7 @@ extern "C" int cafeq_optimize_single(const cafeq_matrix_desc* d, const void* W, 
     bool eval = cfg->eval_every > 0 && (it % cfg->eval_every == 0);
     single_step(st, d, G, W, M, nullptr, nullptr, CAFEQ_OFFSETS_NONE, cfg->loss_kind, kappa, eval, nullptr,
                 loss_history + 2 * (size_t)it, grad, status, s, false, resume || it > 0, opt_state);
+    if (s.err) return s.err;
     if (cfg->optimizer == CAFEQ_OPT_GD) {
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
@@ -1115,6 +1130,8 @@ struct PairWS {
   bool dense;  // the product term runs on the tensor cores (every dimension a multiple of 64)
   uint16_t *W2T, *gVTh, *gVTl;  // [r h, d3]: transposed second factor and transposed split of its gradient
   uint16_t* W1T;                // [d1, h]: transposed first factor (its apply contracts down the rows)
+  bool lean;                    // carved without matrix-sized scratch: only the fused LogSumExp path may run
+  int err;
 };
 
 // Operator gradient of a block-diagonal apply as batched k x k tensor-core products with a two-term split of the
@@ -1149,9 +1166,11 @@ static bool dense_ok(const Geo& G1, const Geo& G2) {
   return G1.d_out % 64 == 0 && G1.d_in % 64 == 0 && G2.d_out % 64 == 0 && G2.d_in % 64 == 0 && G1.k % 32 == 0;
 }
 
-static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool need_R) {
-  carve_matrix(b, G1, &p->m1, true);
-  carve_matrix(b, G2, &p->m2, true);
+static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool need_R, bool lean = false) {
+  p->lean = lean;
+  p->err = CAFEQ_OK;
+  carve_matrix(b, G1, &p->m1, true, lean);
+  carve_matrix(b, G2, &p->m2, true, lean);
   size_t kk = (size_t)G1.nbT * G1.k * G1.k;
   p->Mc = b.take<float>(kk);
   p->Minv = b.take<float>(kk);
@@ -1175,6 +1194,12 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
   return !b.overflow;
 }
 
+static bool lean_pair_ok(const Geo& G1, const Geo& G2, const cafeq_opt_cfg* cfg, const void* W1, const void* W2) {
+  if (!cfg || cfg->loss_kind != CAFEQ_LOSS_LSE || cfg->eval_every != 0) return false;
+  return kk_fast(G1.k) && bd_supported(BD_OUT, G1.d_out, G1.d_in, G1.ld, G1.k, G1.g, W1) &&
+         bd_supported(BD_IN, G2.d_out, G2.d_in, G2.ld, G2.k, G2.g, W2);
+}
+
 static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
                       const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
                       float* losses, float* hist, float* gradM, int32_t* status, PairWS& p, bool force_generic,
@@ -1183,6 +1208,11 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G1.nbT * k * k;
   const float sqrt_h = sqrtf((float)G1.d_out);
+  if (p.lean && (ste || want_pqe || !tc || !bd_supported(BD_OUT, G1.d_out, G1.d_in, G1.ld, k, G1.g, W1) ||
+                 !bd_supported(BD_IN, G2.d_out, G2.d_in, G2.ld, k, G2.g, W2))) {
+    p.err = CAFEQ_ERR_WORKSPACE;  // this mode needs the matrix-sized scratch the workspace was sized without
+    return;
+  }
   if (tc) {
     PrepArgs pa;
     memset(&pa, 0, sizeof(pa));
@@ -1333,6 +1363,31 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
 
 }  // namespace cafeq
 
+extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
+                                    size_t* bytes) {
+  if (!bytes) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg && cfg->struct_size != sizeof(cafeq_opt_cfg)) return CAFEQ_ERR_INVALID_ARG;
+  Geo G1, G2;
+  int rc = make_geo(d1, &G1, false);
+  if (rc) return rc;
+  // the sizes come from the carving code itself, run on a counting allocator
+  Bump b(nullptr, 0);
+  const size_t kk = (size_t)(G1.nbT > 0 ? G1.nbT : 1) * (G1.k > 0 ? G1.k : 1) * (G1.k > 0 ? G1.k : 1);
+  if (!d2) {
+    SingleWS s;
+    carve_single(b, G1, &s, true, G1.k > 0 && lean_single_ok(G1, cfg, nullptr));
+    b.take<float>(kk);  // gradient of the optimise loop / rounded operator of cafeq_rtn
+  } else {
+    if ((rc = make_geo(d2, &G2, false))) return rc;
+    PairWS p;
+    const bool lean = G1.k > 0 && G2.k > 0 && lean_pair_ok(G1, G2, cfg, nullptr, nullptr);
+    carve_pair(b, G1, G2, &p, !lean, lean);
+    b.take<float>(kk);
+  }
+  *bytes = b.used + 256;
+  return CAFEQ_OK;
+}
+
 extern "C" int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
                                   const void* W2, float* P, void* ws, size_t ws_bytes, void* stream) {
   Geo G1, G2;
@@ -1397,7 +1452,7 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   const bool any_pqe = ste || ((P != nullptr) && cfg->eval_every > 0);
   Bump b(ws, ws_bytes);
   PairWS p;
-  if (!carve_pair(b, G1, G2, &p, any_pqe)) return CAFEQ_ERR_WORKSPACE;
+  if (!carve_pair(b, G1, G2, &p, any_pqe, !any_pqe && lean_pair_ok(G1, G2, cfg, W1, W2))) return CAFEQ_ERR_WORKSPACE;
   const long long kk = (long long)G1.nbT * G1.k * G1.k;
   float* grad = b.take<float>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
@@ -1408,6 +1463,7 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
     bool eval = ste || (any_pqe && (it % cfg->eval_every == 0));
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
               grad, status, p, false, resume || it > 0, opt_state, ste);
+    if (p.err) return p.err;
     if (cfg->optimizer == CAFEQ_OPT_GD) {
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
@@ -1495,7 +1551,9 @@ extern "C" int cafeq_rtn_noalloc(const cafeq_matrix_desc* d, const void* W, cons
   Geo Gq;
   int rc = make_geo(d, &Gq, false);
   if (rc) return rc;
-  const size_t need = matrix_scratch_bytes(Gq, false);  // quantisation only: none of the backward scratch
+  if (!W || !codes || !scales) return CAFEQ_ERR_INVALID_ARG;
+  // what cafeq_rtn would carve for this very call (cafeq_rtn_workspace_size gives the same figure for aligned buffers)
+  const size_t need = rtn_scratch(Gq, T != nullptr && Gq.k > 0, W, codes, nullptr, nullptr, nullptr);
   if (need > (size_t)CAFEQ_NOALLOC_SCRATCH_BYTES) return CAFEQ_ERR_TOO_LARGE;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return CAFEQ_ERR_CUDA;

@@ -106,20 +106,41 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait: false when the limit ran out here or in another role (abort flag).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          uint64_t limit_ns = BD_WAIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 63u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > BD_WAIT_NS) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         raise_status(status, CAFEQ_ERR_TIMEOUT);
         return false;
       }
       __nanosleep(32);
     }
+  }
+}
+
+// Self-test of the bounded wait: one thread waits, with the given limit, on a barrier phase that nobody completes
+// (expected: the wait gives up, raises CAFEQ_ERR_TIMEOUT and sets the abort flag), then completes that phase itself
+// and waits again (expected: success).  result[0] = 1 when the first wait gave up, result[1] = 1 when the second
+// succeeded.  Nothing here can block: both waits are bounded and the only arrival is the thread's own.
+__global__ void wait_probe_kernel(uint64_t limit_ns, int32_t* status, int* result) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool first = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, limit_ns);
+    result[0] = first ? 0 : 1;
+    abort_flag = 0;
+    mbar_arrive(smem_u32(&bar));
+    const bool second = mbar_wait(smem_u32(&bar), 0, &abort_flag, nullptr, 1000000000ull);
+    result[1] = second ? 1 : 0;
   }
 }
 

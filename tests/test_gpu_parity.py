@@ -282,7 +282,9 @@ def test_pair_lse_pqe_fwd_bwd(cq, k, r, g1, g2, dims):
 def test_optimize_pair_first_adam_step(cq):
     k, r, h, d1, d3 = 32, 2, 64, 96, 80
     W1b, W2b = syn.weight_student_t(h, d1, 61), syn.weight_student_t(d3, r * h, 62)
-    M0 = syn.haar_blocks(h // k, k, 7)
+    # (a point off the rotations: exactly at M M^T = I the penalty's norm has no gradient and the device, which forms
+    # M M^T in fp32, takes zero below a relative 1e-5)
+    M0 = syn.perturbed_blocks(h // k, k, 7, 0.05)
     W1, W2 = w64(W1b), w64(W2b)
     f = orc.pair_forward(W1, W2, M0, 4, 0, 32, r, 5.0, 0.1, False)
     g = orc.pair_grad_lse(W1, W2, f, 0, 32)
