@@ -156,11 +156,19 @@ int cafeq_rtn_noalloc(const cafeq_matrix_desc* d, const void* W, const float* T,
  *   losses  out fp32[4]: {surrogate (Eq. 4), ||M^-1 Q(MW) - W||_F^2 (Eq. 3), ||W||_F^2, 0};
  *           entries 1,2 only with CAFEQ_FLAG_EXACT_LOSS or loss_kind = CAFEQ_LOSS_L2_STE.
  *   gradM   out [nb,k,k] fp32 gradient of the chosen loss (ignored with CAFEQ_FLAG_NO_GRAD).
+ *   grad_offsets optional out fp32 [d_out,d_in] (row stride d_in): d loss / d offset for soft offsets, only with
+ *           offsets_kind = CAFEQ_OFFSETS_SOFT_F32 and loss_kind = CAFEQ_LOSS_L2_STE (else CAFEQ_ERR_INVALID_ARG).
+ *           With the scales kept at their round-to-nearest values Uhat = s (floor(u/s) + offset), so the gradient is
+ *           s * dL/dUhat = s * 2 M^-T (M^-1 (Uhat - U)).  The paper has no learned offsets (its adaptive rounding
+ *           is Algorithm 1); a caller learns them by a projected step offset <- clip(offset - lr * grad, 0, 1) and
+ *           hardens them at 1/2.
+ * With offsets (either kind) an entry that attains its group's absmax is always coded +-qmax (its quotient is
+ * exactly +-qmax, where floor is discontinuous) and its offset has no effect and no gradient.
  * The operator is M on d->taxis (trole is ignored: the parameter itself is applied). */
 int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* W, const float* M, float* Minv,
                              const void* offsets, int offsets_kind, int loss_kind, float kappa, int flags,
-                             float* losses, float* gradM, int32_t* status, void* ws, size_t ws_bytes,
-                             void* stream);
+                             float* losses, float* gradM, float* grad_offsets, int32_t* status, void* ws,
+                             size_t ws_bytes, void* stream);
 
 /* `cfg->steps` optimisation steps on a single matrix (Section 4.1: gradient descent on Eq. 4 from the
  * caller's initial M; Adam selectable).  M is updated in place (fp32 master parameters).

@@ -97,7 +97,9 @@ def quant_sym(U, bits: int, group: int, offsets=None, dtype=F32):
 
     a = group absmax of fl32(U); s = a/qmax (fp32 division); code
     q = clamp(rne(fl32(U)/s)) (fp32 division), or with `offsets` (same shape as U,
-    values in [0,1]) q = clamp(floor(fl32(U)/s) + offsets).  An all-zero group has
+    values in [0,1]) q = clamp(floor(fl32(U)/s) + offsets), except that an entry attaining its group's
+    absmax is always coded +-qmax (its exact quotient is +-qmax, a point where floor is discontinuous: the fp32
+    quotient lands one ulp above or below depending on the last bits of the maximum).  An all-zero group has
     s = 0 and codes 0.  Returns dict(a, s, idx, q, Uhat) with Uhat = s*q in float64.
     dtype=float64 replaces the normative fp32 steps by float64 ones (finite-difference checks only).
     """
@@ -116,6 +118,9 @@ def quant_sym(U, bits: int, group: int, offsets=None, dtype=F32):
         q = np.rint(x)
     else:
         q = np.floor(x).astype(np.float64) + np.asarray(offsets, dtype=np.float64)
+        a_e = np.repeat(a, g, axis=1)
+        at_max = (np.abs(U32) >= a_e) & (a_e > 0)
+        q = np.where(at_max, np.sign(U32).astype(np.float64) * qm, q)
     q = np.clip(q, -qm, qm)
     Uhat = s_e.astype(np.float64) * q
     if offsets is None:
@@ -237,6 +242,7 @@ def single_forward(W, M, bits: int, group: int, axis: str = "in", kappa=None, of
     out = dict(Mc=Mc, Minv=Minv, U=U, Delta=Delta, E=E, L2=L2, c=c, surrogate=sur,
                kappa=kappa, normW2=float(np.sum(W * W)))
     out.update(Q)
+    out["offsets"] = offsets
     out["rel_l2"] = float(np.sqrt(L2 / out["normW2"])) if out["normW2"] > 0 else 0.0
     return out
 
@@ -291,6 +297,32 @@ def single_grad_ste(W, fwd, bits: int, group: int, axis: str = "in"):
     gU = _route_to_argmax(dL_ds / qm, U, fwd["idx"], group)
     gM = operator_grad(gU, W, k, axis)
     return gM - MinvT @ gMinv @ MinvT
+
+
+def single_grad_offsets(fwd, group: int, axis: str = "in"):
+    """dL2/d rho for soft rounding offsets rho in [0, 1] (not in the paper: the workload statement's learned rounding
+    offsets).  With code q = floor(U/s) + rho and scales kept at their round-to-nearest values,
+    Uhat = s (floor(U/s) + rho), so dUhat/drho = s and dL2/drho = s * dL2/dUhat = s * (2 Minv^T E)  (Eq. 3's
+    residual E = Minv (Uhat - U)).  The entries attaining their group's absmax are coded +-qmax whatever their offset
+    (quant_sym) and have no gradient."""
+    Minv = fwd["Minv"]
+    MinvT = np.transpose(Minv, (0, 2, 1))
+    gUhat = 2.0 * apply_blocks(fwd["E"], MinvT, axis)
+    g = _groups(gUhat.shape[1], group)
+    s_e = np.repeat(fwd["s"].astype(np.float64), g, axis=1)
+    a_e = np.repeat(fwd["a"], g, axis=1)
+    at_max = np.abs(np.asarray(fwd["U"], dtype=np.float64).astype(F32)) >= a_e
+    return np.where(at_max, 0.0, s_e * gUhat)
+
+
+def project_offsets(rho):
+    """Soft offsets live in [0, 1]: projection after a gradient step."""
+    return np.clip(np.asarray(rho, dtype=np.float64), 0.0, 1.0)
+
+
+def harden_offsets(rho):
+    """Soft -> hard: ceil where rho >= 1/2, floor otherwise."""
+    return (np.asarray(rho, dtype=np.float64) >= 0.5).astype(np.float64)
 
 
 # ---------------------------------------------------------------------------

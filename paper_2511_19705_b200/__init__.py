@@ -216,8 +216,8 @@ def cafeq_rtn_noalloc(W, T, codes, scales, *, bits, group, tblock=0, taxis=AXIS_
 
 
 def cafeq_proxy_loss_fwd_bwd(W, M, *, bits, group, taxis=AXIS_IN, loss_kind=LOSS_SURROGATE, kappa=0.0, flags=0,
-                             offsets=None, want_minv=False, Minv=None):
-    """Returns dict(losses[4], gradM or None, Minv or None, status int tensor)."""
+                             offsets=None, want_minv=False, Minv=None, want_grad_offsets=False):
+    """Returns dict(losses[4], gradM or None, Minv or None, status int tensor, grad_offsets or None)."""
     W = _bits_tensor(W)
     M = _f32(M, "M")
     d_out, d_in = W.shape
@@ -235,13 +235,14 @@ def cafeq_proxy_loss_fwd_bwd(W, M, *, bits, group, taxis=AXIS_IN, loss_kind=LOSS
         okind = OFFSETS_HARD_U8 if offsets.dtype == torch.uint8 else OFFSETS_SOFT_F32
         if not offsets.is_contiguous() or tuple(offsets.shape) != (d_out, d_in):
             raise ValueError("offsets must be contiguous [d_out, d_in]")
+    grad_off = torch.empty((d_out, d_in), dtype=torch.float32, device=W.device) if want_grad_offsets else None
     ws = workspace(workspace_size(d), W.device)
     rc = lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(d), _p(W), _p(M), _p(Minv), _p(offsets), ctypes.c_int(okind),
                                         ctypes.c_int(loss_kind), ctypes.c_float(kappa), ctypes.c_int(flags),
-                                        _p(losses), _p(gradM), _p(status), _p(ws), ctypes.c_size_t(ws.numel()),
-                                        _stream())
+                                        _p(losses), _p(gradM), _p(grad_off), _p(status), _p(ws),
+                                        ctypes.c_size_t(ws.numel()), _stream())
     _check(rc, "cafeq_proxy_loss_fwd_bwd")
-    return dict(losses=losses, gradM=gradM, Minv=Minv, status=status)
+    return dict(losses=losses, gradM=gradM, Minv=Minv, status=status, grad_offsets=grad_off)
 
 
 def cafeq_optimize_single(W, M, cfg: OptCfg, *, bits, group, taxis=AXIS_IN, opt_state=None):

@@ -836,7 +836,7 @@ static bool lean_single_ok(const Geo& G, const cafeq_opt_cfg* cfg, const void* W
 static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& G, const void* W, const float* M,
                         float* Minv_out, const void* offsets, int off_kind, int loss_kind, float kappa, bool want_exact,
                         float* losses, float* hist, float* gradM, int32_t* status, SingleWS& s, bool force_generic,
-                        bool warm = false, float* step_counter = nullptr) {
+                        bool warm = false, float* step_counter = nullptr, float* grad_offsets = nullptr) {
   const int k = G.k;
   const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G.nbT * k * k;
@@ -1003,6 +1003,9 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
     CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, s.gMinv, 0.f, kk);
     launch_opgrad(st, s.m.E, G.d_in, s.m.D, 0, G.d_in, G, s.gMinv, 0, 2.f, status);
     launch_apply(st, s.m.E, 0, G.d_in, G, s.Minv, 1, s.m.D, G.d_in, GEMM_STORE, nullptr, status, 2.f);
+    if (grad_offsets)  // s.m.D holds d L2 / d Uhat = 2 Minv^T E
+      CQ_LAUNCH(grad_offsets_kernel, grid_for(G.n), 256, 0, st, s.m.U, s.m.D, (long long)G.d_in, G.d_out, G.d_in, G.g, s.m.a, qm,
+                grad_offsets, status);
     CQ_LAUNCH(ste_scale_path_kernel, (unsigned)(((long long)G.d_out * G.ng * 32 + 255) / 256), 256, 0, st, 
         s.m.U, s.m.D, G.d_in, G.d_out, G.ng, G.g, s.m.a, s.m.usel, qm, offsets, off_kind, G.d_in, s.m.coef, status);
     launch_scatter(st, W, G, s.m.coef, s.m.idx, gradM, 0, status, 0);
@@ -1020,12 +1023,15 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
 
 extern "C" int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* W, const float* M, float* Minv,
                                         const void* offsets, int offsets_kind, int loss_kind, float kappa, int flags,
-                                        float* losses, float* gradM, int32_t* status, void* ws, size_t ws_bytes,
-                                        void* stream) {
+                                        float* losses, float* gradM, float* grad_offsets, int32_t* status, void* ws,
+                                        size_t ws_bytes, void* stream) {
   Geo G;
   int rc = make_geo(d, &G, true);
   if (rc) return rc;
   if (!W || !M || !losses) return CAFEQ_ERR_INVALID_ARG;
+  // the gradient with respect to soft offsets belongs to the straight-through loss evaluated with soft offsets
+  if (grad_offsets && (offsets_kind != CAFEQ_OFFSETS_SOFT_F32 || loss_kind != CAFEQ_LOSS_L2_STE || (flags & CAFEQ_FLAG_NO_GRAD)))
+    return CAFEQ_ERR_INVALID_ARG;
   if (loss_kind != CAFEQ_LOSS_SURROGATE && loss_kind != CAFEQ_LOSS_L2_STE) return CAFEQ_ERR_INVALID_ARG;
   if (offsets_kind < CAFEQ_OFFSETS_NONE || offsets_kind > CAFEQ_OFFSETS_SOFT_F32) return CAFEQ_ERR_INVALID_ARG;
   if (offsets_kind != CAFEQ_OFFSETS_NONE && !offsets) return CAFEQ_ERR_INVALID_ARG;
@@ -1040,7 +1046,7 @@ extern "C" int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* 
   const bool warm = (flags & CAFEQ_FLAG_WARM_MINV) && Minv;
   if (warm) CQ_LAUNCH(copy_f32_kernel, grid_for((long long)G.nbT * G.k * G.k), 256, 0, st, Minv, s.Minv, (long long)G.nbT * G.k * G.k);
   single_step(st, d, G, W, M, Minv, offsets, offsets_kind, loss_kind, kappa, (flags & CAFEQ_FLAG_EXACT_LOSS) != 0, losses,
-              nullptr, want_grad ? gradM : nullptr, status, s, (flags & CAFEQ_FLAG_GENERIC) != 0, warm);
+              nullptr, want_grad ? gradM : nullptr, status, s, (flags & CAFEQ_FLAG_GENERIC) != 0, warm, nullptr, grad_offsets);
   return last_launch();
 }
 

@@ -330,9 +330,12 @@ __global__ void scales_kernel(const float* __restrict__ a, float* __restrict__ s
 // ------------------------------------------------------------------------------------------------
 // quantise: code, dequantised value, residual Delta = Uhat - U
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ float quantise_one(float u, float s, float qmax, float off, int off_kind) {
+// a: the group's absmax.  With rounding offsets an entry attaining it is always coded +-qmax: its exact quotient is
+// +-qmax, where floor is discontinuous and the fp32 quotient lands an ulp above or below.
+__device__ __forceinline__ float quantise_one(float u, float s, float a, float qmax, float off, int off_kind) {
   float x = (s > 0.f) ? __fdiv_rn(u, s) : 0.f;
   float q = (off_kind == CAFEQ_OFFSETS_NONE) ? rintf(x) : floorf(x) + off;
+  if (off_kind != CAFEQ_OFFSETS_NONE && a > 0.f && fabsf(u) >= a) q = copysignf(qmax, u);
   return fminf(fmaxf(q, -qmax), qmax);
 }
 
@@ -346,11 +349,12 @@ __global__ void quant_kernel(const float* __restrict__ U, long long ld, int rows
   for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
     int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
     float u = U[row * ld + col];
-    float s = __fdiv_rn(a[(long long)row * ng + col / g], qmax);
+    const float av = a[(long long)row * ng + col / g];
+    float s = __fdiv_rn(av, qmax);
     float off = 0.f;
     if (off_kind == CAFEQ_OFFSETS_HARD_U8) off = (float)((const uint8_t*)offsets)[e];
     else if (off_kind == CAFEQ_OFFSETS_SOFT_F32) off = ((const float*)offsets)[e];
-    float q = quantise_one(u, s, qmax, off, off_kind);
+    float q = quantise_one(u, s, av, qmax, off, off_kind);
     float uh = s * q;
     if (Delta) Delta[row * ld + col] = uh - u;
     if (Uhat) Uhat[row * ld + col] = uh;
@@ -459,7 +463,7 @@ __global__ void ste_scale_path_kernel(const float* __restrict__ U, const float* 
     float off = 0.f;
     if (off_kind == CAFEQ_OFFSETS_HARD_U8) off = (float)((const uint8_t*)offsets)[(long long)row * cols + col];
     else if (off_kind == CAFEQ_OFFSETS_SOFT_F32) off = ((const float*)offsets)[(long long)row * cols + col];
-    float q = quantise_one(u, s, qmax, off, off_kind);
+    float q = quantise_one(u, s, av, qmax, off, off_kind);
     float x = (s > 0.f) ? __fdiv_rn(u, s) : 0.f;
     sum = fmaf(gD[row * ld + col], q - x, sum);
   }
@@ -468,6 +472,23 @@ __global__ void ste_scale_path_kernel(const float* __restrict__ U, const float* 
     float u = usel[w];
     float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
     coef[w] = sum * sgn / qmax;
+  }
+}
+
+// d loss / d rho for soft rounding offsets: Uhat = s (floor(U/s) + rho) with the scale kept, so d Uhat / d rho = s and
+// the gradient is s * gUhat; entries attaining their group's absmax are coded +-qmax whatever rho and get 0.
+__global__ void grad_offsets_kernel(const float* __restrict__ U, const float* __restrict__ gUhat, long long ld, int rows, int cols,
+                                    int g, const float* __restrict__ a, float qmax, float* __restrict__ out,
+                                    const int32_t* status) {
+  if (status && *status) return;
+  const int ng = cols / g;
+  const long long n = (long long)rows * cols;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const int row = (int)(e / cols), col = (int)(e - (long long)row * cols);
+    const float av = a[(long long)row * ng + col / g];
+    const float s = __fdiv_rn(av, qmax);
+    const float u = U[row * ld + col];
+    out[e] = (av > 0.f && fabsf(u) >= av) ? 0.f : s * gUhat[row * ld + col];
   }
 }
 

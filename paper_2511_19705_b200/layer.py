@@ -39,7 +39,7 @@ class SingleProblem:
         loss_kind = self.loss_kind if loss_kind is None else loss_kind
         rc = lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(self.desc), _p(self.W), _p(self.M), _p(None), _p(None),
                                             ctypes.c_int(OFFSETS_NONE), ctypes.c_int(loss_kind), ctypes.c_float(0.0),
-                                            ctypes.c_int(flags), _p(self.losses), _p(self.grad), _p(self.status),
+                                            ctypes.c_int(flags), _p(self.losses), _p(self.grad), _p(None), _p(self.status),
                                             _p(ws), ctypes.c_size_t(ws.numel()), _stream())
         _check(rc, "cafeq_proxy_loss_fwd_bwd")
 

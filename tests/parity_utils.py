@@ -66,24 +66,31 @@ def assert_codes_tie_aware(q_gpu, s_gpu, Q, U64, group, window=TIE_WINDOW, max_f
 # ---------------------------------------------------------------------------------------------------------
 # inputs without rounding ties
 # ---------------------------------------------------------------------------------------------------------
-def near_tie_mask(U64, bits, group, window):
-    """Entries of a transformed matrix whose quotient U/s lies within `window` * max(1, |x|) of a rounding boundary,
-    and groups whose two largest magnitudes are within 1e-5 relative of each other (either would let fp32 and
-    float64 arithmetic disagree about an integer decision).  Returns a boolean [d_out, d_in] mask."""
+def near_tie_mask(U64, bits, group, window, boundary="round"):
+    """Entries of a transformed matrix whose quotient U/s lies within `window` * max(1, |x|) of a rounding boundary
+    (half-integers for round-to-nearest; integers for boundary="floor", the floor + offset codes; the entries
+    attaining the group's absmax are exempt there, they are coded +-qmax by rule), and groups whose two largest
+    magnitudes are within 1e-5 relative of each other (either would let fp32 and float64 arithmetic disagree about
+    an integer decision).  Returns a boolean [d_out, d_in] mask."""
     from oracle import cafeq_oracle as orc
     Q = orc.quant_sym(U64, bits, group)
     d_out, d_in = U64.shape
     g = d_in if group == 0 else group
     s_e = np.repeat(Q["s"].astype(np.float64), g, axis=1)
     x = np.where(s_e > 0, U64 / np.where(s_e > 0, s_e, 1.0), 0.0)
-    dist = np.abs(np.abs(x - np.floor(x)) - 0.5)
+    if boundary == "floor":
+        dist = np.abs(x - np.rint(x))
+        a_e = np.repeat(Q["a"].astype(np.float64), g, axis=1)
+        dist = np.where(np.abs(U64.astype(np.float32)) >= a_e, 1.0, dist)
+    else:
+        dist = np.abs(np.abs(x - np.floor(x)) - 0.5)
     bad = dist <= window * np.maximum(1.0, np.abs(x))
     A = np.sort(np.abs(U64).reshape(d_out, d_in // g, g), axis=2)
     close = (A[..., -1] - A[..., -2]) <= 1e-5 * A[..., -1]
     return bad | np.repeat(close, g, axis=1)
 
 
-def tie_free_weight(draw, transform, bits, group, redraw, window=2e-4, max_iter=200):
+def tie_free_weight(draw, transform, bits, group, redraw, window=2e-4, max_iter=200, boundary="round"):
     """A seeded weight (bf16 bit patterns) none of whose transformed entries is a near-tie.
 
     draw(i) -> uint16 [d_out, d_in] bit patterns of the i-th independent draw; transform(W64) -> U64;
@@ -94,7 +101,7 @@ def tie_free_weight(draw, transform, bits, group, redraw, window=2e-4, max_iter=
     half-integer."""
     Wb = draw(0).copy()
     for it in range(1, max_iter + 1):
-        mask = near_tie_mask(transform(w64(Wb)), bits, group, window)
+        mask = near_tie_mask(transform(w64(Wb)), bits, group, window, boundary)
         lines = mask.any(axis=1) if redraw == "rows" else mask.any(axis=0)
         if not lines.any():
             return Wb

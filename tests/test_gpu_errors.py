@@ -50,7 +50,7 @@ def test_too_small_workspace_is_refused_before_any_launch(cq):
     n0 = cq.launch_count()
     rc = cq.lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(d), cq._p(Wd), cq._p(M), cq._p(None), cq._p(None), ctypes.c_int(0),
                                            ctypes.c_int(cq.LOSS_SURROGATE), ctypes.c_float(0.0), ctypes.c_int(0),
-                                           cq._p(losses), cq._p(grad), cq._p(status), cq._p(ws), ctypes.c_size_t(ws.numel()),
+                                           cq._p(losses), cq._p(grad), cq._p(None), cq._p(status), cq._p(ws), ctypes.c_size_t(ws.numel()),
                                            cq._stream())
     torch.cuda.synchronize()
     assert rc == 3                                       # CAFEQ_ERR_WORKSPACE
@@ -60,7 +60,7 @@ def test_too_small_workspace_is_refused_before_any_launch(cq):
     big = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
     rc = cq.lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(d), cq._p(Wd), cq._p(M), cq._p(None), cq._p(None), ctypes.c_int(0),
                                            ctypes.c_int(cq.LOSS_SURROGATE), ctypes.c_float(0.0), ctypes.c_int(0),
-                                           cq._p(losses), cq._p(grad), cq._p(status), ctypes.c_void_p(big.data_ptr() + 8),
+                                           cq._p(losses), cq._p(grad), cq._p(None), cq._p(status), ctypes.c_void_p(big.data_ptr() + 8),
                                            ctypes.c_size_t(need), cq._stream())
     assert rc == 3
 

@@ -578,3 +578,32 @@ def test_optimize_pair_composes_the_pinned_pieces():
     assert abs(hist[1, 0] - f1["loss"]) <= 1e-12
     Mz, hz = orc.optimize_pair(W1, W2, M0, 4, 0, 4, r, 3, 0.0, 5.0, 0.1)
     assert np.array_equal(Mz, M0.astype(np.float32).astype(np.float64)) and np.ptp(hz[:, 0]) == 0.0
+
+
+def test_single_grad_offsets_finite_differences():
+    """dL2/drho against central differences of the forward evaluated with perturbed soft offsets (the loss is an
+    exact quadratic in rho as long as no code is clamped), and the projection / hardening conventions."""
+    rng = np.random.default_rng(3)
+    W = rng.standard_normal((6, 8)) * 0.3
+    M = syn.perturbed_blocks(2, 4, 2, 0.2)
+    for axis, shape_nb in (("in", 2),):
+        rho = rng.uniform(0.2, 0.8, size=W.shape)
+        f = orc.single_forward(W, M, 4, 4, axis, offsets=rho)
+        g = orc.single_grad_offsets(f, 4, axis)
+        fd = np.zeros_like(g)
+        eps = 1e-4
+        for i in range(W.shape[0]):
+            for j in range(W.shape[1]):
+                d = np.zeros_like(rho)
+                d[i, j] = eps
+                fd[i, j] = (orc.single_forward(W, M, 4, 4, axis, offsets=rho + d)["L2"] -
+                            orc.single_forward(W, M, 4, 4, axis, offsets=rho - d)["L2"]) / (2 * eps)
+        assert np.allclose(g, fd, rtol=1e-4, atol=1e-7)     # fp32 scales inside the forward limit the agreement
+    assert np.array_equal(orc.project_offsets([-0.2, 0.3, 1.7]), [0.0, 0.3, 1.0])
+    assert np.array_equal(orc.harden_offsets([0.49, 0.5, 0.51]), [0.0, 1.0, 1.0])
+    # soft offsets equal to the fractional part reproduce U exactly: zero loss
+    f0 = orc.single_forward(W, M, 4, 4, "in")
+    s_e = np.repeat(f0["s"].astype(np.float64), 4, axis=1)
+    x = f0["U"] / s_e
+    fz = orc.single_forward(W, M, 4, 4, "in", offsets=x - np.floor(x))
+    assert fz["L2"] <= 1e-10 * f0["L2"]
