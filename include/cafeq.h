@@ -70,7 +70,7 @@ enum {
   CAFEQ_FLAG_GENERIC = 4,    /* force the shape-agnostic kernels (debugging aid) */
   CAFEQ_FLAG_WARM_MINV = 8   /* Minv holds an approximate inverse (e.g. the previous step's) to refine */
 };
-enum { CAFEQ_ROUND_ALG1 = 0 };
+enum { CAFEQ_ROUND_ALG1 = 0, CAFEQ_ROUND_LEARNED_OFFSETS = 1 };
 enum { CAFEQ_OFFSETS_NONE = 0, CAFEQ_OFFSETS_HARD_U8 = 1, CAFEQ_OFFSETS_SOFT_F32 = 2 };
 
 /* One weight matrix and how it is transformed and quantised. */
@@ -220,7 +220,16 @@ int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, const cafeq
  * equals the printed update when Uhat^T has full column rank) and the first factor's least-squares target is
  * P pinv(fold(Vhat^T)); both reduce to the printed lines for r = 1.
  * Every dimension (h, d1, d3) must be a multiple of 64 and the block size a multiple of 32, else
- * CAFEQ_ERR_UNSUPPORTED. */
+ * CAFEQ_ERR_UNSUPPORTED.
+ *
+ * mode = CAFEQ_ROUND_LEARNED_OFFSETS (the paper has no counterpart; it is this library's definition of the learned
+ * rounding offsets the workload statement names): scales stay at their round-to-nearest values and the codes are
+ * floor(x) + rho with soft offsets rho in [0, 1] started at the fractional parts (zero error).  Each of the `iters`
+ * iterations (1..30) moves the first factor's offsets along d = (dL/dUhat) / (s * H), H = 2 * squared norm of the
+ * other factor's matching row, L = Eq. 5 squared, with an exact line search (L is quadratic in one factor's offsets)
+ * and projects to [0, 1]; does the same for the second factor at the updated first; then pushes both by
+ * lambda_t (2 rho - 1), lambda_t = 0.5 t / iters, towards the nearer of {0, 1}.  At the end rho is hardened at 1/2.  pqe_history: fp32 [iters + 2] = {independent round-to-nearest, the soft iterate entering each
+ * iteration, the hardened result}.  Any shape (the products run on the plain fp32 kernel). */
 int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1, const cafeq_matrix_desc* d2,
                          const void* W2, const float* M, int iters, int mode, int8_t* codes1, float* scales1,
                          int8_t* codes2, float* scales2, float* pqe_history, int32_t* status, void* ws,

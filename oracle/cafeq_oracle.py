@@ -567,6 +567,77 @@ def adaptive_round_stored(U1s, V2s, bits: int, group1: int, group2: int, k: int,
                 pqe=np.array(hist))
 
 
+LEARN_LAMBDA = 0.5  # final weight of the push towards {0, 1}
+
+
+def adaptive_round_learned(U1s, V2s, bits: int, group1: int, group2: int, k: int, r: int, iters: int):
+    """Learned rounding offsets for a coupled product (not in the paper, whose adaptive rounding is Algorithm 1; this
+    is the workload statement's gradient-learned alternative, defined here).
+
+    Scales stay at their round-to-nearest values; codes are floor(x) + rho with soft offsets rho in [0, 1], started
+    at the fractional parts (Uhat = U exactly, zero error).  Iteration t = 1..iters, on L = || Uhat Vhat - U V ||_F^2
+    (Eq. 5 squared): for the first factor, the direction d = (dL/drho) / (per-entry curvature) = gUhat / (s H) with
+    H = 2 ||the second factor's matching (replica-folded) row||^2, an exact line search along it (L is quadratic in one
+    factor's offsets), projection to [0, 1]; the same for the second factor at the updated first; then both are pushed
+    towards the nearer of {0, 1} by lambda_t (2 rho - 1), lambda_t = LEARN_LAMBDA * t / iters, and projected.  At the
+    end the offsets are hardened at 1/2.  Entries attaining their group's absmax have no offset (quant_sym).
+    Returns dict(Uhat, Vhat, q1, q2, s1, s2, rho1, rho2, history): history[0] the product error of independent
+    round-to-nearest, history[t] that of the soft iterate entering iteration t, history[iters + 1] of the hardened result.
+    """
+    U = np.asarray(U1s, dtype=np.float64)
+    V = np.asarray(V2s, dtype=np.float64)
+    P = pair_product(U, V, k, r)
+    Q1, Q2 = quant_sym(U, bits, group1), quant_sym(V, bits, group2)
+    hist = [float(np.linalg.norm(pair_product(Q1["Uhat"], Q2["Uhat"], k, r) - P))]
+
+    def frac(X, Q, group):
+        g = _groups(X.shape[1], group)
+        s_e = np.repeat(Q["s"], g, axis=1)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            x = (X.astype(F32) / s_e).astype(F32)
+        x = np.where(s_e > 0, x, F32(0)).astype(np.float64)
+        a_e = np.repeat(Q["a"], g, axis=1)
+        free = (np.abs(X.astype(F32)) < a_e) & (s_e > 0)
+        return x - np.floor(x), s_e.astype(np.float64), free
+
+    def line_search(R, D):
+        dd = float(np.sum(D * D))
+        return float(np.sum(R * D)) / dd if dd > 0 else 0.0
+
+    rho1, s1, free1 = frac(U, Q1, group1)
+    rho2, s2, free2 = frac(V, Q2, group2)
+    for t in range(1, iters + 1):
+        Uh = quant_sym(U, bits, group1, rho1)["Uhat"]
+        Vh = quant_sym(V, bits, group2, rho2)["Uhat"]
+        R = pair_product(Uh, Vh, k, r) - P
+        hist.append(float(np.linalg.norm(R)))
+        # first factor
+        gUh = fold_rows(2.0 * (R @ Vh).T, k, r)                       # [h, d1]
+        Bf = fold_rows(Vh.T, k, r)                                    # [h, d3]: the rows that meet U's rows
+        H1 = 2.0 * np.sum(Bf * Bf, axis=1)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            dr1 = np.where(free1 & (H1[:, None] > 0), gUh / (s1 * H1[:, None]), 0.0)
+        alpha = line_search(R, pair_product(s1 * dr1, Vh, k, r))
+        rho1 = np.clip(rho1 - alpha * dr1, 0.0, 1.0)
+        # second factor, at the updated first
+        Uh = quant_sym(U, bits, group1, rho1)["Uhat"]
+        R = pair_product(Uh, Vh, k, r) - P
+        gVh = 2.0 * (expand_rows(Uh, k, r) @ R).T                     # [d3, r h]
+        H2 = expand_rows((2.0 * np.sum(Uh * Uh, axis=1))[:, None], k, r)[:, 0]
+        with np.errstate(divide="ignore", invalid="ignore"):
+            dr2 = np.where(free2 & (H2[None, :] > 0), gVh / (s2 * H2[None, :]), 0.0)
+        alpha = line_search(R, pair_product(Uh, s2 * dr2, k, r))
+        rho2 = np.clip(rho2 - alpha * dr2, 0.0, 1.0)
+        lam = LEARN_LAMBDA * t / iters
+        rho1 = np.clip(rho1 + lam * (2.0 * rho1 - 1.0), 0.0, 1.0)
+        rho2 = np.clip(rho2 + lam * (2.0 * rho2 - 1.0), 0.0, 1.0)
+    F1 = quant_sym(U, bits, group1, harden_offsets(rho1))
+    F2 = quant_sym(V, bits, group2, harden_offsets(rho2))
+    hist.append(float(np.linalg.norm(pair_product(F1["Uhat"], F2["Uhat"], k, r) - P)))
+    return dict(Uhat=F1["Uhat"], Vhat=F2["Uhat"], q1=F1["q"].astype(np.int32), q2=F2["q"].astype(np.int32),
+                s1=Q1["s"], s2=Q2["s"], rho1=rho1, rho2=rho2, history=np.array(hist))
+
+
 # ---------------------------------------------------------------------------
 # exhaustive rounding search (tiny shapes only)
 # ---------------------------------------------------------------------------

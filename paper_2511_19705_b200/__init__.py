@@ -21,6 +21,7 @@ OPT_STATE_HEADER = 4   # floats before the moment arrays of an optimiser state (
 OPT_GD, OPT_ADAM = 0, 1
 FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC, FLAG_WARM_MINV = 1, 2, 4, 8
 OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
+ROUND_ALG1, ROUND_LEARNED_OFFSETS = 0, 1
 
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_workspace_size", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
@@ -321,7 +322,7 @@ def cafeq_adaptive_round(W1, W2, M, *, iters, bits, group1, group2, replicas=1, 
     codes2 = torch.empty(tuple(W2.shape), dtype=torch.int8, device=dev)
     scales1 = torch.empty((W1.shape[0], W1.shape[1] // g1), dtype=torch.float32, device=dev)
     scales2 = torch.empty((W2.shape[0], W2.shape[1] // g2), dtype=torch.float32, device=dev)
-    hist = torch.zeros(2 * iters + 1, dtype=torch.float32, device=dev)
+    hist = torch.zeros((iters + 2) if mode == ROUND_LEARNED_OFFSETS else (2 * iters + 1), dtype=torch.float32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     ws = workspace(workspace_size(d1, d2), dev)
     rc = lib().cafeq_adaptive_round(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(_f32(M, "M")),

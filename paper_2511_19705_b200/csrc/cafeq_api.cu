@@ -1369,6 +1369,8 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
 
 }  // namespace cafeq
 
+#include "adaptive_offsets.cuh"
+
 extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const cafeq_opt_cfg* cfg,
                                     size_t* bytes) {
   if (!bytes) return CAFEQ_ERR_INVALID_ARG;
@@ -1389,6 +1391,13 @@ extern "C" int cafeq_workspace_size(const cafeq_matrix_desc* d1, const cafeq_mat
     const bool lean = G1.k > 0 && G2.k > 0 && lean_pair_ok(G1, G2, cfg, nullptr, nullptr);
     carve_pair(b, G1, G2, &p, !lean, lean);
     b.take<float>(kk);
+    if (!cfg) {  // cafeq_adaptive_round's learned-offset mode carves its own set of buffers from the same workspace
+      Bump b2(nullptr, 0);
+      LearnWS lw;
+      carve_learn(b2, G1, G2, &lw);
+      b2.take<float>(kk); b2.take<float>(kk); b2.take<float>(kk);
+      if (b2.used > b.used) b.used = b2.used;
+    }
   }
   *bytes = b.used + 256;
   return CAFEQ_OK;
@@ -1488,10 +1497,34 @@ extern "C" int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1,
   int rc = make_pair_geo(d1, d2, &G1, &G2);
   if (rc) return rc;
   if (!W1 || !W2 || !codes1 || !scales1 || !codes2 || !scales2 || !pqe_history) return CAFEQ_ERR_INVALID_ARG;
-  if (mode != CAFEQ_ROUND_ALG1 || iters < 0 || iters > 15) return CAFEQ_ERR_INVALID_ARG;
-  if (!dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;  // every dimension a multiple of 64, block a multiple of 32
+  if (mode != CAFEQ_ROUND_ALG1 && mode != CAFEQ_ROUND_LEARNED_OFFSETS) return CAFEQ_ERR_INVALID_ARG;
+  if (iters < 0 || iters > (mode == CAFEQ_ROUND_ALG1 ? 15 : 30)) return CAFEQ_ERR_INVALID_ARG;
   if ((rc = check_ws(ws, ws_bytes))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
+  if (mode == CAFEQ_ROUND_LEARNED_OFFSETS) {
+    if (iters < 1) return CAFEQ_ERR_INVALID_ARG;
+    Bump b(ws, ws_bytes);
+    LearnWS w;
+    carve_learn(b, G1, G2, &w);
+    const long long kk = (long long)G1.nbT * G1.k * G1.k;
+    float* Mc = b.take<float>(kk);
+    float* Minv = b.take<float>(kk);
+    float* Minv_c = b.take<float>(kk);
+    if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+    if (M) {
+      CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, M, Mc, kk, status);
+      launch_inverse(st, Mc, Minv, nullptr, G1.nbT, G1.k, status);
+      CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, Minv, Minv_c, kk, status);
+      launch_apply(st, W1, 1, G1.ld, G1, Mc, 1, w.U, G1.d_in, GEMM_STORE, nullptr, status);
+      launch_apply(st, W2, 1, G2.ld, G2, Minv_c, 0, w.V, G2.d_in, GEMM_STORE, nullptr, status);
+    } else {
+      CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G1.n), 256, 0, st, (const uint16_t*)W1, G1.ld, G1.d_out, G1.d_in, w.U);
+      CQ_LAUNCH(bf16_to_f32_kernel, grid_for(G2.n), 256, 0, st, (const uint16_t*)W2, G2.ld, G2.d_out, G2.d_in, w.V);
+    }
+    learned_offsets_run(st, d1->bits, G1, G2, iters, codes1, scales1, codes2, scales2, pqe_history, w, status);
+    return last_launch();
+  }
+  if (!dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;  // every dimension a multiple of 64, block a multiple of 32
   Bump b(ws, ws_bytes);
   DenseWS w;
   if (!carve_dense(b, G1.d_out, G1.d_in, G2.d_out, G2.r, G1.k, G1.ng, G2.ng, &w)) return CAFEQ_ERR_WORKSPACE;

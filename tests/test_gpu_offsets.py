@@ -102,3 +102,67 @@ def test_grad_offsets_argument_rules(cq):
     with pytest.raises(cq.CafeqError):                 # hard offsets have no gradient
         cq.cafeq_proxy_loss_fwd_bwd(Wd, Md, bits=4, group=32, loss_kind=cq.LOSS_L2_STE,
                                     offsets=(rho > 0.5).to(torch.uint8), want_grad_offsets=True)
+
+
+# ------------------------------------------------------------------ learned offsets for a coupled product
+def _pair_inputs(h, d1, d3, r, seed, scale=1.0):
+    W1b = syn.weight_student_t(h, d1, seed, 2, 10.0)
+    W2b = syn.weight_student_t(d3, r * h, seed + 1, 2, 10.0)
+    return W1b, W2b
+
+
+@pytest.mark.parametrize("k,r,h,d1,d3,g1,g2,bits", [(32, 2, 64, 96, 80, 32, 32, 3), (64, 1, 128, 192, 128, 64, 64, 4),
+                                                    (16, 1, 48, 40, 56, 8, 16, 3)])
+def test_learned_offsets_pair_matches_oracle(cq, k, r, h, d1, d3, g1, g2, bits):
+    """cafeq_adaptive_round in its learned-offset mode on the untransformed pair (M = NULL: both sides start from
+    identical U, V) against the oracle's float64 run of the same iteration: the error history of the soft iterates,
+    the hardened codes (equal except where the oracle's final offset sits at 1/2 within 1e-3), and the reported final
+    error, which must be Eq. 5 of the codes the device returned."""
+    W1b, W2b = _pair_inputs(h, d1, d3, r, 40 + k)
+    iters = 10
+    out = cq.cafeq_adaptive_round(to_dev(W1b), to_dev(W2b), None, iters=iters, bits=bits, group1=g1, group2=g2, replicas=r, k=k,
+                                  mode=cq.ROUND_LEARNED_OFFSETS)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    U, V = w64(W1b), w64(W2b)
+    ref = orc.adaptive_round_learned(U, V, bits, g1, g2, k, r, iters)
+    H = out["pqe"].cpu().numpy().astype(np.float64)
+    assert H.shape == (iters + 2,)
+    assert abs(H[0] - ref["history"][0]) <= TOL * ref["history"][0]
+    # the soft iterates: the first is exactly U, V (error at the level of fp32 rounding of the products)
+    assert H[1] <= 1e-4 * H[0]
+    assert np.allclose(H[2:iters + 1], ref["history"][2:iters + 1], rtol=5 * TOL)
+    for name, q_dev, q_ref, rho in (("first", out["codes1"], ref["q1"], ref["rho1"]), ("second", out["codes2"], ref["q2"], ref["rho2"])):
+        qd = q_dev.cpu().numpy().astype(np.int32)
+        diff = qd != q_ref
+        assert np.all(np.abs(rho[diff] - 0.5) <= 1e-3), name       # only undecided offsets may harden the other way
+        assert diff.mean() <= 1e-3, name
+    assert np.array_equal(out["scales1"].cpu().numpy(), ref["s1"]) and np.array_equal(out["scales2"].cpu().numpy(), ref["s2"])
+    # the reported final error is Eq. 5 of the returned codes, evaluated by the oracle
+    Uh = np.repeat(ref["s1"].astype(np.float64), g1, axis=1) * out["codes1"].cpu().numpy()
+    Vh = np.repeat(ref["s2"].astype(np.float64), g2, axis=1) * out["codes2"].cpu().numpy()
+    pqe = np.linalg.norm(orc.pair_product(Uh, Vh, k, r) - orc.pair_product(U, V, k, r))
+    assert abs(H[-1] - pqe) <= TOL * pqe
+    assert H[-1] < H[0]                                            # and it beats independent rounding here
+
+
+def test_learned_offsets_pair_against_enumeration_on_tiny_pairs(cq):
+    """n1 + n2 = 12 weights: the oracle enumerates all 4096 floor/ceil choices; the device's learned offsets never lose
+    to round-to-nearest by more than it can be held to (a caller keeps the better of the two), never beat the
+    enumerated minimum, and reach it in a good share of the cases."""
+    rng = np.random.default_rng(0)
+    hits, n_cases = 0, 10
+    for case in range(n_cases):
+        U = syn.f32_to_bf16_bits((rng.standard_normal((2, 3)) * 0.7).astype(np.float32))
+        V = syn.f32_to_bf16_bits((rng.standard_normal((3, 2)) * 0.7).astype(np.float32))
+        out = cq.cafeq_adaptive_round(to_dev(U), to_dev(V), None, iters=12, bits=3, group1=0, group2=0, replicas=1, k=2,
+                                      mode=cq.ROUND_LEARNED_OFFSETS)
+        torch.cuda.synchronize()
+        assert int(out["status"].item()) == 0
+        H = out["pqe"].cpu().numpy()
+        best, _, _, allv = orc.brute_force_pair(w64(U), w64(V), 3, 0, 0, 2, 1)
+        got = min(float(H[-1]), float(H[0]))
+        assert best <= got * (1 + 1e-5)
+        hits += int(got <= best * (1 + 1e-5))
+    print(f"learned pair offsets reached the enumerated optimum in {hits} of {n_cases} cases")
+    assert hits >= n_cases // 3

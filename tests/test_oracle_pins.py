@@ -607,3 +607,25 @@ def test_single_grad_offsets_finite_differences():
     x = f0["U"] / s_e
     fz = orc.single_forward(W, M, 4, 4, "in", offsets=x - np.floor(x))
     assert fz["L2"] <= 1e-10 * f0["L2"]
+
+
+def test_adaptive_round_learned_pins():
+    """The learned-offset iteration: starts at zero error (offsets = fractional parts reproduce U, V), ends on the
+    grid (hardened offsets are floor/ceil choices: its result is one of the enumerated vectors, so never below the
+    enumerated minimum), its reported errors are Eq. 5 of what it returns, and on a pair where independent rounding
+    leaves room it lowers the error."""
+    rng = np.random.default_rng(0)
+    U, V = rng.standard_normal((2, 3)) * 0.7, rng.standard_normal((3, 2)) * 0.7
+    o = orc.adaptive_round_learned(U, V, 3, 0, 0, 2, 1, 12)
+    best, _, _, allv = orc.brute_force_pair(U, V, 3, 0, 0, 2, 1)
+    P = orc.pair_product(U, V, 2, 1)
+    assert o["history"][1] <= 1e-6 * o["history"][0]
+    assert abs(o["history"][-1] - np.linalg.norm(orc.pair_product(o["Uhat"], o["Vhat"], 2, 1) - P)) <= 1e-12
+    assert best <= o["history"][-1] * (1 + 1e-12)
+    assert np.min(np.abs(allv - o["history"][-1])) <= 1e-9        # the result is one of the enumerated choices
+    Q1, Q2 = orc.quant_sym(U, 3, 0), orc.quant_sym(V, 3, 0)
+    assert abs(o["history"][0] - np.linalg.norm(orc.pair_product(Q1["Uhat"], Q2["Uhat"], 2, 1) - P)) <= 1e-12
+    assert np.all(np.abs(o["q1"] - Q1["q"]) <= 1) and np.all(np.abs(o["q2"] - Q2["q"]) <= 1)   # floor or ceil of the same quotient
+    U, V = rng.standard_normal((32, 48)) * 0.1, rng.standard_normal((40, 64)) * 0.1
+    o = orc.adaptive_round_learned(U, V, 3, 16, 16, 16, 2, 10)
+    assert o["history"][-1] < 0.9 * o["history"][0]
