@@ -189,7 +189,7 @@ def cafeq_rtn(W, T=None, *, bits, group, tblock=0, taxis=AXIS_IN, trole=APPLY_T,
     g = group or d_in
     codes = torch.empty((d_out, d_in), dtype=torch.int8, device=W.device)
     scales = torch.empty((d_out, d_in // g), dtype=torch.float32, device=W.device)
-    ws = workspace(workspace_size(d), W.device)
+    ws = workspace(max(rtn_workspace_size(d, T is not None), 256), W.device)
     rc = lib().cafeq_rtn(ctypes.byref(d), _p(W), _p(_f32(T, "T")), _p(codes), _p(scales), _p(ws),
                          ctypes.c_size_t(ws.numel()), _stream())
     _check(rc, "cafeq_rtn")
@@ -237,7 +237,8 @@ def cafeq_proxy_loss_fwd_bwd(W, M, *, bits, group, taxis=AXIS_IN, loss_kind=LOSS
         if not offsets.is_contiguous() or tuple(offsets.shape) != (d_out, d_in):
             raise ValueError("offsets must be contiguous [d_out, d_in]")
     grad_off = torch.empty((d_out, d_in), dtype=torch.float32, device=W.device) if want_grad_offsets else None
-    ws = workspace(workspace_size(d), W.device)
+    lean = loss_kind == LOSS_SURROGATE and not (flags & (FLAG_EXACT_LOSS | FLAG_GENERIC)) and offsets is None
+    ws = workspace(workspace_size(d, None, make_cfg(loss_kind=LOSS_SURROGATE) if lean else None), W.device)
     rc = lib().cafeq_proxy_loss_fwd_bwd(ctypes.byref(d), _p(W), _p(M), _p(Minv), _p(offsets), ctypes.c_int(okind),
                                         ctypes.c_int(loss_kind), ctypes.c_float(kappa), ctypes.c_int(flags),
                                         _p(losses), _p(gradM), _p(grad_off), _p(status), _p(ws),

@@ -1042,11 +1042,28 @@ extern "C" int cafeq_proxy_loss_fwd_bwd(const cafeq_matrix_desc* d, const void* 
   cudaStream_t st = (cudaStream_t)stream;
   Bump b(ws, ws_bytes);
   SingleWS s;
-  if (!carve_single(b, G, &s, true)) return CAFEQ_ERR_WORKSPACE;
+  // Eq. 4 alone on a shape the tensor-core pass covers leaves nothing matrix-sized in scratch (the lean size of
+  // cafeq_workspace_size with a CAFEQ_LOSS_SURROGATE configuration is enough); everything else takes the full carving
+  bool lean = false;
+  if (loss_kind == CAFEQ_LOSS_SURROGATE && !(flags & (CAFEQ_FLAG_EXACT_LOSS | CAFEQ_FLAG_GENERIC)) &&
+      offsets_kind == CAFEQ_OFFSETS_NONE) {
+    cafeq_opt_cfg c0;
+    memset(&c0, 0, sizeof(c0));
+    c0.loss_kind = CAFEQ_LOSS_SURROGATE;
+    lean = lean_single_ok(G, &c0, W);
+    if (lean) {  // a workspace that holds the full carving keeps using it
+      Bump probe(nullptr, 0);
+      SingleWS tmp;
+      carve_single(probe, G, &tmp, true, false);
+      if (probe.used <= ws_bytes) lean = false;
+    }
+  }
+  if (!carve_single(b, G, &s, true, lean)) return CAFEQ_ERR_WORKSPACE;
   const bool warm = (flags & CAFEQ_FLAG_WARM_MINV) && Minv;
   if (warm) CQ_LAUNCH(copy_f32_kernel, grid_for((long long)G.nbT * G.k * G.k), 256, 0, st, Minv, s.Minv, (long long)G.nbT * G.k * G.k);
   single_step(st, d, G, W, M, Minv, offsets, offsets_kind, loss_kind, kappa, (flags & CAFEQ_FLAG_EXACT_LOSS) != 0, losses,
               nullptr, want_grad ? gradM : nullptr, status, s, (flags & CAFEQ_FLAG_GENERIC) != 0, warm, nullptr, grad_offsets);
+  if (s.err) return s.err;
   return last_launch();
 }
 
