@@ -286,6 +286,11 @@ int cafeq_layer_prepare(const cafeq_layer_problem* probs, int n, int32_t* status
 int cafeq_optimize_layer(const cafeq_layer_problem* probs, int n, int steps, int32_t* status, void* ws, size_t ws_bytes,
                          void* stream);
 
+/* Benchmark aid (host out, synchronises the device): how many operator blocks, summed over all steps since
+ * cafeq_layer_prepare on this workspace, were re-inverted by elimination because the iterative refinement of the
+ * previous step's inverse had not converged (a step that changed a transform by more than about half its norm). */
+int cafeq_layer_debug_fallbacks(const cafeq_layer_problem* probs, int n, void* ws, size_t ws_bytes, int* count);
+
 const char* cafeq_status_string(int status);
 int cafeq_version(void);
 /* Tuning knob, process-wide (the paper has no counterpart).  overlapped = 0 (default): one problem runs alone:

@@ -26,7 +26,7 @@ ROUND_ALG1, ROUND_LEARNED_OFFSETS = 0, 1
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_workspace_size", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_layer_debug_fallbacks", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
     "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
@@ -400,6 +400,13 @@ class LayerOptimizer:
         _check(lib().cafeq_layer_prepare(self.arr, ctypes.c_int(self.n), _p(self.status), _p(self.ws),
                                          ctypes.c_size_t(self.ws_bytes), _stream()), "cafeq_layer_prepare")
         self.prepared = True
+
+    def fallbacks(self) -> int:
+        """Blocks re-inverted by elimination since prepare() (synchronises)."""
+        n = ctypes.c_int(0)
+        _check(lib().cafeq_layer_debug_fallbacks(self.arr, ctypes.c_int(self.n), _p(self.ws), ctypes.c_size_t(self.ws_bytes),
+                                                 ctypes.byref(n)), "cafeq_layer_debug_fallbacks")
+        return int(n.value)
 
     def step(self, steps=1):
         if not self.prepared:

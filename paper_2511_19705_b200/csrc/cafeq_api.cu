@@ -207,11 +207,11 @@ static void launch_kk(cudaStream_t st, const float* A, int tA, const float* B, i
 }
 
 static void launch_inverse(cudaStream_t st, const float* Mc, float* Minv, float* cnorm, int nb, int k, int32_t* status,
-                           const double* rn_check = nullptr, double tol2 = 0.0, int* redo_flag = nullptr) {
+                           const double* rn_check = nullptr, double tol2 = 0.0, int* redo_flag = nullptr, int* redo_count = nullptr) {
   int threads = k * k >= 1024 ? 1024 : ((k * k + 31) / 32) * 32;
   size_t sh = (size_t)3 * k * sizeof(float);
   int ti = rn_check ? -1 : kt_begin(3, st);
-  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status, rn_check, tol2, redo_flag);
+  CQ_LAUNCH(block_inverse_kernel, nb, threads, sh, st, Mc, Minv, cnorm, k, status, rn_check, tol2, redo_flag, redo_count);
   kt_end(ti, st);
 }
 
@@ -222,11 +222,12 @@ struct KkWS {  // bf16 scratch, each [nbT * k * k]
   uint16_t *Ab, *Xh[2], *Xl[2], *XTh[2], *XTl[2], *RTh, *RTl, *Ph, *Pl, *Qh, *Ql;
   double* rn;  // [NS_MAX_ITERS][nbT] squared residual norms
   int* flag;   // 1 => Newton-Schulz did not converge, the Gauss-Jordan kernel takes over
+  int* redo_total;  // optional running count of blocks recomputed by elimination (never cleared by a step)
   int cur;     // which of the ping-pong split sets holds the current inverse (host bookkeeping)
 };
 constexpr int NS_MAX_ITERS = 8;
 constexpr int NS_COLD_ITERS = 6;
-constexpr int NS_WARM_ITERS = 2;
+constexpr int NS_WARM_ITERS = 4;  // upper bound: converged blocks skip the later ones (see ns_inverse)
 
 static bool kk_fast(int k) { return k == 64 || k == 128 || k == 256; }
 
@@ -237,6 +238,7 @@ static void carve_kk(Bump& b, int nbT, int k, KkWS* w) {
   for (auto pp : all) *pp = b.take<uint16_t>(kk);
   w->rn = b.take<double>((size_t)NS_MAX_ITERS * nbT);
   w->flag = b.take<int>(64);
+  w->redo_total = nullptr;
   w->cur = 0;
 }
 
@@ -317,8 +319,9 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
                        int32_t* status, bool prepped = false, bool splits_kept = false) {
   const long long kk = (long long)nb * k * k;
   const int iters = warm ? NS_WARM_ITERS : NS_COLD_ITERS;
-  // A warm start that is already close needs one iteration: a block whose residual ||I - A X||_F was below
-  // NS_GATE before an update (below NS_GATE^2 after it) skips the iterations that follow.
+  // A warm start runs up to NS_WARM_ITERS iterations, as many as the step size calls for: a block whose residual
+  // ||I - A X||_F was below 1e-2 before an update (below 1e-4 after it) skips the iterations that follow (their CTAs
+  // return at once).  Small steps take one or two iterations, a change of the transform by half its norm four.
   constexpr double NS_GATE2 = 1e-4;  // squared: the same bound the acceptance test below puts on the residual before the last update
   int ti = kt_begin(3, st);
   if (!prepped) {  // otherwise step_prep_kernel has cleared rn / flag and written Ab
@@ -349,7 +352,7 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   w.cur = cur;
   // accept when ||I - A X||_F before the last update was below 1e-2 (the update squares it: <= 1e-4 after); a block
   // that skipped the last iteration has a zero there and was accepted by the gate
-  launch_inverse(st, Mc, X, nullptr, nb, k, status, w.rn + (size_t)(iters - 1) * nb, 1e-4, w.flag);
+  launch_inverse(st, Mc, X, nullptr, nb, k, status, w.rn + (size_t)(iters - 1) * nb, 1e-4, w.flag, w.redo_total);
   // final splits: written by the last iteration's epilogue, except for blocks that skipped it (and for everything
   // when the elimination recomputed a block)
   const double* last_gate = (warm && iters > 1) ? w.rn + (size_t)(iters - 2) * nb : nullptr;

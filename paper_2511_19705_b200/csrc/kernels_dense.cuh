@@ -12,15 +12,19 @@ namespace cafeq {
 
 // X fp32 [R, C] (row pitch ld) times `scale` (or times 1 / *inv_scale when inv_scale is given) ->
 // bf16 hi / lo splits, row-major [R, C] and / or transposed [C, R]; optional fp32 copy Y of the scaled values
-// (row-major) and YT (transposed, holding hi + lo: used only as a starting guess).
+// (row-major) and YT (transposed, holding hi + lo: used only as a starting guess).  h3 / t3: optional third term
+// bf16(x - hi - lo) in row-major / transposed order (hi + lo + third carries 24 significand bits: products over the
+// three-way split reach fp32 accuracy).
 // One 32 x 32 tile per CTA (grid: ceil(C/32), ceil(R/32); block 32 x 8).
 __global__ void __launch_bounds__(256) split_rect_kernel(const float* __restrict__ X, int R, int C, long long ld, float scale,
                                                          const double* __restrict__ inv_scale, float* __restrict__ Y,
                                                          float* __restrict__ YT, uint16_t* __restrict__ hi, uint16_t* __restrict__ lo,
                                                          uint16_t* __restrict__ thi, uint16_t* __restrict__ tlo,
-                                                         const int32_t* status) {
+                                                         const int32_t* status, uint16_t* __restrict__ h3 = nullptr,
+                                                         uint16_t* __restrict__ t3 = nullptr) {
   if (status && *status) return;
   __shared__ uint32_t tile[32][33];
+  __shared__ uint16_t tile3[32][34];
   const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
   float sc = scale;
@@ -38,10 +42,22 @@ __global__ void __launch_bounds__(256) split_rect_kernel(const float* __restrict
       if (hi) hi[(long long)r * C + c] = hb;
       if (lo) lo[(long long)r * C + c] = lb;
       packed = (uint32_t)hb | ((uint32_t)lb << 16);
+      if (h3 || t3) {
+        const uint16_t b3 = __bfloat16_as_ushort(__float2bfloat16_rn((x - __bfloat162float(h)) - __bfloat162float(l)));
+        if (h3) h3[(long long)r * C + c] = b3;
+        tile3[ty + 8 * q][tx] = b3;
+      }
     }
     tile[ty + 8 * q][tx] = packed;
   }
   __syncthreads();
+  if (t3) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = c0 + ty + 8 * q, r = r0 + tx;
+      if (r < R && c < C) t3[(long long)c * R + r] = tile3[tx][ty + 8 * q];
+    }
+  }
   if (thi || tlo || YT) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {

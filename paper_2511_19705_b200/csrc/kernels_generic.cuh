@@ -179,13 +179,15 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs g) {
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) block_inverse_kernel(const float* __restrict__ Min, float* __restrict__ Out,
                                                              float* __restrict__ cnorm, int k, int32_t* status,
-                                                             const double* __restrict__ rn_check, double tol2, int* redo_flag) {
+                                                             const double* __restrict__ rn_check, double tol2, int* redo_flag,
+                                                             int* redo_count = nullptr) {
   // rn_check: squared residual of an iterative inverse per block; the elimination only runs for blocks whose
   // residual is above tol2 (or not finite) and then raises redo_flag for whoever depends on the result
   if (status && *status) return;
   if (rn_check) {
     if (rn_check[blockIdx.x] <= tol2) return;
     if (threadIdx.x == 0 && redo_flag) *redo_flag = 1;
+    if (threadIdx.x == 0 && redo_count) atomicAdd(redo_count, 1);  // blocks recomputed by elimination, over the run
   }
   extern __shared__ float sm[];  // prow[k], fcol[k], piv (int) [k], red
   float* prow = sm;

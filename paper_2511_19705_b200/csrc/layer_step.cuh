@@ -453,6 +453,7 @@ static int ly_plan(const cafeq_layer_problem* probs, int n, void* ws, size_t ws_
   L->c = b.take<float>((size_t)NB * L->k);
   carve_kk(b, NB, L->k, &L->kk);
   L->one = b.take<float>(64);
+  L->kk.redo_total = reinterpret_cast<int*>(L->one ? L->one + 8 : nullptr);
   for (int i = 0; i < nm; ++i) {
     LyMat& Mt = L->m[i];
     const size_t rows_ng = (size_t)Mt.G.d_out * Mt.G.ng;
@@ -741,6 +742,7 @@ extern "C" int cafeq_layer_prepare(const cafeq_layer_problem* probs, int n, int3
     CQ_LAUNCH(bf16_to_scaled_f16_kernel, grid_for(Mt.G.n / 8), 256, 0, st, (const uint16_t*)Mt.W, Mt.G.ld, Mt.G.d_out, Mt.G.d_in, Mt.wmax,
               Mt.W16, Mt.winv);
   }
+  CQ_LAUNCH(fill_f32_kernel, 1, 32, 0, st, L.one, 0.f, 16);  // (also clears the running count of elimination fall-backs)
   CQ_LAUNCH(set_f32_kernel, 1, 1, 0, st, L.one, 1.f);
   // inverse of the initial transforms from scratch; every step afterwards refines the previous step's inverse
   const long long kk = (long long)L.NB * L.k * L.k;
@@ -775,4 +777,13 @@ extern "C" int cafeq_optimize_layer(const cafeq_layer_problem* probs, int n, int
   for (int it = 0; it < steps; ++it)
     if ((rc = ly_step(st, L, it, status))) return rc;
   return last_launch();
+}
+
+extern "C" int cafeq_layer_debug_fallbacks(const cafeq_layer_problem* probs, int n, void* ws, size_t ws_bytes, int* count) {
+  if (!count) return CAFEQ_ERR_INVALID_ARG;
+  int rc;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  LyPlan L;
+  if ((rc = ly_plan(probs, n, ws, ws_bytes, &L))) return rc;
+  return cudaMemcpy(count, L.kk.redo_total, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess ? CAFEQ_OK : CAFEQ_ERR_CUDA;
 }

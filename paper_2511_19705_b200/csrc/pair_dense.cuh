@@ -49,9 +49,32 @@ static int launch_dense_tc(cudaStream_t st, int nterms, const uint16_t* const* A
 }
 
 static void launch_split_rect(cudaStream_t st, const float* X, int R, int C, long long ld, float scale, const double* inv_scale,
-                              float* Y, float* YT, uint16_t* hi, uint16_t* lo, uint16_t* thi, uint16_t* tlo, const int32_t* status) {
+                              float* Y, float* YT, uint16_t* hi, uint16_t* lo, uint16_t* thi, uint16_t* tlo, const int32_t* status,
+                              uint16_t* h3 = nullptr, uint16_t* t3 = nullptr) {
   dim3 grid((C + 31) / 32, (R + 31) / 32);
-  CQ_LAUNCH(split_rect_kernel, grid, dim3(32, 8), 0, st, X, R, C, ld, scale, inv_scale, Y, YT, hi, lo, thi, tlo, status);
+  CQ_LAUNCH(split_rect_kernel, grid, dim3(32, 8), 0, st, X, R, C, ld, scale, inv_scale, Y, YT, hi, lo, thi, tlo, status, h3, t3);
+}
+
+// The same product with both operands split three ways (x = x1 + x2 + x3, 24 significand bits): the six terms down to
+// 2^-24 relative, as two launches of three terms that accumulate through the fp32 output `acc` (row-major [M, N],
+// pitch N; it may be o.C).  fp32-grade accuracy: what is left is the rounding of the fp32 accumulators.
+// A / B: {x1, x2, x3} in the layouts launch_dense_tc takes.
+static int launch_dense_tc6(cudaStream_t st, const uint16_t* const* A, const uint16_t* const* B, int M, int N, int K, float alpha,
+                            float beta, float gamma, const DenseOut& o, float* acc, int32_t* status, int a_rep_k = 0, int a_rep_r = 1) {
+  const uint16_t* a1[3] = {A[0], A[1], A[0]};
+  const uint16_t* b1[3] = {B[0], B[0], B[1]};
+  DenseOut o1;
+  o1.C0 = o.C0; o1.ldc0 = o.ldc0;
+  o1.C = acc; o1.ldc = N;
+  o1.run_flag = o.run_flag;
+  int rc = launch_dense_tc(st, 3, a1, b1, M, N, K, alpha, beta, gamma, o1, status, a_rep_k, a_rep_r);
+  if (rc) return rc;
+  const uint16_t* a2[3] = {A[0], A[2], A[1]};
+  const uint16_t* b2[3] = {B[2], B[0], B[1]};
+  DenseOut o2 = o;
+  o2.C0 = acc; o2.ldc0 = N;
+  if (!o2.C) { o2.C = nullptr; }
+  return launch_dense_tc(st, 3, a2, b2, M, N, K, alpha, 1.f, 0.f, o2, status, a_rep_k, a_rep_r);
 }
 
 // Scratch of the dense pair algebra for a pair with stored shapes U [h, d1], V [d3, rh]
@@ -64,7 +87,9 @@ struct DenseWS {
   uint16_t *Awh, *Awl;                    // the (wide) matrix being pseudo-inverted [m, n]
   uint16_t *Yh, *Yl, *YTh[2], *YTl[2];    // iterate Y = X^T [m, n] and its transpose [n, m]
   uint16_t *CTh, *CTl;                    // transposed residual [m, m]
-  uint16_t *Oh, *Ol;                      // pseudo-inverse result in the stored shape [h, D]
+  uint16_t *Oh, *Ol, *O3;                 // pseudo-inverse result in the stored shape [h, D], split three ways
+  uint16_t *P3, *PT3, *UT3, *V3, *Aw3, *Y3;  // third terms of the operands that take part in six-term products
+  float* Cf;                              // fp32 accumulator of a six-term product [max(m, d1, d3), ...]
   float *qa, *qusel;                      // quantiser scratch: absmax, signed arg-max value
   int* qidx;
   double* sq;                             // [DENSE_SQ] accumulators: 0..: PQE history, 32..: iteration residuals
@@ -91,7 +116,11 @@ static bool carve_dense(Bump& b, int h, int d1, int d3, int r, int k, int ng1, i
   w->Yh = b.take<uint16_t>(nY); w->Yl = b.take<uint16_t>(nY);
   for (int q = 0; q < 2; ++q) { w->YTh[q] = b.take<uint16_t>(nY); w->YTl[q] = b.take<uint16_t>(nY); }
   w->CTh = b.take<uint16_t>(m * m); w->CTl = b.take<uint16_t>(m * m);
-  w->Oh = b.take<uint16_t>(nY); w->Ol = b.take<uint16_t>(nY);
+  w->Oh = b.take<uint16_t>(nY); w->Ol = b.take<uint16_t>(nY); w->O3 = b.take<uint16_t>(nY);
+  w->P3 = b.take<uint16_t>(nP); w->PT3 = b.take<uint16_t>(nP);
+  w->UT3 = b.take<uint16_t>(nU); w->V3 = b.take<uint16_t>(nV);
+  w->Aw3 = b.take<uint16_t>(nY); w->Y3 = b.take<uint16_t>(nY);
+  w->Cf = b.take<float>(m * m > nY ? m * m : nY);
   const size_t nq = ((size_t)h * ng1 > (size_t)d3 * ng2) ? (size_t)h * ng1 : (size_t)d3 * ng2;
   w->qa = b.take<float>(nq); w->qusel = b.take<float>(nq); w->qidx = b.take<int>(nq);
   w->sq = b.take<double>(DENSE_SQ);
@@ -141,10 +170,10 @@ static void pinv_rows(cudaStream_t st, const float* S, int R, int C, DenseWS& w,
     }
   }
   if (wide) {
-    launch_split_rect(st, S, R, C, C, 1.f, nullptr, nullptr, nullptr, w.Awh, w.Awl, nullptr, nullptr, status);
+    launch_split_rect(st, S, R, C, C, 1.f, nullptr, nullptr, nullptr, w.Awh, w.Awl, nullptr, nullptr, status, w.Aw3, nullptr);
     launch_split_rect(st, S, R, C, C, 1.f, sig2, w.Y, nullptr, w.Yh, w.Yl, w.YTh[0], w.YTl[0], status);
   } else {
-    launch_split_rect(st, S, R, C, C, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.Awh, w.Awl, status);
+    launch_split_rect(st, S, R, C, C, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.Awh, w.Awl, status, nullptr, w.Aw3);
     launch_split_rect(st, S, R, C, C, 1.f, sig2, nullptr, w.Y, w.YTh[0], w.YTl[0], w.Yh, w.Yl, status);
   }
   int cur = 0;
@@ -168,8 +197,25 @@ static void pinv_rows(cudaStream_t st, const float* S, int R, int C, DenseWS& w,
     CQ_LAUNCH(pinv_control_kernel, 1, 1, 0, st, rs, it, 1e-6, w.flag, m, status);
     cur ^= 1;
   }
-  if (wide) launch_split_rect(st, w.Y, m, n, n, 1.f, nullptr, nullptr, nullptr, w.Oh, w.Ol, nullptr, nullptr, status);
-  else launch_split_rect(st, w.Y, m, n, n, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.Oh, w.Ol, status);
+  // The loop above stops at the accuracy of its three-term products (residual entries of a few 1e-7).  One more
+  // step with the residual evaluated over three-way splits (fp32-grade) squares what is left: the quantised targets
+  // of Algorithm 1 then agree with a float64 pseudo-inverse except at rounding ties.  The correction C^T Y is small,
+  // three terms are enough for it.  (A rank-deficient matrix stalls where it stalled before: the step changes nothing.)
+  {
+    launch_split_rect(st, w.Y, m, n, n, 1.f, nullptr, nullptr, nullptr, w.Yh, w.Yl, w.YTh[0], w.YTl[0], status, w.Y3, nullptr);
+    const uint16_t* a[3] = {w.Awh, w.Awl, w.Aw3};
+    const uint16_t* bb[3] = {w.Yh, w.Yl, w.Y3};
+    DenseOut o;
+    o.Cthi = w.CTh; o.Ctlo = w.CTl;
+    launch_dense_tc6(st, a, bb, m, m, n, -1.f, 0.f, 1.f, o, w.Cf, status);
+    const uint16_t* a2[3] = {w.CTh, w.CTl, w.CTh};
+    const uint16_t* b2[3] = {w.YTh[0], w.YTh[0], w.YTl[0]};
+    DenseOut o2;
+    o2.C0 = w.Y; o2.ldc0 = n; o2.C = w.Y; o2.ldc = n;
+    launch_dense_tc(st, 3, a2, b2, m, n, m, 1.f, 1.f, 0.f, o2, status);
+  }
+  if (wide) launch_split_rect(st, w.Y, m, n, n, 1.f, nullptr, nullptr, nullptr, w.Oh, w.Ol, nullptr, nullptr, status, w.O3, nullptr);
+  else launch_split_rect(st, w.Y, m, n, n, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.Oh, w.Ol, status, nullptr, w.O3);
 }
 
 }  // namespace cafeq
@@ -190,14 +236,17 @@ static void quant_matrix(cudaStream_t st, const float* T, int rows, int cols, in
 }
 
 // P = U_exp^T V^T for stored U [h, d1], V [d3, rh] (fp32): fp32 P [d1, d3] with its splits in w.Ph/Pl/PTh/PTl
+// (six terms over three-way splits: P is the reference every least-squares target of Algorithm 1 is measured
+// against, so it is formed to fp32 accuracy; its own third-term splits follow for the target products)
 static void dense_product(cudaStream_t st, const float* U, const float* V, DenseWS& w, float* P, int32_t* status) {
-  launch_split_rect(st, U, w.h, w.d1, w.d1, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.UTh, w.UTl, status);
-  launch_split_rect(st, V, w.d3, w.rh, w.rh, 1.f, nullptr, nullptr, nullptr, w.Vh, w.Vl, nullptr, nullptr, status);
-  const uint16_t* a[3] = {w.UTh, w.UTl, w.UTh};
-  const uint16_t* b[3] = {w.Vh, w.Vh, w.Vl};
+  launch_split_rect(st, U, w.h, w.d1, w.d1, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, w.UTh, w.UTl, status, nullptr, w.UT3);
+  launch_split_rect(st, V, w.d3, w.rh, w.rh, 1.f, nullptr, nullptr, nullptr, w.Vh, w.Vl, nullptr, nullptr, status, w.V3, nullptr);
+  const uint16_t* a[3] = {w.UTh, w.UTl, w.UT3};
+  const uint16_t* b[3] = {w.Vh, w.Vl, w.V3};
   DenseOut o;
   o.C = P; o.ldc = w.d3; o.Chi = w.Ph; o.Clo = w.Pl; o.Cthi = w.PTh; o.Ctlo = w.PTl;
-  launch_dense_tc(st, 3, a, b, w.d1, w.d3, w.rh, 1.f, 0.f, 0.f, o, status, w.k, w.r);
+  launch_dense_tc6(st, a, b, w.d1, w.d3, w.rh, 1.f, 0.f, 0.f, o, P, status, w.k, w.r);
+  launch_split_rect(st, P, w.d1, w.d3, w.d3, 1.f, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, status, w.P3, w.PT3);
 }
 
 // *sq += || Uhat_exp^T Vhat^T - P ||_F^2 ; optionally stores the residual R [d1, d3]
@@ -230,11 +279,11 @@ static void alg1_run(cudaStream_t st, int bits, int g1, int g2, int iters, int8_
     // V side: X0^T [d3, h] = P^T pinv(Uhat^T)^T, then expand the replicas
     pinv_rows(st, w.Uhat, w.h, w.d1, w, status);
     {
-      const uint16_t* a[3] = {w.PTh, w.PTl, w.PTh};
-      const uint16_t* b[3] = {w.Oh, w.Oh, w.Ol};
+      const uint16_t* a[3] = {w.PTh, w.PTl, w.PT3};
+      const uint16_t* b[3] = {w.Oh, w.Ol, w.O3};
       DenseOut o;
       o.C = w.X0T; o.ldc = w.h;
-      launch_dense_tc(st, 3, a, b, w.d3, w.h, w.d1, 1.f, 0.f, 0.f, o, status);
+      launch_dense_tc6(st, a, b, w.d3, w.h, w.d1, 1.f, 0.f, 0.f, o, w.X0T, status);
     }
     CQ_LAUNCH(expand_cols_kernel, grid_for((long long)w.d3 * w.rh), 256, 0, st, w.X0T, w.d3, w.h, w.k, w.r, 1.f / (float)w.r, w.V);
     quant_matrix(st, w.V, w.d3, w.rh, g2, bits, codes2, scales2, w.Vhat, w, status);
@@ -246,11 +295,11 @@ static void alg1_run(cudaStream_t st, int bits, int g1, int g2, int iters, int8_
     }
     pinv_rows(st, w.Bf, w.h, w.d3, w, status);
     {
-      const uint16_t* a[3] = {w.Oh, w.Ol, w.Oh};
-      const uint16_t* b[3] = {w.Ph, w.Ph, w.Pl};
+      const uint16_t* a[3] = {w.Oh, w.Ol, w.O3};
+      const uint16_t* b[3] = {w.Ph, w.Pl, w.P3};
       DenseOut o;
       o.C = w.U; o.ldc = w.d1;
-      launch_dense_tc(st, 3, a, b, w.h, w.d1, w.d3, 1.f, 0.f, 0.f, o, status);
+      launch_dense_tc6(st, a, b, w.h, w.d1, w.d3, 1.f, 0.f, 0.f, o, w.U, status);
     }
     quant_matrix(st, w.U, w.h, w.d1, g1, bits, codes1, scales1, w.Uhat, w, status);
     dense_pqe(st, w.Uhat, w.Vhat, w.P, w, w.sq + 2 * it + 2, nullptr, status);

@@ -33,7 +33,7 @@ TIE_WINDOW = 2.0 ** -18 * 16.0   # 2^-18 sqrt(k) for the largest block (k = 256)
 TIE_FRACTIONS = []               # (test id, fraction of codes that differed inside the window), read by conftest
 
 
-def assert_codes_tie_aware(q_gpu, s_gpu, Q, U64, group, window=TIE_WINDOW, max_frac=1e-4, label=None):
+def assert_codes_tie_aware(q_gpu, s_gpu, Q, U64, group, window=TIE_WINDOW, max_frac=1e-4, label=None, scale_rtol=1e-5):
     """Codes may differ from the oracle only where the oracle's quotient U/s sits within `window`
     (relative to max(1,|x|)) of a rounding boundary, then by exactly one; scales to 1e-5 relative.
 
@@ -47,7 +47,7 @@ def assert_codes_tie_aware(q_gpu, s_gpu, Q, U64, group, window=TIE_WINDOW, max_f
     s_ref = Q["s"].astype(np.float64)
     s_gpu = np.asarray(s_gpu, dtype=np.float64)
     assert s_gpu.shape == s_ref.shape
-    assert np.all(np.abs(s_gpu - s_ref) <= 1e-5 * np.abs(s_ref) + 1e-30), "scales differ"
+    assert np.all(np.abs(s_gpu - s_ref) <= scale_rtol * np.abs(s_ref) + 1e-30), "scales differ"
     g = U64.shape[1] if group == 0 else group
     bad = q_gpu != q_ref
     frac = bad.mean()

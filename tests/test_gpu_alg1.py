@@ -2,17 +2,17 @@
 against the CPU oracle.
 
 The oracle takes its pseudo-inverses from a float64 SVD; the device iterates Newton-Schulz on the tensor cores
-with three-term bf16 splits (about 2^-16 per product).  The least-squares targets therefore agree to roughly
-1e-4 relative, which moves a code only where the target sits that close to a rounding boundary.  Checked here:
-independent rounding (iters = 0) bit-exact; after the first update (identical inputs on both sides) codes one
-step apart at most on under 1 % of the entries; the error history within 1-2 % of the oracle's; and the device's
-reported error equal (1e-3) to the error recomputed in float64 from the codes and scales the device returned."""
+with three-term bf16 splits and finishes with one step whose residual is formed over three-way splits (fp32-grade),
+and forms the product W1 W2 and the least-squares targets over three-way splits too.  Checked here: independent
+rounding (iters = 0) bit-exact; each half-step of the first iteration from identical inputs (teacher forcing) with
+codes equal except inside the tie window; the error history at 1e-3; and the device's reported error equal (1e-3)
+to the error recomputed in float64 from the codes and scales the device returned."""
 import numpy as np
 import pytest
 
 import cafeq_synth as syn
 from oracle import cafeq_oracle as orc
-from parity_utils import f32_dev, rel_err, to_dev, w64
+from parity_utils import assert_codes_tie_aware, device_inverse, f32_dev, rel_err, to_dev, w64
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -36,13 +36,35 @@ def _recomputed_pqe(out, U, V, k, r, g1, g2):
     return float(np.linalg.norm(orc.pair_product(Uh, Vh, k, r) - P))
 
 
-# (h, d1, d3, k, r, g1, g2): tall and wide first factors, with and without replicas, and a square second factor
+# (h, d1, d3, k, r, g1, g2): tall and wide first factors, with and without replicas, a square second factor, an
+# inner dimension four times the outer ones (the up / down aspect ratio) and a grouped-query pair like v-o
 ALG1_CASES = [(128, 192, 256, 64, 2, 64, 64), (256, 128, 192, 64, 1, 64, 128), (128, 256, 192, 128, 1, 128, 64),
-              (128, 256, 128, 128, 1, 128, 64)]
+              (128, 256, 128, 128, 1, 128, 64), (512, 128, 128, 128, 1, 128, 128), (128, 256, 256, 64, 2, 64, 64)]
+# The least-squares targets are solutions of systems whose condition number reaches a few hundred here; computed with
+# fp32-grade arithmetic they carry a relative error of about (condition number) x 2^-24 x sqrt(terms), up to ~1e-4.
+# Scales (a target's group maximum / qmax) are held to that; codes to the usual tie window.
+ALG1_SCALE_RTOL = 3e-4
+
+
+def _half_steps_from_device(out, U, V, bits, g1, g2, k, r):
+    """The oracle's two half-steps of Algorithm 1's first iteration, the second one started from the codes the
+    device returned for the second factor (teacher forcing: a rounding algorithm's later steps depend on every
+    earlier code, so each update is compared from identical inputs)."""
+    P = orc.pair_product(U, V, k, r)
+    Q1 = orc.quant_sym(U, bits, g1)
+    T2 = (orc.pinv(orc.expand_rows(Q1["Uhat"], k, r).T) @ P).T                   # [d3, r h]
+    Vh_dev = out["codes2"].cpu().numpy().astype(np.float64) * np.repeat(out["scales2"].cpu().numpy().astype(np.float64), g2, axis=1)
+    T1 = (P @ orc.pinv(orc.fold_rows(Vh_dev.T, k, r))).T                         # [h, d1]
+    e1 = np.linalg.norm(orc.pair_product(Q1["Uhat"], Vh_dev, k, r) - P)
+    return T2, T1, e1
 
 
 @pytest.mark.parametrize("h,d1,d3,k,r,g1,g2", ALG1_CASES)
 def test_alg1_untransformed_pair(cq, h, d1, d3, k, r, g1, g2):
+    """Algorithm 1 on the device against the oracle's (SVD pseudo-inverse, float64).  The device's pseudo-inverse is
+    an iteration finished with one fp32-grade step, and the products that form the least-squares targets run over
+    three-way bf16 splits, so a target differs from the oracle's by a few 1e-6 relative on well-conditioned factors:
+    codes may differ only where the target's quotient lies within the tie window of a rounding boundary, then by one."""
     W1b = syn.weight_student_t(h, d1, 81, 2, 10.0)
     W2b = syn.weight_student_t(d3, r * h, 82, 2, 10.0)
     U, V = w64(W1b), w64(W2b)
@@ -57,38 +79,28 @@ def test_alg1_untransformed_pair(cq, h, d1, d3, k, r, g1, g2):
     assert np.array_equal(out0["scales1"].cpu().numpy(), Q1["s"]) and np.array_equal(out0["scales2"].cpu().numpy(), Q2["s"])
     ref = orc.adaptive_round_stored(U, V, bits, g1, g2, k, r, 2)
     assert abs(float(out0["pqe"][0].item()) - ref["pqe"][0]) <= 1e-3 * ref["pqe"][0]
-    # one full iteration.  The second factor's update starts from bit-identical inputs, so its codes may differ
-    # only where the least-squares target sits within the pseudo-inverse's accuracy of a rounding boundary.  The
-    # first factor's update then starts from those (slightly different) codes, so its comparison is looser; and
-    # when the inner dimension reaches the outer ones (h >= d3) its least-squares problem is rank-deficient or nearly so
-    # and both implementations' quantised results are sensitive to the last digits of the pseudo-inverse.
-    well_posed = h <= 0.75 * min(d1, d3)   # the aspect ratio of the real v-o pair is 0.57
+    # one full iteration, each half-step from identical inputs
     out1 = cq.cafeq_adaptive_round(to_dev(W1b), to_dev(W2b), None, iters=1, bits=bits, group1=g1, group2=g2, replicas=r, k=k)
     torch.cuda.synchronize()
-    ref1 = orc.adaptive_round_stored(U, V, bits, g1, g2, k, r, 1)
+    assert int(out1["status"].item()) == 0
+    T2, T1, e1 = _half_steps_from_device(out1, U, V, bits, g1, g2, k, r)
+    f2 = assert_codes_tie_aware(out1["codes2"].cpu().numpy(), out1["scales2"].cpu().numpy(), orc.quant_sym(T2, bits, g2), T2, g2,
+                                scale_rtol=ALG1_SCALE_RTOL)
+    f1 = assert_codes_tie_aware(out1["codes1"].cpu().numpy(), out1["scales1"].cpu().numpy(), orc.quant_sym(T1, bits, g1), T1, g1,
+                                scale_rtol=ALG1_SCALE_RTOL)
     h1 = out1["pqe"].cpu().numpy().astype(np.float64)
-    assert np.all(np.abs(h1[:2] - ref1["pqe"][:2]) <= 1e-2 * ref1["pqe"][:2]), (h1, ref1["pqe"])
-    assert abs(h1[2] - ref1["pqe"][2]) <= (1e-2 if well_posed else 0.5) * ref1["pqe"][2], (h1, ref1["pqe"])
-    assert abs(h1[-1] - _recomputed_pqe(out1, U, V, k, r, g1, g2)) <= 1e-3 * h1[-1]
-    if well_posed:
-        d2 = np.abs(out1["codes2"].cpu().numpy().astype(np.int64) - ref1["q2"])
-        assert d2.max() <= 1 and (d2 != 0).mean() <= 0.01, (d2.max(), (d2 != 0).mean())
-        assert rel_err(out1["scales2"].cpu().numpy(), ref1["s2"]) <= 1e-3
-        d1c = np.abs(out1["codes1"].cpu().numpy().astype(np.int64) - ref1["q1"])
-        assert (d1c != 0).mean() <= 0.10, (d1c.max(), (d1c != 0).mean())
-    # two full iterations: the trajectories of a rounding algorithm separate once a code differs, the error level
-    # they reach does not
+    assert abs(h1[1] - e1) <= 1e-3 * e1, (h1, e1)
+    assert abs(h1[2] - _recomputed_pqe(out1, U, V, k, r, g1, g2)) <= 1e-3 * h1[2]
+    # against the oracle's free-running history: the second factor's update starts from bit-identical inputs
+    assert abs(h1[1] - ref["pqe"][1]) <= 1e-3 * ref["pqe"][1] + 1e-2 * f2 * ref["pqe"][1], (h1, ref["pqe"], f2, f1)
+    # two full iterations: the reported errors are the errors of what was returned, and the run helps
     out = cq.cafeq_adaptive_round(to_dev(W1b), to_dev(W2b), None, iters=2, bits=bits, group1=g1, group2=g2, replicas=r, k=k)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
     hist = out["pqe"].cpu().numpy().astype(np.float64)
     assert hist.shape == (5,)
-    assert np.all(np.abs(hist[:2] - ref["pqe"][:2]) <= 1e-2 * ref["pqe"][:2]), (hist, ref["pqe"])
-    if well_posed:
-        assert np.all(np.abs(hist - ref["pqe"]) <= 0.15 * ref["pqe"]), (hist, ref["pqe"])
-        assert hist[1:].min() < hist[0]
-    # the reported error is the error of what was returned
     assert abs(hist[-1] - _recomputed_pqe(out, U, V, k, r, g1, g2)) <= 1e-3 * hist[-1]
+    assert hist[1:].min() < hist[0]
 
 
 def test_alg1_after_learned_transform(cq):
@@ -99,11 +111,14 @@ def test_alg1_after_learned_transform(cq):
     out = cq.cafeq_adaptive_round(to_dev(W1b), to_dev(W2b), f32_dev(M), iters=1, bits=bits, group1=g1, group2=g2, replicas=r)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
-    f = orc.pair_forward(w64(W1b), w64(W2b), M, bits, g1, g2, r, 5.0, 0.0, False)
+    # identical transform parameters on both sides: the second factor's operator is bf16 of the inverse as this call
+    # computes it (elimination)
+    Minv_c = orc.round_bf16(device_inverse(cq, M, generic=True))
+    f = orc.pair_forward(w64(W1b), w64(W2b), M, bits, g1, g2, r, 5.0, 0.0, False, Minv_c=Minv_c)
     ref = orc.adaptive_round_stored(f["U"], f["V"], bits, g1, g2, k, r, 1)
     hist = out["pqe"].cpu().numpy().astype(np.float64)
-    assert np.all(np.abs(hist - ref["pqe"]) <= 2e-2 * ref["pqe"]), (hist, ref["pqe"])
-    assert abs(hist[-1] - _recomputed_pqe(out, f["U"], f["V"], k, r, g1, g2)) <= 2e-3 * hist[-1]
+    assert np.all(np.abs(hist - ref["pqe"]) <= 2e-3 * ref["pqe"]), (hist, ref["pqe"])
+    assert abs(hist[-1] - _recomputed_pqe(out, f["U"], f["V"], k, r, g1, g2)) <= 1e-3 * hist[-1]
 
 
 def test_alg1_unsupported_shape_is_refused(cq):
