@@ -35,13 +35,14 @@ UNIT = "steps/s"
 
 
 def profiled_traffic():
-    """DRAM bytes per launch of the transform pass from the committed ncu summary, or None once the kernel source
-    differs from the one that was profiled."""
+    """DRAM bytes per launch (mean over the transform-pass and backward launches of a step) from the committed ncu
+    summaries, or None once a kernel source differs from the one that was profiled."""
     import hashlib
     import re
     try:
-        txt = open(os.path.join(ROOT, "profiles", "bd_pass_9b_layer.md")).read()
-        src = open(os.path.join(ROOT, "paper_2511_19705_b200", "csrc", "kernels_fused.cuh"), "rb").read()
+        txt = open(os.path.join(ROOT, "profiles", "bd_bwd_kernel_9b_layer.md")).read()
+        src = b"".join(open(os.path.join(ROOT, "paper_2511_19705_b200", "csrc", f), "rb").read()
+                       for f in ("kernels_fused.cuh", "kernels_bwd.cuh"))
         sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]+)", txt).group(1)
         if hashlib.sha256(src).hexdigest() != sha:
             return None
@@ -159,15 +160,19 @@ def cpu_threads():
 def measure_extras(cq, torch, devS, devP, bits, group, peaks):
     """Round-to-nearest (with and without a transform) and packing on the largest single matrix against the HBM
     roofline, and one iteration of Algorithm 1 / of the learned-offset rounding on the first pair.  Every timed call is
-    preceded by a write of a buffer larger than L2."""
+    preceded by a pass over a buffer larger than L2 (read, not written: dirty lines of a written flush buffer would be
+    written back during the timed kernel and charged to it)."""
     out = {}
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=devS[0][1].device if devS else devP[0][1].device)
+    flush.fill_(1)
+    flush_sink = torch.zeros((), dtype=torch.int64, device=flush.device)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def timed(fn, reps=5):
         best = None
         for _ in range(reps + 1):
-            flush.fill_(1)
+            for _ in range(3):  # (three passes keep the device busy while the host prepares the timed call)
+                flush_sink.copy_(flush.sum(dtype=torch.int64))
             e0.record()
             r = fn()
             e1.record()
@@ -470,7 +475,8 @@ def main():
         else:
             ach = byts / t_fb / 1e9
             roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
-        roof.update(traffic=profiled_traffic(),
+        roof.update(traffic=profiled_traffic() if (use_layer and args.config == 3) else None,
+                    algorithmic_bytes_per_launch=byts * 2 / n_launch if n_launch else None,
                     kernel="transform pass + sparse backward (bd_pass_kernel + bd_bwd_kernel), the forward+backward of one step",
                     peak_source=peaks["source"] + ((" burst (SM clock stayed at its maximum through the timed region)" if at_max
                                                     else " sustained (SM clock sagged under load)") if bound_is_tensor else ""),
