@@ -368,7 +368,8 @@ def orth_penalty(M):
 
 
 def pair_forward(W1s, W2s, M, bits: int, group1: int, group2: int, r: int = 1,
-                 t: float = 5.0, lam: float = 0.0, want_pqe: bool = True, prec: str = "bf16", Minv_c=None):
+                 t: float = 5.0, lam: float = 0.0, want_pqe: bool = True, prec: str = "bf16", Minv_c=None,
+                 objective: str = "lse"):
     """Forward for a coupled pair.
 
     Stored W1s is [h, d1] (the paper's W1 transposed), stored W2s is [d3, r*h].
@@ -380,6 +381,10 @@ def pair_forward(W1s, W2s, M, bits: int, group1: int, group2: int, r: int = 1,
     which way an entry of an inverse rounds to bf16 depends on its last bits, so two computations of
     bf16(inv(M_c)) can differ in single entries by one bf16 step; a caller that compares integer codes
     passes the operator that was actually applied).  Gradients still differentiate through inv(M_c).
+    objective: "lse" (Section 4.2), or the alternatives of Appendix D.1 over the same group maxima:
+    "sumsq" = mean of the squared maxima of U + mean of the squared maxima of V; "sumsq_weighted" =
+    ||V||_F * mean(squared maxima of U) + ||U||_F * mean(squared maxima of V) (an error in one factor is magnified by
+    the norm of the other).  out["surrogate"] holds the chosen objective's value, out["loss"] adds lam * penalty.
     """
     W1s = np.asarray(W1s, dtype=np.float64)
     W2s = np.asarray(W2s, dtype=np.float64)
@@ -404,8 +409,22 @@ def pair_forward(W1s, W2s, M, bits: int, group1: int, group2: int, r: int = 1,
     wu = np.exp(t * (au - amax)) / Z                             # softmax weights = dLSE/da
     wv = np.exp(t * (av - amax)) / Z
     pen, gpen = orth_penalty(np.asarray(M, dtype=np.float64))
+    if objective == "lse":
+        sur = lse
+    else:
+        su, sv = float(np.mean(au * au)), float(np.mean(av * av))
+        nu, nv = float(np.sqrt(np.sum(U * U))), float(np.sqrt(np.sum(V * V)))
+        if objective == "sumsq":
+            sur, wu, wv = su + sv, 2.0 * au / au.size, 2.0 * av / av.size      # w = d objective / d maximum
+        elif objective == "sumsq_weighted":
+            sur, wu, wv = nv * su + nu * sv, nv * 2.0 * au / au.size, nu * 2.0 * av / av.size
+        else:
+            raise ValueError("objective")
     out = dict(Mc=Mc, Minv=Minv, Minv_c=Minv_c, U=U, V=V, QU=QU, QV=QV, lse=float(lse), wu=wu, wv=wv,
-               orth=pen, gorth=gpen, loss=float(lse + lam * pen), k=k, r=r, lam=lam, t=t)
+               orth=pen, gorth=gpen, loss=float(sur + lam * pen), surrogate=float(sur), objective=objective,
+               k=k, r=r, lam=lam, t=t)
+    if objective == "sumsq_weighted":
+        out.update(su=su, sv=sv, nu=nu, nv=nv)
     if want_pqe:
         P = pair_product(W1s, W2s, k, r)
         R = pair_product(QU["Uhat"], QV["Uhat"], k, r) - P
@@ -425,9 +444,14 @@ def _pair_chain(W1s, W2s, fwd, gU, gV):
 
 
 def pair_grad_lse(W1s, W2s, fwd, group1: int, group2: int):
-    """Gradient of LSE + lam*orth: softmax weights routed to the arg-max entries."""
+    """Gradient of the pair surrogate + lam*orth: d objective / d group maximum (the softmax weights for
+    LogSumExp, 2 a / count [times the other factor's norm] for the sums of squares of Appendix D.1) routed to the
+    arg-max entries; the weighted form adds the dense terms mean(a_U^2) V / ||V||_F and mean(a_V^2) U / ||U||_F."""
     gU = _route_to_argmax(fwd["wu"], fwd["U"], fwd["QU"]["idx"], group1)
     gV = _route_to_argmax(fwd["wv"], fwd["V"], fwd["QV"]["idx"], group2)
+    if fwd.get("objective") == "sumsq_weighted":
+        gU = gU + fwd["sv"] * fwd["U"] / fwd["nu"]
+        gV = gV + fwd["su"] * fwd["V"] / fwd["nv"]
     return _pair_chain(np.asarray(W1s, np.float64), np.asarray(W2s, np.float64), fwd, gU, gV) \
         + fwd["lam"] * fwd["gorth"]
 
@@ -473,6 +497,21 @@ def adam_step(M, g, state, lr: float, beta1: float = 0.1, beta2: float = 0.999, 
     return np.asarray(M, dtype=np.float64) - lr * mh / (np.sqrt(vh) + eps), (m, v, step)
 
 
+def cayley_step(M, g, momentum, lr: float, beta: float = 0.1):
+    """One step of stochastic gradient descent on the rotations by the Cayley transform (Appendix D.2's strictly
+    orthonormal baseline), per block: momentum V <- beta V + g; A = V M^T - M V^T (skew-symmetric: the direction in
+    the tangent space); M <- (I + lr/2 A)^-1 (I - lr/2 A) M, which is a rotation times M, so an orthonormal M stays
+    orthonormal to rounding.  Returns (M_new, V)."""
+    M = np.asarray(M, dtype=np.float64)
+    V = beta * np.asarray(momentum, dtype=np.float64) + np.asarray(g, dtype=np.float64)
+    A = V @ np.transpose(M, (0, 2, 1)) - M @ np.transpose(V, (0, 2, 1))
+    eye = np.eye(M.shape[1])
+    out = np.empty_like(M)
+    for b in range(M.shape[0]):
+        out[b] = np.linalg.solve(eye + 0.5 * lr * A[b], (eye - 0.5 * lr * A[b]) @ M[b])
+    return out, V
+
+
 def optimize_single(W, M0, bits: int, group: int, axis: str, steps: int, lr: float, kappa=None):
     """Gradient descent on the surrogate; returns (M, history[steps, 2] = surrogate, L2)."""
     M = np.asarray(M0, dtype=np.float32).astype(np.float64)
@@ -487,17 +526,23 @@ def optimize_single(W, M0, bits: int, group: int, axis: str, steps: int, lr: flo
 
 def optimize_pair(W1s, W2s, M0, bits: int, group1: int, group2: int, r: int, steps: int, lr: float,
                   t: float = 5.0, lam: float = 0.1, beta1: float = 0.1, beta2: float = 0.999,
-                  eps: float = 1e-8, want_pqe: bool = False):
-    """Adam on LSE + lam*orth; returns (M, history[steps, 2] = loss, PQE or nan)."""
+                  eps: float = 1e-8, want_pqe: bool = False, objective: str = "lse", optimizer: str = "adam"):
+    """Adam (or Cayley SGD with momentum beta1) on the pair surrogate + lam*orth; returns (M, history[steps, 2] =
+    loss, PQE or nan)."""
     M = np.asarray(M0, dtype=np.float32).astype(np.float64)
     st = (np.zeros_like(M), np.zeros_like(M), 0)
+    mom = np.zeros_like(M)
     hist = np.full((steps, 2), np.nan)
     for it in range(steps):
-        f = pair_forward(W1s, W2s, M, bits, group1, group2, r, t, lam, want_pqe)
+        f = pair_forward(W1s, W2s, M, bits, group1, group2, r, t, lam, want_pqe, objective=objective)
         hist[it, 0] = f["loss"]
         if want_pqe:
             hist[it, 1] = f["pqe"]
-        M, st = adam_step(M, pair_grad_lse(W1s, W2s, f, group1, group2), st, lr, beta1, beta2, eps)
+        g = pair_grad_lse(W1s, W2s, f, group1, group2)
+        if optimizer == "cayley":
+            M, mom = cayley_step(M, g, mom, lr, beta1)
+        else:
+            M, st = adam_step(M, g, st, lr, beta1, beta2, eps)
         M = M.astype(np.float32).astype(np.float64)
     return M, hist
 

@@ -629,3 +629,49 @@ def test_adaptive_round_learned_pins():
     U, V = rng.standard_normal((32, 48)) * 0.1, rng.standard_normal((40, 64)) * 0.1
     o = orc.adaptive_round_learned(U, V, 3, 16, 16, 16, 2, 10)
     assert o["history"][-1] < 0.9 * o["history"][0]
+
+
+@pytest.mark.parametrize("objective", ["sumsq", "sumsq_weighted"])
+def test_pair_sum_of_squares_objectives(objective):
+    """Appendix D.1's alternatives to LogSumExp: the value from its definition written out with plain loops over the
+    group maxima, and the gradient against central finite differences (no rounding of the operators, jittered inputs:
+    no arg-max ties)."""
+    rng = np.random.default_rng(11)
+    k, r, h, d1, d3 = 4, 2, 8, 6, 5
+    W1, W2 = rng.standard_normal((h, d1)), rng.standard_normal((d3, r * h))
+    M = syn.perturbed_blocks(h // k, k, 5, 0.2).astype(np.float64)
+
+    def value(Mx):
+        return orc.pair_forward(W1, W2, Mx, 4, 3, 4, r, 5.0, 0.0, False, prec="exact", objective=objective)
+
+    f = value(M)
+    U, V = f["U"], f["V"]
+    mu = [max(abs(U[i, 3 * G:3 * G + 3])) for i in range(h) for G in range(d1 // 3)]
+    mv = [max(abs(V[j, 4 * G:4 * G + 4])) for j in range(d3) for G in range(r * h // 4)]
+    su, sv = sum(x * x for x in mu) / len(mu), sum(x * x for x in mv) / len(mv)
+    want = su + sv if objective == "sumsq" else np.linalg.norm(V) * su + np.linalg.norm(U) * sv
+    assert f["surrogate"] == pytest.approx(want, rel=1e-12)
+    g = orc.pair_grad_lse(W1, W2, f, 3, 4)
+    fd = _fd(lambda Mx: value(Mx)["surrogate"], M)
+    assert np.allclose(g, fd, rtol=2e-5, atol=1e-8)
+
+
+def test_cayley_step_pins():
+    """The Cayley update keeps rotations rotations, moves along minus the skew part of the gradient to first order,
+    and carries momentum."""
+    rng = np.random.default_rng(2)
+    M = np.stack([np.linalg.qr(rng.standard_normal((6, 6)))[0] for _ in range(2)])   # rotations to float64 accuracy
+    g = rng.standard_normal(M.shape)
+    M1, V = orc.cayley_step(M, g, np.zeros_like(M), 1e-2, 0.1)
+    I = np.eye(6)
+    assert np.allclose(M1 @ np.transpose(M1, (0, 2, 1)), I, atol=1e-12)
+    assert np.array_equal(V, g)
+    A = g @ np.transpose(M, (0, 2, 1)) - M @ np.transpose(g, (0, 2, 1))
+    M_small, _ = orc.cayley_step(M, g, np.zeros_like(M), 1e-6, 0.1)
+    assert np.allclose((M_small - M) / 1e-6, -A @ M, atol=1e-4)
+    _, V2 = orc.cayley_step(M1, g, V, 1e-2, 0.1)
+    assert np.allclose(V2, 1.1 * g)
+    # descent: a linear loss <C, M> decreases along the step
+    C = rng.standard_normal(M.shape)
+    M2, _ = orc.cayley_step(M, C, np.zeros_like(M), 1e-2, 0.0)
+    assert np.sum(C * M2) < np.sum(C * M)
