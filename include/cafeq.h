@@ -59,9 +59,15 @@ enum {
   CAFEQ_LOSS_SURROGATE = 0, /* single: Eq. 4 */
   CAFEQ_LOSS_L2_STE = 1,    /* single: Eq. 3 with a straight-through rounding derivative */
   CAFEQ_LOSS_LSE = 2,       /* pair: LogSumExp of group maxima (+ orthonormality penalty) */
-  CAFEQ_LOSS_PQE_STE = 3    /* pair: Eq. 5 squared, straight-through */
+  CAFEQ_LOSS_PQE_STE = 3,   /* pair: Eq. 5 squared, straight-through */
+  CAFEQ_LOSS_SUMSQ = 4,     /* pair, Appendix D.1: mean of the squared group maxima of U + the same of V */
+  CAFEQ_LOSS_SUMSQ_WEIGHTED = 5 /* pair, Appendix D.1: ||V||_F mean(sq. maxima of U) + ||U||_F mean(sq. maxima of V) */
 };
-enum { CAFEQ_OPT_GD = 0, CAFEQ_OPT_ADAM = 1 };
+/* CAFEQ_OPT_CAYLEY (pairs only, Appendix D.2's strictly orthonormal baseline): momentum V <- beta1 V + grad,
+ * A = V M^T - M V^T, M <- (I + lr/2 A)^-1 (I - lr/2 A) M per block (solved by five fixed-point rounds: choose lr so
+ * that lr ||A|| stays well below 1); a rotation stays a rotation.  The momentum lives in the optimiser state's
+ * first-moment slot. */
+enum { CAFEQ_OPT_GD = 0, CAFEQ_OPT_ADAM = 1, CAFEQ_OPT_CAYLEY = 2 };
 #define CAFEQ_OPT_STATE_HEADER 4 /* floats before the moment arrays of an optimiser state */
 /* flags for the forward/backward calls */
 enum {
@@ -195,7 +201,9 @@ int cafeq_pair_product(const cafeq_matrix_desc* d1, const void* W1, const cafeq_
  *   P       optional fp32 [d1, d3] from cafeq_pair_product; needed for PQE.
  *   losses  out fp32[4]: {LSE + lambda*orth, LSE, orth penalty, PQE^2 (Eq. 5 squared) or 0}.
  *   gradM   out [h/k, k, k].
- * loss_kind CAFEQ_LOSS_LSE is the surrogate of App. D.  CAFEQ_LOSS_PQE_STE differentiates Eq. 5 squared itself with
+ * loss_kind CAFEQ_LOSS_LSE is the surrogate of Section 4.2 / App. D; CAFEQ_LOSS_SUMSQ and CAFEQ_LOSS_SUMSQ_WEIGHTED are the
+ * alternatives of App. D.1 over the same group maxima (losses[1] then holds their value instead of the LogSumExp).
+ * CAFEQ_LOSS_PQE_STE differentiates Eq. 5 squared itself with
  * the quantiser passed straight through (only the scale's dependence on its group's arg-max entry is kept): P is
  * required, losses[0] = losses[3] = PQE^2, lambda_orth is ignored (losses[2] = 0), and every dimension must be
  * a multiple of 64 with k a multiple of 32 (CAFEQ_ERR_UNSUPPORTED otherwise); its products run on the tensor cores. */

@@ -16,9 +16,9 @@ LIB_PATH = os.path.join(_HERE, "libcafeq.so")
 
 AXIS_IN, AXIS_OUT = 0, 1
 APPLY_T, APPLY_TT = 0, 1
-LOSS_SURROGATE, LOSS_L2_STE, LOSS_LSE, LOSS_PQE_STE = 0, 1, 2, 3
+LOSS_SURROGATE, LOSS_L2_STE, LOSS_LSE, LOSS_PQE_STE, LOSS_SUMSQ, LOSS_SUMSQ_WEIGHTED = 0, 1, 2, 3, 4, 5
 OPT_STATE_HEADER = 4   # floats before the moment arrays of an optimiser state (CAFEQ_OPT_STATE_HEADER)
-OPT_GD, OPT_ADAM = 0, 1
+OPT_GD, OPT_ADAM, OPT_CAYLEY = 0, 1, 2
 FLAG_EXACT_LOSS, FLAG_NO_GRAD, FLAG_GENERIC, FLAG_WARM_MINV = 1, 2, 4, 8
 OFFSETS_NONE, OFFSETS_HARD_U8, OFFSETS_SOFT_F32 = 0, 1, 2
 ROUND_ALG1, ROUND_LEARNED_OFFSETS = 0, 1
@@ -303,7 +303,7 @@ def cafeq_optimize_pair(W1, W2, M, cfg: OptCfg, *, bits, group1, group2, replica
     d1, d2 = _pair_descs(W1, W2, M.shape[-1], bits, group1, group2, replicas)
     hist = torch.zeros((max(cfg.steps, 1), 2), dtype=torch.float32, device=W1.device)
     status = torch.zeros(1, dtype=torch.int32, device=W1.device)
-    if cfg.optimizer == OPT_ADAM and opt_state is None:
+    if cfg.optimizer in (OPT_ADAM, OPT_CAYLEY) and opt_state is None:
         opt_state = torch.zeros(OPT_STATE_HEADER + 3 * M.numel(), dtype=torch.float32, device=W1.device)
     ws = workspace(workspace_size(d1, d2, cfg), W1.device)
     rc = lib().cafeq_optimize_pair(ctypes.byref(d1), _p(W1), ctypes.byref(d2), _p(W2), _p(M), _p(opt_state),

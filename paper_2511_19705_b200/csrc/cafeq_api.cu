@@ -1150,6 +1150,7 @@ static void launch_pair_product(cudaStream_t st, const void* A1, int a1_bf16, lo
 struct PairWS {
   MatWS m1, m2;
   float *Mc, *Minv, *Minv_c, *gMinv, *tmp, *RM, *amax, *R;
+  float *G1, *G2, *T1, *T2;  // Appendix D.1's weighted objective: block Grams of the two weights, G1 Mc, Minv_c G2
   double* acc;
   KkWS kk;
   DenseWS dn;
@@ -1204,6 +1205,7 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
   p->gMinv = b.take<float>(kk);
   p->tmp = b.take<float>(kk);
   p->RM = b.take<float>(kk);
+  p->G1 = b.take<float>(kk); p->G2 = b.take<float>(kk); p->T1 = b.take<float>(kk); p->T2 = b.take<float>(kk);
   p->amax = b.take<float>(64);
   p->acc = b.take<double>(8);
   p->R = need_R ? b.take<float>((size_t)G1.d_in * G2.d_out) : nullptr;
@@ -1221,15 +1223,58 @@ static bool carve_pair(Bump& b, const Geo& G1, const Geo& G2, PairWS* p, bool ne
 }
 
 static bool lean_pair_ok(const Geo& G1, const Geo& G2, const cafeq_opt_cfg* cfg, const void* W1, const void* W2) {
-  if (!cfg || cfg->loss_kind != CAFEQ_LOSS_LSE || cfg->eval_every != 0) return false;
+  if (!cfg || cfg->eval_every != 0) return false;
+  if (cfg->loss_kind != CAFEQ_LOSS_LSE && cfg->loss_kind != CAFEQ_LOSS_SUMSQ && cfg->loss_kind != CAFEQ_LOSS_SUMSQ_WEIGHTED) return false;
   return kk_fast(G1.k) && bd_supported(BD_OUT, G1.d_out, G1.d_in, G1.ld, G1.k, G1.g, W1) &&
          bd_supported(BD_IN, G2.d_out, G2.d_in, G2.ld, G2.k, G2.g, W2);
+}
+
+// Block Grams of a pair's weights (constants of a run): G1[b][i][j] = sum_x W1[b k + i, x] W1[b k + j, x] and
+// G2[b][i][j] = sum over the r replicas and the rows y of W2[y, (b r + rep) k + i] W2[y, (b r + rep) k + j].
+static void pair_grams(cudaStream_t st, const void* W1, const Geo& G1, const void* W2, const Geo& G2, PairWS& p, const int32_t* status) {
+  const int k = G1.k;
+  const long long kk = (long long)G1.nbT * k * k;
+  GemmArgs g = gemm_defaults(status);
+  g.M = k; g.N = k; g.K = G1.d_in; g.batch = G1.nbT;
+  g.A = W1; g.a_bf16 = 1; g.sAm = G1.ld; g.sAk = 1; g.sAb = (long long)k * G1.ld;
+  g.B = W1; g.b_bf16 = 1; g.sBk = 1; g.sBn = G1.ld; g.sBb = (long long)k * G1.ld;
+  g.C = p.G1; g.sCm = k; g.sCn = 1; g.sCb = (long long)k * k;
+  g.mode = GEMM_STORE;
+  launch_gemm(st, g);
+  CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.G2, 0.f, kk);
+  GemmArgs h = gemm_defaults(status);
+  h.M = k; h.N = k; h.K = G2.d_out; h.batch = G2.nbq;
+  h.A = W2; h.a_bf16 = 1; h.sAm = 1; h.sAk = G2.ld; h.sAb = k;
+  h.B = W2; h.b_bf16 = 1; h.sBk = G2.ld; h.sBn = 1; h.sBb = k;
+  h.C = p.G2; h.sCm = k; h.sCn = 1; h.sCb = (long long)k * k; h.divC = G2.r;
+  h.mode = GEMM_STORE | GEMM_ATOMIC;
+  launch_gemm(st, h);
+}
+
+// One Cayley step on the rotations (Appendix D.2's strictly orthonormal baseline): V <- beta V + g,
+// A = V M^T - M V^T, M <- (I + lr/2 A)^-1 (I - lr/2 A) M, the solve by the fixed-point iteration
+// Y <- M - lr/2 A (M + Y) from Y = M - lr A M (five rounds: the error falls by lr/2 ||A|| per round).
+static void cayley_update(cudaStream_t st, float* M, const float* grad, float* V, float lr, float beta, int nb, int k, PairWS& p,
+                          const int32_t* status) {
+  const long long kk = (long long)nb * k * k;
+  float *A = p.tmp, *Y = p.RM, *S = p.gMinv, *Pm = p.Minv_c;
+  CQ_LAUNCH(momentum_kernel, grid_for(kk), 256, 0, st, V, beta, grad, kk, status);
+  launch_kk(st, V, 0, M, 1, S, nb, k, 1.f, GEMM_STORE, status);            // V M^T
+  CQ_LAUNCH(skew_blocks_kernel, grid_for(kk), 256, 0, st, S, A, k, kk);    // A = V M^T - M V^T
+  launch_kk(st, A, 0, M, 0, Pm, nb, k, 1.f, GEMM_STORE, status);
+  CQ_LAUNCH(lincomb_kernel, grid_for(kk), 256, 0, st, Y, M, -lr, Pm, kk, status);
+  for (int it = 0; it < 5; ++it) {
+    CQ_LAUNCH(lincomb_kernel, grid_for(kk), 256, 0, st, S, M, 1.f, Y, kk, status);
+    launch_kk(st, A, 0, S, 0, Pm, nb, k, 1.f, GEMM_STORE, status);
+    CQ_LAUNCH(lincomb_kernel, grid_for(kk), 256, 0, st, Y, M, -0.5f * lr, Pm, kk, status);
+  }
+  CQ_LAUNCH(copy_f32_kernel, grid_for(kk), 256, 0, st, Y, M, kk);
 }
 
 static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_matrix_desc* d2, const Geo& G1, const Geo& G2,
                       const void* W1, const void* W2, const float* M, const float* P, float t, float lambda, bool want_pqe,
                       float* losses, float* hist, float* gradM, int32_t* status, PairWS& p, bool force_generic,
-                      bool warm = false, float* step_counter = nullptr, bool ste = false) {
+                      bool warm = false, float* step_counter = nullptr, bool ste = false, int objective = 0) {
   const int k = G1.k;
   const bool tc = kk_fast(k) && !force_generic;
   const long long kk = (long long)G1.nbT * k * k;
@@ -1271,6 +1316,18 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   const long long n1 = (long long)G1.d_out * G1.ng, n2 = (long long)G2.d_out * G2.ng;
   CQ_LAUNCH(max2_f32_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, n1, p.m2.a, n2, p.amax, status);
   CQ_LAUNCH(sumexp2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, n1, p.m2.a, n2, p.amax, t, p.acc + 0, status);
+  if (objective) {
+    // Appendix D.1: sums of the squared group maxima; for the weighted form also ||U||_F^2 = <G1 Mc, Mc> and
+    // ||V||_F^2 = <Minv_c G2, Minv_c> from the block Grams of the weights (computed once per call)
+    CQ_LAUNCH(sqsum_f32_kernel, grid_for(n1), 256, 0, st, p.m1.a, n1, p.acc + 3);
+    CQ_LAUNCH(sqsum_f32_kernel, grid_for(n2), 256, 0, st, p.m2.a, n2, p.acc + 4);
+    if (objective == 2) {
+      launch_kk(st, p.G1, 0, p.Mc, 0, p.T1, G1.nbT, k, 1.f, GEMM_STORE, status);
+      launch_kk(st, p.Minv_c, 0, p.G2, 0, p.T2, G1.nbT, k, 1.f, GEMM_STORE, status);
+      CQ_LAUNCH(dot_f32_kernel, grid_for(kk), 256, 0, st, p.T1, p.Mc, kk, p.acc + 5);
+      CQ_LAUNCH(dot_f32_kernel, grid_for(kk), 256, 0, st, p.T2, p.Minv_c, kk, p.acc + 6);
+    }
+  }
   // orthonormality penalty on the fp32 parameters: R = M M^T - I (not part of the straight-through PQE loss)
   if (ste) {
   } else if (tc) {
@@ -1300,7 +1357,8 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
     CQ_LAUNCH(resid_sq_kernel, grid_for((long long)G1.d_in * G2.d_out), 256, 0, st, p.R, P, (long long)G1.d_in * G2.d_out, p.acc + 2,
                                                                              status);
   }
-  CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, ste ? 2 : (want_pqe ? 1 : 0));
+  CQ_LAUNCH(finalize_pair_kernel, 1, 1, 0, st, p.acc, p.amax, t, lambda, sqrt_h, losses, hist, ste ? 2 : (want_pqe ? 1 : 0), objective,
+            (double)n1, (double)n2);
   if (!gradM) return;
   if (ste) {
     // Straight-through gradient of ||Uhat_exp^T Vhat^T - P||_F^2 (Eq. 5 squared): the residual R [d1, d3] and
@@ -1365,8 +1423,12 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
     }
     return;
   }
-  CQ_LAUNCH(lse_coef2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, p.m1.usel, p.m1.coef, n1, p.m2.a, p.m2.usel, p.m2.coef, n2,
-            p.amax, t, p.acc + 0, status);
+  if (objective)
+    CQ_LAUNCH(sumsq_coef2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, p.m1.usel, p.m1.coef, n1, p.m2.a, p.m2.usel, p.m2.coef, n2,
+              p.acc, objective == 2 ? 1 : 0, status);
+  else
+    CQ_LAUNCH(lse_coef2_kernel, grid_for(n1 + n2), 256, 0, st, p.m1.a, p.m1.usel, p.m1.coef, n1, p.m2.a, p.m2.usel, p.m2.coef, n2,
+              p.amax, t, p.acc + 0, status);
   if (!tc) {
     CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, gradM, 0.f, kk);
     CQ_LAUNCH(fill_f32_kernel, grid_for(kk), 256, 0, st, p.gMinv, 0.f, kk);
@@ -1375,6 +1437,11 @@ static void pair_step(cudaStream_t st, const cafeq_matrix_desc* d1, const cafeq_
   launch_scatter(st, W1, G1, p.m1.coef, p.m1.idx, gradM, 1, status, f1 ? 1 : 0);
   // V side: gradient with respect to Minv, then through the inverse
   launch_scatter(st, W2, G2, p.m2.coef, p.m2.idx, p.gMinv, 0, status, f2 ? 1 : 0);
+  if (objective == 2) {
+    // mean(a_V^2) d||U||_F/dM = mean(a_V^2) G1 Mc / ||U||_F ; mean(a_U^2) d||V||_F/dMinv = mean(a_U^2) Minv_c G2 / ||V||_F
+    CQ_LAUNCH(axpy_norm_kernel, grid_for(kk), 256, 0, st, gradM, p.T1, kk, p.acc, 4, (double)n2, 5, status);
+    CQ_LAUNCH(axpy_norm_kernel, grid_for(kk), 256, 0, st, p.gMinv, p.T2, kk, p.acc, 3, (double)n1, 6, status);
+  }
   if (tc) {
     minv_path_tc(st, p.gMinv, gradM, G1.nbT, k, true, p.kk, status);
   } else {
@@ -1453,7 +1520,8 @@ extern "C" int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* 
   if (rc) return rc;
   if (!W1 || !W2 || !M || !losses) return CAFEQ_ERR_INVALID_ARG;
   const bool ste = loss_kind == CAFEQ_LOSS_PQE_STE;
-  if (!ste && loss_kind != CAFEQ_LOSS_LSE) return CAFEQ_ERR_INVALID_ARG;
+  const int objective = loss_kind == CAFEQ_LOSS_SUMSQ ? 1 : (loss_kind == CAFEQ_LOSS_SUMSQ_WEIGHTED ? 2 : 0);
+  if (!ste && !objective && loss_kind != CAFEQ_LOSS_LSE) return CAFEQ_ERR_INVALID_ARG;
   if (ste && !dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;
   if (!(lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
   const bool want_grad = !(flags & CAFEQ_FLAG_NO_GRAD);
@@ -1464,8 +1532,9 @@ extern "C" int cafeq_pair_loss_fwd_bwd(const cafeq_matrix_desc* d1, const void* 
   Bump b(ws, ws_bytes);
   PairWS p;
   if (!carve_pair(b, G1, G2, &p, want_pqe)) return CAFEQ_ERR_WORKSPACE;
+  if (objective == 2) pair_grams((cudaStream_t)stream, W1, G1, W2, G2, p, status);
   pair_step((cudaStream_t)stream, d1, d2, G1, G2, W1, W2, M, P, lse_t, lambda_orth, want_pqe, losses, nullptr,
-            want_grad ? gradM : nullptr, status, p, (flags & CAFEQ_FLAG_GENERIC) != 0, false, nullptr, ste);
+            want_grad ? gradM : nullptr, status, p, (flags & CAFEQ_FLAG_GENERIC) != 0, false, nullptr, ste, objective);
   return last_launch();
 }
 
@@ -1477,11 +1546,13 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   if (rc) return rc;
   if (!W1 || !W2 || !M || !cfg || cfg->struct_size != sizeof(cafeq_opt_cfg) || !loss_history) return CAFEQ_ERR_INVALID_ARG;
   const bool ste = cfg->loss_kind == CAFEQ_LOSS_PQE_STE;
-  if ((!ste && cfg->loss_kind != CAFEQ_LOSS_LSE) || cfg->steps < 0 || !(cfg->lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
+  const int objective = cfg->loss_kind == CAFEQ_LOSS_SUMSQ ? 1 : (cfg->loss_kind == CAFEQ_LOSS_SUMSQ_WEIGHTED ? 2 : 0);
+  if ((!ste && !objective && cfg->loss_kind != CAFEQ_LOSS_LSE) || cfg->steps < 0 || !(cfg->lse_t > 0.f)) return CAFEQ_ERR_INVALID_ARG;
   if (ste && !P) return CAFEQ_ERR_INVALID_ARG;
   if (ste && !dense_ok(G1, G2)) return CAFEQ_ERR_UNSUPPORTED;
-  if (cfg->optimizer == CAFEQ_OPT_ADAM && !opt_state) return CAFEQ_ERR_INVALID_ARG;
-  if (cfg->optimizer != CAFEQ_OPT_ADAM && cfg->optimizer != CAFEQ_OPT_GD) return CAFEQ_ERR_INVALID_ARG;
+  const bool cayley = cfg->optimizer == CAFEQ_OPT_CAYLEY;
+  if ((cfg->optimizer == CAFEQ_OPT_ADAM || cayley) && !opt_state) return CAFEQ_ERR_INVALID_ARG;
+  if (cfg->optimizer != CAFEQ_OPT_ADAM && cfg->optimizer != CAFEQ_OPT_GD && !cayley) return CAFEQ_ERR_INVALID_ARG;
   if ((rc = check_ws(ws, ws_bytes))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const bool any_pqe = ste || ((P != nullptr) && cfg->eval_every > 0);
@@ -1494,12 +1565,16 @@ extern "C" int cafeq_optimize_pair(const cafeq_matrix_desc* d1, const void* W1, 
   // the inverse of the last step's transform lives in the optimiser state, so a resumed run refines it
   const bool resume = cfg->resume && opt_state;
   if (opt_state) p.Minv = opt_state + CAFEQ_OPT_STATE_HEADER + 2 * kk;
+  if (objective == 2) pair_grams(st, W1, G1, W2, G2, p, status);
   for (int it = 0; it < cfg->steps; ++it) {
     bool eval = ste || (any_pqe && (it % cfg->eval_every == 0));
     pair_step(st, d1, d2, G1, G2, W1, W2, M, P, cfg->lse_t, cfg->lambda_orth, eval, nullptr, loss_history + 2 * (size_t)it,
-              grad, status, p, false, resume || it > 0, opt_state, ste);
+              grad, status, p, false, resume || it > 0, opt_state, ste, objective);
     if (p.err) return p.err;
-    if (cfg->optimizer == CAFEQ_OPT_GD) {
+    if (cayley) {
+      // momentum in the state's first-moment slot
+      cayley_update(st, M, grad, opt_state + CAFEQ_OPT_STATE_HEADER, cfg->lr, cfg->beta1, G1.nbT, G1.k, p, status);
+    } else if (cfg->optimizer == CAFEQ_OPT_GD) {
       CQ_LAUNCH(gd_update_kernel, grid_for(kk), 256, 0, st, M, grad, cfg->lr, kk, status);
     } else {
       CQ_LAUNCH(adam_update_kernel, grid_for(kk), 256, 0, st, M, grad, opt_state, cfg->lr, cfg->beta1, cfg->beta2, cfg->eps, kk,

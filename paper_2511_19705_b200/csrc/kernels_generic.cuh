@@ -1154,10 +1154,66 @@ __global__ void finalize_single_kernel(const double* acc, float* losses, float* 
   }
 }
 
-// pair: acc = {Z, ||R_orth||^2, PQE^2}; amax = running max
+// Appendix D.1's sums of squares over the group maxima: coef = w * 2 a sign(U at the arg-max) / count, with
+// w = the other factor's Frobenius norm in the weighted form (acc[5] = ||U||_F^2, acc[6] = ||V||_F^2), else 1
+__global__ void sumsq_coef2_kernel(const float* __restrict__ a1, const float* __restrict__ u1, float* __restrict__ c1, long long n1,
+                                   const float* __restrict__ a2, const float* __restrict__ u2, float* __restrict__ c2, long long n2,
+                                   const double* __restrict__ acc, int weighted, const int32_t* status) {
+  if (status && *status) return;
+  const float w1 = (weighted ? (float)sqrt(acc[6]) : 1.f) * 2.f / (float)n1;
+  const float w2 = (weighted ? (float)sqrt(acc[5]) : 1.f) * 2.f / (float)n2;
+  const long long n = n1 + n2;
+  for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < n; w += (long long)gridDim.x * blockDim.x) {
+    const bool first = w < n1;
+    const long long i = first ? w : w - n1;
+    const float u = first ? u1[i] : u2[i];
+    const float av = first ? a1[i] : a2[i];
+    const float sgn = (u > 0.f) ? 1.f : ((u < 0.f) ? -1.f : 0.f);
+    if (first) c1[i] = w1 * av * sgn; else c2[i] = w2 * av * sgn;
+  }
+}
+
+// dst += (acc[num] / count) / sqrt(acc[den]) * src   (the dense terms of the weighted form: mean(a^2) d||X||_F)
+__global__ void axpy_norm_kernel(float* __restrict__ dst, const float* __restrict__ src, long long n, const double* __restrict__ acc,
+                                 int num, double count, int den, const int32_t* status) {
+  if (status && *status) return;
+  const double d = sqrt(acc[den]);
+  const float f = d > 0.0 ? (float)(acc[num] / count / d) : 0.f;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    dst[i] = fmaf(f, src[i], dst[i]);
+}
+
+// out = T - T^T per block (the skew part that drives a Cayley step)
+__global__ void skew_blocks_kernel(const float* __restrict__ T, float* __restrict__ out, int k, long long n) {
+  const long long kk = (long long)k * k;
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const long long b = e / kk, q = e - b * kk;
+    const int i = (int)(q / k), j = (int)(q - (long long)i * k);
+    out[e] = T[e] - T[b * kk + (long long)j * k + i];
+  }
+}
+
+// out = x + alpha * y  /  x = beta * x + y
+__global__ void lincomb_kernel(float* __restrict__ out, const float* __restrict__ x, float alpha, const float* __restrict__ y,
+                               long long n, const int32_t* status) {
+  if (status && *status) return;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    out[i] = fmaf(alpha, y[i], x[i]);
+}
+__global__ void momentum_kernel(float* __restrict__ v, float beta, const float* __restrict__ g, long long n, const int32_t* status) {
+  if (status && *status) return;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    v[i] = fmaf(beta, v[i], g[i]);
+}
+
+// pair: acc = {Z, ||R_orth||^2, PQE^2, sum a_U^2, sum a_V^2, ||U||_F^2, ||V||_F^2}; amax = running max.
+// objective 0: LogSumExp; 1: mean of squared maxima; 2: the norm-weighted form (counts n1, n2 of group maxima)
 __global__ void finalize_pair_kernel(const double* acc, const float* amax, float t, float lambda, float sqrt_h,
-                                     float* losses, float* hist, int want_pqe) {
+                                     float* losses, float* hist, int want_pqe, int objective = 0, double n1 = 1.0,
+                                     double n2 = 1.0) {
   float lse = *amax + (float)(log(acc[0]) / (double)t);
+  if (objective == 1) lse = (float)(acc[3] / n1 + acc[4] / n2);
+  if (objective == 2) lse = (float)(sqrt(acc[6]) * acc[3] / n1 + sqrt(acc[5]) * acc[4] / n2);
   float orth = (float)(sqrt(acc[1]) / (double)sqrt_h);
   // want_pqe == 2: the squared product error is the loss being minimised (straight-through mode)
   const float loss = (want_pqe == 2) ? (float)acc[2] : lse + lambda * orth;
