@@ -299,6 +299,14 @@ int cafeq_optimize_layer(const cafeq_layer_problem* probs, int n, int steps, int
  * previous step's inverse had not converged (a step that changed a transform by more than about half its norm). */
 int cafeq_layer_debug_fallbacks(const cafeq_layer_problem* probs, int n, void* ws, size_t ws_bytes, int* count);
 
+/* Tuning knob of the layer step, process-wide (the paper has no counterpart; results do not depend on it).
+ * dual = 1 (default): when a layer has matrices on both axes, their transform passes share one persistent launch and
+ * their sparse backwards another; dual = 0: one launch per axis.  pass_out_pct / bwd_out_pct (> 0, default 150 / 120):
+ * cost of an output-axis tile in percent of an input-axis tile of the same bytes, which sets how the 148 CTAs of a
+ * shared launch are divided between the two lists; <= 0 keeps the current value.  Returns CAFEQ_ERR_INVALID_ARG
+ * unless dual is 0 or 1 and the percentages are at most 1000. */
+int cafeq_debug_set_layer_launch(int dual, int pass_out_pct, int bwd_out_pct);
+
 const char* cafeq_status_string(int status);
 int cafeq_version(void);
 /* Tuning knob, process-wide (the paper has no counterpart).  overlapped = 0 (default): one problem runs alone:

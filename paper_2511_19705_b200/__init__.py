@@ -26,7 +26,7 @@ ROUND_ALG1, ROUND_LEARNED_OFFSETS = 0, 1
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_workspace_size", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_layer_debug_fallbacks", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_layer_debug_fallbacks", "cafeq_debug_set_layer_launch", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
     "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
@@ -91,6 +91,13 @@ def set_overlap_mode(overlapped: bool) -> None:
     """Process-wide launch-shape rule: True when several problems run concurrently in different streams (kernels
     then take fewer CTAs: fewer SM-microseconds each), False (default) when one problem runs alone (lowest latency)."""
     _check(lib().cafeq_set_overlap_mode(ctypes.c_int(1 if overlapped else 0)), "cafeq_set_overlap_mode")
+
+
+def set_layer_launch(dual: bool = True, pass_out_pct: int = 0, bwd_out_pct: int = 0) -> None:
+    """Process-wide launch rule of the layer step: both axes' matrices in one pass launch and one backward launch
+    (dual), and the cost of an output-axis tile in percent of an input-axis tile (0 keeps the current value)."""
+    _check(lib().cafeq_debug_set_layer_launch(ctypes.c_int(1 if dual else 0), ctypes.c_int(pass_out_pct), ctypes.c_int(bwd_out_pct)),
+           "cafeq_debug_set_layer_launch")
 
 
 def launch_count() -> int:

@@ -224,6 +224,8 @@ struct KkWS {  // bf16 scratch, each [nbT * k * k]
   int* flag;   // 1 => Newton-Schulz did not converge, the Gauss-Jordan kernel takes over
   int* redo_total;  // optional running count of blocks recomputed by elimination (never cleared by a step)
   int cur;     // which of the ping-pong split sets holds the current inverse (host bookkeeping)
+  bool mn;     // the inverse was refined on row-major arrays only (whole-block products with MN-major operands): the
+               // transposed splits XTh / XTl are not maintained
 };
 constexpr int NS_MAX_ITERS = 8;
 constexpr int NS_COLD_ITERS = 6;
@@ -240,13 +242,14 @@ static void carve_kk(Bump& b, int nbT, int k, KkWS* w) {
   w->flag = b.take<int>(64);
   w->redo_total = nullptr;
   w->cur = 0;
+  w->mn = false;
 }
 
 // C[b] = alpha * sum_t A_t[b] B_t[b]^T + beta * C0[b] + gamma * I for nb blocks of k x k; operands bf16 [nb*k, k]
 static int launch_kk_tc(cudaStream_t st, int nterms, const uint16_t* const* A, const uint16_t* const* B, int nb, int k,
                         float alpha, float beta, float gamma, const float* C0, float* C, uint16_t* Chi, uint16_t* Clo,
                         uint16_t* Cthi, uint16_t* Ctlo, double* sq, const int* run_flag, int32_t* status, int sq_stride = 1,
-                        const double* gate = nullptr, double gate_tol = 0.0) {
+                        const double* gate = nullptr, double gate_tol = 0.0, int a_mn = 0, int b_mn = 0) {
   TgOperand oa[TG_MAX_TERMS], ob[TG_MAX_TERMS];
   for (int t = 0; t < nterms; ++t) {
     oa[t] = TgOperand{A[t], (long long)nb * k, k, k};
@@ -271,6 +274,11 @@ static int launch_kk_tc(cudaStream_t st, int nterms, const uint16_t* const* A, c
   p.gate_tol = gate_tol;
   p.status = status;
   g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (g_tb_enable.load(std::memory_order_relaxed) && tb_supported(k, nterms)) {
+    const int rc = tb_launch(st, nterms, A, B, a_mn, b_mn, (long long)nb * k, (long long)nb * k, k, p);
+    if (rc != CAFEQ_ERR_UNSUPPORTED) return rc;
+  }
+  if (a_mn || b_mn) return CAFEQ_ERR_UNSUPPORTED;  // the tiled kernel takes K-major operands only
   return tg_launch(st, oa, ob, p);
 }
 
@@ -330,23 +338,38 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   }
   if (!warm) CQ_LAUNCH(transpose_blocks_kernel, grid_for(kk), 256, 0, st, Mc, X, k, kk);
   int cur = 0;
+  // Block sizes with the whole-block product kernel run the iteration on row-major arrays only (MN-major operands):
+  // no transposed split of X or R is written.
+  const bool mn = g_tb_enable.load(std::memory_order_relaxed) && tb_supported(k, 2);
+  w.mn = mn;
   // (splits_kept: the splits of X that the previous call left in set 0 are still there)
-  if (!(warm && splits_kept))
-    launch_split(st, X, k, kk, w.Xh[cur], iters > 0 ? nullptr : w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
+  if (!(warm && splits_kept)) {
+    if (mn) launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], nullptr, nullptr, nullptr, status);
+    else launch_split(st, X, k, kk, w.Xh[cur], iters > 0 ? nullptr : w.Xl[cur], w.XTh[cur], w.XTl[cur], nullptr, status);
+  }
   for (int it = 0; it < iters; ++it) {
     const double* gate = (warm && it > 0) ? w.rn + (size_t)(it - 1) * nb : nullptr;
     // R = I - A X needs X to full precision (the product cancels against I): two terms over the split of X.
-    const uint16_t* a1[2] = {w.Ab, w.Ab};
-    const uint16_t* b1[2] = {w.XTh[cur], w.XTl[cur]};
-    launch_kk_tc(st, 2, a1, b1, nb, k, -1.f, 0.f, 1.f, nullptr, nullptr, nullptr, nullptr, w.RTh, nullptr, w.rn + (size_t)it * nb,
-                 nullptr, status, 1, gate, NS_GATE2);
     // X += X R: the correction is small and the iteration corrects its own errors, so one bf16 term is enough
     // (the error it leaves is 2^-8 |R| relative, below 4e-5 for every accepted residual).
+    const uint16_t* a1[2] = {w.Ab, w.Ab};
     const uint16_t* a2[1] = {w.Xh[cur]};
-    const uint16_t* b2[1] = {w.RTh};
-    // (the row-major low half is only read after the last iteration, by the M^-1 path of the gradient)
-    launch_kk_tc(st, 1, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], (it == iters - 1) ? w.Xl[cur ^ 1] : nullptr,
-                 w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr, nullptr, status, 1, gate, NS_GATE2);
+    if (mn) {
+      const uint16_t* b1[2] = {w.Xh[cur], w.Xl[cur]};  // X stored [l][n]
+      launch_kk_tc(st, 2, a1, b1, nb, k, -1.f, 0.f, 1.f, nullptr, nullptr, w.RTh, nullptr, nullptr, nullptr, w.rn + (size_t)it * nb,
+                   nullptr, status, 1, gate, NS_GATE2, 0, 1);
+      const uint16_t* b2[1] = {w.RTh};                  // bf16(R), row-major here
+      launch_kk_tc(st, 1, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], w.Xl[cur ^ 1], nullptr, nullptr, nullptr, nullptr, status,
+                   1, gate, NS_GATE2, 0, 1);
+    } else {
+      const uint16_t* b1[2] = {w.XTh[cur], w.XTl[cur]};
+      launch_kk_tc(st, 2, a1, b1, nb, k, -1.f, 0.f, 1.f, nullptr, nullptr, nullptr, nullptr, w.RTh, nullptr, w.rn + (size_t)it * nb,
+                   nullptr, status, 1, gate, NS_GATE2);
+      const uint16_t* b2[1] = {w.RTh};
+      // (the row-major low half is only read after the last iteration, by the M^-1 path of the gradient)
+      launch_kk_tc(st, 1, a2, b2, nb, k, 1.f, 1.f, 0.f, X, X, w.Xh[cur ^ 1], (it == iters - 1) ? w.Xl[cur ^ 1] : nullptr,
+                   w.XTh[cur ^ 1], w.XTl[cur ^ 1], nullptr, nullptr, status, 1, gate, NS_GATE2);
+    }
     cur ^= 1;
   }
   w.cur = cur;
@@ -356,7 +379,8 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   // final splits: written by the last iteration's epilogue, except for blocks that skipped it (and for everything
   // when the elimination recomputed a block)
   const double* last_gate = (warm && iters > 1) ? w.rn + (size_t)(iters - 2) * nb : nullptr;
-  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], w.flag, status, last_gate, NS_GATE2);
+  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], mn ? nullptr : w.XTh[cur], mn ? nullptr : w.XTl[cur], w.flag, status, last_gate,
+               NS_GATE2);
   if (cnorm) {
     dim3 grid((k + 127) / 128, nb);
     CQ_LAUNCH(colnorm_kernel, grid, 128, 0, st, X, k, nb, cnorm);
@@ -369,11 +393,20 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
 static void minv_path_tc(cudaStream_t st, const float* Gx, float* G, int nb, int k, bool accumulate, KkWS& w, int32_t* status) {
   const long long kk = (long long)nb * k * k;
   const int c = w.cur;
-  launch_split(st, Gx, k, kk, nullptr, nullptr, w.Ph, w.Pl, nullptr, status);  // Gx^T splits
-  // T1 = X^T Gx : T1[i][j] = sum_l XT[i][l] * GxT[j][l]
-  const uint16_t* a1[3] = {w.XTh[c], w.XTl[c], w.XTh[c]};
-  const uint16_t* b1[3] = {w.Ph, w.Ph, w.Pl};
-  launch_kk_tc(st, 3, a1, b1, nb, k, 1.f, 0.f, 0.f, nullptr, nullptr, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status);
+  if (w.mn) {
+    // T1 = X^T Gx with both operands read from their row-major arrays: A_op[i][l] = X[l][i], B_op[j][l] = Gx[l][j]
+    launch_split(st, Gx, k, kk, w.Ph, w.Pl, nullptr, nullptr, nullptr, status);
+    const uint16_t* a1[3] = {w.Xh[c], w.Xl[c], w.Xh[c]};
+    const uint16_t* b1[3] = {w.Ph, w.Ph, w.Pl};
+    launch_kk_tc(st, 3, a1, b1, nb, k, 1.f, 0.f, 0.f, nullptr, nullptr, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status, 1, nullptr,
+                 0.0, 1, 1);
+  } else {
+    launch_split(st, Gx, k, kk, nullptr, nullptr, w.Ph, w.Pl, nullptr, status);  // Gx^T splits
+    // T1 = X^T Gx : T1[i][j] = sum_l XT[i][l] * GxT[j][l]
+    const uint16_t* a1[3] = {w.XTh[c], w.XTl[c], w.XTh[c]};
+    const uint16_t* b1[3] = {w.Ph, w.Ph, w.Pl};
+    launch_kk_tc(st, 3, a1, b1, nb, k, 1.f, 0.f, 0.f, nullptr, nullptr, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status);
+  }
   // G -= T1 X^T : [i][j] = sum_l T1[i][l] * X[j][l]
   const uint16_t* a2[3] = {w.Qh, w.Ql, w.Qh};
   const uint16_t* b2[3] = {w.Xh[c], w.Xh[c], w.Xl[c]};
@@ -936,9 +969,16 @@ static void single_step(cudaStream_t st, const cafeq_matrix_desc* d, const Geo& 
       tg_launch(st, oa, ob, p);
     }
     {  // N = Minv^T Minv (fp32 in s.Nf, splits in w.Qh / w.Ql)
-      const uint16_t* a1[3] = {w.XTh[c], w.XTl[c], w.XTh[c]};
-      const uint16_t* b1[3] = {w.XTh[c], w.XTh[c], w.XTl[c]};
-      launch_kk_tc(st, 3, a1, b1, G.nbT, k, 1.f, 0.f, 0.f, nullptr, s.Nf, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status);
+      if (w.mn) {  // both operands are X read transposed from its row-major splits
+        const uint16_t* a1[3] = {w.Xh[c], w.Xl[c], w.Xh[c]};
+        const uint16_t* b1[3] = {w.Xh[c], w.Xh[c], w.Xl[c]};
+        launch_kk_tc(st, 3, a1, b1, G.nbT, k, 1.f, 0.f, 0.f, nullptr, s.Nf, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status, 1,
+                     nullptr, 0.0, 1, 1);
+      } else {
+        const uint16_t* a1[3] = {w.XTh[c], w.XTl[c], w.XTh[c]};
+        const uint16_t* b1[3] = {w.XTh[c], w.XTh[c], w.XTl[c]};
+        launch_kk_tc(st, 3, a1, b1, G.nbT, k, 1.f, 0.f, 0.f, nullptr, s.Nf, w.Qh, w.Ql, nullptr, nullptr, nullptr, nullptr, status);
+      }
     }
     CQ_LAUNCH(dot_f32_kernel, grid_for(kk), 256, 0, st, s.Nf, s.tmp, kk, s.acc + 1);
     CQ_LAUNCH(sqsum_bf16_kernel, grid_for(G.n), 256, 0, st, (const uint16_t*)W, G.ld, G.d_out, G.d_in, s.acc + 2, status);

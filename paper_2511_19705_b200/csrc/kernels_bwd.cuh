@@ -103,14 +103,14 @@ __device__ __forceinline__ uint32_t bw_s_offset(int target, int kk) {
 // SWAP = 0: accumulator rows = targets i, columns = j (coalesced when the output is stored transposed);
 // SWAP = 1: rows = j, columns = i (coalesced for the plain layout).
 template <int FORM, int K, int SWAP, int F16>
-__global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_constant__ BwMaps maps, const __grid_constant__ BwMulti mp) {
+__device__ __forceinline__ void bd_bwd_body(const BwMaps& maps, const BwMulti& mp, const int cta, const int ncta) {
   using C = BwCfg<K, F16>;
   static_assert(K == 128 || K == 256, "block size");
   int32_t* const status = mp.p[0].status;
   if (status && *status) return;
   const int total_tiles = mp.tile_end[mp.n - 1];
-  const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
-  const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
+  const int t_begin = (int)(((long long)cta * total_tiles) / ncta);
+  const int t_end = (int)(((long long)(cta + 1) * total_tiles) / ncta);
   if (t_begin >= t_end) return;
   int s_first = 0;
   while (mp.tile_end[s_first] <= t_begin) ++s_first;
@@ -385,6 +385,21 @@ __global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_cons
   }
 }
 
+template <int FORM, int K, int SWAP, int F16>
+__global__ void __launch_bounds__(BW_THREADS, 1) bd_bwd_kernel(const __grid_constant__ BwMaps maps, const __grid_constant__ BwMulti mp) {
+  bd_bwd_body<FORM, K, SWAP, F16>(maps, mp, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// Input-axis and output-axis matrices in one launch (fp16 single-term form): the first n_in CTAs run the input-axis
+// list, the others the output-axis list.
+template <int K, int SWAP_IN, int SWAP_OUT>
+__global__ void __launch_bounds__(BW_THREADS, 1)
+bd_bwd_dual_kernel(const __grid_constant__ BwMaps maps_in, const __grid_constant__ BwMulti mp_in,
+                   const __grid_constant__ BwMaps maps_out, const __grid_constant__ BwMulti mp_out, const int n_in) {
+  if ((int)blockIdx.x < n_in) bd_bwd_body<BW_IN, K, SWAP_IN, 1>(maps_in, mp_in, (int)blockIdx.x, n_in);
+  else bd_bwd_body<BW_OUT, K, SWAP_OUT, 1>(maps_out, mp_out, (int)blockIdx.x - n_in, (int)gridDim.x - n_in);
+}
+
 // host side ------------------------------------------------------------------------------------------------
 static bool bw_supported(int axis_in, int d_out, int d_in, long long ld, int k, int g, const void* W) {
   if (!(k == 128 || k == 256)) return false;
@@ -493,6 +508,69 @@ static int bw_launch_many(cudaStream_t st, int axis_in, int k, int transpose_out
   for (int s = n; s < BW_MAX_SUB; ++s) maps.w[s] = maps.w[0];
   mp.n = n;
   return bw_dispatch(st, axis_in, k, transpose_out ? 0 : 1, f16, maps, mp, 6);
+}
+
+template <int K, int SWAP_IN, int SWAP_OUT>
+static int bw_launch_dual_t(cudaStream_t st, const BwMaps& mi, BwMulti pi, const BwMaps& mo, BwMulti po) {
+  using C = BwCfg<K, 1>;
+  static std::atomic<unsigned long long> done{0};
+  if (!opt_in_smem(bd_bwd_dual_kernel<K, SWAP_IN, SWAP_OUT>, C::SMEM, done)) return CAFEQ_ERR_CUDA;
+  long long ti = 0, to = 0, maj_i = 0, maj_o = 0;
+  for (int s = 0; s < pi.n; ++s) {
+    bw_fill_tiles(pi.p[s], 1, K);
+    ti += (long long)pi.p[s].n_major * pi.p[s].n_minor;
+    maj_i += pi.p[s].n_major;
+    pi.tile_end[s] = (int)ti;
+  }
+  for (int s = pi.n; s < BW_MAX_SUB; ++s) pi.tile_end[s] = (int)ti;
+  for (int s = 0; s < po.n; ++s) {
+    bw_fill_tiles(po.p[s], 0, K);
+    to += (long long)po.p[s].n_major * po.p[s].n_minor;
+    maj_o += po.p[s].n_major;
+    po.tile_end[s] = (int)to;
+  }
+  for (int s = po.n; s < BW_MAX_SUB; ++s) po.tile_end[s] = (int)to;
+  // tiles of the two forms hold the same bytes (64 x K entries)
+  const int n_in = dual_split(ti, to, g_dual_bwd_pct.load(std::memory_order_relaxed));
+  bd_bwd_dual_kernel<K, SWAP_IN, SWAP_OUT><<<148, BW_THREADS, C::SMEM, st>>>(mi, pi, mo, po, n_in);
+  return CAFEQ_OK;
+}
+
+// fp16 single-term form only; each list holds at least 148 * 6 tiles (the caller checks with bw_dual_ok)
+static bool bw_dual_ok(int k) { return k == 128 || k == 256; }
+static int bw_launch_dual(cudaStream_t st, int k, int tr_in, const BwSub* in, int n_in, int tr_out, const BwSub* out, int n_out) {
+  if (n_in < 1 || n_in > BW_MAX_SUB || n_out < 1 || n_out > BW_MAX_SUB || !bw_dual_ok(k)) return CAFEQ_ERR_INVALID_ARG;
+  BwMaps mi, mo;
+  BwMulti pi, po;
+  memset(&pi, 0, sizeof(pi));
+  memset(&po, 0, sizeof(po));
+  for (int s = 0; s < n_in; ++s) {
+    if (!make_map_bf16(&mi.w[s], in[s].W16, in[s].p.d_in, in[s].p.d_out, in[s].ld, 64)) return CAFEQ_ERR_UNSUPPORTED;
+    pi.p[s] = in[s].p;
+    pi.p[s].transpose_out = tr_in;
+  }
+  for (int s = n_in; s < BW_MAX_SUB; ++s) mi.w[s] = mi.w[0];
+  for (int s = 0; s < n_out; ++s) {
+    if (!make_map_bf16(&mo.w[s], out[s].W16, out[s].p.d_in, out[s].p.d_out, out[s].ld, k)) return CAFEQ_ERR_UNSUPPORTED;
+    po.p[s] = out[s].p;
+    po.p[s].transpose_out = tr_out;
+  }
+  for (int s = n_out; s < BW_MAX_SUB; ++s) mo.w[s] = mo.w[0];
+  pi.n = n_in;
+  po.n = n_out;
+  const int si = tr_in ? 0 : 1, so = tr_out ? 0 : 1;
+#define BW_DUAL(KK, SI, SO) \
+  if (k == KK && si == SI && so == SO) return bw_launch_dual_t<KK, SI, SO>(st, mi, pi, mo, po);
+  BW_DUAL(128, 0, 0)
+  BW_DUAL(128, 0, 1)
+  BW_DUAL(128, 1, 0)
+  BW_DUAL(128, 1, 1)
+  BW_DUAL(256, 0, 0)
+  BW_DUAL(256, 0, 1)
+  BW_DUAL(256, 1, 0)
+  BW_DUAL(256, 1, 1)
+#undef BW_DUAL
+  return CAFEQ_ERR_UNSUPPORTED;
 }
 
 }  // namespace cafeq

@@ -253,9 +253,10 @@ struct BdCfg {
   static constexpr int SMEM = 1024 + T_BYTES + NSTAGE * BD_STAGE_BYTES + 256;
 };
 
+// The body takes the CTA's index and the number of CTAs that share its tile list, so that one launch can run two
+// lists side by side (bd_pass_dual_kernel below).
 template <int FORM, int K, int G>
-__global__ void __launch_bounds__(BD_THREADS, 1)
-bd_pass_kernel(const __grid_constant__ BdMaps maps, const __grid_constant__ BdMulti mp) {
+__device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& mp, const int cta, const int ncta) {
   using C = BdCfg<FORM, K, G>;
   static_assert(K == 64 || K == 128 || K == 256, "block size");
   static_assert(FORM == BD_IN || K >= 128, "output-axis form needs k >= 128");
@@ -266,8 +267,8 @@ bd_pass_kernel(const __grid_constant__ BdMaps maps, const __grid_constant__ BdMu
   // persistent CTA: a contiguous run of tiles in (sub-problem, major, minor) order; the operator block is reloaded
   // when the run crosses into the next major or the next sub-problem
   const int total_tiles = mp.tile_end[mp.n - 1];
-  const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
-  const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
+  const int t_begin = (int)(((long long)cta * total_tiles) / ncta);
+  const int t_end = (int)(((long long)(cta + 1) * total_tiles) / ncta);
   if (t_begin >= t_end) return;
   int s_first = 0;
   while (mp.tile_end[s_first] <= t_begin) ++s_first;
@@ -715,6 +716,23 @@ bd_pass_kernel(const __grid_constant__ BdMaps maps, const __grid_constant__ BdMu
   }
 }
 
+template <int FORM, int K, int G>
+__global__ void __launch_bounds__(BD_THREADS, 1)
+bd_pass_kernel(const __grid_constant__ BdMaps maps, const __grid_constant__ BdMulti mp) {
+  bd_pass_body<FORM, K, G>(maps, mp, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// Both forms in one launch: the first n_in CTAs run the input-axis list, the others the output-axis list (a layer
+// has matrices of both forms; two launches pay the fixed cost of a persistent kernel -- operator load, pipeline
+// fill, the tail of the slowest CTA -- twice, and the smaller list alone cannot fill the memory system).
+template <int K, int G>
+__global__ void __launch_bounds__(BD_THREADS, 1)
+bd_pass_dual_kernel(const __grid_constant__ BdMaps maps_in, const __grid_constant__ BdMulti mp_in,
+                    const __grid_constant__ BdMaps maps_out, const __grid_constant__ BdMulti mp_out, const int n_in) {
+  if ((int)blockIdx.x < n_in) bd_pass_body<BD_IN, K, G>(maps_in, mp_in, (int)blockIdx.x, n_in);
+  else bd_pass_body<BD_OUT, K, G>(maps_out, mp_out, (int)blockIdx.x - n_in, (int)gridDim.x - n_in);
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side: tensor maps and launch
 // ------------------------------------------------------------------------------------------------
@@ -868,6 +886,74 @@ static int bd_launch_many(cudaStream_t st, int form, int k, int g, const BdSub* 
   for (int s = n; s < BD_MAX_SUB; ++s) { maps.x[s] = maps.x[0]; maps.t[s] = maps.t[0]; }
   mp.n = n;
   return bd_dispatch(st, form, k, g, maps, mp, 1);
+}
+
+// relative cost of an output-axis tile against an input-axis tile of the same bytes (measured per-tile times of
+// the two forms): sets how the CTAs of a dual launch are divided
+static std::atomic<int> g_dual_pass_pct{150}, g_dual_bwd_pct{120};
+
+static int dual_split(long long tiles_in, long long tiles_out, int out_weight_pct) {
+  const double wi = (double)tiles_in, wo = (double)tiles_out * out_weight_pct / 100.0;
+  int n_in = (int)(148.0 * wi / (wi + wo) + 0.5);
+  if (n_in < 1) n_in = 1;
+  if (n_in > 147) n_in = 147;
+  return n_in;
+}
+
+template <int K, int G>
+static int bd_launch_dual_t(cudaStream_t st, const BdMaps& mi, BdMulti pi, const BdMaps& mo, BdMulti po) {
+  constexpr int SMEM = BdCfg<BD_IN, K, G>::SMEM > BdCfg<BD_OUT, K, G>::SMEM ? BdCfg<BD_IN, K, G>::SMEM : BdCfg<BD_OUT, K, G>::SMEM;
+  static std::atomic<unsigned long long> done{0};
+  if (!opt_in_smem(bd_pass_dual_kernel<K, G>, SMEM, done)) return CAFEQ_ERR_CUDA;
+  long long ti = 0, to = 0;
+  for (int s = 0; s < pi.n; ++s) {
+    bd_fill_tiles<BD_IN, K, G>(pi.p[s]);
+    ti += (long long)pi.p[s].n_major * pi.p[s].n_minor;
+    pi.tile_end[s] = (int)ti;
+  }
+  for (int s = pi.n; s < BD_MAX_SUB; ++s) pi.tile_end[s] = (int)ti;
+  for (int s = 0; s < po.n; ++s) {
+    bd_fill_tiles<BD_OUT, K, G>(po.p[s]);
+    to += (long long)po.p[s].n_major * po.p[s].n_minor;
+    po.tile_end[s] = (int)to;
+  }
+  for (int s = po.n; s < BD_MAX_SUB; ++s) po.tile_end[s] = (int)to;
+  const int n_in = dual_split(ti, to, g_dual_pass_pct.load(std::memory_order_relaxed));
+  bd_pass_dual_kernel<K, G><<<148, BD_THREADS, SMEM, st>>>(mi, pi, mo, po, n_in);
+  return CAFEQ_OK;
+}
+
+// Input-axis and output-axis matrices of one block size and group size in ONE persistent launch (both lists
+// non-empty, each at least 148 tiles so that every CTA has work; otherwise the caller launches them separately).
+static bool bd_dual_ok(int k, int g) { return (k == 128 || k == 256) && (g == 64 || g == 128); }
+static int bd_launch_dual(cudaStream_t st, int k, int g, const BdSub* in, int n_in, const BdSub* out, int n_out) {
+  if (n_in < 1 || n_in > BD_MAX_SUB || n_out < 1 || n_out > BD_MAX_SUB || !bd_dual_ok(k, g)) return CAFEQ_ERR_INVALID_ARG;
+  BdMaps mi, mo;
+  BdMulti pi, po;
+  memset(&pi, 0, sizeof(pi));
+  memset(&po, 0, sizeof(po));
+  for (int s = 0; s < n_in; ++s) {
+    if (!make_map_bf16(&mi.x[s], in[s].X, in[s].p.d_in, in[s].p.d_out, in[s].ld, 128)) return CAFEQ_ERR_UNSUPPORTED;
+    if (!make_map_bf16(&mi.t[s], in[s].Tb, k, (long long)in[s].nbT * k, k, k)) return CAFEQ_ERR_UNSUPPORTED;
+    pi.p[s] = in[s].p;
+  }
+  for (int s = n_in; s < BD_MAX_SUB; ++s) { mi.x[s] = mi.x[0]; mi.t[s] = mi.t[0]; }
+  for (int s = 0; s < n_out; ++s) {
+    if (!make_map_bf16(&mo.x[s], out[s].X, out[s].p.d_in, out[s].p.d_out, out[s].ld, 128)) return CAFEQ_ERR_UNSUPPORTED;
+    if (!make_map_bf16(&mo.t[s], out[s].Tb, k, (long long)out[s].nbT * k, k, k)) return CAFEQ_ERR_UNSUPPORTED;
+    po.p[s] = out[s].p;
+  }
+  for (int s = n_out; s < BD_MAX_SUB; ++s) { mo.x[s] = mo.x[0]; mo.t[s] = mo.t[0]; }
+  pi.n = n_in;
+  po.n = n_out;
+#define BD_DUAL(KK, GG) \
+  if (k == KK && g == GG) return bd_launch_dual_t<KK, GG>(st, mi, pi, mo, po);
+  BD_DUAL(128, 64)
+  BD_DUAL(128, 128)
+  BD_DUAL(256, 64)
+  BD_DUAL(256, 128)
+#undef BD_DUAL
+  return CAFEQ_ERR_UNSUPPORTED;
 }
 
 // fp32 operator blocks -> bf16 in applied orientation (transposed when the role asks for T^T)

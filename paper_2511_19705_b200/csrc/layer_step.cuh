@@ -18,6 +18,7 @@
 namespace cafeq {
 
 constexpr int LY_MAX_PROBS = 8;
+static std::atomic<int> g_ly_dual{1};  // both forms of a layer in one pass launch and one backward launch
 constexpr int LY_MAX_MATS = 2 * LY_MAX_PROBS;
 
 // ------------------------------------------------------------------------------------------------
@@ -566,25 +567,18 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
       else CQ_LAUNCH(cw_out_kernel, (G.d_out + 127) / 128, 128, 0, st, L.c + (size_t)P.blk0 * k, G.d_out, G.g, k, G.r, Mt.cw);
     }
   }
-  // transform passes: all matrices of one form in one launch
-  for (int form = 0; form < 2; ++form) {
-    BdSub subs[BD_MAX_SUB];
-    int ns = 0;
-    auto flush = [&]() -> int {
-      if (!ns) return CAFEQ_OK;
-      int ti = kt_begin(5, st);
-      g_launches.fetch_add(1, std::memory_order_relaxed);
-      int rc = bd_launch_many(st, form, k, L.g, subs, ns);
-      kt_end(ti, st);
-      ns = 0;
-      return rc;
-    };
+  // transform passes: all matrices of a form in one launch, and both forms in the same launch when each has
+  // enough tiles for its share of the CTAs
+  {
+    BdSub subs[2][LY_MAX_MATS];
+    int ns[2] = {0, 0};
+    long long ntile[2] = {0, 0};
     for (int i = 0; i < L.nm; ++i) {
       const LyMat& Mt = L.m[i];
-      if ((Mt.G.axis == CAFEQ_AXIS_IN ? BD_IN : BD_OUT) != form) continue;
+      const int form = (Mt.G.axis == CAFEQ_AXIS_IN) ? BD_IN : BD_OUT;
       const LyProb& P = L.p[Mt.prob];
       const long long off = (long long)P.blk0 * kk1;
-      BdSub& s = subs[ns];
+      BdSub& s = subs[form][ns[form]++];
       memset(&s, 0, sizeof(s));
       s.X = Mt.W; s.ld = Mt.G.ld; s.nbT = P.nb;
       BdParams& p = s.p;
@@ -602,10 +596,27 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
         s.Tb = (Mt.side == 0) ? w.Qh + off : w.Xh[w.cur] + off;  // bf16(M)^T for U = W1 M, bf16(M^-1) for V = M^-1 W2
         p.epi = EPI_ABSMAX;
       }
-      if (++ns == BD_MAX_SUB) { int rc = flush(); if (rc) return rc; }
+      ntile[form] += (long long)Mt.G.n / 32768;  // tiles hold 32768 entries in both forms
     }
-    int rc = flush();
-    if (rc) return rc;
+    const bool dual = g_ly_dual.load(std::memory_order_relaxed) && ns[0] >= 1 && ns[1] >= 1 && ns[0] <= BD_MAX_SUB &&
+                      ns[1] <= BD_MAX_SUB && bd_dual_ok(k, L.g) && ntile[0] >= 148 && ntile[1] >= 148;
+    if (dual) {
+      int ti = kt_begin(5, st);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      int rc = bd_launch_dual(st, k, L.g, subs[0], ns[0], subs[1], ns[1]);
+      kt_end(ti, st);
+      if (rc) return rc;
+    } else {
+      for (int form = 0; form < 2; ++form)
+        for (int c0 = 0; c0 < ns[form]; c0 += BD_MAX_SUB) {
+          const int n = (ns[form] - c0 < BD_MAX_SUB) ? ns[form] - c0 : BD_MAX_SUB;
+          int ti = kt_begin(5, st);
+          g_launches.fetch_add(1, std::memory_order_relaxed);
+          int rc = bd_launch_many(st, form, k, L.g, subs[form] + c0, n);
+          kt_end(ti, st);
+          if (rc) return rc;
+        }
+    }
   }
   // LogSumExp of the pairs
   {
@@ -629,19 +640,22 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
     g.status = status;
     if (np) CQ_LAUNCH(layer_lse_kernel, dim3(grid_for(nmax, 256, 148 * 4), np), 256, 0, st, g);
   }
-  // sparse backward: all matrices of one (axis, orientation) in one launch, fp16 single-term form
-  for (int axis = 0; axis < 2; ++axis)
-    for (int tr = 0; tr < 2; ++tr) {
-      int list[LY_MAX_MATS], cnt = 0;
-      ly_lists(L, axis, tr, list, &cnt);
-      for (int c0 = 0; c0 < cnt; c0 += BW_MAX_SUB) {
-        BwSub subs[BW_MAX_SUB];
-        const int ns = (cnt - c0 < BW_MAX_SUB) ? cnt - c0 : BW_MAX_SUB;
-        for (int j = 0; j < ns; ++j) {
-          const LyMat& Mt = L.m[list[c0 + j]];
+  // sparse backward, fp16 single-term form: all matrices of one (axis, orientation) in one launch; when the layer has
+  // exactly one input-axis and one output-axis group, both in the same launch
+  {
+    BwSub subs[4][LY_MAX_MATS];
+    int cnt[4] = {0, 0, 0, 0};
+    long long ntile[4] = {0, 0, 0, 0};
+    for (int axis = 0; axis < 2; ++axis)
+      for (int tr = 0; tr < 2; ++tr) {
+        const int c = axis * 2 + tr;
+        int list[LY_MAX_MATS];
+        ly_lists(L, axis, tr, list, &cnt[c]);
+        for (int j = 0; j < cnt[c]; ++j) {
+          const LyMat& Mt = L.m[list[j]];
           const LyProb& P = L.p[Mt.prob];
           const long long off = (long long)P.blk0 * kk1;
-          BwSub& s = subs[j];
+          BwSub& s = subs[c][j];
           memset(&s, 0, sizeof(s));
           s.W16 = Mt.W16; s.ld = Mt.G.d_in;
           BwParams& p = s.p;
@@ -658,14 +672,35 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
             p.coefmax = L.one;   // the largest exp(t (a - max)) is 1
             p.out_div = P.acc;   // Z
           }
+          ntile[c] += (long long)Mt.G.n / (64 * k);
         }
-        int ti = kt_begin(2, st);
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-        int rc = bw_launch_many(st, axis == CAFEQ_AXIS_IN, k, tr, 1, subs, ns);
-        kt_end(ti, st);
-        if (rc) return rc;
       }
+    const int c_in0 = CAFEQ_AXIS_IN * 2, c_out0 = CAFEQ_AXIS_OUT * 2;
+    int ci = -1, co = -1;
+    bool dual = g_ly_dual.load(std::memory_order_relaxed) && bw_dual_ok(k);
+    if (cnt[c_in0] && cnt[c_in0 + 1]) dual = false;
+    if (cnt[c_out0] && cnt[c_out0 + 1]) dual = false;
+    ci = cnt[c_in0] ? c_in0 : c_in0 + 1;
+    co = cnt[c_out0] ? c_out0 : c_out0 + 1;
+    if (!cnt[ci] || !cnt[co] || cnt[ci] > BW_MAX_SUB || cnt[co] > BW_MAX_SUB || ntile[ci] < 148 * 6 || ntile[co] < 148 * 6) dual = false;
+    if (dual) {
+      int ti = kt_begin(2, st);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      int rc = bw_launch_dual(st, k, ci & 1, subs[ci], cnt[ci], co & 1, subs[co], cnt[co]);
+      kt_end(ti, st);
+      if (rc) return rc;
+    } else {
+      for (int c = 0; c < 4; ++c)
+        for (int c0 = 0; c0 < cnt[c]; c0 += BW_MAX_SUB) {
+          const int ns = (cnt[c] - c0 < BW_MAX_SUB) ? cnt[c] - c0 : BW_MAX_SUB;
+          int ti = kt_begin(2, st);
+          g_launches.fetch_add(1, std::memory_order_relaxed);
+          int rc = bw_launch_many(st, (c >> 1) == CAFEQ_AXIS_IN, k, c & 1, 1, subs[c] + c0, ns);
+          kt_end(ti, st);
+          if (rc) return rc;
+        }
     }
+  }
   // dL/dMinv of Eq. 4 for the singles, then grad -= Minv^T (dL/dMinv) Minv^T over all blocks
   if (L.pair_blk0 > 0) {
     LyGminvArgs ga;
@@ -777,6 +812,14 @@ extern "C" int cafeq_optimize_layer(const cafeq_layer_problem* probs, int n, int
   for (int it = 0; it < steps; ++it)
     if ((rc = ly_step(st, L, it, status))) return rc;
   return last_launch();
+}
+
+extern "C" int cafeq_debug_set_layer_launch(int dual, int pass_out_pct, int bwd_out_pct) {
+  if ((dual != 0 && dual != 1) || pass_out_pct > 1000 || bwd_out_pct > 1000) return CAFEQ_ERR_INVALID_ARG;
+  g_ly_dual.store(dual, std::memory_order_relaxed);
+  if (pass_out_pct > 0) g_dual_pass_pct.store(pass_out_pct, std::memory_order_relaxed);
+  if (bwd_out_pct > 0) g_dual_bwd_pct.store(bwd_out_pct, std::memory_order_relaxed);
+  return CAFEQ_OK;
 }
 
 extern "C" int cafeq_layer_debug_fallbacks(const cafeq_layer_problem* probs, int n, void* ws, size_t ws_bytes, int* count) {
