@@ -301,7 +301,7 @@ int cafeq_layer_debug_fallbacks(const cafeq_layer_problem* probs, int n, void* w
 
 /* Tuning knob of the layer step, process-wide (the paper has no counterpart; results do not depend on it).
  * dual = 1 (default): when a layer has matrices on both axes, their transform passes share one persistent launch and
- * their sparse backwards another; dual = 0: one launch per axis.  pass_out_pct / bwd_out_pct (> 0, default 150 / 120):
+ * their sparse backwards another; dual = 0: one launch per axis.  pass_out_pct / bwd_out_pct (> 0, default 130 / 80):
  * cost of an output-axis tile in percent of an input-axis tile of the same bytes, which sets how the 148 CTAs of a
  * shared launch are divided between the two lists; <= 0 keeps the current value.  Returns CAFEQ_ERR_INVALID_ARG
  * unless dual is 0 or 1 and the percentages are at most 1000. */

@@ -890,7 +890,7 @@ static int bd_launch_many(cudaStream_t st, int form, int k, int g, const BdSub* 
 
 // relative cost of an output-axis tile against an input-axis tile of the same bytes (measured per-tile times of
 // the two forms): sets how the CTAs of a dual launch are divided
-static std::atomic<int> g_dual_pass_pct{150}, g_dual_bwd_pct{120};
+static std::atomic<int> g_dual_pass_pct{130}, g_dual_bwd_pct{80};
 
 static int dual_split(long long tiles_in, long long tiles_out, int out_weight_pct) {
   const double wi = (double)tiles_in, wo = (double)tiles_out * out_weight_pct / 100.0;

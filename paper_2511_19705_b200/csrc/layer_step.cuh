@@ -487,6 +487,31 @@ static int ly_plan(const cafeq_layer_problem* probs, int n, void* ws, size_t ws_
   return CAFEQ_OK;
 }
 
+// Side stream of the layer step with its fork / join events, one set per host thread and device (two threads that
+// enqueue steps on the same device must not share the events), created on first use.
+struct LyAux {
+  cudaStream_t stream;
+  cudaEvent_t fork, join;
+};
+static LyAux* ly_aux() {
+  static thread_local LyAux slots[64];
+  static thread_local bool made[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!made[dev]) {
+    LyAux a;
+    if (cudaStreamCreateWithFlags(&a.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&a.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&a.join, cudaEventDisableTiming) != cudaSuccess)
+      return nullptr;
+    slots[dev] = a;
+    made[dev] = true;
+  }
+  return &slots[dev];
+}
+// block sizes whose inverse refinement runs on row-major arrays (the transposed split arrays are then free)
+static bool w_mn_expected(int k) { return g_tb_enable.load(std::memory_order_relaxed) && tb_supported(k, 2); }
+
 static void ly_lists(const LyPlan& L, int axis, int transpose, int* out, int* cnt) {
   // matrices whose backward shares (axis, output orientation): singles store gradT plainly, a pair's first factor
   // (operator M^T) stores it transposed, its second factor feeds dL/dMinv plainly
@@ -524,21 +549,36 @@ static int ly_step(cudaStream_t st, LyPlan& L, int hist_row, int32_t* status) {
   }
   bool any_lambda = false;
   for (int q = 0; q < L.n; ++q) any_lambda |= (L.p[q].pair && L.p[q].cfg.lambda_orth != 0.f);
+  // The pair blocks' penalty chain (splits of the parameters, R = M M^T - I, R M) does not depend on the inverse:
+  // it runs on a side stream beside the Newton-Schulz chain (both are chains of short, latency-bound launches that
+  // leave SMs idle) and joins before the transform pass, which reads bf16(M)^T.  Event record / wait pairs only, so
+  // the fork and the join are captured with the step when the caller's stream is being captured.
+  LyAux* aux = (nbP > 0 && g_ly_dual.load(std::memory_order_relaxed) && w_mn_expected(k)) ? ly_aux() : nullptr;
+  cudaStream_t so = st;
+  if (aux) {
+    if (cudaEventRecord(aux->fork, st) != cudaSuccess || cudaStreamWaitEvent(aux->stream, aux->fork, 0) != cudaSuccess) return CAFEQ_ERR_CUDA;
+    so = aux->stream;
+  }
   if (nbP > 0) {
     // pair blocks: splits of the fp32 parameters (the transposed high halves are bf16(M)^T, the operator of the
-    // first factors' pass), R = M M^T - I with ||R_b||_F^2 per block, and R M for the penalty's gradient
-    launch_split(st, L.Mf, k, (long long)nbP * kk1, w.Ph + offP, w.Pl + offP, w.Qh + offP, w.Ql + offP, nullptr, status);
+    // first factors' pass), R = M M^T - I with ||R_b||_F^2 per block, and R M for the penalty's gradient.
+    // On the side stream R's splits live in the transposed-split arrays, which the row-major refinement leaves unused
+    // (the Newton-Schulz chain writes its own residual into RTh meanwhile).
+    uint16_t* Rh = (aux ? w.XTh[0] : w.RTh) + offP;
+    uint16_t* Rl = (aux ? w.XTl[0] : w.RTl) + offP;
+    launch_split(so, L.Mf, k, (long long)nbP * kk1, w.Ph + offP, w.Pl + offP, w.Qh + offP, w.Ql + offP, nullptr, status);
     const uint16_t* a1[3] = {w.Ph + offP, w.Pl + offP, w.Ph + offP};
     const uint16_t* b1[3] = {w.Ph + offP, w.Ph + offP, w.Pl + offP};
-    launch_kk_tc(st, 3, a1, b1, nbP, k, 1.f, 0.f, -1.f, nullptr, nullptr, w.RTh + offP, w.RTl + offP, nullptr, nullptr, L.orth_sq,
-                 nullptr, status, 1);
+    launch_kk_tc(so, 3, a1, b1, nbP, k, 1.f, 0.f, -1.f, nullptr, nullptr, Rh, Rl, nullptr, nullptr, L.orth_sq, nullptr, status, 1);
     if (any_lambda) {
-      const uint16_t* a2[3] = {w.RTh + offP, w.RTl + offP, w.RTh + offP};
+      const uint16_t* a2[3] = {Rh, Rl, Rh};
       const uint16_t* b2[3] = {w.Qh + offP, w.Qh + offP, w.Ql + offP};
-      launch_kk_tc(st, 3, a2, b2, nbP, k, 1.f, 0.f, 0.f, nullptr, L.RM, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, status);
+      launch_kk_tc(so, 3, a2, b2, nbP, k, 1.f, 0.f, 0.f, nullptr, L.RM, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, status);
     }
   }
+  if (aux && cudaEventRecord(aux->join, aux->stream) != cudaSuccess) return CAFEQ_ERR_CUDA;
   ns_inverse(st, L.Mc, L.Minv, nullptr, NB, k, true, w, status, true, true);
+  if (aux && cudaStreamWaitEvent(st, aux->join, 0) != cudaSuccess) return CAFEQ_ERR_CUDA;
   // Eq. 4 weights of the single matrices (they own the first pair_blk0 blocks)
   if (L.pair_blk0 > 0) {
     LyColArgs ca;
