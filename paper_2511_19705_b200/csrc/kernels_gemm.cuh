@@ -347,12 +347,14 @@ struct TbMaps {
   CUtensorMap b[TB_MAX_ARR];
   CUtensorMap c0, c;    // fp32 [nb * k, k], box 32 x 32, 128-byte swizzle
   CUtensorMap chi, clo; // bf16 [nb * k, k], box 32 x 32, 64-byte swizzle
+  CUtensorMap chl;      // hi and lo as the two planes of one 3-D view (when lo lies a fixed distance after hi): one store
 };
 struct TbTerms {
   int na, nb;                 // distinct A / B arrays
   int nterms;
   int ta[TG_MAX_TERMS], tb[TG_MAX_TERMS];  // term t multiplies a[ta[t]] by b[tb[t]]
   int a_mn, b_mn;             // the A / B arrays are stored [l][m] / [l][n] (MN-major operands)
+  int hl3d;                   // Chi and Clo are stored with one 3-D bulk copy through maps.chl
 };
 
 template <int K>
@@ -371,6 +373,11 @@ struct TbCfg {
 __device__ __forceinline__ void fence_proxy_async_smem_tb() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y),
+               "r"(z)
                : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
@@ -407,8 +414,11 @@ tc_block_kernel(const __grid_constant__ TbMaps maps, const TbTerms tt, const TgP
   if (threadIdx.x == 32) {
     if (p.C0) tma_prefetch_desc(&maps.c0);
     if (p.C) tma_prefetch_desc(&maps.c);
-    if (p.Chi) tma_prefetch_desc(&maps.chi);
-    if (p.Clo) tma_prefetch_desc(&maps.clo);
+    if (tt.hl3d) tma_prefetch_desc(&maps.chl);
+    else {
+      if (p.Chi) tma_prefetch_desc(&maps.chi);
+      if (p.Clo) tma_prefetch_desc(&maps.clo);
+    }
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::NSLOT; ++s) {
@@ -514,18 +524,6 @@ tc_block_kernel(const __grid_constant__ TbMaps maps, const TbTerms tt, const TgP
         tile_of(i, mh, ch);
         const int row0 = b * K + mh * 128 + q * 32, col0 = ch * 32;
         const uint32_t tCi = tC + (uint32_t)(i & 1) * 4096;
-        if (lane == 0) {
-          // the stores of the previous tile have read their shared memory (the other fp32 buffer and hi / lo)
-          tma_store_wait_read();
-          if (p.C0 && i + 1 < NU) {
-            int mh2, ch2;
-            tile_of(i + 1, mh2, ch2);
-            const uint32_t bn = bc0 + 8 * ((i + 1) & 1);
-            mbar_expect_tx(bn, 4096);
-            tma_load_2d(tC + (uint32_t)((i + 1) & 1) * 4096, &maps.c0, ch2 * 32, b * K + mh2 * 128 + q * 32, bn);
-          }
-        }
-        __syncwarp();
         float v[32];
         tc_ld32(taddr + mh * K + ch * 32, v);
 #pragma unroll
@@ -554,6 +552,20 @@ tc_block_kernel(const __grid_constant__ TbMaps maps, const TbTerms tt, const TgP
 #pragma unroll
           for (int e = 0; e < 32; ++e) sq4[e & 3] = fmaf(v[e], v[e], sq4[e & 3]);
         }
+        // Only now, with this tile's values in registers: wait until the stores of the previous tile have read their
+        // shared memory (the other fp32 buffer, hi, lo), then fetch the next C0 tile into that other buffer (it is needed
+        // one tile from now).
+        if (lane == 0) {
+          tma_store_wait_read();
+          if (p.C0 && i + 1 < NU) {
+            int mh2, ch2;
+            tile_of(i + 1, mh2, ch2);
+            const uint32_t bn = bc0 + 8 * ((i + 1) & 1);
+            mbar_expect_tx(bn, 4096);
+            tma_load_2d(tC + (uint32_t)((i + 1) & 1) * 4096, &maps.c0, ch2 * 32, b * K + mh2 * 128 + q * 32, bn);
+          }
+        }
+        __syncwarp();
         if (p.C) {
 #pragma unroll
           for (int c = 0; c < 8; ++c)
@@ -588,8 +600,12 @@ tc_block_kernel(const __grid_constant__ TbMaps maps, const TbTerms tt, const TgP
         __syncwarp();
         if (lane == 0) {
           if (p.C) tma_store_2d(&maps.c, tCi, col0, row0);
-          if (p.Chi) tma_store_2d(&maps.chi, tH, col0, row0);
-          if (p.Clo) tma_store_2d(&maps.clo, tL, col0, row0);
+          if (tt.hl3d) {
+            tma_store_3d(&maps.chl, tH, col0, row0, 0);  // the lo tile follows the hi tile in shared memory
+          } else {
+            if (p.Chi) tma_store_2d(&maps.chi, tH, col0, row0);
+            if (p.Clo) tma_store_2d(&maps.clo, tL, col0, row0);
+          }
           tma_store_commit();
         }
       }
@@ -712,6 +728,16 @@ static int tb_launch(cudaStream_t st, int nterms, const uint16_t* const* A, cons
   if (p.Clo) okm = okm && make_map_2d(&maps.clo, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.Clo, k, rowsC, k, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
   if (!okm) return CAFEQ_ERR_UNSUPPORTED;
   if (p.Clo && !p.Chi) return CAFEQ_ERR_UNSUPPORTED;
+  if (p.Chi && p.Clo && p.Clo > p.Chi && (((uintptr_t)p.Clo - (uintptr_t)p.Chi) & 15) == 0) {
+    EncodeTiledFn enc = get_encode_tiled();
+    cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rowsC, 2};
+    cuuint64_t strides[2] = {(cuuint64_t)k * 2, (cuuint64_t)((uintptr_t)p.Clo - (uintptr_t)p.Chi)};
+    cuuint32_t box[3] = {32, 32, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (enc && enc(&maps.chl, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, p.Chi, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+      tt.hl3d = 1;
+  }
   return k == 256 ? tb_launch_t<256>(st, maps, tt, p) : tb_launch_t<128>(st, maps, tt, p);
 }
 
