@@ -313,9 +313,10 @@ __global__ void colnorm_kernel(const float* __restrict__ X, int k, int nb, float
 
 static void launch_split(cudaStream_t st, const float* X, int k, long long n, uint16_t* hi, uint16_t* lo, uint16_t* thi,
                          uint16_t* tlo, const int* run_flag, const int32_t* status, const double* gate = nullptr,
-                         double gate_tol = 0.0) {
+                         double gate_tol = 0.0, int parity_iters = 0, int parity_nb = 0) {
   dim3 grid(k / 32, k / 32, (unsigned)(n / ((long long)k * k)));
-  CQ_LAUNCH(split_bf16_kernel, grid, dim3(32, 8), 0, st, X, k, hi, lo, thi, tlo, run_flag, status, gate, gate_tol);
+  CQ_LAUNCH(split_bf16_kernel, grid, dim3(32, 8), 0, st, X, k, hi, lo, thi, tlo, run_flag, status, gate, gate_tol, parity_iters,
+            parity_nb);
 }
 
 // Minv = inv(bf16(M)) by Newton-Schulz iteration X <- X + X (I - A X) on the tensor cores, from X0 = A^T
@@ -378,9 +379,15 @@ static void ns_inverse(cudaStream_t st, const float* Mc, float* X, float* cnorm,
   launch_inverse(st, Mc, X, nullptr, nb, k, status, w.rn + (size_t)(iters - 1) * nb, 1e-4, w.flag, w.redo_total);
   // final splits: written by the last iteration's epilogue, except for blocks that skipped it (and for everything
   // when the elimination recomputed a block)
-  const double* last_gate = (warm && iters > 1) ? w.rn + (size_t)(iters - 2) * nb : nullptr;
-  launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], mn ? nullptr : w.XTh[cur], mn ? nullptr : w.XTl[cur], w.flag, status, last_gate,
-               NS_GATE2);
+  if (mn) {
+    // every iteration writes both row-major splits, so a block that stopped early needs this only when its newest
+    // splits are in the other set
+    launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], nullptr, nullptr, w.flag, status, (warm && iters > 1) ? w.rn : nullptr, NS_GATE2,
+                 iters, nb);
+  } else {
+    const double* last_gate = (warm && iters > 1) ? w.rn + (size_t)(iters - 2) * nb : nullptr;
+    launch_split(st, X, k, kk, w.Xh[cur], w.Xl[cur], w.XTh[cur], w.XTl[cur], w.flag, status, last_gate, NS_GATE2);
+  }
   if (cnorm) {
     dim3 grid((k + 127) / 128, nb);
     CQ_LAUNCH(colnorm_kernel, grid, 128, 0, st, X, k, nb, cnorm);

@@ -746,12 +746,25 @@ static int tb_launch(cudaStream_t st, int nterms, const uint16_t* const* A, cons
 __global__ void __launch_bounds__(256) split_bf16_kernel(const float* __restrict__ X, int k, uint16_t* __restrict__ hi,
                                                          uint16_t* __restrict__ lo, uint16_t* __restrict__ thi,
                                                          uint16_t* __restrict__ tlo, const int* run_flag, const int32_t* status,
-                                                         const double* gate = nullptr, double gate_tol = 0.0) {
+                                                         const double* gate = nullptr, double gate_tol = 0.0,
+                                                         int parity_iters = 0, int parity_nb = 0) {
   // runs for every block by default; with run_flag and / or gate: only when *run_flag != 0, or for the blocks
-  // with gate[block] <= gate_tol
+  // with gate[block] <= gate_tol.  parity_iters > 0: `gate` is the base of the residual table [iteration][block] of
+  // a gated iteration that writes its splits alternately into two sets; the block is split again only when the
+  // number of iterations it ran (iteration i runs iff the residual of iteration i - 1 exceeds gate_tol) left its
+  // newest splits in the other set than parity_iters iterations would have.
   if (status && *status) return;
   if (run_flag || gate) {
-    const bool run = (run_flag && *run_flag != 0) || (gate && gate[blockIdx.z] <= gate_tol);
+    bool run = run_flag && *run_flag != 0;
+    if (!run && gate) {
+      if (parity_iters > 0) {
+        int ran = 1;
+        while (ran < parity_iters && gate[(size_t)(ran - 1) * parity_nb + blockIdx.z] > gate_tol) ++ran;
+        run = ((ran ^ parity_iters) & 1) != 0;
+      } else {
+        run = gate[blockIdx.z] <= gate_tol;
+      }
+    }
     if (!run) return;
   }
   __shared__ uint32_t tile[32][33];
