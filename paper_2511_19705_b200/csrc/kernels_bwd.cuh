@@ -255,14 +255,20 @@ __device__ __forceinline__ void bd_bwd_body(const BwMaps& maps, const BwMulti& m
     // ---------------------------------------------------------------- operand builders (one record per thread and tile) and flush
     const int bt = threadIdx.x - 64;
     const int q = warp & 3, hw = (warp - 2) >> 2;
-    float cfN = 0.f;
-    int tgN = -1, kkN = 0;
+    // The record of the NEXT tile is requested one tile ahead and only its raw words are kept: nothing may depend on
+    // them before the next iteration, or the thread would sit out the whole memory latency here, once per tile.
+    float rawC = 0.f;     // coefficient word
+    int rawI = 0;         // arg-max word
+    int rawBase = -1;     // input axis: column offset of this thread's group inside the block; output axis: first
+                          // column of the group minus the tile's first column; -1: no record for this thread
+    int rawKK = 0;        // input axis: contraction index (row inside the tile); output axis: target row
+    float rawScale = 1.f;
     auto load_rec = [&](int sub, int tile) {
       const BwParams& p = mp.p[sub];
       const int major = tile / p.n_minor, t = tile - major * p.n_minor;
-      cfN = 0.f;
-      tgN = -1;
-      kkN = 0;
+      rawBase = -1;
+      rawC = 0.f;
+      rawI = 0;
       if constexpr (FORM == BW_IN) {
         const int rl = bt & 63, qq = bt >> 6;
         const int row = t * 64 + rl;
@@ -270,29 +276,38 @@ __device__ __forceinline__ void bd_bwd_body(const BwMaps& maps, const BwMulti& m
         const int G = G0 + qq;
         if (qq < p.NG && row < p.d_out && G < p.ng) {
           const long long pi = p.gm ? (long long)G * p.d_out + row : (long long)row * p.ng + G;
-          const float c = __ldg(p.coef + pi);
-          const int col = qq * p.g + __ldg(p.idx + pi) + (G0 * p.g - major * K);
-          if (c != 0.f && (unsigned)col < (unsigned)K) {
-            cfN = c;
-            tgN = col;
-            kkN = rl;
-          }
+          rawC = __ldg(p.coef + pi);
+          rawI = __ldg(p.idx + pi);
+          rawBase = qq * p.g + (G0 * p.g - major * K) + (1 << 20);  // kept non-negative: the offset can be below zero
+          rawKK = rl;
         }
       } else {
         if (bt < K) {
           const int row = major * K + bt;
           const int G = (t * 64) / p.g;
           const long long pi = p.gm ? (long long)G * p.d_out + row : (long long)row * p.ng + G;
-          const float c = __ldg(p.coef + pi);
-          const int col = G * p.g + __ldg(p.idx + pi) - t * 64;
-          if (c != 0.f && (unsigned)col < 64u) {
-            cfN = c;
-            tgN = bt;
-            kkN = col;
-          }
+          rawC = __ldg(p.coef + pi);
+          rawI = __ldg(p.idx + pi);
+          rawBase = G * p.g - t * 64 + (1 << 20);
+          rawKK = bt;
         }
       }
-      if constexpr (F16) cfN *= bw_coef_scale(p.coefmax);
+      if constexpr (F16) rawScale = bw_coef_scale(p.coefmax);
+    };
+    // the record requested one iteration ago, decoded: coefficient, target row, contraction index (tg < 0: none)
+    auto take_rec = [&](float& cf, int& tg, int& kk) {
+      cf = 0.f;
+      tg = -1;
+      kk = 0;
+      if (rawBase >= 0) {
+        const int col = rawBase - (1 << 20) + rawI;
+        if constexpr (FORM == BW_IN) {
+          if (rawC != 0.f && (unsigned)col < (unsigned)K) { cf = rawC; tg = col; kk = rawKK; }
+        } else {
+          if (rawC != 0.f && (unsigned)col < 64u) { cf = rawC; tg = rawKK; kk = col; }
+        }
+      }
+      if constexpr (F16) cf *= rawScale;
     };
     // flush of one block: accumulators -> global memory, coalesced atomic adds straight from the registers
     // (accumulator row m = this thread's lane, 32 consecutive columns n per load)
@@ -333,8 +348,9 @@ __device__ __forceinline__ void bd_bwd_body(const BwMaps& maps, const BwMulti& m
       while (gt >= mp.tile_end[sub]) ++sub;
       const int tile = gt - (sub ? mp.tile_end[sub - 1] : 0);
       const int major = tile / mp.p[sub].n_minor;
-      const float cf = cfN;
-      const int tg = tgN, kk = kkN;
+      float cf;
+      int tg, kk;
+      take_rec(cf, tg, kk);
       if (gt + 1 < t_end) {
         int sn = sub;
         while (gt + 1 >= mp.tile_end[sn]) ++sn;
