@@ -249,6 +249,26 @@ int cafeq_adaptive_round(const cafeq_matrix_desc* d1, const void* W1, const cafe
  * library's.  d_in*bits must be a multiple of 8. */
 int cafeq_pack(const cafeq_matrix_desc* d, const int8_t* codes, uint8_t* packed, void* stream);
 
+/* ---- inference side (Section 4.1's cost argument and its table of extra FLOPs / wall-clock time) -------------
+ * A matrix quantised as Q(W o T) on its input axis is used as  y = W x = (W o T) (T^-T x): the activations are
+ * multiplied by the block-diagonal inverse before the (dequantised) matrix product.  cafeq_apply_transform does that
+ * multiplication on a bf16 activation matrix X [d_out = tokens, d_in] (row pitch d->ld):
+ *     Y[o, B k + i] = sum_j P[B][i][j] X[o, B k + j],   P = T (d->trole = CAFEQ_APPLY_T) or T^T (CAFEQ_APPLY_TT),
+ * (CAFEQ_AXIS_OUT: the operator acts on the row index instead), with the operator rounded to bf16, fp32
+ * accumulation, and Y written as bf16 [d_out, d_in], dense (row pitch d_in).  T: fp32 [d_in / k, k, k] on the device.
+ * d->group and d->bits are not used.  Shapes the tensor-core pass covers (k in {64, 128, 256}, d_in a multiple of
+ * 256, 16-byte aligned rows) run in one kernel; all others on the shape-agnostic kernels with an fp32 copy of Y in
+ * the workspace.  Workspace: cafeq_apply_workspace_size bytes (sized for 16-byte aligned rows; CAFEQ_ERR_WORKSPACE
+ * otherwise).  Device status word as elsewhere (may be NULL). */
+int cafeq_apply_workspace_size(const cafeq_matrix_desc* d, size_t* bytes);
+int cafeq_apply_transform(const cafeq_matrix_desc* d, const void* X, const float* T, void* Y, int32_t* status, void* ws,
+                          size_t ws_bytes, void* stream);
+
+/* Unpack the bit stream written by cafeq_pack and dequantise: What[o, c] = bf16(scales[o, c / group] * q[o, c]),
+ * What bf16 [d_out, d_in] with row pitch ldo >= d_in (elements).  d_in must be a multiple of 8. */
+int cafeq_dequant(const cafeq_matrix_desc* d, const uint8_t* packed, const float* scales, void* What, long long ldo,
+                  void* stream);
+
 /* ---- one decoder layer at a time --------------------------------------------------------------------------
  * Section 6 quantises a model layer by layer; within a layer every matrix (block-diagonal transform, Section 4.1)
  * and every coupled pair (Section 4.2) is an independent optimisation problem.  The calls below advance all

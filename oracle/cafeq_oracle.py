@@ -767,3 +767,24 @@ def unpack_codes(p, bits: int, d_in: int):
             pos = i * bits + b
             u[:, i] |= ((p[:, pos // 8].astype(np.int64) >> (pos % 8)) & 1) << b
     return (u - qmax_of(bits)).astype(np.int32)
+
+
+# ---------------------------------------------------------------------------
+# inference side (Section 4.1: the transform is undone on the activations; the table of extra FLOPs / time)
+# ---------------------------------------------------------------------------
+def inference_apply(X, T, axis: str = "in", transpose: bool = False):
+    """The activation-side multiplication that goes with a matrix quantised as Q(W o T) on its input axis:
+    y = W x = (W o T)(T^-T x), so the activations X [tokens, d_in] are sent through P = T^-T, i.e. the inverse's
+    blocks applied transposed.  This function applies a given block operator P = T (or T^T with transpose=True),
+    rounded to bf16 as deployed, on the chosen axis in float64."""
+    P = round_bf16(np.asarray(T, dtype=np.float32)).astype(np.float64)
+    if transpose:
+        P = np.transpose(P, (0, 2, 1))
+    return apply_blocks(np.asarray(X, dtype=np.float64), P, axis, 1)
+
+
+def dequant(packed, scales, bits: int, group: int, d_in: int):
+    """What = scale * code from the packed stream (the layout of pack_codes) and the per-group scales [d_out, d_in/group]."""
+    q = unpack_codes(packed, bits, d_in).astype(np.float64)
+    s = np.repeat(np.asarray(scales, dtype=np.float64), group, axis=1)
+    return s * q

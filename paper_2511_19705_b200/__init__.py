@@ -26,7 +26,7 @@ ROUND_ALG1, ROUND_LEARNED_OFFSETS = 0, 1
 EXPORTS = [
     "cafeq_workspace_size", "cafeq_rtn", "cafeq_rtn_workspace_size", "cafeq_rtn_noalloc", "cafeq_proxy_loss_fwd_bwd", "cafeq_optimize_single",
     "cafeq_pair_product", "cafeq_pair_loss_fwd_bwd", "cafeq_optimize_pair", "cafeq_adaptive_round",
-    "cafeq_pack", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_layer_debug_fallbacks", "cafeq_debug_set_layer_launch", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
+    "cafeq_pack", "cafeq_apply_workspace_size", "cafeq_apply_transform", "cafeq_dequant", "cafeq_layer_workspace_size", "cafeq_layer_prepare", "cafeq_optimize_layer", "cafeq_layer_debug_fallbacks", "cafeq_debug_set_layer_launch", "cafeq_set_overlap_mode", "cafeq_debug_wait_probe", "cafeq_debug_timer_begin", "cafeq_debug_timer_read",
     "cafeq_debug_launch_count",
     "cafeq_status_string", "cafeq_version",
 ]
@@ -349,6 +349,33 @@ def cafeq_pack(codes, *, bits):
     rc = lib().cafeq_pack(ctypes.byref(d), _p(codes), _p(packed), _stream())
     _check(rc, "cafeq_pack")
     return packed
+
+
+def cafeq_apply_transform(X, T, *, taxis=AXIS_IN, trole=APPLY_T, status=None):
+    """Y = P o X on one axis of a bf16 activation matrix X [tokens, d_in] (P = T or T^T, rounded to bf16): the
+    inference-side multiplication by the block-diagonal inverse.  Returns bf16 Y [tokens, d_in]."""
+    if X.dtype != torch.bfloat16 or not X.is_cuda or X.stride(1) != 1:
+        raise ValueError("X must be a CUDA bf16 matrix with unit column stride")
+    d_out, d_in = X.shape
+    k = T.shape[-1]
+    d = make_desc(d_out, d_in, 4, 128 if d_in % 128 == 0 else d_in, k, taxis, trole, 1, X.stride(0))
+    n = ctypes.c_size_t(0)
+    _check(lib().cafeq_apply_workspace_size(ctypes.byref(d), ctypes.byref(n)), "cafeq_apply_workspace_size")
+    ws = torch.empty(max(int(n.value), 256), dtype=torch.uint8, device=X.device)
+    Y = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=X.device)
+    rc = lib().cafeq_apply_transform(ctypes.byref(d), _p(X), _p(T), _p(Y), _p(status), _p(ws), ctypes.c_size_t(ws.numel()), _stream())
+    _check(rc, "cafeq_apply_transform")
+    return Y
+
+
+def cafeq_dequant(packed, scales, *, bits, group, d_in):
+    """bf16 [d_out, d_in] = scales * codes from the bit stream of cafeq_pack."""
+    d_out = packed.shape[0]
+    d = make_desc(d_out, d_in, bits, group)
+    out = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=packed.device)
+    rc = lib().cafeq_dequant(ctypes.byref(d), _p(packed), _p(scales), _p(out), ctypes.c_longlong(d_in), _stream())
+    _check(rc, "cafeq_dequant")
+    return out
 
 
 # ----------------------------------------------------------------------------- one layer at a time

@@ -832,6 +832,74 @@ extern "C" int cafeq_rtn(const cafeq_matrix_desc* d, const void* W, const float*
 }
 
 // ------------------------------------------------------------------------------------------------
+// inference side: apply a block-diagonal operator to activations, dequantise packed weights
+// ------------------------------------------------------------------------------------------------
+static size_t apply_scratch(const Geo& G, bool fused) {
+  const size_t kk = (size_t)G.nbT * G.k * G.k;
+  return 1024 + kk * 6 + (fused ? 0 : (size_t)G.n * 4 + 256);
+}
+static Geo apply_geo(Geo G) {
+  // the store epilogue ignores the quantisation groups: any group width the pass is built for will do
+  if (G.d_in % 128 == 0) { G.g = 128; G.ng = G.d_in / 128; }
+  return G;
+}
+
+extern "C" int cafeq_apply_workspace_size(const cafeq_matrix_desc* d, size_t* bytes) {
+  Geo G;
+  int rc = make_geo(d, &G, false);
+  if (rc) return rc;
+  if (!bytes || G.k <= 0) return CAFEQ_ERR_INVALID_ARG;
+  const Geo Ga = apply_geo(G);
+  // (X itself is not known here: 16-byte aligned rows are assumed; a call whose X does not qualify returns
+  // CAFEQ_ERR_WORKSPACE)
+  const bool fused = bd_supported(G.axis == CAFEQ_AXIS_IN ? BD_IN : BD_OUT, Ga.d_out, Ga.d_in, Ga.ld, Ga.k, Ga.g, nullptr);
+  *bytes = apply_scratch(G, fused);
+  return CAFEQ_OK;
+}
+
+extern "C" int cafeq_apply_transform(const cafeq_matrix_desc* d, const void* X, const float* T, void* Y, int32_t* status, void* ws,
+                                     size_t ws_bytes, void* stream) {
+  Geo G;
+  int rc = make_geo(d, &G, false);
+  if (rc) return rc;
+  if (!X || !T || !Y || G.k <= 0) return CAFEQ_ERR_INVALID_ARG;
+  if ((rc = check_ws(ws, ws_bytes))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const long long kk = (long long)G.nbT * G.k * G.k;
+  Bump b(ws, ws_bytes);
+  float* Tc = b.take<float>(kk);
+  uint16_t* Tb = b.take<uint16_t>(kk);
+  if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  // the deployed operator is the bf16 rounding of the given one (what the tensor cores apply)
+  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, T, Tc, kk, nullptr);
+  const int transposed = d->trole == CAFEQ_APPLY_TT;
+  {
+    const Geo Ga = apply_geo(G);
+    BdParams p;
+    memset(&p, 0, sizeof(p));
+    p.epi = EPI_STORE;
+    p.delta = reinterpret_cast<uint16_t*>(Y);
+    if (fused_pass(st, X, G.ld, Ga, Tc, transposed, Tb, p, status, nullptr)) return last_launch();
+  }
+  float* U = b.take<float>(G.n);
+  if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  launch_apply(st, X, 1, G.ld, G, Tc, transposed, U, G.d_in, GEMM_STORE, nullptr, status);
+  CQ_LAUNCH(f32_to_bf16_kernel, grid_for(G.n), 256, 0, st, U, reinterpret_cast<uint16_t*>(Y), (long long)G.n);
+  return last_launch();
+}
+
+extern "C" int cafeq_dequant(const cafeq_matrix_desc* d, const uint8_t* packed, const float* scales, void* What, long long ldo,
+                             void* stream) {
+  Geo G;
+  int rc = make_geo(d, &G, false);
+  if (rc) return rc;
+  if (!packed || !scales || !What || ldo < G.d_in || (G.d_in % 8)) return CAFEQ_ERR_INVALID_ARG;
+  CQ_LAUNCH(dequant_kernel, grid_for(G.n / 8), 256, 0, (cudaStream_t)stream, packed, scales, reinterpret_cast<uint16_t*>(What), G.d_out,
+            G.d_in, d->bits, G.g, ldo);
+  return last_launch();
+}
+
+// ------------------------------------------------------------------------------------------------
 // single matrix forward + backward
 // ------------------------------------------------------------------------------------------------
 namespace cafeq {

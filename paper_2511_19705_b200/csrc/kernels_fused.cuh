@@ -26,7 +26,7 @@
 namespace cafeq {
 
 enum { BD_IN = 0, BD_OUT = 1 };
-enum { EPI_ABSMAX = 1, EPI_DELTA = 2, EPI_CODES = 4, EPI_SQSUM = 8, EPI_SURR = 16 };
+enum { EPI_ABSMAX = 1, EPI_DELTA = 2, EPI_CODES = 4, EPI_SQSUM = 8, EPI_SURR = 16, EPI_STORE = 32 };
 
 struct BdParams {
   int d_out, d_in;     // shape of X
@@ -40,7 +40,7 @@ struct BdParams {
   float* a;            // [d_in / G, d_out] group absmax
   float* usel;         // signed value at the arg-max
   int* idx;            // arg-max position inside the group
-  uint16_t* delta;     // bf16 [d_out, d_in], row stride d_in
+  uint16_t* delta;     // bf16 [d_out, d_in], row stride d_in (EPI_STORE: U itself is written here instead of the residual)
   uint16_t* delta_lo;  // optional second bf16 term of the residual (delta + delta_lo carries 16 mantissa bits)
   int8_t* codes;       // [d_out, d_in]
   float* scales;       // [d_out, d_in / G]
@@ -485,7 +485,23 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
       int bidx[NG];
 #pragma unroll
       for (int gi = 0; gi < NG; ++gi) { best[gi] = -1.f; bval[gi] = 0.f; bidx[gi] = 0; }
-      if (p.epi == EPI_SQSUM) {
+      if (p.epi == EPI_STORE) {
+        // the transformed matrix itself, rounded to bf16 (inference-side apply of a block-diagonal operator)
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          tc_ld32(taddr + ch * 32, v);
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2)
+            pk[e >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e])) |
+                         ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[e + 1])) << 16);
+          if (valid) {
+            uint4* dst = reinterpret_cast<uint4*>(p.delta + (long long)row * p.d_in + col0 + ch * 32);
+#pragma unroll
+            for (int w4 = 0; w4 < 4; ++w4) dst[w4] = make_uint4(pk[4 * w4], pk[4 * w4 + 1], pk[4 * w4 + 2], pk[4 * w4 + 3]);
+          }
+        }
+      } else if (p.epi == EPI_SQSUM) {
         // sum of squares only (second pass of the l2 proxy)
         float sq4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll

@@ -1248,6 +1248,36 @@ __global__ void pack_kernel(const int8_t* __restrict__ codes, uint8_t* __restric
   }
 }
 
+// The inverse of pack_kernel followed by the dequantisation: out[row][c] = bf16(scale(row, c / g) * (field - qmax)),
+// one thread per 8 consecutive codes (`bits` bytes of the stream); cols % 8 == 0, out row pitch ldo elements.
+__global__ void __launch_bounds__(256) dequant_kernel(const uint8_t* __restrict__ packed, const float* __restrict__ scales,
+                                                      uint16_t* __restrict__ out, int rows, int cols, int bits, int g, long long ldo) {
+  const long long chunks_per_row = cols / 8;
+  const long long n = (long long)rows * chunks_per_row;
+  const int qmax = (1 << (bits - 1)) - 1;
+  const unsigned mask = (1u << bits) - 1u;
+  const int ng = cols / g;
+  for (long long c = blockIdx.x * (long long)blockDim.x + threadIdx.x; c < n; c += (long long)gridDim.x * blockDim.x) {
+    const long long row = c / chunks_per_row, ch = c - row * chunks_per_row;
+    const uint8_t* src = packed + row * ((long long)cols * bits / 8) + ch * bits;
+    unsigned long long v = 0;
+    for (int b = 0; b < bits; ++b) v |= (unsigned long long)src[b] << (8 * b);
+    uint16_t* dst = out + row * ldo + ch * 8;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int col = (int)ch * 8 + i;
+      const float s = __ldg(scales + row * ng + col / g);
+      const int q = (int)((v >> (bits * i)) & mask) - qmax;
+      dst[i] = __bfloat16_as_ushort(__float2bfloat16_rn(s * (float)q));
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) f32_to_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, long long n) {
+  for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x)
+    out[e] = __bfloat16_as_ushort(__float2bfloat16_rn(in[e]));
+}
+
 // The same stream, 32 codes per thread: 32 b-bit fields are exactly b 32-bit words, so a thread reads two 16-byte
 // vectors of codes and writes whole words (cols % 32 == 0, codes 16-byte aligned, packed 4-byte aligned).
 template <int BITS>

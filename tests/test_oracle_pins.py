@@ -675,3 +675,53 @@ def test_cayley_step_pins():
     C = rng.standard_normal(M.shape)
     M2, _ = orc.cayley_step(M, C, np.zeros_like(M), 1e-2, 0.0)
     assert np.sum(C * M2) < np.sum(C * M)
+
+
+# ---------------------------------------------------------------------------
+# inference side (Section 4.1): function preservation, special operators, dequantisation against its definition
+# ---------------------------------------------------------------------------
+def test_inference_apply_preserves_the_product_and_special_cases():
+    rng = np.random.default_rng(11)
+    k, nb = 4, 3
+    W, X = rng.standard_normal((5, nb * k)), rng.standard_normal((7, nb * k))
+    M = orc.round_bf16(rng.standard_normal((nb, k, k)).astype(np.float32)).astype(np.float64)
+    # y = W x = (W o M)(M^-T x): the activations go through the inverse's blocks applied transposed
+    Minv = orc.round_bf16(np.linalg.inv(M).astype(np.float32)).astype(np.float64)     # deployed in bf16
+    U = orc.apply_blocks(W, M, "in", 1)
+    Xp = orc.inference_apply(X, Minv, "in", transpose=True)
+    exact = W @ X.T
+    assert np.abs(U @ Xp.T - exact).max() <= 2.0 ** -7 * np.abs(exact).max() * k      # only the bf16 rounding of M^-1
+    # with an operator that bf16 holds exactly (a signed permutation) the identity is exact
+    P = np.zeros((nb, k, k))
+    for b in range(nb):
+        perm = rng.permutation(k)
+        P[b, np.arange(k), perm] = rng.choice([-1.0, 1.0], k)
+    Up = orc.apply_blocks(W, P, "in", 1)
+    Xq = orc.inference_apply(X, np.linalg.inv(P), "in", transpose=True)
+    assert np.array_equal(Up @ Xq.T, W @ X.T) or np.abs(Up @ Xq.T - W @ X.T).max() < 1e-13
+    # the identity operator returns the input; transpose=True with a symmetric operator changes nothing
+    eye = np.broadcast_to(np.eye(k), (nb, k, k))
+    assert np.array_equal(orc.inference_apply(X, eye), X)
+    S = M + np.transpose(M, (0, 2, 1))
+    assert np.array_equal(orc.inference_apply(X, S, "in", True), orc.inference_apply(X, S, "in", False))
+    # one entry by hand: Y[o, B k + i] = sum_j P[B][i][j] X[o, B k + j]
+    Y = orc.inference_apply(X, M)
+    o, B, i = 3, 1, 2
+    assert abs(Y[o, B * k + i] - sum(M[B, i, j] * X[o, B * k + j] for j in range(k))) < 1e-14
+
+
+def test_dequant_inverts_pack_and_matches_the_quantiser_output():
+    rng = np.random.default_rng(12)
+    U = rng.standard_normal((6, 32)) * np.array([1, 10, 0.1, 1, 3, 1])[:, None]
+    for bits in (3, 4):
+        out = orc.quant_sym(U, bits, 16)
+        q, s, Uhat = out["q"], out["s"], out["Uhat"]
+        packed = orc.pack_codes(q, bits)
+        What = orc.dequant(packed, s, bits, 16, 32)
+        assert np.allclose(What, np.asarray(Uhat, dtype=np.float64), rtol=1e-6, atol=0)   # the quantiser's own s * q
+        # one entry by hand from the bit stream: code i of a row sits at bits [bits * i, bits * i + bits)
+        r, i = 2, 5
+        pos = bits * i
+        word = int(packed[r, pos // 8]) | (int(packed[r, pos // 8 + 1]) << 8)
+        u = (word >> (pos % 8)) & ((1 << bits) - 1)
+        assert abs(What[r, i] - float(s[r, i // 16]) * (u - (2 ** (bits - 1) - 1))) < 1e-12
