@@ -40,7 +40,7 @@ def profiled_traffic():
     import hashlib
     import re
     try:
-        txt = open(os.path.join(ROOT, "profiles", "bd_bwd_kernel_9b_layer.md")).read()
+        txt = open(os.path.join(ROOT, "profiles", "bd_bwd_dual_kernel_9b_layer.md")).read()
         src = b"".join(open(os.path.join(ROOT, "paper_2511_19705_b200", "csrc", f), "rb").read()
                        for f in ("kernels_fused.cuh", "kernels_bwd.cuh"))
         sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]+)", txt).group(1)
@@ -207,7 +207,30 @@ def measure_extras(cq, torch, devS, devP, bits, group, peaks):
                                                        mode=cq.ROUND_LEARNED_OFFSETS), reps=0)
         H = o["pqe"].cpu().numpy()
         out["learned_offsets"] = dict(pair=n, ms_total_2_iterations=t2_ * 1e3, pqe_independent=float(H[0]), pqe_hardened=float(H[-1]))
+    out["inference_apply"] = measure_inference_apply(cq, torch, timed, hbm)
     return out
+
+
+def measure_inference_apply(cq, torch, timed, hbm, tokens=8192, d_in=9216, d_out=2304):
+    """The extra wall-clock time of the block-diagonal multiplication against the product it accompanies, on the shape
+    of Section 4.1's table (down projection of the 2B model: 9216 -> 2304; the operator acts on the 2304-wide side,
+    which is what the table's extra-FLOPs row, k / 9216, counts).  The product is torch's bf16 matmul (library code,
+    used as the yardstick only)."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234)
+    X = torch.randn((tokens, d_in), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    W = (torch.randn((d_out, d_in), generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    t_mm, Y = timed(lambda: X @ W.t())
+    res = dict(tokens=tokens, d_in=d_in, d_out=d_out, matmul_ms=t_mm * 1e3, matmul_tflops=2.0 * tokens * d_in * d_out / t_mm / 1e12,
+               yardstick="torch bf16 matmul", blocks={})
+    for k in (64, 128, 256):
+        T = torch.linalg.qr(torch.randn((d_out // k, k, k), generator=gen, device=dev))[0].contiguous()
+        t, _ = timed(lambda: cq.cafeq_apply_transform(Y, T))
+        by = 2.0 * 2.0 * tokens * d_out                     # bf16 in, bf16 out
+        res["blocks"][str(k)] = dict(ms=t * 1e3, extra_time_pct=100.0 * t / t_mm, extra_flops_pct=100.0 * k / d_in,
+                                     gbs=by / t / 1e9, frac_of_hbm=by / t / 1e9 / hbm)
+    return res
 
 
 # ------------------------------------------------------------------------------------------ main
@@ -477,7 +500,7 @@ def main():
             roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
         roof.update(traffic=profiled_traffic() if (use_layer and args.config == 3) else None,
                     algorithmic_bytes_per_launch=byts * 2 / n_launch if n_launch else None,
-                    kernel="transform pass + sparse backward (bd_pass_kernel + bd_bwd_kernel), the forward+backward of one step",
+                    kernel="transform pass + sparse backward (bd_pass_dual_kernel + bd_bwd_dual_kernel: one launch each for both axes; bd_pass_kernel + bd_bwd_kernel per axis on layers with one axis only), the forward+backward of one step",
                     peak_source=peaks["source"] + ((" burst (SM clock stayed at its maximum through the timed region)" if at_max
                                                     else " sustained (SM clock sagged under load)") if bound_is_tensor else ""),
                     launches_per_step=n_launch, ms_per_step=t_fb * 1e3,

@@ -870,8 +870,8 @@ extern "C" int cafeq_apply_transform(const cafeq_matrix_desc* d, const void* X, 
   float* Tc = b.take<float>(kk);
   uint16_t* Tb = b.take<uint16_t>(kk);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
-  // the deployed operator is the bf16 rounding of the given one (what the tensor cores apply)
-  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, T, Tc, kk, nullptr);
+  // the deployed operator is the bf16 rounding of the given one (what the tensor cores apply; the pass converts it
+  // itself, the shape-agnostic kernels take the rounded fp32 copy)
   const int transposed = d->trole == CAFEQ_APPLY_TT;
   {
     const Geo Ga = apply_geo(G);
@@ -879,10 +879,11 @@ extern "C" int cafeq_apply_transform(const cafeq_matrix_desc* d, const void* X, 
     memset(&p, 0, sizeof(p));
     p.epi = EPI_STORE;
     p.delta = reinterpret_cast<uint16_t*>(Y);
-    if (fused_pass(st, X, G.ld, Ga, Tc, transposed, Tb, p, status, nullptr)) return last_launch();
+    if (fused_pass(st, X, G.ld, Ga, T, transposed, Tb, p, status, nullptr)) return last_launch();
   }
   float* U = b.take<float>(G.n);
   if (b.overflow) return CAFEQ_ERR_WORKSPACE;
+  CQ_LAUNCH(round_bf16_kernel, grid_for(kk), 256, 0, st, T, Tc, kk, nullptr);
   launch_apply(st, X, 1, G.ld, G, Tc, transposed, U, G.d_in, GEMM_STORE, nullptr, status);
   CQ_LAUNCH(f32_to_bf16_kernel, grid_for(G.n), 256, 0, st, U, reinterpret_cast<uint16_t*>(Y), (long long)G.n);
   return last_launch();
