@@ -225,6 +225,33 @@ def test_randomised_hadamard_baseline_and_learning(cq):
     assert e_learned < e_h
 
 
+def test_randomised_hadamard_block_1024_baseline(cq):
+    """The RANDOM column of Section 4.1's table: a randomised Hadamard transform with diagonal blocks of 1024.  The
+    tensor-core pass stops at k = 256; this block size runs on the shape-agnostic kernels (product, group maxima,
+    quantiser, elimination inverse of the 1024 x 1024 blocks).  Codes tie-aware against the oracle, the relative l2
+    error at 1e-3, and the table's ordering against plain round-to-nearest on heavy-tailed weights."""
+    k, d_out, d_in, bits, group = 1024, 192, 2048, 3, 128
+    Wb = syn.weight_student_t(d_out, d_in, seed=2026, n_outlier_channels=4, mult=15.0)
+    Wd, W = to_dev(Wb), w64(Wb)
+    H = syn.hadamard_blocks(d_in // k, k, 37)
+    assert np.array_equal(orc.round_bf16(H), H.astype(np.float64))          # +-1/32: exact in bf16
+    assert np.allclose(H[0].astype(np.float64) @ H[0].astype(np.float64).T, np.eye(k), atol=1e-12)
+    codes, scales = cq.cafeq_rtn(Wd, f32_dev(H), bits=bits, group=group, tblock=k)
+    U = orc.apply_blocks(W, H.astype(np.float64), "in")
+    assert_codes_tie_aware(codes.cpu().numpy(), scales.cpu().numpy(), orc.quant_sym(U, bits, group), U, group)
+
+    def rel_l2(M, kk):
+        o = cq.cafeq_proxy_loss_fwd_bwd(Wd, f32_dev(M), bits=bits, group=group, flags=cq.FLAG_EXACT_LOSS | cq.FLAG_NO_GRAD)
+        assert int(o["status"].item()) == 0
+        L = o["losses"].cpu().numpy()
+        return float(np.sqrt(L[1] / L[2]))
+
+    e_id, e_h = rel_l2(syn.identity_blocks(d_in // 256, 256), 256), rel_l2(H, k)
+    f = orc.single_forward(W, H, bits, group, "in")
+    assert abs(e_h - np.sqrt(f["L2"] / f["normW2"])) <= 1e-3 * e_h
+    assert e_h < 0.9 * e_id
+
+
 def test_fused_full_size_k_matrix_straight_through(cq):
     """k of the 9B-shaped layer (2048 x 3584, k = 256, 3-bit, g = 128) in the straight-through mode, on the launch
     configuration the benchmark's `--loss ste` run times: losses and the whole gradient against the oracle."""
