@@ -3,7 +3,8 @@ the activations (cafeq_apply_transform) and the dequantisation of packed weights
 
 The device writes bf16; both sides therefore round to bf16 at the end.  The fp32 accumulation order differs from the
 oracle's float64 sum, so an output whose exact value lies next to a bf16 rounding boundary may land on the other
-side: such entries must be exactly one bf16 step away and must be rare."""
+side: such entries must be rare, and every entry must lie within half a bf16 step of the exact value plus a bound on
+the fp32 sum's error (which, where the terms cancel, can exceed a bf16 step of the small result)."""
 import numpy as np
 import pytest
 
