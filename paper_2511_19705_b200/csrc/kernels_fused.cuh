@@ -640,41 +640,52 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
             // code = rne(fl32(u / s)).  The IEEE division is a long dependent sequence with a slow-path branch per
             // element; u * (1 / s) differs from the exact quotient by less than 1.5 ulp, and from fl32(u / s) by
             // less than 2 ulp, i.e. by less than (qmax + 1) * 2.4e-7, so it rounds to the same integer unless the
-            // quotient lies within that distance of a half-integer.  Those (rare) chunks are redone with the division.
+            // quotient lies within that distance of a half-integer: those (rare: the transformed values are not on a
+            // coarse grid) chunks are redone with the division.
+            // The rounding itself uses no conversion instruction: t = x + 1.5 * 2^23 holds rne(x) in its low mantissa
+            // bits (the fp32 add rounds to nearest even, as rintf does) and, 0x4B400000 having a zero low byte, the low
+            // byte of t's pattern is the two's-complement code; |x| <= qmax (1 + 3 * 2^-23), so nothing is clamped.
             float qv[32];
+            uint32_t cb[32];
             {
+              constexpr float MAGIC = 12582912.f;
               const float rs = (s > 0.f) ? __frcp_rn(s) : 0.f;
-              const float win = 0.5f - (p.qmax + 1.f) * 1.0e-6f;
-              bool near_half = !(rs < 3.0e38f);  // a scale so small that its reciprocal overflows: take the division
+              const uint32_t winb = __float_as_uint(0.5f - (p.qmax + 1.f) * 1.0e-6f);
+              uint32_t dmax = 0u;  // largest |x - rne(x)| of the chunk, as a bit pattern
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 const float x = v[e] * rs;
-                const float q = rintf(x);
-                near_half |= fabsf(x - q) > win;
-                qv[e] = q;
+                const float t = x + MAGIC;
+                qv[e] = t - MAGIC;
+                cb[e] = __float_as_uint(t);
+                dmax = max(dmax, __float_as_uint(x - qv[e]) & 0x7FFFFFFFu);
               }
-              if (near_half) {
+              // (also: a scale so small that its reciprocal overflows)
+              if (dmax > winb || !(rs < 3.0e38f)) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) qv[e] = (s > 0.f) ? rintf(__fdiv_rn(v[e], s)) : 0.f;
+                for (int e = 0; e < 32; ++e) {
+                  float q = (s > 0.f) ? rintf(__fdiv_rn(v[e], s)) : 0.f;
+                  q = fminf(fmaxf(q, -p.qmax), p.qmax);
+                  qv[e] = q;
+                  cb[e] = (uint32_t)((int)q);
+                }
               }
             }
+            if (want_d) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              const float q0 = fminf(fmaxf(qv[e], -p.qmax), p.qmax);
-              const float q1 = fminf(fmaxf(qv[e + 1], -p.qmax), p.qmax);
-              if (want_d) {
-                const float d0 = s * q0 - v[e], d1 = s * q1 - v[e + 1];
+              for (int e = 0; e < 32; e += 2) {
+                const float d0 = s * qv[e] - v[e], d1 = s * qv[e + 1] - v[e + 1];
                 const __nv_bfloat16 b0 = __float2bfloat16_rn(d0), b1 = __float2bfloat16_rn(d1);
                 dpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
                 if (want_dl)
                   lpk[e >> 1] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d0 - __bfloat162float(b0))) |
                                 ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(d1 - __bfloat162float(b1))) << 16);
               }
-              if (want_c) {
-                const uint32_t c0 = (uint32_t)((int)q0) & 0xFFu, c1 = (uint32_t)((int)q1) & 0xFFu;
-                if ((e & 2) == 0) cpk[e >> 2] = c0 | (c1 << 8);
-                else cpk[e >> 2] |= (c0 << 16) | (c1 << 24);
-              }
+            }
+            if (want_c) {
+#pragma unroll
+              for (int w = 0; w < 8; ++w)
+                cpk[w] = __byte_perm(__byte_perm(cb[4 * w], cb[4 * w + 1], 0x0040), __byte_perm(cb[4 * w + 2], cb[4 * w + 3], 0x0040), 0x5410);
             }
             if (valid && (p.epi & EPI_DELTA)) {
               uint4* dst = reinterpret_cast<uint4*>(p.delta + (long long)row * p.d_in + col0 + ch * 32);
