@@ -278,14 +278,15 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
   uint8_t* sT = smem;
   uint8_t* sStage = smem + C::T_BYTES;
   uint64_t* bars = (uint64_t*)(sStage + C::NSTAGE * BD_STAGE_BYTES);
-  // barrier slots: full[NSTAGE], empty[NSTAGE], tfull, accf[2], acce[2], tfree
+  // barrier slots: full[NSTAGE], empty[NSTAGE], tfull[4] (one per 64-column chunk of the operator: the products on the
+  // first stage of a new block start when a quarter of it has arrived), accf[2], acce[2], tfree
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8 * C::NSTAGE;
   const uint32_t bar_tfull = bar_empty + 8 * C::NSTAGE;
-  const uint32_t bar_accf = bar_tfull + 8;
+  const uint32_t bar_accf = bar_tfull + 32;
   const uint32_t bar_acce = bar_accf + 16;
   const uint32_t bar_tfree = bar_acce + 16;
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 6);
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::NSTAGE + 9);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -297,7 +298,7 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
-    mbar_init(bar_tfull, 1);
+    for (int c = 0; c < 4; ++c) mbar_init(bar_tfull + 8 * c, 1);
     mbar_init(bar_tfree, 1);
     mbar_init(bar_accf, 1);
     mbar_init(bar_accf + 8, 1);
@@ -335,11 +336,13 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
           if (major != cur_major) {
             // the products of the previous operator block must have finished reading it
             if (tloads > 0 && !mbar_wait(bar_tfree, (tloads - 1) & 1u, abort_flag, status)) { ok = false; break; }
-            mbar_expect_tx(bar_tfull, C::T_BYTES);
             for (int bi = 0; bi < C::NBLK; ++bi) {
               const int tb = (FORM == BD_IN) ? (major * C::NBLK + bi) / p.r : major / p.r;
-              for (int ci = 0; ci < K / 64; ++ci)
-                tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), tmT, ci * 64, tb * K, bar_tfull);
+              for (int ci = 0; ci < K / 64; ++ci) {
+                const uint32_t bq = bar_tfull + 8 * (bi * (K / 64) + ci);  // at most four chunks: NBLK * K = 256 or NBLK = 1
+                mbar_expect_tx(bq, K * 128);
+                tma_load_2d(smem_u32(sT + bi * K * K * 2 + ci * K * 128), tmT, ci * 64, tb * K, bq);
+              }
             }
             cur_major = major;
             ++tloads;
@@ -380,8 +383,13 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
         int cur_major = -1;
         for (int tile = lo; tile < hi && ok; ++tile, ++tl) {
           const int major = tile / n_minor;
-          if (major != cur_major) {
-            if (!mbar_wait(bar_tfull, tfulls & 1u, abort_flag, status)) { ok = false; break; }
+          const bool fresh = major != cur_major;  // first tile on a newly loaded operator block
+          const uint32_t tph = tfulls & 1u;
+          if (fresh) {
+            if constexpr (FORM == BD_OUT) {
+              for (int c = 0; c < K / 64 && ok; ++c) ok = mbar_wait(bar_tfull + 8 * c, tph, abort_flag, status);
+              if (!ok) break;
+            }
             ++tfulls;
             cur_major = major;
           }
@@ -393,6 +401,8 @@ __device__ __forceinline__ void bd_pass_body(const BdMaps& maps, const BdMulti& 
             for (int sidx = 0; sidx < BD_STAGES_PER_TILE; ++sidx, ++it) {
               const uint32_t s = it % C::NSTAGE, ph = (it / C::NSTAGE) & 1u;
               if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, status)) { ok = false; break; }
+              // stage sidx multiplies the operator's chunk sidx
+              if (fresh && !mbar_wait(bar_tfull + 8 * sidx, tph, abort_flag, status)) { ok = false; break; }
               tc_fence_after();
               const uint32_t stage = sSt_u + s * BD_STAGE_BYTES;
               const int bi = (sidx * 64) / K, ci = ((sidx * 64) % K) / 64;
